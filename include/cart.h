@@ -1,0 +1,170 @@
+/*
+ * cart.h -- C ABI of the B200 Cartridge decode-attention library (libcart.so).
+ *
+ * The library serves the attention part of decoding with Cartridges (arXiv 2506.06266): every
+ * request attends over a trained, compact KV cache (a Cartridge of p key/value tokens per layer,
+ * Sec. 3.2; possibly several Cartridges concatenated, Sec. 3.1 / Sec. 5.4; possibly shared by many
+ * requests and stored once) followed by the request's own growing suffix KV (Sec. 2.3), exactly as
+ * "a request with a prefix of length p" (Sec. 3.3).
+ *
+ * Conventions that hold for every entry point
+ *   - Returns a cart_status.  Out-parameters are written only on CART_OK.  Nothing throws, aborts
+ *     or exits.  cart_last_error(ctx) gives a one-line reason for the last failure on that context.
+ *   - Arguments are validated on the host before anything is launched; a failing call changes no
+ *     state.
+ *   - "device" pointers are CUDA device pointers on the context's device; "host" pointers are
+ *     ordinary host memory.  Each parameter says which.
+ *   - All device memory comes from the caller: the arena handed to cart_create and the q / k / v /
+ *     out tensors passed per call.  The library itself never allocates device memory.  The arena
+ *     stays owned by the caller and must outlive the context.
+ *   - Calls that take a stream enqueue work on it and return without synchronising.  A context is
+ *     meant to be driven from one host thread on one stream at a time; to switch streams the caller
+ *     orders them (event or synchronise).
+ *   - Tensors are bf16 (upper half of IEEE binary32), head_dim = 128, dense row-major in the stated
+ *     index order.  Device tensor pointers must be 16-byte aligned.
+ *   - Query head h reads KV head h / (n_q_heads / n_kv_heads) (contiguous groups).
+ *   - Keys are stored as given (already position-encoded by the caller); the library applies no
+ *     positional transform and no causal mask: the single decode query of a request sees its whole
+ *     cache [Cartridge(s) ; suffix].
+ */
+#ifndef CART_H_
+#define CART_H_
+
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define CART_API __attribute__((visibility("default")))
+#else
+#define CART_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct cart_ctx cart_ctx; /* opaque */
+typedef int32_t cart_id;          /* Cartridge handle (registered or composed) */
+typedef int32_t cart_req;         /* request handle (owns one suffix KV buffer) */
+#define CART_NONE (-1)            /* "no Cartridge": the request attends to its suffix only */
+
+typedef enum {
+    CART_OK = 0,
+    CART_ERR_INVALID_ARG = 1, /* NULL / misaligned pointer, negative size, bad flag */
+    CART_ERR_SHAPE = 2,       /* head_dim != 128, n_q_heads not a multiple of n_kv_heads, group > 8 */
+    CART_ERR_BAD_HANDLE = 3,  /* unknown, closed or released handle; layer out of range */
+    CART_ERR_CAPACITY = 4,    /* suffix buffer full, handle table full, too many parts */
+    CART_ERR_OOM = 5,         /* the arena has no room left */
+    CART_ERR_EMPTY = 6,       /* a request has no KV token at all in the layer asked for */
+    CART_ERR_IN_USE = 7,      /* releasing a Cartridge that an open request or composition uses */
+    CART_ERR_CUDA = 8,        /* a CUDA runtime / driver call failed (see cart_last_error) */
+    CART_ERR_TIMEOUT = 9      /* a bounded device-side wait ran out (reported by cart_sync_status) */
+} cart_status;
+
+typedef struct {
+    int32_t n_layers;       /* L >= 1 */
+    int32_t n_q_heads;      /* Hq */
+    int32_t n_kv_heads;     /* Hkv; Hq % Hkv == 0 and Hq / Hkv <= 8 */
+    int32_t head_dim;       /* must be 128 */
+    int32_t max_requests;   /* size of the request table (>= 1) */
+    int32_t max_cartridges; /* size of the Cartridge table, compositions included (>= 1) */
+    int32_t max_parts;      /* most registered Cartridges one composition may hold; 0 => 8 */
+    float softmax_scale;    /* multiplies q.k before the softmax; 0 => 1/sqrt(head_dim) (Eq. 1) */
+    void *arena;            /* device; 256-byte aligned; holds every Cartridge, suffix and scratch */
+    uint64_t arena_bytes;
+    int32_t device;         /* CUDA device ordinal the arena lives on */
+} cart_config;
+
+/* Bytes of the arena the library reserves for its own scratch (work lists, split partials) under
+ * this configuration; the rest is available to Cartridges and suffix buffers.  Pure host
+ * arithmetic, needs no device.  *out_bytes is a multiple of 256. */
+CART_API cart_status cart_scratch_bytes(const cart_config *cfg /*host*/, uint64_t *out_bytes /*host*/);
+
+/* Creates a context on cfg->device over the caller's arena.  Makes cfg->device current, builds the
+ * tensor map the kernels use to fetch KV tiles from the arena, allocates small pinned host staging
+ * buffers.  Errors: INVALID_ARG, SHAPE, OOM (arena smaller than the scratch), CUDA. */
+CART_API cart_status cart_create(const cart_config *cfg /*host*/, cart_ctx **out /*host*/);
+
+/* Synchronises the device, frees host-side state.  The arena is untouched.  NULL is accepted. */
+CART_API cart_status cart_destroy(cart_ctx *ctx);
+
+/* Sec. 3.2 / Sec. 3.3: make a trained Cartridge resident ("loaded into the KV cache slots") and
+ * addressable by handle.  k and v are device bf16 [n_layers][n_kv_heads][p][128]; they are copied
+ * into the arena on `stream` (the caller may free them once the stream has passed this point).
+ * p >= 1, the same in every layer.  A Cartridge is stored once however many requests open on it.
+ * Errors: INVALID_ARG, CAPACITY (table full), OOM, CUDA. */
+CART_API cart_status cart_register_cartridge(cart_ctx *ctx, const void *k /*device*/, const void *v /*device*/,
+                                    int32_t p, void *stream /*cudaStream_t*/, cart_id *out /*host*/);
+
+/* Sec. 3.1 ("capable of composition"), Sec. 5.4: the handle returned stands for the concatenation
+ * [Z_1, Z_2, ...] of the parts along the token axis, in list order, with no retraining, no copy and
+ * no re-encoding of positions.  Parts may themselves be compositions (flattened).  The parts stay
+ * referenced until the composition is released.  parts is a host array.
+ * Errors: INVALID_ARG (n_parts < 1), BAD_HANDLE, CAPACITY (more than max_parts registered parts
+ * after flattening, or table full). */
+CART_API cart_status cart_compose(cart_ctx *ctx, const cart_id *parts /*host*/, int32_t n_parts,
+                         cart_id *out /*host*/);
+
+/* Drops a Cartridge or composition.  Its arena space becomes reusable for later registrations; the
+ * caller makes sure no enqueued decode still reads it.  Errors: BAD_HANDLE, IN_USE. */
+CART_API cart_status cart_release_cartridge(cart_ctx *ctx, cart_id id);
+
+/* Opens a request that attends to `cartridge` (or CART_NONE) followed by its own suffix, and
+ * reserves a suffix buffer of suffix_capacity tokens per layer in the arena (Sec. 3.3: per-user KV
+ * caches next to the shared prefix).  suffix_capacity >= 0; it is rounded up to a multiple of 64.
+ * Errors: BAD_HANDLE, CAPACITY (table full), OOM. */
+CART_API cart_status cart_request_open(cart_ctx *ctx, cart_id cartridge, int32_t suffix_capacity,
+                              cart_req *out /*host*/);
+
+/* Closes a request and returns its suffix buffer to the arena.  Errors: BAD_HANDLE. */
+CART_API cart_status cart_request_close(cart_ctx *ctx, cart_req req);
+
+/* Sec. 2.3, decode phase ("append to the KV cache"): for i < n_reqs, writes token i of k_new / v_new
+ * (device bf16 [n_reqs][n_kv_heads][128]) at the end of request reqs[i]'s suffix in `layer`, and
+ * advances that length by one.  reqs is a host array; a handle may appear at most once.
+ * Errors: INVALID_ARG, BAD_HANDLE, CAPACITY (some suffix is full; nothing is appended), CUDA. */
+CART_API cart_status cart_append_kv(cart_ctx *ctx, int32_t layer, const cart_req *reqs /*host*/, int32_t n_reqs,
+                           const void *k_new /*device*/, const void *v_new /*device*/, void *stream);
+
+/* Sec. 2.3, prefill of the user's message: appends n_tokens consecutive tokens to one request's
+ * suffix in `layer`.  k and v are device bf16 [n_tokens][n_kv_heads][128] (token-major, as a
+ * projection over the message's tokens produces them).
+ * Errors: INVALID_ARG, BAD_HANDLE, CAPACITY, CUDA. */
+CART_API cart_status cart_extend_kv(cart_ctx *ctx, int32_t layer, cart_req req, const void *k /*device*/,
+                           const void *v /*device*/, int32_t n_tokens, void *stream);
+
+/* Eq. 1 (Sec. 2.3) at the last position, for a batch: for i < n_reqs and every query head h,
+ *     out[i][h] = sum_j softmax_j(scale * <q[i][h], K*_j>) V*_j,   lse[i][h] = ln sum_j exp(scale * <q[i][h], K*_j>)
+ * where K*, V* are KV head h / G of request reqs[i]'s cache in `layer`: its Cartridge(s) in
+ * composition order, then its suffix (layout of Sec. 3.2).  q and out are device bf16
+ * [n_reqs][n_q_heads][128]; lse is device fp32 [n_reqs][n_q_heads] or NULL.  Products and sums are
+ * accumulated in fp32; out is rounded to nearest-even bf16.  reqs is a host array (duplicates
+ * allowed).  The result does not depend on how the library splits the cache across thread blocks
+ * beyond fp32 rounding, and is bitwise reproducible for the same batch and lengths.
+ * Errors: INVALID_ARG, BAD_HANDLE, EMPTY, CAPACITY (batch larger than max_requests), CUDA. */
+CART_API cart_status cart_decode_attention(cart_ctx *ctx, int32_t layer, const cart_req *reqs /*host*/,
+                                  int32_t n_reqs, const void *q /*device*/, void *out /*device*/,
+                                  float *lse /*device or NULL*/, void *stream);
+
+/* Current suffix length of a request in a layer (host-side mirror). */
+CART_API cart_status cart_suffix_len(cart_ctx *ctx, cart_req req, int32_t layer, int32_t *out_len /*host*/);
+
+/* KV bytes a request attends to, summed over layers (Sec. 3.2: a Cartridge costs what a p-token
+ * prompt costs).  logical counts every Cartridge token as if private; unique_private counts only
+ * the request's own suffix tokens (what is not shared with other requests). */
+CART_API cart_status cart_kv_bytes(cart_ctx *ctx, cart_req req, uint64_t *logical /*host*/,
+                          uint64_t *unique_private /*host*/);
+
+/* Synchronises `stream` and reports the device-side status word: CART_OK, or CART_ERR_TIMEOUT if a
+ * kernel gave up on a bounded wait since the last call (the word is then cleared). */
+CART_API cart_status cart_sync_status(cart_ctx *ctx, void *stream);
+
+/* Number of kernels this context has launched so far (for the benchmark's launch count). */
+CART_API uint64_t cart_launch_count(const cart_ctx *ctx);
+
+CART_API const char *cart_status_string(cart_status s);
+CART_API const char *cart_last_error(const cart_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CART_H_ */

@@ -1,0 +1,84 @@
+/*
+ * cart_plan.h -- the host-side work planner of libcart.so, exported so that it can be tested
+ * without a device.  cart_decode_attention calls it once per (batch, lengths) and reuses the result
+ * for every layer of a decode step.
+ *
+ * The paper gives no schedule (Sec. 3.3 only says a Cartridge is served like a cached prefix of
+ * length p); this split is the library's own.  The KV cache of a (request, KV head) pair -- a "row
+ * group": the G = Hq/Hkv query heads that read the same K/V (GQA) -- is the concatenation of its
+ * segments (Cartridge parts in composition order, then the suffix; Sec. 3.2 layout).  Each segment
+ * is cut into tiles of `tile_tokens` tokens (the last one ragged).  The tiles of all row groups,
+ * laid end to end in batch order, are divided into `n_cta` contiguous, equal (+-1 tile) ranges, one
+ * per persistent thread block.  Where a range boundary falls inside a row group, that row group is
+ * "split": each block holding a piece writes a partial (o, lse) into its own slot and the pieces
+ * are merged by log-sum-exp afterwards (softmax over a union of token sets, from Eq. 1).  A row
+ * group held entirely by one block is written directly.
+ */
+#ifndef CART_PLAN_H_
+#define CART_PLAN_H_
+
+#include <stdint.h>
+#include "cart.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* One KV segment of a request, as rows of 128 bf16 (256 bytes) counted from the arena base. */
+typedef struct {
+    uint32_t k_row;        /* row of token 0, KV head 0, layer 0 (keys) */
+    uint32_t v_row;        /* same for values */
+    uint32_t head_stride;  /* rows between consecutive KV heads (p, or the suffix capacity) */
+    uint32_t layer_stride; /* rows between consecutive layers (n_kv_heads * head_stride) */
+    uint32_t n_tok;        /* tokens in the segment (> 0) */
+} cart_plan_seg;
+
+#define CART_ITEM_BEGIN 1u  /* first item of a row-group piece in this block: load q, reset state */
+#define CART_ITEM_END 2u    /* last item of the piece: combine the warps' states and write */
+#define CART_ITEM_DIRECT 4u /* the piece is the whole row group: write out / lse, not a partial */
+
+/* A run of consecutive tiles of one segment of one row group, processed by one block. */
+typedef struct {
+    uint32_t k_row;        /* first row of the run for layer 0 (KV head already applied) */
+    uint32_t v_row;
+    uint32_t layer_stride; /* add layer * layer_stride to both rows */
+    uint32_t n_tok;        /* tokens in the run (> 0); only the last tile may be ragged */
+    uint32_t row_group;    /* batch index * n_kv_heads + KV head */
+    uint32_t flags;        /* CART_ITEM_* */
+    uint32_t slot;         /* partial slot (meaningful with END and without DIRECT) */
+    uint32_t reserved;
+} cart_work_item;
+
+/* A split row group: its partials are slots slot_begin .. slot_end-1. */
+typedef struct {
+    uint32_t row_group;
+    uint32_t slot_begin;
+    uint32_t slot_end;
+    uint32_t reserved;
+} cart_merge_item;
+
+/*
+ * Builds the plan.  All pointers are host memory.
+ *   segs, seg_begin   request i of the batch owns segs[seg_begin[i] .. seg_begin[i+1]-1], in cache
+ *                     order; every request must own at least one token
+ *   n_cta             persistent blocks available (>= 1)
+ *   tile_tokens       tokens per tile (>= 1)
+ *   items / items_cap work items, grouped by block; block c owns items[cta_begin[c] .. cta_begin[c+1]-1]
+ *   cta_begin         [n_cta + 1]
+ *   merges / merges_cap  one entry per split row group
+ *   n_cta_used        blocks that received work (<= n_cta); blocks beyond it own no item
+ *   n_slots           partial slots used
+ *   total_tiles       tiles in the whole batch
+ * Errors: INVALID_ARG, EMPTY (a request without tokens), CAPACITY (items_cap / merges_cap too small).
+ */
+CART_API cart_status cart_plan_build(const cart_plan_seg *segs, const int32_t *seg_begin, int32_t n_reqs,
+                            int32_t n_kv_heads, int32_t n_cta, int32_t tile_tokens,
+                            cart_work_item *items, int32_t items_cap, int32_t *n_items,
+                            uint32_t *cta_begin, cart_merge_item *merges, int32_t merges_cap,
+                            int32_t *n_merges, int32_t *n_cta_used, int32_t *n_slots,
+                            int64_t *total_tiles);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CART_PLAN_H_ */

@@ -1,0 +1,672 @@
+// Host side of libcart.so: handle tables, the arena allocator, plan caching and kernel launches.
+// The contract of every entry point is stated in include/cart.h.
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "cart.h"
+#include "cart_internal.h"
+
+namespace {
+
+using namespace cart;
+
+constexpr int kMaxCta = 1024;   // upper bound on persistent blocks (device independent)
+constexpr int kPlanSlots = 4;   // ring of uploaded plans
+constexpr uint64_t kAlign = 256;
+
+uint64_t round_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
+
+struct ScratchLayout {
+    uint64_t status_off, plan_off, plan_slot_bytes, cta_begin_off, merges_off, items_off;
+    uint64_t part_o_off, part_lse_off, total;
+    int items_cap, slots_cap;
+};
+
+ScratchLayout scratch_layout(const cart_config &c)
+{
+    ScratchLayout s{};
+    const int parts = c.max_parts > 0 ? c.max_parts : 8;
+    const int group = c.n_q_heads / c.n_kv_heads;
+    s.items_cap = c.max_requests * c.n_kv_heads * (parts + 1) + kMaxCta;
+    s.slots_cap = 2 * kMaxCta;
+    s.status_off = 0;
+    s.plan_off = kAlign;
+    // one plan slot: [cta_begin][merges][items]
+    s.cta_begin_off = 0;
+    s.merges_off = round_up((uint64_t)(kMaxCta + 1) * 4, kAlign);
+    s.items_off = s.merges_off + round_up((uint64_t)kMaxCta * sizeof(cart_merge_item), kAlign);
+    s.plan_slot_bytes = s.items_off + round_up((uint64_t)s.items_cap * sizeof(cart_work_item), kAlign);
+    s.part_o_off = s.plan_off + (uint64_t)kPlanSlots * s.plan_slot_bytes;
+    s.part_lse_off = s.part_o_off + round_up((uint64_t)s.slots_cap * group * kHeadDim * 4, kAlign);
+    s.total = s.part_lse_off + round_up((uint64_t)s.slots_cap * kMaxGroup * 4, kAlign);
+    return s;
+}
+
+cart_status check_config(const cart_config *c)
+{
+    if (!c) return CART_ERR_INVALID_ARG;
+    if (c->n_layers < 1 || c->n_q_heads < 1 || c->n_kv_heads < 1 || c->max_requests < 1 ||
+        c->max_cartridges < 1 || c->max_parts < 0 || !(c->softmax_scale >= 0.f))
+        return CART_ERR_INVALID_ARG;
+    if (c->head_dim != kHeadDim || c->n_q_heads % c->n_kv_heads != 0 ||
+        c->n_q_heads / c->n_kv_heads > kMaxGroup)
+        return CART_ERR_SHAPE;
+    return CART_OK;
+}
+
+struct FreeBlock { uint64_t start, len; };  // in rows of 256 bytes
+
+struct Cartridge {
+    bool live = false;
+    bool composed = false;
+    int32_t p = 0;                 // tokens (sum over parts for a composition)
+    uint64_t k_row = 0, v_row = 0; // registered only
+    uint64_t alloc_start = 0, alloc_rows = 0;
+    std::vector<int32_t> parts;    // composed: registered ids, flattened, in order
+    int32_t refs = 0;              // open requests + compositions that hold it
+};
+
+struct Request {
+    bool live = false;
+    int32_t cart = CART_NONE;
+    int32_t cap = 0;
+    uint64_t k_row = 0, v_row = 0;
+    uint64_t alloc_start = 0, alloc_rows = 0;
+    std::vector<int32_t> len;  // per layer
+    uint64_t stamp = 0;
+};
+
+struct PlanSlot {
+    uint8_t *host = nullptr;   // pinned
+    uint8_t *dev = nullptr;    // inside the arena scratch
+    cudaEvent_t ev = nullptr;
+    bool ev_recorded = false;
+    bool valid = false;
+    cudaStream_t last_stream = nullptr;
+    std::vector<uint32_t> key;
+    uint64_t epoch = 0;
+    int32_t n_items = 0, n_merges = 0, n_cta_used = 0, n_slots = 0;
+};
+
+}  // namespace
+
+struct cart_ctx {
+    cart_config cfg{};
+    ScratchLayout lay{};
+    int group = 1;
+    float scale = 0.f;
+    int n_cta = 0;
+    uint64_t n_rows = 0;
+    alignas(64) CUtensorMap tmap;
+    std::vector<FreeBlock> free_list;
+    std::vector<Cartridge> carts;
+    std::vector<Request> reqs;
+    PlanSlot slots[kPlanSlots];
+    int cur_slot = -1;
+    uint64_t epoch = 1;
+    uint64_t stamp = 0;
+    uint64_t launches = 0;
+    std::vector<cart_plan_seg> seg_tmp;
+    std::vector<int32_t> seg_begin_tmp;
+    std::vector<uint32_t> key_tmp;
+    char err[256] = {0};
+};
+
+namespace {
+
+cart_status fail(cart_ctx *ctx, cart_status st, const char *fmt, ...)
+{
+    if (ctx) {
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(ctx->err, sizeof ctx->err, fmt, ap);
+        va_end(ap);
+    }
+    return st;
+}
+
+#define CART_CUDA(ctx, call)                                                                        \
+    do {                                                                                            \
+        cudaError_t e_ = (call);                                                                    \
+        if (e_ != cudaSuccess)                                                                      \
+            return fail(ctx, CART_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e_));        \
+    } while (0)
+
+bool arena_alloc(cart_ctx *ctx, uint64_t rows, uint64_t *start)
+{
+    for (size_t i = 0; i < ctx->free_list.size(); ++i) {
+        FreeBlock &b = ctx->free_list[i];
+        if (b.len >= rows) {
+            *start = b.start;
+            b.start += rows;
+            b.len -= rows;
+            if (b.len == 0) ctx->free_list.erase(ctx->free_list.begin() + (long)i);
+            return true;
+        }
+    }
+    return false;
+}
+
+void arena_free(cart_ctx *ctx, uint64_t start, uint64_t rows)
+{
+    if (rows == 0) return;
+    auto &fl = ctx->free_list;
+    size_t i = 0;
+    while (i < fl.size() && fl[i].start < start) ++i;
+    fl.insert(fl.begin() + (long)i, FreeBlock{start, rows});
+    if (i + 1 < fl.size() && fl[i].start + fl[i].len == fl[i + 1].start) {
+        fl[i].len += fl[i + 1].len;
+        fl.erase(fl.begin() + (long)i + 1);
+    }
+    if (i > 0 && fl[i - 1].start + fl[i - 1].len == fl[i].start) {
+        fl[i - 1].len += fl[i].len;
+        fl.erase(fl.begin() + (long)i);
+    }
+}
+
+bool aligned16(const void *p) { return p && (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+Cartridge *get_cart(cart_ctx *ctx, cart_id id)
+{
+    if (id < 0 || (size_t)id >= ctx->carts.size() || !ctx->carts[(size_t)id].live) return nullptr;
+    return &ctx->carts[(size_t)id];
+}
+
+Request *get_req(cart_ctx *ctx, cart_req r)
+{
+    if (r < 0 || (size_t)r >= ctx->reqs.size() || !ctx->reqs[(size_t)r].live) return nullptr;
+    return &ctx->reqs[(size_t)r];
+}
+
+uint8_t *arena_ptr(cart_ctx *ctx, uint64_t row) { return static_cast<uint8_t *>(ctx->cfg.arena) + row * kRowBytes; }
+
+cart_status encode_tensor_map(cart_ctx *ctx)
+{
+    typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                 const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                 CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                 CUtensorMapFloatOOBfill);
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    CART_CUDA(ctx, cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+    if (!fn || qres != cudaDriverEntryPointSuccess)
+        return fail(ctx, CART_ERR_CUDA, "the driver does not provide cuTensorMapEncodeTiled");
+    // The whole arena as a matrix of rows of 128 bf16; a KV tile is 64 consecutive rows, fetched as
+    // two boxes of 64 rows x 64 elements (128 bytes, the widest row a 128-byte swizzle allows).
+    const cuuint64_t gdim[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)ctx->n_rows};
+    const cuuint64_t gstride[1] = {(cuuint64_t)kRowBytes};
+    const cuuint32_t box[2] = {64u, (cuuint32_t)kTileTokens};
+    const cuuint32_t estride[2] = {1u, 1u};
+    CUresult r = reinterpret_cast<EncodeFn>(fn)(&ctx->tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ctx->cfg.arena,
+                                                gdim, gstride, box, estride, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(ctx, CART_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+    return CART_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *cart_status_string(cart_status s)
+{
+    switch (s) {
+    case CART_OK: return "CART_OK";
+    case CART_ERR_INVALID_ARG: return "CART_ERR_INVALID_ARG";
+    case CART_ERR_SHAPE: return "CART_ERR_SHAPE";
+    case CART_ERR_BAD_HANDLE: return "CART_ERR_BAD_HANDLE";
+    case CART_ERR_CAPACITY: return "CART_ERR_CAPACITY";
+    case CART_ERR_OOM: return "CART_ERR_OOM";
+    case CART_ERR_EMPTY: return "CART_ERR_EMPTY";
+    case CART_ERR_IN_USE: return "CART_ERR_IN_USE";
+    case CART_ERR_CUDA: return "CART_ERR_CUDA";
+    case CART_ERR_TIMEOUT: return "CART_ERR_TIMEOUT";
+    }
+    return "CART_ERR_UNKNOWN";
+}
+
+const char *cart_last_error(const cart_ctx *ctx) { return ctx ? ctx->err : "no context"; }
+
+uint64_t cart_launch_count(const cart_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+cart_status cart_scratch_bytes(const cart_config *cfg, uint64_t *out_bytes)
+{
+    if (!out_bytes) return CART_ERR_INVALID_ARG;
+    cart_status st = check_config(cfg);
+    if (st != CART_OK) return st;
+    *out_bytes = scratch_layout(*cfg).total;
+    return CART_OK;
+}
+
+cart_status cart_create(const cart_config *cfg, cart_ctx **out)
+{
+    if (!out) return CART_ERR_INVALID_ARG;
+    cart_status st = check_config(cfg);
+    if (st != CART_OK) return st;
+    if (!cfg->arena || (reinterpret_cast<uintptr_t>(cfg->arena) & (kAlign - 1)) != 0 || cfg->device < 0)
+        return CART_ERR_INVALID_ARG;
+    const ScratchLayout lay = scratch_layout(*cfg);
+    if (cfg->arena_bytes < lay.total + kRowBytes) return CART_ERR_OOM;
+    if (cfg->arena_bytes / kRowBytes >= (1ull << 31)) return CART_ERR_INVALID_ARG;
+
+    cart_ctx *ctx = new (std::nothrow) cart_ctx();
+    if (!ctx) return CART_ERR_OOM;
+    ctx->cfg = *cfg;
+    if (ctx->cfg.max_parts == 0) ctx->cfg.max_parts = 8;
+    ctx->lay = lay;
+    ctx->group = cfg->n_q_heads / cfg->n_kv_heads;
+    ctx->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / std::sqrt((float)cfg->head_dim);
+    ctx->n_rows = cfg->arena_bytes / kRowBytes;
+
+    auto bail = [&](cart_status s) {
+        for (auto &sl : ctx->slots) {
+            if (sl.host) cudaFreeHost(sl.host);
+            if (sl.ev) cudaEventDestroy(sl.ev);
+        }
+        delete ctx;
+        return s;
+    };
+    cudaError_t e = cudaSetDevice(cfg->device);
+    if (e != cudaSuccess) return bail(CART_ERR_CUDA);
+    int sms = 0;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, cfg->device);
+    if (e != cudaSuccess || sms < 1) return bail(CART_ERR_CUDA);
+    ctx->n_cta = std::min(sms, kMaxCta);
+    if (prepare_kernels() != cudaSuccess) return bail(CART_ERR_CUDA);
+    if (encode_tensor_map(ctx) != CART_OK) return bail(CART_ERR_CUDA);
+    for (int i = 0; i < kPlanSlots; ++i) {
+        PlanSlot &sl = ctx->slots[i];
+        if (cudaHostAlloc(reinterpret_cast<void **>(&sl.host), lay.plan_slot_bytes, cudaHostAllocDefault) != cudaSuccess)
+            return bail(CART_ERR_CUDA);
+        if (cudaEventCreateWithFlags(&sl.ev, cudaEventDisableTiming) != cudaSuccess) return bail(CART_ERR_CUDA);
+        sl.dev = static_cast<uint8_t *>(cfg->arena) + lay.plan_off + (uint64_t)i * lay.plan_slot_bytes;
+    }
+    if (cudaMemset(static_cast<uint8_t *>(cfg->arena) + lay.status_off, 0, kAlign) != cudaSuccess)
+        return bail(CART_ERR_CUDA);
+
+    const uint64_t first_row = lay.total / kRowBytes;
+    ctx->free_list.push_back(FreeBlock{first_row, ctx->n_rows - first_row});
+    ctx->carts.resize((size_t)cfg->max_cartridges);
+    ctx->reqs.resize((size_t)cfg->max_requests);
+    *out = ctx;
+    return CART_OK;
+}
+
+cart_status cart_destroy(cart_ctx *ctx)
+{
+    if (!ctx) return CART_OK;
+    cudaSetDevice(ctx->cfg.device);
+    cudaDeviceSynchronize();
+    for (auto &sl : ctx->slots) {
+        if (sl.host) cudaFreeHost(sl.host);
+        if (sl.ev) cudaEventDestroy(sl.ev);
+    }
+    delete ctx;
+    return CART_OK;
+}
+
+cart_status cart_register_cartridge(cart_ctx *ctx, const void *k, const void *v, int32_t p, void *stream,
+                                    cart_id *out)
+{
+    if (!ctx) return CART_ERR_INVALID_ARG;
+    if (!out || !aligned16(k) || !aligned16(v) || p < 1)
+        return fail(ctx, CART_ERR_INVALID_ARG, "register: null/misaligned pointer or p < 1");
+    int32_t id = -1;
+    for (size_t i = 0; i < ctx->carts.size(); ++i)
+        if (!ctx->carts[i].live) { id = (int32_t)i; break; }
+    if (id < 0) return fail(ctx, CART_ERR_CAPACITY, "register: Cartridge table full (%d)", ctx->cfg.max_cartridges);
+    const uint64_t rows_one = (uint64_t)ctx->cfg.n_layers * ctx->cfg.n_kv_heads * (uint64_t)p;
+    uint64_t start = 0;
+    if (!arena_alloc(ctx, 2 * rows_one, &start))
+        return fail(ctx, CART_ERR_OOM, "register: arena has no room for %llu bytes",
+                    (unsigned long long)(2 * rows_one * kRowBytes));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(arena_ptr(ctx, start), k, rows_one * kRowBytes, cudaMemcpyDeviceToDevice, s);
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(arena_ptr(ctx, start + rows_one), v, rows_one * kRowBytes, cudaMemcpyDeviceToDevice, s);
+    if (e != cudaSuccess) {
+        arena_free(ctx, start, 2 * rows_one);
+        return fail(ctx, CART_ERR_CUDA, "register: copy failed: %s", cudaGetErrorString(e));
+    }
+    Cartridge &c = ctx->carts[(size_t)id];
+    c = Cartridge();
+    c.live = true;
+    c.p = p;
+    c.k_row = start;
+    c.v_row = start + rows_one;
+    c.alloc_start = start;
+    c.alloc_rows = 2 * rows_one;
+    ++ctx->epoch;
+    *out = id;
+    return CART_OK;
+}
+
+cart_status cart_compose(cart_ctx *ctx, const cart_id *parts, int32_t n_parts, cart_id *out)
+{
+    if (!ctx) return CART_ERR_INVALID_ARG;
+    if (!parts || !out || n_parts < 1) return fail(ctx, CART_ERR_INVALID_ARG, "compose: no parts");
+    std::vector<int32_t> flat;
+    int64_t total = 0;
+    for (int32_t i = 0; i < n_parts; ++i) {
+        Cartridge *c = get_cart(ctx, parts[i]);
+        if (!c) return fail(ctx, CART_ERR_BAD_HANDLE, "compose: part %d is not a live Cartridge", i);
+        if (c->composed) flat.insert(flat.end(), c->parts.begin(), c->parts.end());
+        else flat.push_back(parts[i]);
+        total += c->p;
+    }
+    if ((int32_t)flat.size() > ctx->cfg.max_parts)
+        return fail(ctx, CART_ERR_CAPACITY, "compose: %d parts exceed max_parts = %d", (int)flat.size(), ctx->cfg.max_parts);
+    if (total > INT32_MAX) return fail(ctx, CART_ERR_CAPACITY, "compose: too many tokens");
+    int32_t id = -1;
+    for (size_t i = 0; i < ctx->carts.size(); ++i)
+        if (!ctx->carts[i].live) { id = (int32_t)i; break; }
+    if (id < 0) return fail(ctx, CART_ERR_CAPACITY, "compose: Cartridge table full");
+    for (int32_t b : flat) ++ctx->carts[(size_t)b].refs;
+    Cartridge &c = ctx->carts[(size_t)id];
+    c = Cartridge();
+    c.live = true;
+    c.composed = true;
+    c.p = (int32_t)total;
+    c.parts = flat;
+    ++ctx->epoch;
+    *out = id;
+    return CART_OK;
+}
+
+cart_status cart_release_cartridge(cart_ctx *ctx, cart_id id)
+{
+    if (!ctx) return CART_ERR_INVALID_ARG;
+    Cartridge *c = get_cart(ctx, id);
+    if (!c) return fail(ctx, CART_ERR_BAD_HANDLE, "release: not a live Cartridge");
+    if (c->refs > 0) return fail(ctx, CART_ERR_IN_USE, "release: %d users still hold the Cartridge", c->refs);
+    if (c->composed) {
+        for (int32_t b : c->parts) --ctx->carts[(size_t)b].refs;
+    } else {
+        arena_free(ctx, c->alloc_start, c->alloc_rows);
+    }
+    *c = Cartridge();
+    ++ctx->epoch;
+    return CART_OK;
+}
+
+cart_status cart_request_open(cart_ctx *ctx, cart_id cartridge, int32_t suffix_capacity, cart_req *out)
+{
+    if (!ctx) return CART_ERR_INVALID_ARG;
+    if (!out || suffix_capacity < 0) return fail(ctx, CART_ERR_INVALID_ARG, "open: bad argument");
+    if (cartridge != CART_NONE && !get_cart(ctx, cartridge))
+        return fail(ctx, CART_ERR_BAD_HANDLE, "open: not a live Cartridge");
+    int32_t id = -1;
+    for (size_t i = 0; i < ctx->reqs.size(); ++i)
+        if (!ctx->reqs[i].live) { id = (int32_t)i; break; }
+    if (id < 0) return fail(ctx, CART_ERR_CAPACITY, "open: request table full (%d)", ctx->cfg.max_requests);
+    const int64_t cap = ((int64_t)suffix_capacity + kTileTokens - 1) / kTileTokens * kTileTokens;
+    const uint64_t rows_one = (uint64_t)ctx->cfg.n_layers * ctx->cfg.n_kv_heads * (uint64_t)cap;
+    uint64_t start = 0;
+    if (rows_one > 0 && !arena_alloc(ctx, 2 * rows_one, &start))
+        return fail(ctx, CART_ERR_OOM, "open: arena has no room for a suffix of %lld tokens", (long long)cap);
+    Request &r = ctx->reqs[(size_t)id];
+    r = Request();
+    r.live = true;
+    r.cart = cartridge;
+    r.cap = (int32_t)cap;
+    r.k_row = start;
+    r.v_row = start + rows_one;
+    r.alloc_start = start;
+    r.alloc_rows = 2 * rows_one;
+    r.len.assign((size_t)ctx->cfg.n_layers, 0);
+    if (cartridge != CART_NONE) ++ctx->carts[(size_t)cartridge].refs;
+    ++ctx->epoch;
+    *out = id;
+    return CART_OK;
+}
+
+cart_status cart_request_close(cart_ctx *ctx, cart_req req)
+{
+    if (!ctx) return CART_ERR_INVALID_ARG;
+    Request *r = get_req(ctx, req);
+    if (!r) return fail(ctx, CART_ERR_BAD_HANDLE, "close: not an open request");
+    if (r->cart != CART_NONE) --ctx->carts[(size_t)r->cart].refs;
+    arena_free(ctx, r->alloc_start, r->alloc_rows);
+    *r = Request();
+    ++ctx->epoch;
+    return CART_OK;
+}
+
+cart_status cart_append_kv(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int32_t n_reqs, const void *k_new,
+                           const void *v_new, void *stream)
+{
+    if (!ctx) return CART_ERR_INVALID_ARG;
+    if (!reqs || n_reqs < 1 || !aligned16(k_new) || !aligned16(v_new))
+        return fail(ctx, CART_ERR_INVALID_ARG, "append: null/misaligned pointer or empty batch");
+    if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, CART_ERR_BAD_HANDLE, "append: layer out of range");
+    const uint64_t stamp = ++ctx->stamp;
+    for (int32_t i = 0; i < n_reqs; ++i) {
+        Request *r = get_req(ctx, reqs[i]);
+        if (!r) return fail(ctx, CART_ERR_BAD_HANDLE, "append: reqs[%d] is not an open request", i);
+        if (r->stamp == stamp) return fail(ctx, CART_ERR_INVALID_ARG, "append: reqs[%d] appears twice", i);
+        r->stamp = stamp;
+        if (r->len[(size_t)layer] >= r->cap)
+            return fail(ctx, CART_ERR_CAPACITY, "append: suffix of reqs[%d] is full (%d tokens)", i, r->cap);
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int Hkv = ctx->cfg.n_kv_heads;
+    static_assert(sizeof(AppendParams) <= 4096, "append parameters must fit the kernel parameter space");
+    AppendParams ap;
+    for (int32_t b0 = 0; b0 < n_reqs; b0 += kAppendBatch) {
+        const int32_t n = std::min(kAppendBatch, n_reqs - b0);
+        for (int32_t i = 0; i < n; ++i) {
+            const Request &r = ctx->reqs[(size_t)reqs[b0 + i]];
+            const uint64_t off = (uint64_t)layer * Hkv * (uint64_t)r.cap + (uint64_t)r.len[(size_t)layer];
+            ap.e[i].k_row = (uint32_t)(r.k_row + off);
+            ap.e[i].v_row = (uint32_t)(r.v_row + off);
+            ap.e[i].head_stride = (uint32_t)r.cap;
+        }
+        ap.arena = ctx->cfg.arena;
+        ap.k_new = static_cast<const uint8_t *>(k_new) + (uint64_t)b0 * Hkv * kRowBytes;
+        ap.v_new = static_cast<const uint8_t *>(v_new) + (uint64_t)b0 * Hkv * kRowBytes;
+        ap.n = n;
+        ap.n_kv_heads = Hkv;
+        CART_CUDA(ctx, launch_append(ap, s));
+        ++ctx->launches;
+    }
+    for (int32_t i = 0; i < n_reqs; ++i) ++ctx->reqs[(size_t)reqs[i]].len[(size_t)layer];
+    return CART_OK;
+}
+
+cart_status cart_extend_kv(cart_ctx *ctx, int32_t layer, cart_req req, const void *k, const void *v,
+                           int32_t n_tokens, void *stream)
+{
+    if (!ctx) return CART_ERR_INVALID_ARG;
+    if (!aligned16(k) || !aligned16(v) || n_tokens < 1)
+        return fail(ctx, CART_ERR_INVALID_ARG, "extend: null/misaligned pointer or n_tokens < 1");
+    if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, CART_ERR_BAD_HANDLE, "extend: layer out of range");
+    Request *r = get_req(ctx, req);
+    if (!r) return fail(ctx, CART_ERR_BAD_HANDLE, "extend: not an open request");
+    if ((int64_t)r->len[(size_t)layer] + n_tokens > r->cap)
+        return fail(ctx, CART_ERR_CAPACITY, "extend: %d + %d tokens exceed the capacity %d", r->len[(size_t)layer],
+                    n_tokens, r->cap);
+    ExtendParams ep;
+    const uint64_t off = (uint64_t)layer * ctx->cfg.n_kv_heads * (uint64_t)r->cap + (uint64_t)r->len[(size_t)layer];
+    ep.arena = ctx->cfg.arena;
+    ep.k = k;
+    ep.v = v;
+    ep.k_row = (uint32_t)(r->k_row + off);
+    ep.v_row = (uint32_t)(r->v_row + off);
+    ep.head_stride = (uint32_t)r->cap;
+    ep.n_tokens = n_tokens;
+    ep.n_kv_heads = ctx->cfg.n_kv_heads;
+    CART_CUDA(ctx, launch_extend(ep, static_cast<cudaStream_t>(stream)));
+    ++ctx->launches;
+    r->len[(size_t)layer] += n_tokens;
+    return CART_OK;
+}
+
+cart_status cart_decode_attention(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int32_t n_reqs, const void *q,
+                                  void *out, float *lse, void *stream)
+{
+    if (!ctx) return CART_ERR_INVALID_ARG;
+    if (!reqs || n_reqs < 1 || !aligned16(q) || !aligned16(out) || (lse && (reinterpret_cast<uintptr_t>(lse) & 3u)))
+        return fail(ctx, CART_ERR_INVALID_ARG, "decode: null/misaligned pointer or empty batch");
+    if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, CART_ERR_BAD_HANDLE, "decode: layer out of range");
+    if (n_reqs > ctx->cfg.max_requests)
+        return fail(ctx, CART_ERR_CAPACITY, "decode: batch %d exceeds max_requests %d", n_reqs, ctx->cfg.max_requests);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int Hkv = ctx->cfg.n_kv_heads;
+
+    // The plan depends on which requests are in the batch and on their lengths in this layer.
+    std::vector<uint32_t> &key = ctx->key_tmp;
+    key.clear();
+    key.push_back((uint32_t)n_reqs);
+    for (int32_t i = 0; i < n_reqs; ++i) {
+        Request *r = get_req(ctx, reqs[i]);
+        if (!r) return fail(ctx, CART_ERR_BAD_HANDLE, "decode: reqs[%d] is not an open request", i);
+        const int32_t len = r->len[(size_t)layer];
+        if (len == 0 && r->cart == CART_NONE)
+            return fail(ctx, CART_ERR_EMPTY, "decode: reqs[%d] has no KV token in layer %d", i, layer);
+        key.push_back((uint32_t)reqs[i]);
+        key.push_back((uint32_t)len);
+    }
+
+    PlanSlot *sl = ctx->cur_slot >= 0 ? &ctx->slots[ctx->cur_slot] : nullptr;
+    if (!(sl && sl->valid && sl->epoch == ctx->epoch && sl->key == key)) {
+        // Build a new plan in the next ring slot.
+        if (sl && sl->valid) {
+            CART_CUDA(ctx, cudaEventRecord(sl->ev, sl->last_stream));
+            sl->ev_recorded = true;
+        }
+        const int next = (ctx->cur_slot + 1) % kPlanSlots;
+        PlanSlot &ns = ctx->slots[next];
+        if (ns.ev_recorded) {
+            CART_CUDA(ctx, cudaEventSynchronize(ns.ev));
+            ns.ev_recorded = false;
+        }
+        ns.valid = false;
+        auto &segs = ctx->seg_tmp;
+        auto &sb = ctx->seg_begin_tmp;
+        segs.clear();
+        sb.clear();
+        sb.push_back(0);
+        for (int32_t i = 0; i < n_reqs; ++i) {
+            const Request &r = ctx->reqs[(size_t)reqs[i]];
+            auto push_cart = [&](const Cartridge &c) {
+                cart_plan_seg sg;
+                sg.k_row = (uint32_t)c.k_row;
+                sg.v_row = (uint32_t)c.v_row;
+                sg.head_stride = (uint32_t)c.p;
+                sg.layer_stride = (uint32_t)((uint64_t)Hkv * c.p);
+                sg.n_tok = (uint32_t)c.p;
+                segs.push_back(sg);
+            };
+            if (r.cart != CART_NONE) {
+                const Cartridge &c = ctx->carts[(size_t)r.cart];
+                if (c.composed) for (int32_t b : c.parts) push_cart(ctx->carts[(size_t)b]);
+                else push_cart(c);
+            }
+            const int32_t len = r.len[(size_t)layer];
+            if (len > 0) {
+                cart_plan_seg sg;
+                sg.k_row = (uint32_t)r.k_row;
+                sg.v_row = (uint32_t)r.v_row;
+                sg.head_stride = (uint32_t)r.cap;
+                sg.layer_stride = (uint32_t)((uint64_t)Hkv * r.cap);
+                sg.n_tok = (uint32_t)len;
+                segs.push_back(sg);
+            }
+            sb.push_back((int32_t)segs.size());
+        }
+        const ScratchLayout &lay = ctx->lay;
+        int64_t total_tiles = 0;
+        cart_status st = cart_plan_build(
+            segs.data(), sb.data(), n_reqs, Hkv, ctx->n_cta, kTileTokens,
+            reinterpret_cast<cart_work_item *>(ns.host + lay.items_off), lay.items_cap, &ns.n_items,
+            reinterpret_cast<uint32_t *>(ns.host + lay.cta_begin_off),
+            reinterpret_cast<cart_merge_item *>(ns.host + lay.merges_off), kMaxCta, &ns.n_merges, &ns.n_cta_used,
+            &ns.n_slots, &total_tiles);
+        if (st != CART_OK) return fail(ctx, st, "decode: planning failed (%s)", cart_status_string(st));
+        if (ns.n_slots > lay.slots_cap) return fail(ctx, CART_ERR_CAPACITY, "decode: too many partial slots");
+        const uint64_t bytes = lay.items_off + (uint64_t)ns.n_items * sizeof(cart_work_item);
+        CART_CUDA(ctx, cudaMemcpyAsync(ns.dev, ns.host, bytes, cudaMemcpyHostToDevice, s));
+        ns.key = key;
+        ns.epoch = ctx->epoch;
+        ns.valid = true;
+        ctx->cur_slot = next;
+        sl = &ns;
+    }
+    sl->last_stream = s;
+
+    uint8_t *arena = static_cast<uint8_t *>(ctx->cfg.arena);
+    DecodeParams dp;
+    dp.cta_begin = reinterpret_cast<const uint32_t *>(sl->dev + ctx->lay.cta_begin_off);
+    dp.items = reinterpret_cast<const cart_work_item *>(sl->dev + ctx->lay.items_off);
+    dp.q = q;
+    dp.out = out;
+    dp.lse = lse;
+    dp.part_o = reinterpret_cast<float *>(arena + ctx->lay.part_o_off);
+    dp.part_lse2 = reinterpret_cast<float *>(arena + ctx->lay.part_lse_off);
+    dp.status = reinterpret_cast<uint32_t *>(arena + ctx->lay.status_off);
+    dp.layer = layer;
+    dp.group = ctx->group;
+    dp.scale_log2 = ctx->scale * 1.4426950408889634f;
+    CART_CUDA(ctx, launch_decode(ctx->tmap, dp, sl->n_cta_used, s));
+    ++ctx->launches;
+    if (sl->n_merges > 0) {
+        MergeParams mp;
+        mp.merges = reinterpret_cast<const cart_merge_item *>(sl->dev + ctx->lay.merges_off);
+        mp.part_o = dp.part_o;
+        mp.part_lse2 = dp.part_lse2;
+        mp.out = out;
+        mp.lse = lse;
+        mp.group = ctx->group;
+        CART_CUDA(ctx, launch_merge(mp, sl->n_merges, s));
+        ++ctx->launches;
+    }
+    return CART_OK;
+}
+
+cart_status cart_suffix_len(cart_ctx *ctx, cart_req req, int32_t layer, int32_t *out_len)
+{
+    if (!ctx) return CART_ERR_INVALID_ARG;
+    if (!out_len) return fail(ctx, CART_ERR_INVALID_ARG, "suffix_len: null out");
+    Request *r = get_req(ctx, req);
+    if (!r || layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, CART_ERR_BAD_HANDLE, "suffix_len: bad handle");
+    *out_len = r->len[(size_t)layer];
+    return CART_OK;
+}
+
+cart_status cart_kv_bytes(cart_ctx *ctx, cart_req req, uint64_t *logical, uint64_t *unique_private)
+{
+    if (!ctx) return CART_ERR_INVALID_ARG;
+    if (!logical || !unique_private) return fail(ctx, CART_ERR_INVALID_ARG, "kv_bytes: null out");
+    Request *r = get_req(ctx, req);
+    if (!r) return fail(ctx, CART_ERR_BAD_HANDLE, "kv_bytes: not an open request");
+    const uint64_t per_token = 2ull * ctx->cfg.n_kv_heads * kRowBytes;  // K and V, all KV heads, one layer
+    uint64_t suffix = 0;
+    for (int32_t l : r->len) suffix += (uint64_t)l;
+    const uint64_t cart_tokens = r->cart == CART_NONE ? 0ull : (uint64_t)ctx->carts[(size_t)r->cart].p;
+    *unique_private = suffix * per_token;
+    *logical = (cart_tokens * (uint64_t)ctx->cfg.n_layers + suffix) * per_token;
+    return CART_OK;
+}
+
+cart_status cart_sync_status(cart_ctx *ctx, void *stream)
+{
+    if (!ctx) return CART_ERR_INVALID_ARG;
+    CART_CUDA(ctx, cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+    uint32_t word = 0;
+    uint8_t *st = static_cast<uint8_t *>(ctx->cfg.arena) + ctx->lay.status_off;
+    CART_CUDA(ctx, cudaMemcpy(&word, st, 4, cudaMemcpyDeviceToHost));
+    if (word != 0) {
+        CART_CUDA(ctx, cudaMemset(st, 0, 4));
+        return fail(ctx, CART_ERR_TIMEOUT, "a device-side wait ran out (status word 0x%x)", word);
+    }
+    return CART_OK;
+}
+
+}  // extern "C"

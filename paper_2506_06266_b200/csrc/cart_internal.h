@@ -1,0 +1,82 @@
+// Internal declarations shared by the host API (cart_api.cc) and the kernels (cart_kernels.cu).
+#ifndef CART_INTERNAL_H_
+#define CART_INTERNAL_H_
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "cart_plan.h"
+
+namespace cart {
+
+constexpr int kHeadDim = 128;
+constexpr int kRowBytes = kHeadDim * 2;  // one token of one KV head: 128 bf16
+constexpr int kTileTokens = 64;          // tokens per shared-memory stage
+constexpr int kMaxGroup = 8;             // query heads per KV head the kernels support
+constexpr int kAppendBatch = 256;        // requests one append launch takes (kernel-parameter budget)
+
+// bits of the device status word
+constexpr uint32_t kStatusTimeoutProducer = 1u;
+constexpr uint32_t kStatusTimeoutConsumer = 2u;
+
+struct DecodeParams {
+    const uint32_t *cta_begin;   // [grid + 1]
+    const cart_work_item *items;
+    const void *q;               // bf16 [n_reqs][Hq][128]
+    void *out;                   // bf16 [n_reqs][Hq][128]
+    float *lse;                  // fp32 [n_reqs][Hq] or null
+    float *part_o;               // fp32 [slot][G][128], normalised partial outputs
+    float *part_lse2;            // fp32 [slot][kMaxGroup], base-2 log-sum-exp of a partial
+    uint32_t *status;
+    int32_t layer;
+    int32_t group;               // G
+    float scale_log2;            // softmax scale * log2(e)
+};
+
+struct MergeParams {
+    const cart_merge_item *merges;
+    const float *part_o;
+    const float *part_lse2;
+    void *out;
+    float *lse;
+    int32_t group;
+};
+
+struct AppendEntry {
+    uint32_t k_row;        // destination row of KV head 0 (layer and position applied)
+    uint32_t v_row;
+    uint32_t head_stride;  // rows between KV heads
+};
+
+struct AppendParams {
+    AppendEntry e[kAppendBatch];
+    void *arena;
+    const void *k_new;  // bf16 [n][Hkv][128], already offset to the first request of this launch
+    const void *v_new;
+    int32_t n;
+    int32_t n_kv_heads;
+};
+
+struct ExtendParams {
+    void *arena;
+    const void *k;  // bf16 [T][Hkv][128]
+    const void *v;
+    uint32_t k_row; // destination row of KV head 0, first new token
+    uint32_t v_row;
+    uint32_t head_stride;
+    int32_t n_tokens;
+    int32_t n_kv_heads;
+};
+
+// Launchers (defined in cart_kernels.cu).  Each returns the cudaError_t of the launch.
+size_t decode_smem_bytes();
+int decode_threads();
+cudaError_t prepare_kernels();  // sets the dynamic shared-memory attribute; call once per device
+cudaError_t launch_decode(const CUtensorMap &tmap, const DecodeParams &p, int grid, cudaStream_t s);
+cudaError_t launch_merge(const MergeParams &p, int n_merges, cudaStream_t s);
+cudaError_t launch_append(const AppendParams &p, cudaStream_t s);
+cudaError_t launch_extend(const ExtendParams &p, cudaStream_t s);
+
+}  // namespace cart
+#endif

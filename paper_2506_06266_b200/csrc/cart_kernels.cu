@@ -1,0 +1,531 @@
+// sm_100a kernels of libcart.so: split-KV decode attention over [Cartridge(s) ; suffix], the
+// log-sum-exp merge of split row groups, and the KV append / extend scatters.
+//
+// Decode kernel in one paragraph.  One persistent block per SM walks its list of work items (runs
+// of 64-token tiles of one KV segment of one (request, KV head) row group).  A producer warp streams
+// K and V tiles from HBM into a ring of shared-memory stages with TMA (cp.async.bulk.tensor, 128-byte
+// swizzle, completion on mbarriers); eight consumer warps each take whole tiles round-robin.  A
+// consumer multiplies the group's G query heads (padded to the 16 rows of an m16n8k16 bf16 MMA, so
+// a K/V tile is read once per group) with the tile, keeps an fp32 online softmax (running max, sum,
+// rescaled output) in registers, and multiplies the probabilities with V.  At the end of a row-group
+// piece the warps' states are combined through shared memory and written either as the final bf16
+// output + lse (piece = whole row group) or as an fp32 partial that the merge kernel combines.
+// Arithmetic follows Eq. 1 of the paper evaluated at the last position; the split and the merge use
+// that a softmax over a union of token sets is the lse-weighted mix of the softmaxes over the sets.
+#include <cuda_bf16.h>
+
+#include "cart_internal.h"
+
+namespace cart {
+namespace {
+
+constexpr int kStages = 6;
+constexpr int kConsumerWarps = 8;
+constexpr int kConsumerThreads = kConsumerWarps * 32;
+constexpr int kThreads = kConsumerThreads + 32;
+constexpr uint32_t kHalfBytes = kTileTokens * 128;    // 64 tokens x 64 dims of bf16
+constexpr uint32_t kTileBytes = 2 * kHalfBytes;       // K or V tile: 64 tokens x 128 dims
+constexpr uint32_t kStageBytes = 2 * kTileBytes;      // K tile then V tile
+constexpr int kScratchStride = 132;                   // floats per scratch row (128 + pad)
+constexpr uint32_t kScratchOBytes = kConsumerWarps * kMaxGroup * kScratchStride * 4;
+constexpr uint32_t kScratchMLBytes = kConsumerWarps * kMaxGroup * 2 * 4;
+constexpr uint32_t kBarrierBytes = 3 * kStages * 8;
+constexpr uint32_t kSmemUsed = kStages * kStageBytes + kScratchOBytes + kScratchMLBytes + kBarrierBytes + 16;
+constexpr uint32_t kSmemBytes = kSmemUsed + 1024;     // slack to align the stages to 1024 bytes
+static_assert(kSmemBytes <= 232448, "shared memory budget of one sm_100 block exceeded");
+
+constexpr uint64_t kWaitLimitNs = 2000000000ull;      // a wait gives up after about two seconds
+
+// ---- small PTX wrappers ---------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p)
+{
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ uint64_t global_timer_ns()
+{
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false if the block has given up (this wait ran out, or another warp's did).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag,
+                                          uint32_t *status, uint32_t code)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    const uint64_t t0 = global_timer_ns();
+    uint32_t spins = 0;
+    for (;;) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((++spins & 0xFFu) == 0) {
+            if (*abort_flag) return false;
+            if (global_timer_ns() - t0 > kWaitLimitNs) {
+                *abort_flag = 1;
+                atomicOr(status, code);
+                return false;
+            }
+        }
+    }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tmap, int32_t x, int32_t y,
+                                            uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr)
+                 : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr)
+                 : "memory");
+}
+// D += A(16x16, row) * B(16x8, col); rows 8..15 of A are zero here, so a1 = a3 = 0.
+__device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1)
+{
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ float fast_exp2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+__device__ __forceinline__ void consumer_bar()
+{
+    asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory");
+}
+
+// Online-softmax state of one warp for one row-group piece.  Thread (lane) owns query row lane/4
+// (valid when < G) and, per 8-wide column tile, columns 2*(lane%4) and 2*(lane%4)+1.
+struct WarpState {
+    float o[16][4];  // output accumulator, 16 tiles of 8 dims; [.][2..3] belong to the zero rows 8..15
+    float m;         // running maximum of the scaled scores (base-2 units)
+    float l;         // this thread's share of the running sum of 2^(score - m)
+};
+
+// One 64-token tile: scores, online softmax update, probabilities times V.
+__device__ __forceinline__ void process_tile(WarpState &st, const uint32_t (&qa0)[8], const uint32_t (&qa2)[8],
+                                             uint32_t kbase, uint32_t vbase, uint32_t full_k, uint32_t full_v,
+                                             uint32_t parity, int valid, float scale_log2, int lane,
+                                             volatile uint32_t *abort_flag, uint32_t *status, bool &ok)
+{
+    const int l7 = lane & 7;
+    const int lm = lane >> 3;
+    ok = mbar_wait(full_k, parity, abort_flag, status, kStatusTimeoutConsumer);
+    if (!ok) return;
+
+    // ---- S = Q K^T : 16 (padded heads) x 64 tokens, fp32 ------------------------------------
+    float s[8][4];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
+#pragma unroll
+    for (int kp = 0; kp < 4; ++kp) {  // 32 dims per step
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {  // 8 tokens per column tile
+            const uint32_t addr = kbase + (uint32_t)(kp >> 1) * kHalfBytes + (uint32_t)(8 * j + l7) * 128u +
+                                  (uint32_t)(((4 * (kp & 1) + lm) ^ l7) << 4);
+            uint32_t b0, b1, b2, b3;
+            ldmatrix_x4(addr, b0, b1, b2, b3);
+            mma_bf16(s[j], qa0[2 * kp], qa2[2 * kp], b0, b1);
+            mma_bf16(s[j], qa0[2 * kp + 1], qa2[2 * kp + 1], b2, b3);
+        }
+    }
+
+    // ---- online softmax on the valid rows (c0, c1 of every column tile) ------------------------
+    const int col0 = 2 * (lane & 3);
+    float mx = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        float x0 = s[j][0] * scale_log2, x1 = s[j][1] * scale_log2;
+        if (valid < kTileTokens) {  // ragged last tile of a segment: tokens >= valid do not exist
+            if (8 * j + col0 >= valid) x0 = -INFINITY;
+            if (8 * j + col0 + 1 >= valid) x1 = -INFINITY;
+        }
+        s[j][0] = x0;
+        s[j][1] = x1;
+        mx = fmaxf(mx, fmaxf(x0, x1));
+    }
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+    const float m_new = fmaxf(st.m, mx);
+    const float alpha = fast_exp2(st.m - m_new);  // 0 on the first tile (st.m = -inf)
+    st.m = m_new;
+    float psum = 0.f;
+    uint32_t pa0[4], pa2[4];  // probabilities as the A operand of the second MMA, 16 tokens per step
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+        const float p00 = fast_exp2(s[2 * t][0] - m_new), p01 = fast_exp2(s[2 * t][1] - m_new);
+        const float p10 = fast_exp2(s[2 * t + 1][0] - m_new), p11 = fast_exp2(s[2 * t + 1][1] - m_new);
+        psum += (p00 + p01) + (p10 + p11);
+        pa0[t] = pack_bf16(p00, p01);
+        pa2[t] = pack_bf16(p10, p11);
+    }
+    st.l = st.l * alpha + psum;
+#pragma unroll
+    for (int d = 0; d < 16; ++d) {
+        st.o[d][0] *= alpha;
+        st.o[d][1] *= alpha;
+    }
+
+    // ---- O += P V ---------------------------------------------------------------------------------
+    ok = mbar_wait(full_v, parity, abort_flag, status, kStatusTimeoutConsumer);
+    if (!ok) return;
+    int ksteps = 4;
+    if (valid < kTileTokens) {
+        // Rows past the segment's end hold whatever follows it in memory.  Their probability is zero,
+        // but 0 * NaN would poison the sum, so clear the rows that the last 16-token step still reads.
+        ksteps = (valid + 15) >> 4;
+        const int row_end = ksteps << 4;
+        for (int idx = lane; idx < (row_end - valid) * 16; idx += 32) {
+            const int r = valid + (idx >> 4), c = idx & 15;
+            const uint32_t a = vbase + (uint32_t)(c >> 3) * kHalfBytes + (uint32_t)r * 128u + (uint32_t)((c & 7) << 4);
+            asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0u) : "memory");
+        }
+        __syncwarp();
+    }
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+        if (t < ksteps) {
+#pragma unroll
+            for (int dp = 0; dp < 8; ++dp) {  // two 8-dim column tiles per load
+                const uint32_t addr = vbase + (uint32_t)(dp >> 2) * kHalfBytes +
+                                      (uint32_t)(16 * t + 8 * (lm & 1) + l7) * 128u +
+                                      (uint32_t)(((2 * (dp & 3) + (lm >> 1)) ^ l7) << 4);
+                uint32_t b0, b1, b2, b3;
+                ldmatrix_x4_trans(addr, b0, b1, b2, b3);
+                mma_bf16(st.o[2 * dp], pa0[t], pa2[t], b0, b1);
+                mma_bf16(st.o[2 * dp + 1], pa0[t], pa2[t], b2, b3);
+            }
+        }
+    }
+    if (valid < kTileTokens) {
+        // the zeroing above wrote through the generic proxy; order it before the next TMA write
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeParams p)
+{
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t *smem = smem_raw + (base - raw);
+    const uint32_t stages = base;
+    float *scratch_o = reinterpret_cast<float *>(smem + kStages * kStageBytes);
+    float *scratch_ml = reinterpret_cast<float *>(smem + kStages * kStageBytes + kScratchOBytes);
+    const uint32_t bars = base + kStages * kStageBytes + kScratchOBytes + kScratchMLBytes;
+    volatile uint32_t *abort_flag =
+        reinterpret_cast<volatile uint32_t *>(smem + kStages * kStageBytes + kScratchOBytes + kScratchMLBytes + kBarrierBytes);
+    auto full_k = [&](int s) { return bars + (uint32_t)s * 8u; };
+    auto full_v = [&](int s) { return bars + (uint32_t)(kStages + s) * 8u; };
+    auto empty = [&](int s) { return bars + (uint32_t)(2 * kStages + s) * 8u; };
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(full_k(s), 1);
+            mbar_init(full_v(s), 1);
+            mbar_init(empty(s), 1);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    const uint32_t item_begin = p.cta_begin[blockIdx.x];
+    const uint32_t item_end = p.cta_begin[blockIdx.x + 1];
+
+    if (warp == kConsumerWarps) {
+        // ================= producer: one thread feeds the ring ====================================
+        if (lane == 0) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap)) : "memory");
+            uint32_t t = 0;  // tiles issued by this block so far
+            bool ok = true;
+            for (uint32_t it = item_begin; it < item_end && ok; ++it) {
+                const cart_work_item w = p.items[it];
+                const uint32_t k_row = w.k_row + (uint32_t)p.layer * w.layer_stride;
+                const uint32_t v_row = w.v_row + (uint32_t)p.layer * w.layer_stride;
+                const uint32_t ntiles = (w.n_tok + kTileTokens - 1) / kTileTokens;
+                for (uint32_t j = 0; j < ntiles; ++j, ++t) {
+                    const int s = (int)(t % kStages);
+                    const uint32_t round = t / kStages;
+                    ok = mbar_wait(empty(s), (round & 1u) ^ 1u, abort_flag, p.status, kStatusTimeoutProducer);
+                    if (!ok) break;
+                    const uint32_t kdst = stages + (uint32_t)s * kStageBytes;
+                    const uint32_t vdst = kdst + kTileBytes;
+                    const int32_t yk = (int32_t)(k_row + j * kTileTokens);
+                    const int32_t yv = (int32_t)(v_row + j * kTileTokens);
+                    mbar_expect_tx(full_k(s), kTileBytes);
+                    tma_load_2d(kdst, &tmap, 0, yk, full_k(s));
+                    tma_load_2d(kdst + kHalfBytes, &tmap, 64, yk, full_k(s));
+                    mbar_expect_tx(full_v(s), kTileBytes);
+                    tma_load_2d(vdst, &tmap, 0, yv, full_v(s));
+                    tma_load_2d(vdst + kHalfBytes, &tmap, 64, yv, full_v(s));
+                }
+            }
+            if (!ok) {
+                // Gave up: no new copies are issued; wait (bounded) for those still in flight so that
+                // none lands in shared memory after the block has gone.
+                const uint32_t issued = t;
+                for (uint32_t u = (issued > (uint32_t)kStages ? issued - kStages : 0u); u < issued; ++u) {
+                    const int s = (int)(u % kStages);
+                    const uint32_t par = (u / kStages) & 1u;
+                    const uint64_t t0 = global_timer_ns();
+                    while (!mbar_try_wait(full_k(s), par) && global_timer_ns() - t0 < kWaitLimitNs) {}
+                    while (!mbar_try_wait(full_v(s), par) && global_timer_ns() - t0 < kWaitLimitNs) {}
+                }
+            }
+        }
+        return;
+    }
+
+    // ===================== consumers ==============================================================
+    const int G = p.group;
+    const int row = lane >> 2;  // query head inside the group that this thread's c0/c1 belong to
+    const __nv_bfloat16 *q = reinterpret_cast<const __nv_bfloat16 *>(p.q);
+    WarpState st;
+    uint32_t qa0[8], qa2[8];
+    uint32_t t = 0;       // tiles seen by this block so far (same count as the producer's)
+    uint32_t piece = 0;   // tiles seen in the current row-group piece
+    bool alive = true;    // false once the block has given up
+
+    for (uint32_t it = item_begin; it < item_end; ++it) {
+        const cart_work_item w = p.items[it];
+        if (w.flags & CART_ITEM_BEGIN) {
+            piece = 0;
+            st.m = -INFINITY;
+            st.l = 0.f;
+#pragma unroll
+            for (int d = 0; d < 16; ++d) st.o[d][0] = st.o[d][1] = st.o[d][2] = st.o[d][3] = 0.f;
+            if (row < G) {
+                const uint32_t *qrow = reinterpret_cast<const uint32_t *>(
+                    q + ((size_t)w.row_group * G + row) * kHeadDim);
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    qa0[kk] = __ldg(qrow + kk * 8 + (lane & 3));
+                    qa2[kk] = __ldg(qrow + kk * 8 + 4 + (lane & 3));
+                }
+            } else {
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) qa0[kk] = qa2[kk] = 0u;
+            }
+        }
+        const uint32_t ntiles = (w.n_tok + kTileTokens - 1) / kTileTokens;
+        // this warp takes the tiles whose index within the piece is congruent to its number
+        uint32_t j = (uint32_t)((warp + kConsumerWarps - (int)(piece % kConsumerWarps)) % kConsumerWarps);
+        for (; j < ntiles; j += kConsumerWarps) {
+            if (!alive) break;
+            const uint32_t tt = t + j;
+            const int s = (int)(tt % kStages);
+            const uint32_t parity = (tt / kStages) & 1u;
+            const uint32_t kbase = stages + (uint32_t)s * kStageBytes;
+            const int valid = min((int)kTileTokens, (int)(w.n_tok - j * kTileTokens));
+            bool ok;
+            process_tile(st, qa0, qa2, kbase, kbase + kTileBytes, full_k(s), full_v(s), parity, valid,
+                         p.scale_log2, lane, abort_flag, p.status, ok);
+            if (!ok) { alive = false; break; }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty(s));
+        }
+        t += ntiles;
+        piece += ntiles;
+
+        if (w.flags & CART_ITEM_END) {
+            // ---- combine the eight warps' states -------------------------------------------------
+            float lsum = st.l;
+            lsum += __shfl_xor_sync(0xffffffffu, lsum, 1);
+            lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);
+            if (row < G) {
+                float *so = scratch_o + ((size_t)warp * kMaxGroup + row) * kScratchStride + 2 * (lane & 3);
+#pragma unroll
+                for (int d = 0; d < 16; ++d)
+                    *reinterpret_cast<float2 *>(so + 8 * d) = make_float2(st.o[d][0], st.o[d][1]);
+                if ((lane & 3) == 0) {
+                    scratch_ml[(warp * kMaxGroup + row) * 2 + 0] = st.m;
+                    scratch_ml[(warp * kMaxGroup + row) * 2 + 1] = lsum;
+                }
+            }
+            consumer_bar();
+            if (*abort_flag) alive = false;
+            for (int idx = threadIdx.x; idx < G * 64; idx += kConsumerThreads) {
+                const int r = idx >> 6, dpair = idx & 63;
+                float M = -INFINITY;
+#pragma unroll
+                for (int wv = 0; wv < kConsumerWarps; ++wv) M = fmaxf(M, scratch_ml[(wv * kMaxGroup + r) * 2]);
+                float L = 0.f, a0 = 0.f, a1 = 0.f;
+#pragma unroll
+                for (int wv = 0; wv < kConsumerWarps; ++wv) {
+                    const float wgt = fast_exp2(scratch_ml[(wv * kMaxGroup + r) * 2] - M);
+                    L += wgt * scratch_ml[(wv * kMaxGroup + r) * 2 + 1];
+                    const float2 v = *reinterpret_cast<const float2 *>(
+                        scratch_o + ((size_t)wv * kMaxGroup + r) * kScratchStride + 2 * dpair);
+                    a0 += wgt * v.x;
+                    a1 += wgt * v.y;
+                }
+                const float inv = 1.f / L;
+                const float lse2 = M + log2f(L);
+                if (alive) {
+                    if (w.flags & CART_ITEM_DIRECT) {
+                        const size_t orow = (size_t)w.row_group * G + r;
+                        __nv_bfloat162 *op = reinterpret_cast<__nv_bfloat162 *>(
+                            reinterpret_cast<__nv_bfloat16 *>(p.out) + orow * kHeadDim + 2 * dpair);
+                        *op = __floats2bfloat162_rn(a0 * inv, a1 * inv);
+                        if (dpair == 0 && p.lse) p.lse[orow] = lse2 * 0.6931471805599453f;
+                    } else {
+                        float2 *pp = reinterpret_cast<float2 *>(
+                            p.part_o + ((size_t)w.slot * G + r) * kHeadDim + 2 * dpair);
+                        *pp = make_float2(a0 * inv, a1 * inv);
+                        if (dpair == 0) p.part_lse2[(size_t)w.slot * kMaxGroup + r] = lse2;
+                    }
+                }
+            }
+            consumer_bar();  // the scratch may be overwritten by the next piece from here on
+        }
+    }
+}
+
+// One block per split row group: out = sum_c 2^(lse_c - lse) o_c, lse = log2 sum_c 2^lse_c.
+__global__ void __launch_bounds__(128) cart_merge_kernel(const MergeParams p)
+{
+    const cart_merge_item mi = p.merges[blockIdx.x];
+    const int G = p.group;
+    const int d = threadIdx.x;  // 128 threads, one per dim
+    for (int r = 0; r < G; ++r) {
+        float M = -INFINITY;
+        for (uint32_t c = mi.slot_begin; c < mi.slot_end; ++c)
+            M = fmaxf(M, p.part_lse2[(size_t)c * kMaxGroup + r]);
+        float L = 0.f, acc = 0.f;
+        for (uint32_t c = mi.slot_begin; c < mi.slot_end; ++c) {
+            const float wgt = fast_exp2(p.part_lse2[(size_t)c * kMaxGroup + r] - M);
+            L += wgt;
+            acc += wgt * p.part_o[((size_t)c * G + r) * kHeadDim + d];
+        }
+        const size_t orow = (size_t)mi.row_group * G + r;
+        reinterpret_cast<__nv_bfloat16 *>(p.out)[orow * kHeadDim + d] = __float2bfloat16_rn(acc / L);
+        if (d == 0 && p.lse) p.lse[orow] = (M + log2f(L)) * 0.6931471805599453f;
+    }
+}
+
+// One block per request: copy the new token's K and V rows (Hkv x 256 bytes each) to the suffix end.
+__global__ void __launch_bounds__(128) cart_append_kernel(const __grid_constant__ AppendParams p)
+{
+    const int i = blockIdx.x;
+    const AppendEntry e = p.e[i];
+    const int chunks = p.n_kv_heads * 16;  // 16-byte chunks per tensor
+    uint4 *arena = reinterpret_cast<uint4 *>(p.arena);
+    const uint4 *ks = reinterpret_cast<const uint4 *>(p.k_new) + (size_t)i * chunks;
+    const uint4 *vs = reinterpret_cast<const uint4 *>(p.v_new) + (size_t)i * chunks;
+    for (int c = threadIdx.x; c < 2 * chunks; c += blockDim.x) {
+        const bool is_v = c >= chunks;
+        const int cc = is_v ? c - chunks : c;
+        const int h = cc >> 4, part = cc & 15;
+        const size_t row = (size_t)(is_v ? e.v_row : e.k_row) + (size_t)h * e.head_stride;
+        arena[row * 16 + part] = is_v ? vs[cc] : ks[cc];
+    }
+}
+
+// Token-major [T][Hkv][128] -> head-major suffix rows; one thread per 16-byte chunk.
+__global__ void __launch_bounds__(256) cart_extend_kernel(const ExtendParams p)
+{
+    const size_t chunks = (size_t)p.n_tokens * p.n_kv_heads * 16;
+    uint4 *arena = reinterpret_cast<uint4 *>(p.arena);
+    const uint4 *ks = reinterpret_cast<const uint4 *>(p.k);
+    const uint4 *vs = reinterpret_cast<const uint4 *>(p.v);
+    for (size_t c = (size_t)blockIdx.x * blockDim.x + threadIdx.x; c < 2 * chunks;
+         c += (size_t)gridDim.x * blockDim.x) {
+        const bool is_v = c >= chunks;
+        const size_t cc = is_v ? c - chunks : c;
+        const int part = (int)(cc & 15);
+        const size_t th = cc >> 4;  // token * Hkv + head
+        const size_t tok = th / p.n_kv_heads, h = th % p.n_kv_heads;
+        const size_t row = (size_t)(is_v ? p.v_row : p.k_row) + h * p.head_stride + tok;
+        arena[row * 16 + part] = is_v ? vs[cc] : ks[cc];
+    }
+}
+
+}  // namespace
+
+size_t decode_smem_bytes() { return kSmemBytes; }
+int decode_threads() { return kThreads; }
+
+cudaError_t prepare_kernels()
+{
+    return cudaFuncSetAttribute(cart_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+}
+
+cudaError_t launch_decode(const CUtensorMap &tmap, const DecodeParams &p, int grid, cudaStream_t s)
+{
+    cart_decode_kernel<<<grid, kThreads, kSmemBytes, s>>>(tmap, p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_merge(const MergeParams &p, int n_merges, cudaStream_t s)
+{
+    cart_merge_kernel<<<n_merges, 128, 0, s>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_append(const AppendParams &p, cudaStream_t s)
+{
+    cart_append_kernel<<<p.n, 128, 0, s>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_extend(const ExtendParams &p, cudaStream_t s)
+{
+    const size_t chunks = 2ull * (size_t)p.n_tokens * p.n_kv_heads * 16;
+    int grid = (int)((chunks + 255) / 256);
+    if (grid > 148 * 8) grid = 148 * 8;
+    if (grid < 1) grid = 1;
+    cart_extend_kernel<<<grid, 256, 0, s>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace cart
