@@ -4,7 +4,7 @@
 // Decode kernel in one paragraph.  One persistent block per SM walks its list of work items (runs
 // of 64-token tiles of one KV segment of one (request, KV head) row group).  A producer warp streams
 // K and V tiles from HBM into a ring of shared-memory stages with TMA (cp.async.bulk.tensor, 128-byte
-// swizzle, completion on mbarriers); eight consumer warps each take whole tiles round-robin.  A
+// swizzle, completion on mbarriers); each stage has its own consumer warp, which takes whole tiles.  A
 // consumer multiplies the group's G query heads (padded to the 16 rows of an m16n8k16 bf16 MMA, so
 // a K/V tile is read once per group) with the tile, keeps an fp32 online softmax (running max, sum,
 // rescaled output) in registers, and multiplies the probabilities with V.  At the end of a row-group
@@ -20,7 +20,11 @@ namespace cart {
 namespace {
 
 constexpr int kStages = 6;
-constexpr int kConsumerWarps = 8;
+// One consumer warp per stage: warp w is the only reader of stage w, so its waits on that stage's
+// barriers follow one another round by round.  (With several warps sharing a stage, a warp two
+// rounds ahead would mistake an older completed phase for its own: an mbarrier only tells the
+// current phase from the one before.)
+constexpr int kConsumerWarps = kStages;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
 constexpr int kThreads = kConsumerThreads + 32;
 constexpr uint32_t kHalfBytes = kTileTokens * 128;    // 64 tokens x 64 dims of bf16
@@ -333,13 +337,11 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeParams 
     WarpState st;
     uint32_t qa0[8], qa2[8];
     uint32_t t = 0;       // tiles seen by this block so far (same count as the producer's)
-    uint32_t piece = 0;   // tiles seen in the current row-group piece
     bool alive = true;    // false once the block has given up
 
     for (uint32_t it = item_begin; it < item_end; ++it) {
         const cart_work_item w = p.items[it];
         if (w.flags & CART_ITEM_BEGIN) {
-            piece = 0;
             st.m = -INFINITY;
             st.l = 0.f;
 #pragma unroll
@@ -358,12 +360,12 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeParams 
             }
         }
         const uint32_t ntiles = (w.n_tok + kTileTokens - 1) / kTileTokens;
-        // this warp takes the tiles whose index within the piece is congruent to its number
-        uint32_t j = (uint32_t)((warp + kConsumerWarps - (int)(piece % kConsumerWarps)) % kConsumerWarps);
-        for (; j < ntiles; j += kConsumerWarps) {
+        // this warp takes the tiles that land in its own stage: block-wide tile index = warp (mod stages)
+        uint32_t j = (uint32_t)((warp + kStages - (int)(t % kStages)) % kStages);
+        for (; j < ntiles; j += kStages) {
             if (!alive) break;
             const uint32_t tt = t + j;
-            const int s = (int)(tt % kStages);
+            const int s = warp;
             const uint32_t parity = (tt / kStages) & 1u;
             const uint32_t kbase = stages + (uint32_t)s * kStageBytes;
             const int valid = min((int)kTileTokens, (int)(w.n_tok - j * kTileTokens));
@@ -375,10 +377,9 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeParams 
             if (lane == 0) mbar_arrive(empty(s));
         }
         t += ntiles;
-        piece += ntiles;
 
         if (w.flags & CART_ITEM_END) {
-            // ---- combine the eight warps' states -------------------------------------------------
+            // ---- combine the consumer warps' states ---------------------------------------------
             float lsum = st.l;
             lsum += __shfl_xor_sync(0xffffffffu, lsum, 1);
             lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);

@@ -142,12 +142,14 @@ def workload_arena_bytes(w: synth.Workload, extra_capacity: int = 0) -> int:
 
 
 def load_workload(w: synth.Workload, extra_capacity: int = 0, with_oracle: bool = True,
-                  gen_device: str = "cuda:0", **kw) -> tuple:
+                  gen_device: str = "cuda:0", extra_bytes: int = 0, extra_requests: int = 0,
+                  extra_cartridges: int = 0, **kw) -> tuple:
     """Creates a Session for ``w``: registers its Cartridges, opens one request per batch entry
     (composing pool members where the workload says so) and fills the suffixes.  Returns
     (session, request handles)."""
-    sess = Session(w.n_layers, w.n_q_heads, w.n_kv_heads, workload_arena_bytes(w, extra_capacity),
-                   max_requests=max(w.batch, 1), max_cartridges=w.n_cartridges + w.batch + 1,
+    sess = Session(w.n_layers, w.n_q_heads, w.n_kv_heads, workload_arena_bytes(w, extra_capacity) + extra_bytes,
+                   max_requests=max(w.batch, 1) + extra_requests,
+                   max_cartridges=w.n_cartridges + w.batch + 1 + extra_cartridges,
                    with_oracle=with_oracle, **kw)
     cids = []
     for c in range(w.n_cartridges):

@@ -64,7 +64,7 @@ def test_config3_shape_shared_cartridge_with_decode_appends():
 
 def test_config4_shape_composed_pairs_equal_physical_concatenation():
     w = synth.shrink(synth.config4(), n_layers=2, batch=10, pool=5)
-    sess, reqs = H.load_workload(w)
+    sess, reqs = H.load_workload(w, extra_bytes=3 * (40 << 20), extra_requests=3, extra_cartridges=3)
     try:
         check_all_layers(sess, reqs, w)
         # compose(A, B) must equal one Cartridge that physically holds A || B  (Sec. 3.1, Sec. 5.4)
@@ -167,7 +167,7 @@ def test_composition_of_eight_parts_and_nested_compose():
 
 def test_duplicate_requests_in_a_batch_and_null_lse():
     w = synth.Workload("dup", 9, 1, 24, 8, 2, 100, 10, 10)
-    sess, reqs = H.load_workload(w)
+    sess, reqs = H.load_workload(w, extra_requests=1)
     try:
         q = w.queries(0, "cuda:0")[0]
         batch = [reqs[0], reqs[1], reqs[0]]
