@@ -1,0 +1,370 @@
+#!/usr/bin/env python
+"""Benchmark of Cartridge decode attention on B200 (one JSON line on stdout).
+
+A "step" is one decode step of the whole hot path over one batch of synthetic input: for every
+layer, append each request's new KV token and attend over [Cartridge(s) ; suffix] (projections,
+MLP and sampling of a real model are outside the path and not timed).  Cartridges are registered
+before the timed region (the paper's throughput protocol pre-loads them, App. A.3).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl ours|reference]
+
+N > 1 is launched with torch.distributed.run: every rank runs an independent replica on its own
+GPU (the path has no exchange step), timing is the maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2506_06266_b200 import synth
+
+METRIC = "decode_attention_tokens_per_s"
+UNIT = "tokens/s"
+
+WORKLOADS = {
+    "c1": synth.config1, "c2": synth.config2, "c3": synth.config3, "c4": synth.config4,
+    "c5_full": synth.config5_full, "c5_cartridge": synth.config5_cartridge,
+}
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the decode kernel, from the ncu capture
+# summarised under profiles/ (a smaller case of the same kernel, scaled by KV bytes); None = not captured.
+NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = {}
+
+
+def measured_peak_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_max_mhz": float(max(mx)) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def dist_setup(n_gpus: int):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    return rank, world, local
+
+
+def barrier(world: int):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+def max_over_ranks(x: float, world: int, dev) -> float:
+    if world == 1:
+        return x
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+# ------------------------------------------------------------------------------------------------
+def oracle_sample(w: synth.Workload, lw, layers, q_host_bits, reps_target_s: float = 10.0):
+    """Times the CPU oracle, as it stands, on `layers` of the loaded workload (all requests)."""
+    import oracle
+    segs = {layer: [lw.host_segments(layer, b) for b in range(w.batch)] for layer in layers}
+    oracle.decode_layer(q_host_bits[layers[0]][:1], [segs[layers[0]][0]], w.scale)   # load the library
+    t0 = time.perf_counter()
+    reps = 0
+    while True:
+        for layer in layers:
+            oracle.decode_layer(q_host_bits[layer], segs[layer], w.scale)
+        reps += 1
+        el = time.perf_counter() - t0
+        if el >= reps_target_s or reps >= 400:
+            break
+    per_layer = el / (reps * len(layers))
+    return {"value": w.batch / (per_layer * w.n_layers), "unit": UNIT, "cores": oracle.num_threads(),
+            "kind": "oracle",
+            "sample": "layers %s of %d, all %d requests, %d repetition(s), %.1f s of CPU time; "
+                      "extrapolated to %d layers" % (list(layers), w.n_layers, w.batch, reps, el, w.n_layers),
+            "s_per_layer": per_layer}
+
+
+def run_ours(args):
+    from paper_2506_06266_b200 import binding, runner
+    rank, world, local = dist_setup(args.gpus)
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    w = WORKLOADS[args.workload]()
+    if args.layers:
+        w = synth.shrink(w, n_layers=args.layers)
+    L, B = w.n_layers, w.batch
+    total_steps = args.warmup + args.steps + (0 if args.no_e2e else args.warmup + args.e2e_steps) + 2
+    sample_layers = list(range(min(args.cpu_layers, L))) if (rank == 0 and world == 1 and not args.no_cpu) else []
+    stream = torch.cuda.current_stream(dev)
+    lw = runner.LoadedWorkload(w, dev, extra_capacity=total_steps, keep_layers=sample_layers, stream=stream)
+    ctx = lw.ctx
+
+    q = w.queries(0, dev)
+    k_new, v_new = w.appended_kv(0, dev)
+    out = torch.empty_like(q)
+    lse = torch.empty((L, B, w.n_q_heads), dtype=torch.float32, device=dev)
+    torch.cuda.synchronize(dev)
+
+    # ---- device-resident timing ------------------------------------------------------------
+    for _ in range(args.warmup):
+        lw.step(q, k_new, v_new, out, lse)
+    binding.cart_sync_status(ctx, stream)
+    barrier(world)
+    torch.cuda.synchronize(dev)
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    binding.cart_set_timing(ctx, True)
+    launches0 = binding.cart_launch_count(ctx)
+    bytes_layer_sum = 0
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        lw.step(q, k_new, v_new, out, lse)
+        bytes_layer_sum += lw.algorithmic_bytes_per_layer()
+    e1.record(stream)
+    torch.cuda.synchronize(dev)
+    barrier(world)
+    clocks = sampler.stop() if rank == 0 else None
+    ms = e0.elapsed_time(e1)
+    launches = binding.cart_launch_count(ctx) - launches0
+    kern_ms, kern_n = binding.cart_get_timing(ctx)
+    binding.cart_set_timing(ctx, False)
+    binding.cart_sync_status(ctx, stream)
+    ms_max = max_over_ranks(ms, world, dev)
+    value = world * B * args.steps / (ms_max * 1e-3)
+
+    # ---- roofline of the dominant kernel (split-KV decode attention) -------------------------
+    peak, peak_kind = measured_peak_gbs()
+    bytes_per_launch = bytes_layer_sum / args.steps          # one launch = one layer of one step
+    avg_kernel_s = kern_ms * 1e-3 / max(kern_n, 1)
+    achieved = bytes_per_launch / avg_kernel_s / 1e9
+    ratio = NCU_TRAFFIC_PER_ALGORITHMIC_BYTE.get(args.workload)
+    roofline = {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
+                "frac": round(achieved / peak, 4), "peak_kind": "of " + peak_kind,
+                "frac_of_8TBs_nominal": round(achieved / 8000.0, 4),
+                "traffic": None if ratio is None else int(ratio * bytes_per_launch),
+                "kernel": "cart_decode_kernel", "launches_timed": kern_n,
+                "avg_kernel_us": round(avg_kernel_s * 1e6, 2),
+                "algorithmic_bytes_per_launch": int(bytes_per_launch)}
+
+    # ---- end to end through the C ABI from pinned host buffers -------------------------------
+    e2e = None
+    if not args.no_e2e:
+        hq = q.cpu().pin_memory()
+        hk, hv = k_new.cpu().pin_memory(), v_new.cpu().pin_memory()
+        hout = torch.empty(out.shape, dtype=out.dtype).pin_memory()
+        hlse = torch.empty(lse.shape, dtype=lse.dtype).pin_memory()
+        dq, dk, dv = torch.empty_like(q), torch.empty_like(k_new), torch.empty_like(v_new)
+
+        def e2e_step():
+            for layer in range(L):
+                dq[layer].copy_(hq[layer], non_blocking=True)
+                dk[layer].copy_(hk[layer], non_blocking=True)
+                dv[layer].copy_(hv[layer], non_blocking=True)
+                binding.cart_append_kv(ctx, layer, lw.req_list, dk[layer], dv[layer], stream)
+                binding.cart_decode_attention(ctx, layer, lw.req_list, dq[layer], out[layer], lse[layer], stream)
+                hout[layer].copy_(out[layer], non_blocking=True)
+                hlse[layer].copy_(lse[layer], non_blocking=True)
+            lw.appended += 1
+
+        for _ in range(args.warmup):
+            e2e_step()
+        torch.cuda.synchronize(dev)
+        barrier(world)
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record(stream)
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        f1.record(stream)
+        torch.cuda.synchronize(dev)
+        barrier(world)
+        ems = max_over_ranks(f0.elapsed_time(f1), world, dev)
+        h2d = L * (hq[0].numel() * 2 + hk[0].numel() * 2 + hv[0].numel() * 2)
+        d2h = L * (hout[0].numel() * 2 + hlse[0].numel() * 4)
+        e2e = {"value": round(world * B * args.e2e_steps / (ems * 1e-3), 1), "unit": UNIT,
+               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": args.e2e_steps,
+               "ms_per_step": round(ems / args.e2e_steps, 4)}
+        binding.cart_sync_status(ctx, stream)
+
+    # ---- CPU oracle on a bounded sample (rank 0, N = 1 only) ---------------------------------
+    cpu = None
+    if sample_layers:
+        cpu = oracle_sample(w, lw, sample_layers, synth.bits(q))
+        cpu["value"] = round(cpu["value"], 3)
+
+    logical, private = binding.cart_kv_bytes(ctx, lw.reqs[0])
+    kv_tokens = lw.kv_tokens()
+    lw.close()
+    if rank != 0:
+        return
+    line = {
+        "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(ms_max / args.steps, 4), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "batch_per_gpu": B, "layers": L, "q_heads": w.n_q_heads,
+                   "kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "cartridge_tokens": w.p,
+                   "cartridges": w.cartridges, "suffix": "uniform[%d,%d]" % (w.suffix_lo, w.suffix_hi),
+                   "mean_kv_tokens": round(float(kv_tokens.mean()), 1),
+                   "step": "per layer: append 1 KV token per request, then decode attention",
+                   "l2": "inputs larger than L2 (%.0f MB of KV per layer, %.1f GB per step)"
+                         % (bytes_per_launch / 1e6, bytes_per_launch * L / 1e9),
+                   "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "attention_us_per_layer": round(ms_max * 1e3 / args.steps / L, 2),
+                   "kv_bytes_per_request": int(logical), "kv_bytes_private_per_request": int(private)},
+        "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
+        "clocks": clocks,
+    }
+    print(json.dumps(line))
+
+
+def run_reference(args):
+    """The reference arm is the CPU oracle, as it stands, timed on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    w = WORKLOADS[args.workload]()
+    L, B = w.n_layers, w.batch
+    n_layers = min(args.ref_layers, L)
+    suffix = w.suffix_lengths()
+    parts = w.request_parts()
+    # the same seeded inputs as the GPU arm, generated on the host for the sampled layers only
+    carts = {}
+    for b in range(B):
+        for c in parts[b]:
+            if c not in carts:
+                k, v = synth.shrink(w, n_layers=n_layers).cartridge_kv(c, "cpu")
+                carts[c] = (synth.bits(k), synth.bits(v))
+    segs = [[] for _ in range(n_layers)]
+    ws = synth.shrink(w, n_layers=n_layers)
+    for b in range(B):
+        ks, vs = ws.suffix_kv(b, int(suffix[b]), "cpu")
+        kb, vb = synth.bits(ks), synth.bits(vs)
+        for layer in range(n_layers):
+            s = [(carts[c][0][layer], carts[c][1][layer]) for c in parts[b]]
+            s.append((np.ascontiguousarray(np.transpose(kb[layer], (1, 0, 2))),
+                      np.ascontiguousarray(np.transpose(vb[layer], (1, 0, 2)))))
+            segs[layer].append(s)
+    q = synth.bits(ws.queries(0, "cpu"))
+
+    def step():
+        for layer in range(n_layers):
+            oracle.decode_layer(q[layer], segs[layer], w.scale)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    el = time.perf_counter() - t0
+    per_step_full = el / args.steps * (L / n_layers)
+    value = B / per_step_full
+    sample = ("each step = layers 0..%d of %d, all %d requests (inputs of the GPU arm's recipe, "
+              "generated per sampled layer); extrapolated to %d layers" % (n_layers - 1, L, B, L))
+    line = {"impl": "reference", "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(per_step_full * 1e3, 3),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": {"workload": w.name, "batch_per_gpu": B, "layers": L},
+            "cpu_baseline": {"value": round(value, 3), "unit": UNIT, "cores": oracle.num_threads(),
+                             "kind": "oracle", "sample": sample},
+            "e2e": {"value": round(value, 3), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2", choices=sorted(WORKLOADS))
+    ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling small cases)")
+    ap.add_argument("--e2e-steps", type=int, default=10)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--cpu-layers", type=int, default=4, help="layers the CPU oracle sample covers")
+    ap.add_argument("--ref-layers", type=int, default=2, help="layers per step of the reference arm")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -158,6 +158,14 @@ CART_API cart_status cart_kv_bytes(cart_ctx *ctx, cart_req req, uint64_t *logica
  * kernel gave up on a bounded wait since the last call (the word is then cleared). */
 CART_API cart_status cart_sync_status(cart_ctx *ctx, void *stream);
 
+/* Kernel timing for the benchmark's roofline line.  With timing enabled, every decode-attention
+ * kernel launch (the split-KV kernel alone, not the merge) is bracketed by a pair of CUDA events on
+ * its stream.  cart_get_timing synchronises the recorded events, returns the summed kernel time in
+ * milliseconds and the number of launches since the last call, and forgets them.  At most 8192
+ * launches are remembered between two reads; later ones go untimed.  Errors: INVALID_ARG, CUDA. */
+CART_API cart_status cart_set_timing(cart_ctx *ctx, int32_t enable);
+CART_API cart_status cart_get_timing(cart_ctx *ctx, double *total_ms /*host*/, uint64_t *n_launches /*host*/);
+
 /* Number of kernels this context has launched so far (for the benchmark's launch count). */
 CART_API uint64_t cart_launch_count(const cart_ctx *ctx);
 

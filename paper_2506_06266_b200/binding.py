@@ -28,7 +28,7 @@ STATUS_NAMES = ["CART_OK", "CART_ERR_INVALID_ARG", "CART_ERR_SHAPE", "CART_ERR_B
 EXPORTS = ["cart_scratch_bytes", "cart_create", "cart_destroy", "cart_register_cartridge",
            "cart_compose", "cart_release_cartridge", "cart_request_open", "cart_request_close",
            "cart_append_kv", "cart_extend_kv", "cart_decode_attention", "cart_suffix_len",
-           "cart_kv_bytes", "cart_sync_status", "cart_launch_count", "cart_status_string",
+           "cart_kv_bytes", "cart_sync_status", "cart_set_timing", "cart_get_timing", "cart_launch_count", "cart_status_string",
            "cart_last_error", "cart_plan_build"]
 
 
@@ -98,6 +98,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.cart_suffix_len.argtypes = [vp, i32, i32, i32p]
     lib.cart_kv_bytes.argtypes = [vp, i32, u64p, u64p]
     lib.cart_sync_status.argtypes = [vp, vp]
+    lib.cart_set_timing.argtypes = [vp, i32]
+    lib.cart_get_timing.argtypes = [vp, ctypes.POINTER(ctypes.c_double), u64p]
     lib.cart_launch_count.argtypes = [vp]
     lib.cart_launch_count.restype = ctypes.c_uint64
     lib.cart_status_string.argtypes = [ctypes.c_int]
@@ -242,6 +244,16 @@ def cart_kv_bytes(ctx: int, req: int) -> Tuple[int, int]:
 
 def cart_sync_status(ctx: int, stream=None) -> None:
     _check(load_library().cart_sync_status(ctx, _stream(stream)), "cart_sync_status", ctx)
+
+
+def cart_set_timing(ctx: int, enable: bool) -> None:
+    _check(load_library().cart_set_timing(ctx, 1 if enable else 0), "cart_set_timing", ctx)
+
+
+def cart_get_timing(ctx: int) -> Tuple[float, int]:
+    ms, n = ctypes.c_double(0.0), ctypes.c_uint64(0)
+    _check(load_library().cart_get_timing(ctx, ctypes.byref(ms), ctypes.byref(n)), "cart_get_timing", ctx)
+    return float(ms.value), int(n.value)
 
 
 def cart_launch_count(ctx: int) -> int:

@@ -19,6 +19,7 @@ using namespace cart;
 constexpr int kMaxCta = 1024;   // upper bound on persistent blocks (device independent)
 constexpr int kPlanSlots = 4;   // ring of uploaded plans
 constexpr uint64_t kAlign = 256;
+constexpr size_t kMaxTimedLaunches = 8192;
 
 uint64_t round_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
 
@@ -115,6 +116,9 @@ struct cart_ctx {
     std::vector<cart_plan_seg> seg_tmp;
     std::vector<int32_t> seg_begin_tmp;
     std::vector<uint32_t> key_tmp;
+    bool timing = false;
+    std::vector<cudaEvent_t> ev_pool;  // pairs: start, stop
+    size_t ev_used = 0;
     char err[256] = {0};
 };
 
@@ -308,7 +312,32 @@ cart_status cart_destroy(cart_ctx *ctx)
         if (sl.host) cudaFreeHost(sl.host);
         if (sl.ev) cudaEventDestroy(sl.ev);
     }
+    for (cudaEvent_t e : ctx->ev_pool) cudaEventDestroy(e);
     delete ctx;
+    return CART_OK;
+}
+
+cart_status cart_set_timing(cart_ctx *ctx, int32_t enable)
+{
+    if (!ctx) return CART_ERR_INVALID_ARG;
+    ctx->timing = enable != 0;
+    return CART_OK;
+}
+
+cart_status cart_get_timing(cart_ctx *ctx, double *total_ms, uint64_t *n_launches)
+{
+    if (!ctx) return CART_ERR_INVALID_ARG;
+    if (!total_ms || !n_launches) return fail(ctx, CART_ERR_INVALID_ARG, "get_timing: null out");
+    double sum = 0.0;
+    for (size_t i = 0; i + 1 < ctx->ev_used; i += 2) {
+        CART_CUDA(ctx, cudaEventSynchronize(ctx->ev_pool[i + 1]));
+        float ms = 0.f;
+        CART_CUDA(ctx, cudaEventElapsedTime(&ms, ctx->ev_pool[i], ctx->ev_pool[i + 1]));
+        sum += (double)ms;
+    }
+    *total_ms = sum;
+    *n_launches = ctx->ev_used / 2;
+    ctx->ev_used = 0;
     return CART_OK;
 }
 
@@ -614,8 +643,21 @@ cart_status cart_decode_attention(cart_ctx *ctx, int32_t layer, const cart_req *
     dp.layer = layer;
     dp.group = ctx->group;
     dp.scale_log2 = ctx->scale * 1.4426950408889634f;
+    const bool timed = ctx->timing && ctx->ev_used + 2 <= kMaxTimedLaunches * 2;
+    if (timed) {
+        while (ctx->ev_pool.size() < ctx->ev_used + 2) {
+            cudaEvent_t e;
+            CART_CUDA(ctx, cudaEventCreate(&e));
+            ctx->ev_pool.push_back(e);
+        }
+        CART_CUDA(ctx, cudaEventRecord(ctx->ev_pool[ctx->ev_used], s));
+    }
     CART_CUDA(ctx, launch_decode(ctx->tmap, dp, sl->n_cta_used, s));
     ++ctx->launches;
+    if (timed) {
+        CART_CUDA(ctx, cudaEventRecord(ctx->ev_pool[ctx->ev_used + 1], s));
+        ctx->ev_used += 2;
+    }
     if (sl->n_merges > 0) {
         MergeParams mp;
         mp.merges = reinterpret_cast<const cart_merge_item *>(sl->dev + ctx->lay.merges_off);
