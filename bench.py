@@ -28,7 +28,7 @@ if ROOT not in sys.path:
 import numpy as np
 import torch
 
-from paper_2506_06266_b200 import synth
+from paper_2506_06266_b200 import replicas, synth
 
 METRIC = "decode_attention_tokens_per_s"
 UNIT = "tokens/s"
@@ -40,7 +40,7 @@ WORKLOADS = {
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the decode kernel, from the ncu capture
 # summarised under profiles/ (a smaller case of the same kernel, scaled by KV bytes); None = not captured.
-NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = {}
+NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = {"c2": 622.56 / 608.27}   # profiles/decode_kernel_c2.md
 
 
 def measured_peak_gbs():
@@ -106,32 +106,6 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def dist_setup(n_gpus: int):
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if world > 1:
-        import torch.distributed as dist
-        torch.cuda.set_device(local)
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    return rank, world, local
-
-
-def barrier(world: int):
-    if world > 1:
-        import torch.distributed as dist
-        dist.barrier()
-
-
-def max_over_ranks(x: float, world: int, dev) -> float:
-    if world == 1:
-        return x
-    import torch.distributed as dist
-    t = torch.tensor([x], dtype=torch.float64, device=dev)
-    dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    return float(t.item())
-
-
 # ------------------------------------------------------------------------------------------------
 def oracle_sample(w: synth.Workload, lw, layers, q_host_bits, reps_target_s: float = 10.0):
     """Times the CPU oracle, as it stands, on `layers` of the loaded workload (all requests)."""
@@ -157,7 +131,7 @@ def oracle_sample(w: synth.Workload, lw, layers, q_host_bits, reps_target_s: flo
 
 def run_ours(args):
     from paper_2506_06266_b200 import binding, runner
-    rank, world, local = dist_setup(args.gpus)
+    rank, world, local = replicas.setup()
     dev = torch.device("cuda", local)
     torch.cuda.set_device(dev)
     w = WORKLOADS[args.workload]()
@@ -180,7 +154,7 @@ def run_ours(args):
     for _ in range(args.warmup):
         lw.step(q, k_new, v_new, out, lse)
     binding.cart_sync_status(ctx, stream)
-    barrier(world)
+    replicas.barrier(world)
     torch.cuda.synchronize(dev)
     sampler = ClockSampler(local)
     if rank == 0:
@@ -195,15 +169,14 @@ def run_ours(args):
         bytes_layer_sum += lw.algorithmic_bytes_per_layer()
     e1.record(stream)
     torch.cuda.synchronize(dev)
-    barrier(world)
+    replicas.barrier(world)
     clocks = sampler.stop() if rank == 0 else None
     ms = e0.elapsed_time(e1)
     launches = binding.cart_launch_count(ctx) - launches0
     kern_ms, kern_n = binding.cart_get_timing(ctx)
     binding.cart_set_timing(ctx, False)
     binding.cart_sync_status(ctx, stream)
-    ms_max = max_over_ranks(ms, world, dev)
-    value = world * B * args.steps / (ms_max * 1e-3)
+    value, ms_max = replicas.whole_job_tokens_per_s(B * args.steps, ms, world, dev)
 
     # ---- roofline of the dominant kernel (split-KV decode attention) -------------------------
     peak, peak_kind = measured_peak_gbs()
@@ -242,18 +215,18 @@ def run_ours(args):
         for _ in range(args.warmup):
             e2e_step()
         torch.cuda.synchronize(dev)
-        barrier(world)
+        replicas.barrier(world)
         f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         f0.record(stream)
         for _ in range(args.e2e_steps):
             e2e_step()
         f1.record(stream)
         torch.cuda.synchronize(dev)
-        barrier(world)
-        ems = max_over_ranks(f0.elapsed_time(f1), world, dev)
+        replicas.barrier(world)
+        e2e_value, ems = replicas.whole_job_tokens_per_s(B * args.e2e_steps, f0.elapsed_time(f1), world, dev)
         h2d = L * (hq[0].numel() * 2 + hk[0].numel() * 2 + hv[0].numel() * 2)
         d2h = L * (hout[0].numel() * 2 + hlse[0].numel() * 4)
-        e2e = {"value": round(world * B * args.e2e_steps / (ems * 1e-3), 1), "unit": UNIT,
+        e2e = {"value": round(e2e_value, 1), "unit": UNIT,
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": args.e2e_steps,
                "ms_per_step": round(ems / args.e2e_steps, 4)}
         binding.cart_sync_status(ctx, stream)
@@ -267,6 +240,9 @@ def run_ours(args):
     logical, private = binding.cart_kv_bytes(ctx, lw.reqs[0])
     kv_tokens = lw.kv_tokens()
     lw.close()
+    if world > 1:
+        replicas.barrier(world)
+        replicas.shutdown()
     if rank != 0:
         return
     line = {
