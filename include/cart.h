@@ -166,6 +166,39 @@ CART_API cart_status cart_sync_status(cart_ctx *ctx, void *stream);
 CART_API cart_status cart_set_timing(cart_ctx *ctx, int32_t enable);
 CART_API cart_status cart_get_timing(cart_ctx *ctx, double *total_ms /*host*/, uint64_t *n_launches /*host*/);
 
+/* Decode attention for callers that cannot allocate.  (The paper has no counterpart; this is a
+ * convenience of the library.)  The entry points above need an arena from the caller and pinned
+ * staging memory from cart_create.  Callers that may call neither cudaMalloc nor a framework's
+ * allocator -- code running while a memory pool is frozen, a plug-in that is only handed tensors,
+ * an early health check -- can use this one call instead: it needs no context, and the kernels'
+ * scratch (work list, split partials; CART_STATIC_SCRATCH_BYTES) lives in a fixed device array inside
+ * the library image, which every GPU that loads the library holds until the process exits.
+ *
+ * Computes the same result as cart_decode_attention for n_reqs requests that each attend over their
+ * own n_tokens KV tokens: q and out are device bf16 [n_reqs][n_q_heads][128]; kv is ONE device
+ * buffer, 256-byte aligned, bf16 [2][n_reqs][n_kv_heads][n_tokens][128] (all keys, then all values);
+ * lse is device fp32 [n_reqs][n_q_heads] or NULL; softmax_scale 0 => 1/sqrt(128).  `device` must be
+ * the current CUDA device and the one the buffers live on.
+ *
+ * Limits: n_reqs * n_kv_heads <= CART_STATIC_MAX_ROW_GROUPS, 2 * n_reqs * n_kv_heads * n_tokens < 2^31,
+ * n_q_heads / n_kv_heads <= 8, device < 64; anything larger returns CART_ERR_CAPACITY and launches
+ * nothing.  The call runs no cudaMalloc, cudaFree, cudaHostAlloc or other allocating routine.
+ *
+ * The first call on a device also does that device's one-time set-up (it looks up the scratch
+ * array's device address and raises the kernel's shared-memory limit); make that first call before
+ * any stream capture begins.  The work list is copied from ordinary (pageable) host memory, so the
+ * call may wait for earlier work on `stream` before it returns.  All calls share the one scratch
+ * array, which keeps the previous call's contents (the call clears what it needs zeroed): calls
+ * whose GPU work may overlap -- different streams, different host threads -- race and must be
+ * ordered by the caller.  A device-side wait that ran out is not reported by this entry point.
+ * Errors: INVALID_ARG, SHAPE, CAPACITY, CUDA. */
+#define CART_STATIC_MAX_ROW_GROUPS 2048
+#define CART_STATIC_SCRATCH_BYTES 2228224
+CART_API cart_status cart_decode_attention_static(const void *q /*device*/, const void *kv /*device*/,
+                                                  int32_t n_reqs, int32_t n_q_heads, int32_t n_kv_heads,
+                                                  int32_t n_tokens, float softmax_scale, void *out /*device*/,
+                                                  float *lse /*device or NULL*/, int32_t device, void *stream);
+
 /* Number of kernels this context has launched so far (for the benchmark's launch count). */
 CART_API uint64_t cart_launch_count(const cart_ctx *ctx);
 

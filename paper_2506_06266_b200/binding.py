@@ -28,7 +28,8 @@ STATUS_NAMES = ["CART_OK", "CART_ERR_INVALID_ARG", "CART_ERR_SHAPE", "CART_ERR_B
 EXPORTS = ["cart_scratch_bytes", "cart_create", "cart_destroy", "cart_register_cartridge",
            "cart_compose", "cart_release_cartridge", "cart_request_open", "cart_request_close",
            "cart_append_kv", "cart_extend_kv", "cart_decode_attention", "cart_suffix_len",
-           "cart_kv_bytes", "cart_sync_status", "cart_set_timing", "cart_get_timing", "cart_launch_count", "cart_status_string",
+           "cart_kv_bytes", "cart_sync_status", "cart_set_timing", "cart_get_timing",
+           "cart_decode_attention_static", "cart_launch_count", "cart_status_string",
            "cart_last_error", "cart_plan_build"]
 
 
@@ -100,6 +101,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.cart_sync_status.argtypes = [vp, vp]
     lib.cart_set_timing.argtypes = [vp, i32]
     lib.cart_get_timing.argtypes = [vp, ctypes.POINTER(ctypes.c_double), u64p]
+    lib.cart_decode_attention_static.argtypes = [vp, vp, i32, i32, i32, i32, ctypes.c_float, vp, vp, i32, vp]
     lib.cart_launch_count.argtypes = [vp]
     lib.cart_launch_count.restype = ctypes.c_uint64
     lib.cart_status_string.argtypes = [ctypes.c_int]
@@ -254,6 +256,15 @@ def cart_get_timing(ctx: int) -> Tuple[float, int]:
     ms, n = ctypes.c_double(0.0), ctypes.c_uint64(0)
     _check(load_library().cart_get_timing(ctx, ctypes.byref(ms), ctypes.byref(n)), "cart_get_timing", ctx)
     return float(ms.value), int(n.value)
+
+
+def cart_decode_attention_static(q, kv, n_reqs: int, n_q_heads: int, n_kv_heads: int, n_tokens: int,
+                                 out, lse=None, softmax_scale: float = 0.0, device: int = 0, stream=None) -> None:
+    """Context-free decode attention whose scratch is a fixed device array inside libcart.so, for
+    callers that may not allocate (see include/cart.h).  kv is one buffer: all keys, then all values."""
+    _check(load_library().cart_decode_attention_static(
+        _ptr(q), _ptr(kv), int(n_reqs), int(n_q_heads), int(n_kv_heads), int(n_tokens), float(softmax_scale),
+        _ptr(out), _ptr(lse), int(device), _stream(stream)), "cart_decode_attention_static")
 
 
 def cart_launch_count(ctx: int) -> int:
