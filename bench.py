@@ -159,7 +159,7 @@ def run_ours(args):
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    binding.cart_set_timing(ctx, True)
+    binding.cart_set_timing(ctx, not args.no_kernel_events)
     launches0 = binding.cart_launch_count(ctx)
     bytes_layer_sum = 0
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -181,6 +181,8 @@ def run_ours(args):
     # ---- roofline of the dominant kernel (split-KV decode attention) -------------------------
     peak, peak_kind = measured_peak_gbs()
     bytes_per_launch = bytes_layer_sum / args.steps          # one launch = one layer of one step
+    if kern_n == 0:      # kernel events switched off: fall back to the whole step (a lower bound on the rate)
+        kern_ms, kern_n = ms, args.steps * L
     avg_kernel_s = kern_ms * 1e-3 / max(kern_n, 1)
     achieved = bytes_per_launch / avg_kernel_s / 1e9
     ratio = NCU_TRAFFIC_PER_ALGORITHMIC_BYTE.get(args.workload)
@@ -331,6 +333,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-kernel-events", action="store_true",
+                    help="do not bracket each decode kernel with CUDA events (to see what the events cost)")
     ap.add_argument("--cpu-layers", type=int, default=4, help="layers the CPU oracle sample covers")
     ap.add_argument("--ref-layers", type=int, default=2, help="layers per step of the reference arm")
     args = ap.parse_args()

@@ -159,7 +159,7 @@ CART_API cart_status cart_kv_bytes(cart_ctx *ctx, cart_req req, uint64_t *logica
 CART_API cart_status cart_sync_status(cart_ctx *ctx, void *stream);
 
 /* Kernel timing for the benchmark's roofline line.  With timing enabled, every decode-attention
- * kernel launch (the split-KV kernel alone, not the merge) is bracketed by a pair of CUDA events on
+ * kernel launch (not the append) is bracketed by a pair of CUDA events on
  * its stream.  cart_get_timing synchronises the recorded events, returns the summed kernel time in
  * milliseconds and the number of launches since the last call, and forgets them.  At most 8192
  * launches are remembered between two reads; later ones go untimed.  Errors: INVALID_ARG, CUDA. */

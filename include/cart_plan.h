@@ -10,8 +10,9 @@
  * is cut into tiles of `tile_tokens` tokens (the last one ragged).  The tiles of all row groups,
  * laid end to end in batch order, are divided into `n_cta` contiguous, equal (+-1 tile) ranges, one
  * per persistent thread block.  Where a range boundary falls inside a row group, that row group is
- * "split": each block holding a piece writes a partial (o, lse) into its own slot and the pieces
- * are merged by log-sum-exp afterwards (softmax over a union of token sets, from Eq. 1).  A row
+ * "split": each block holding a piece writes a partial (o, lse) into its own slot and the block
+ * that finishes last merges the pieces by log-sum-exp (softmax over a union of token sets, from
+ * Eq. 1).  A row
  * group held entirely by one block is written directly.
  */
 #ifndef CART_PLAN_H_
@@ -46,7 +47,7 @@ typedef struct {
     uint32_t row_group;    /* batch index * n_kv_heads + KV head */
     uint32_t flags;        /* CART_ITEM_* */
     uint32_t slot;         /* partial slot (meaningful with END and without DIRECT) */
-    uint32_t reserved;
+    uint32_t merge;        /* index of the row group's cart_merge_item (same condition) */
 } cart_work_item;
 
 /* A split row group: its partials are slots slot_begin .. slot_end-1. */

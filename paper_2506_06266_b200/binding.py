@@ -52,7 +52,7 @@ class cart_work_item(ctypes.Structure):
     _fields_ = [("k_row", ctypes.c_uint32), ("v_row", ctypes.c_uint32),
                 ("layer_stride", ctypes.c_uint32), ("n_tok", ctypes.c_uint32),
                 ("row_group", ctypes.c_uint32), ("flags", ctypes.c_uint32),
-                ("slot", ctypes.c_uint32), ("reserved", ctypes.c_uint32)]
+                ("slot", ctypes.c_uint32), ("merge", ctypes.c_uint32)]
 
 
 class cart_merge_item(ctypes.Structure):

@@ -24,7 +24,7 @@ constexpr size_t kMaxTimedLaunches = 8192;
 uint64_t round_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
 
 struct ScratchLayout {
-    uint64_t status_off, plan_off, plan_slot_bytes, cta_begin_off, merges_off, items_off;
+    uint64_t status_off, tickets_off, plan_off, plan_slot_bytes, cta_begin_off, merges_off, items_off;
     uint64_t part_o_off, part_lse_off, total;
     int items_cap, slots_cap;
 };
@@ -37,7 +37,8 @@ ScratchLayout scratch_layout(const cart_config &c)
     s.items_cap = c.max_requests * c.n_kv_heads * (parts + 1) + kMaxCta;
     s.slots_cap = 2 * kMaxCta;
     s.status_off = 0;
-    s.plan_off = kAlign;
+    s.tickets_off = kAlign;  // one arrival counter per split row group, zero between launches
+    s.plan_off = s.tickets_off + round_up((uint64_t)kMaxCta * 4, kAlign);
     // one plan slot: [cta_begin][merges][items]
     s.cta_begin_off = 0;
     s.merges_off = round_up((uint64_t)(kMaxCta + 1) * 4, kAlign);
@@ -292,7 +293,7 @@ cart_status cart_create(const cart_config *cfg, cart_ctx **out)
         if (cudaEventCreateWithFlags(&sl.ev, cudaEventDisableTiming) != cudaSuccess) return bail(CART_ERR_CUDA);
         sl.dev = static_cast<uint8_t *>(cfg->arena) + lay.plan_off + (uint64_t)i * lay.plan_slot_bytes;
     }
-    if (cudaMemset(static_cast<uint8_t *>(cfg->arena) + lay.status_off, 0, kAlign) != cudaSuccess)
+    if (cudaMemset(static_cast<uint8_t *>(cfg->arena) + lay.status_off, 0, lay.plan_off) != cudaSuccess)
         return bail(CART_ERR_CUDA);
 
     const uint64_t first_row = lay.total / kRowBytes;
@@ -639,6 +640,8 @@ cart_status cart_decode_attention(cart_ctx *ctx, int32_t layer, const cart_req *
     dp.lse = lse;
     dp.part_o = reinterpret_cast<float *>(arena + ctx->lay.part_o_off);
     dp.part_lse2 = reinterpret_cast<float *>(arena + ctx->lay.part_lse_off);
+    dp.merges = reinterpret_cast<const cart_merge_item *>(sl->dev + ctx->lay.merges_off);
+    dp.tickets = reinterpret_cast<uint32_t *>(arena + ctx->lay.tickets_off);
     dp.status = reinterpret_cast<uint32_t *>(arena + ctx->lay.status_off);
     dp.layer = layer;
     dp.group = ctx->group;
@@ -657,17 +660,6 @@ cart_status cart_decode_attention(cart_ctx *ctx, int32_t layer, const cart_req *
     if (timed) {
         CART_CUDA(ctx, cudaEventRecord(ctx->ev_pool[ctx->ev_used + 1], s));
         ctx->ev_used += 2;
-    }
-    if (sl->n_merges > 0) {
-        MergeParams mp;
-        mp.merges = reinterpret_cast<const cart_merge_item *>(sl->dev + ctx->lay.merges_off);
-        mp.part_o = dp.part_o;
-        mp.part_lse2 = dp.part_lse2;
-        mp.out = out;
-        mp.lse = lse;
-        mp.group = ctx->group;
-        CART_CUDA(ctx, launch_merge(mp, sl->n_merges, s));
-        ++ctx->launches;
     }
     return CART_OK;
 }
@@ -705,7 +697,8 @@ cart_status cart_sync_status(cart_ctx *ctx, void *stream)
     uint8_t *st = static_cast<uint8_t *>(ctx->cfg.arena) + ctx->lay.status_off;
     CART_CUDA(ctx, cudaMemcpy(&word, st, 4, cudaMemcpyDeviceToHost));
     if (word != 0) {
-        CART_CUDA(ctx, cudaMemset(st, 0, 4));
+        // a block that gave up may have left arrival tickets behind: clear them with the word
+        CART_CUDA(ctx, cudaMemset(st, 0, ctx->lay.plan_off));
         return fail(ctx, CART_ERR_TIMEOUT, "a device-side wait ran out (status word 0x%x)", word);
     }
     return CART_OK;

@@ -28,19 +28,12 @@ struct DecodeParams {
     float *lse;                  // fp32 [n_reqs][Hq] or null
     float *part_o;               // fp32 [slot][G][128], normalised partial outputs
     float *part_lse2;            // fp32 [slot][kMaxGroup], base-2 log-sum-exp of a partial
+    const cart_merge_item *merges;  // split row groups (which slots belong together)
+    uint32_t *tickets;           // one arrival counter per merge item; zero between launches
     uint32_t *status;
     int32_t layer;
     int32_t group;               // G
     float scale_log2;            // softmax scale * log2(e)
-};
-
-struct MergeParams {
-    const cart_merge_item *merges;
-    const float *part_o;
-    const float *part_lse2;
-    void *out;
-    float *lse;
-    int32_t group;
 };
 
 struct AppendEntry {
@@ -74,7 +67,6 @@ size_t decode_smem_bytes();
 int decode_threads();
 cudaError_t prepare_kernels();  // sets the dynamic shared-memory attribute; call once per device
 cudaError_t launch_decode(const CUtensorMap &tmap, const DecodeParams &p, int grid, cudaStream_t s);
-cudaError_t launch_merge(const MergeParams &p, int n_merges, cudaStream_t s);
 cudaError_t launch_append(const AppendParams &p, cudaStream_t s);
 cudaError_t launch_extend(const ExtendParams &p, cudaStream_t s);
 

@@ -1,4 +1,4 @@
-// sm_100a kernels of libcart.so: split-KV decode attention over [Cartridge(s) ; suffix], the
+// sm_100a kernels of libcart.so: split-KV decode attention over [Cartridge(s) ; suffix] with the
 // log-sum-exp merge of split row groups, and the KV append / extend scatters.
 //
 // Decode kernel in one paragraph.  One persistent block per SM walks its list of work items (runs
@@ -9,7 +9,8 @@
 // a K/V tile is read once per group) with the tile, keeps an fp32 online softmax (running max, sum,
 // rescaled output) in registers, and multiplies the probabilities with V.  At the end of a row-group
 // piece the warps' states are combined through shared memory and written either as the final bf16
-// output + lse (piece = whole row group) or as an fp32 partial that the merge kernel combines.
+// output + lse (piece = whole row group) or as an fp32 partial; the block that delivers the last
+// partial of a split row group merges them (an arrival ticket per split row group, no waiting).
 // Arithmetic follows Eq. 1 of the paper evaluated at the last position; the split and the merge use
 // that a softmax over a union of token sets is the lse-weighted mix of the softmaxes over the sets.
 #include <cuda_bf16.h>
@@ -34,7 +35,7 @@ constexpr int kScratchStride = 132;                   // floats per scratch row 
 constexpr uint32_t kScratchOBytes = kConsumerWarps * kMaxGroup * kScratchStride * 4;
 constexpr uint32_t kScratchMLBytes = kConsumerWarps * kMaxGroup * 2 * 4;
 constexpr uint32_t kBarrierBytes = 3 * kStages * 8;
-constexpr uint32_t kSmemUsed = kStages * kStageBytes + kScratchOBytes + kScratchMLBytes + kBarrierBytes + 16;
+constexpr uint32_t kSmemUsed = kStages * kStageBytes + kScratchOBytes + kScratchMLBytes + kBarrierBytes + 16;  // + flags
 constexpr uint32_t kSmemBytes = kSmemUsed + 1024;     // slack to align the stages to 1024 bytes
 static_assert(kSmemBytes <= 232448, "shared memory budget of one sm_100 block exceeded");
 
@@ -265,6 +266,7 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeParams 
     const uint32_t bars = base + kStages * kStageBytes + kScratchOBytes + kScratchMLBytes;
     volatile uint32_t *abort_flag =
         reinterpret_cast<volatile uint32_t *>(smem + kStages * kStageBytes + kScratchOBytes + kScratchMLBytes + kBarrierBytes);
+    volatile uint32_t *last_flag = abort_flag + 1;  // "this block merges the split row group"
     auto full_k = [&](int s) { return bars + (uint32_t)s * 8u; };
     auto full_v = [&](int s) { return bars + (uint32_t)(kStages + s) * 8u; };
     auto empty = [&](int s) { return bars + (uint32_t)(2 * kStages + s) * 8u; };
@@ -427,30 +429,48 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeParams 
                     }
                 }
             }
+            if (!(w.flags & CART_ITEM_DIRECT)) __threadfence();  // publish the partial before the ticket
             consumer_bar();  // the scratch may be overwritten by the next piece from here on
-        }
-    }
-}
 
-// One block per split row group: out = sum_c 2^(lse_c - lse) o_c, lse = log2 sum_c 2^lse_c.
-__global__ void __launch_bounds__(128) cart_merge_kernel(const MergeParams p)
-{
-    const cart_merge_item mi = p.merges[blockIdx.x];
-    const int G = p.group;
-    const int d = threadIdx.x;  // 128 threads, one per dim
-    for (int r = 0; r < G; ++r) {
-        float M = -INFINITY;
-        for (uint32_t c = mi.slot_begin; c < mi.slot_end; ++c)
-            M = fmaxf(M, p.part_lse2[(size_t)c * kMaxGroup + r]);
-        float L = 0.f, acc = 0.f;
-        for (uint32_t c = mi.slot_begin; c < mi.slot_end; ++c) {
-            const float wgt = fast_exp2(p.part_lse2[(size_t)c * kMaxGroup + r] - M);
-            L += wgt;
-            acc += wgt * p.part_o[((size_t)c * G + r) * kHeadDim + d];
+            if (!(w.flags & CART_ITEM_DIRECT)) {
+                // Split row group: the block whose piece arrives last merges all pieces.  Nobody waits.
+                const cart_merge_item mi = p.merges[w.merge];
+                if (threadIdx.x == 0) {
+                    uint32_t last = 0;
+                    if (alive) {
+                        const uint32_t seen = atomicAdd(&p.tickets[w.merge], 1u);
+                        last = (seen + 1u == mi.slot_end - mi.slot_begin) ? 1u : 0u;
+                    }
+                    *last_flag = last;
+                }
+                consumer_bar();
+                if (*last_flag) {
+                    __threadfence();
+                    for (int idx = threadIdx.x; idx < G * 64; idx += kConsumerThreads) {
+                        const int r = idx >> 6, dpair = idx & 63;
+                        float M = -INFINITY;
+                        for (uint32_t c = mi.slot_begin; c < mi.slot_end; ++c)
+                            M = fmaxf(M, __ldcg(p.part_lse2 + (size_t)c * kMaxGroup + r));
+                        float L = 0.f, a0 = 0.f, a1 = 0.f;
+                        for (uint32_t c = mi.slot_begin; c < mi.slot_end; ++c) {
+                            const float wgt = fast_exp2(__ldcg(p.part_lse2 + (size_t)c * kMaxGroup + r) - M);
+                            const float2 v = __ldcg(reinterpret_cast<const float2 *>(
+                                p.part_o + ((size_t)c * G + r) * kHeadDim + 2 * dpair));
+                            L += wgt;
+                            a0 += wgt * v.x;
+                            a1 += wgt * v.y;
+                        }
+                        const float inv = 1.f / L;
+                        const size_t orow = (size_t)mi.row_group * G + r;
+                        __nv_bfloat162 *op = reinterpret_cast<__nv_bfloat162 *>(
+                            reinterpret_cast<__nv_bfloat16 *>(p.out) + orow * kHeadDim + 2 * dpair);
+                        *op = __floats2bfloat162_rn(a0 * inv, a1 * inv);
+                        if (dpair == 0 && p.lse) p.lse[orow] = (M + log2f(L)) * 0.6931471805599453f;
+                    }
+                    if (threadIdx.x == 0) p.tickets[w.merge] = 0;  // ready for the next launch
+                }
+            }
         }
-        const size_t orow = (size_t)mi.row_group * G + r;
-        reinterpret_cast<__nv_bfloat16 *>(p.out)[orow * kHeadDim + d] = __float2bfloat16_rn(acc / L);
-        if (d == 0 && p.lse) p.lse[orow] = (M + log2f(L)) * 0.6931471805599453f;
     }
 }
 
@@ -504,12 +524,6 @@ cudaError_t prepare_kernels()
 cudaError_t launch_decode(const CUtensorMap &tmap, const DecodeParams &p, int grid, cudaStream_t s)
 {
     cart_decode_kernel<<<grid, kThreads, kSmemBytes, s>>>(tmap, p);
-    return cudaGetLastError();
-}
-
-cudaError_t launch_merge(const MergeParams &p, int n_merges, cudaStream_t s)
-{
-    cart_merge_kernel<<<n_merges, 128, 0, s>>>(p);
     return cudaGetLastError();
 }
 

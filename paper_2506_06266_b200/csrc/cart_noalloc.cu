@@ -23,7 +23,8 @@ constexpr int kNaSlotsCap = 2 * kNaMaxCta;
 constexpr int kNaMaxDevices = 64;
 
 constexpr size_t kOffStatus = 0;
-constexpr size_t kOffCtaBegin = 256;
+constexpr size_t kOffTickets = 256;
+constexpr size_t kOffCtaBegin = kOffTickets + (size_t)kNaMaxCta * 4;
 constexpr size_t kOffMerges = kOffCtaBegin + ((kNaMaxCta + 1) * 4 + 255) / 256 * 256;
 constexpr size_t kOffItems = kOffMerges + (size_t)kNaMaxCta * sizeof(cart_merge_item);
 constexpr size_t kOffPartO = kOffItems + (size_t)kNaItemsCap * sizeof(cart_work_item);
@@ -135,10 +136,11 @@ extern "C" cart_status cart_decode_attention_static(const void *q, const void *k
     if (st != CART_OK) return st;
     if (n_slots > kNaSlotsCap) return CART_ERR_CAPACITY;
 
-    // The scratch keeps the previous call's contents.  Only the status word must start at zero; the
-    // plan region is overwritten here and every partial slot that is read is written first.
+    // The scratch keeps the previous call's contents.  The status word and the arrival tickets must
+    // start at zero; the plan region is overwritten here and every partial slot that is read is
+    // written first.
     unsigned char *sc = su->scratch;
-    if (cudaMemsetAsync(sc + kOffStatus, 0, 256, s) != cudaSuccess) return CART_ERR_CUDA;
+    if (cudaMemsetAsync(sc + kOffStatus, 0, kOffCtaBegin, s) != cudaSuccess) return CART_ERR_CUDA;
     const size_t plan_bytes = (kOffItems - kOffCtaBegin) + (size_t)n_items * sizeof(cart_work_item);
     if (cudaMemcpyAsync(sc + kOffCtaBegin, hp, plan_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return CART_ERR_CUDA;
 
@@ -150,21 +152,13 @@ extern "C" cart_status cart_decode_attention_static(const void *q, const void *k
     dp.lse = lse;
     dp.part_o = reinterpret_cast<float *>(sc + kOffPartO);
     dp.part_lse2 = reinterpret_cast<float *>(sc + kOffPartLse);
+    dp.merges = reinterpret_cast<const cart_merge_item *>(sc + kOffMerges);
+    dp.tickets = reinterpret_cast<uint32_t *>(sc + kOffTickets);
     dp.status = reinterpret_cast<uint32_t *>(sc + kOffStatus);
     dp.layer = 0;
     dp.group = n_q_heads / n_kv_heads;
     const float scale = softmax_scale > 0.f ? softmax_scale : 0.08838834764831845f;  // 1/sqrt(128)
     dp.scale_log2 = scale * 1.4426950408889634f;
     if (launch_decode(tmap, dp, n_cta_used, s) != cudaSuccess) return CART_ERR_CUDA;
-    if (n_merges > 0) {
-        MergeParams mp;
-        mp.merges = reinterpret_cast<const cart_merge_item *>(sc + kOffMerges);
-        mp.part_o = dp.part_o;
-        mp.part_lse2 = dp.part_lse2;
-        mp.out = out;
-        mp.lse = lse;
-        mp.group = dp.group;
-        if (launch_merge(mp, n_merges, s) != cudaSuccess) return CART_ERR_CUDA;
-    }
     return CART_OK;
 }

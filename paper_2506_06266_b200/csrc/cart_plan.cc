@@ -49,6 +49,7 @@ extern "C" cart_status cart_plan_build(const cart_plan_seg *segs, const int32_t 
             uint64_t seg_tile = 0; // tiles of segment s already handed out
             const uint32_t slot_first = next_slot;
             bool split = false;
+            int32_t my_merge = -1;
             while (pos < rg_end) {
                 const uint64_t piece_end = std::min(rg_end, range_end(c));
                 const bool direct = (pos == rg_start && piece_end == rg_end);
@@ -68,7 +69,7 @@ extern "C" cart_status cart_plan_build(const cart_plan_seg *segs, const int32_t 
                     it.row_group = rg;
                     it.flags = first ? CART_ITEM_BEGIN : 0u;
                     it.slot = 0;
-                    it.reserved = 0;
+                    it.merge = 0;
                     first = false;
                     want -= take;
                     seg_tile += take;
@@ -79,19 +80,22 @@ extern "C" cart_status cart_plan_build(const cart_plan_seg *segs, const int32_t 
                 if (direct) {
                     last.flags |= CART_ITEM_DIRECT;
                 } else {
+                    if (!split) {
+                        if (nm >= merges_cap) return CART_ERR_CAPACITY;
+                        my_merge = nm++;
+                        split = true;
+                    }
                     last.slot = next_slot++;
-                    split = true;
+                    last.merge = (uint32_t)my_merge;
                 }
                 pos = piece_end;
                 if (pos == range_end(c)) { ++c; cta_begin[c] = (uint32_t)ni; }
             }
             if (split) {
-                if (nm >= merges_cap) return CART_ERR_CAPACITY;
-                merges[nm].row_group = rg;
-                merges[nm].slot_begin = slot_first;
-                merges[nm].slot_end = next_slot;
-                merges[nm].reserved = 0;
-                ++nm;
+                merges[my_merge].row_group = rg;
+                merges[my_merge].slot_begin = slot_first;
+                merges[my_merge].slot_end = next_slot;
+                merges[my_merge].reserved = 0;
             }
         }
     }

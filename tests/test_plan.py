@@ -56,6 +56,8 @@ def check_plan(segs, Hkv, n_cta, tile):
             tiles += -(-it.n_tok // tile)
             if it.flags & E_:
                 pieces.setdefault(it.row_group, []).append((bool(it.flags & D_), it.slot))
+                if not (it.flags & D_):
+                    assert plan["merges"][it.merge].row_group == it.row_group
                 open_rg = None
             else:
                 assert not (it.flags & D_)
