@@ -1,0 +1,126 @@
+"""GPU parity at the full sizes of the benchmark workloads, in the launch configuration the
+benchmark times (the same loader, the same per-layer append + decode calls): the CUDA path against the
+float64 CPU oracle on sampled (layer, request) outputs, which the oracle computes one by one, plus
+properties that hold at any size (finite outputs, lse bounds, bitwise reproducibility).
+
+The two largest workloads hold 77 GB and 105 GB of KV; they are skipped when the device has less free
+memory than they need."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2506_06266_b200 import binding, runner, synth
+
+import cart_harness as H
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+
+
+def need_bytes(w, extra_capacity, slack=12 << 30):
+    """Arena plus the generator's temporaries (one Cartridge's K and V and a float32 chunk)."""
+    one_cart = 2 * w.n_layers * w.n_kv_heads * w.p * w.head_dim * 2
+    return runner.arena_bytes_for(w, extra_capacity) + 2 * one_cart + slack
+
+
+def skip_unless_fits(w, extra_capacity):
+    free, _ = torch.cuda.mem_get_info(torch.device(DEV))
+    need = need_bytes(w, extra_capacity)
+    if free < need:
+        pytest.skip("needs %.0f GB of device memory, %.0f GB free" % (need / 1e9, free / 1e9))
+
+
+def sampled_check(lw, w, q, out, lse, layers, requests, appended):
+    """Oracle on the sampled (layer, request) pairs.  `appended` lists, oldest first, the (k_new, v_new)
+    tensors [L][B][Hkv][D] of the decode steps taken so far."""
+    worst = 0.0
+    for layer in layers:
+        segs, rows = [], []
+        for b in requests:
+            s = list(lw.host_segments(layer, b))
+            if appended:
+                ka = np.stack([synth.bits(k[layer, b]) for (k, _) in appended], axis=1)   # [Hkv][steps][D]
+                va = np.stack([synth.bits(v[layer, b]) for (_, v) in appended], axis=1)
+                s.append((ka, va))
+            segs.append(s)
+            rows.append(b)
+        ro, rl = oracle.decode_layer(synth.bits(q[layer][rows]), segs, w.scale)
+        r = H.assert_close(out[layer][rows], lse[layer][rows], ro, rl,
+                           "%s layer %d requests %s" % (w.name, layer, rows))
+        worst = max(worst, r["rel_fro"])
+    return worst
+
+
+def any_size_properties(w, lw, out, lse):
+    """Every output is finite.  With N(0,1) queries and keys the scaled scores are close to N(0,1), so
+    the lse of n tokens sits near ln n + 1/2 (checked loosely, and only without outlier channels).
+    Outputs are convex combinations of N(0,1) draws, so none exceeds the largest magnitude drawn."""
+    assert torch.isfinite(out.float()).all()
+    assert torch.isfinite(lse).all()
+    n = torch.from_numpy(lw.kv_tokens()).to(lse.device).double()
+    centred = lse.double() - torch.log(n)[None, :, None]
+    if w.outlier_prob == 0.0:
+        assert float(centred.min()) > -0.5 and float(centred.max()) < 6.0
+    assert float(out.float().abs().max()) < 8.0
+
+
+def run_steps(w, steps, check_steps, layers, requests):
+    skip_unless_fits(w, steps)
+    dev = torch.device(DEV)
+    torch.cuda.set_device(dev)
+    stream = torch.cuda.current_stream(dev)
+    lw = runner.LoadedWorkload(w, dev, extra_capacity=steps, keep_layers=layers, keep_requests=requests,
+                               stream=stream)
+    try:
+        L, B = w.n_layers, w.batch
+        out = torch.empty((L, B, w.n_q_heads, 128), dtype=torch.bfloat16, device=dev)
+        lse = torch.empty((L, B, w.n_q_heads), dtype=torch.float32, device=dev)
+        appended = []
+        for step in range(steps):
+            q = w.queries(step, dev)
+            kn, vn = w.appended_kv(step, dev)
+            out.fill_(float("nan"))
+            lse.fill_(float("nan"))
+            lw.step(q, kn, vn, out, lse)
+            binding.cart_sync_status(lw.ctx, stream)
+            appended.append((kn, vn))
+            if step + 1 in check_steps:
+                sampled_check(lw, w, q, out, lse, layers, requests, appended)
+                any_size_properties(w, lw, out, lse)
+                if step + 1 == check_steps[-1]:
+                    # the same step's attention again (no append): bitwise equal
+                    out2, lse2 = torch.empty_like(out), torch.empty_like(lse)
+                    for layer in layers:
+                        binding.cart_decode_attention(lw.ctx, layer, lw.req_list, q[layer], out2[layer],
+                                                      lse2[layer], stream)
+                    binding.cart_sync_status(lw.ctx, stream)
+                    for layer in layers:
+                        assert torch.equal(out[layer], out2[layer]) and torch.equal(lse[layer], lse2[layer])
+        for b in requests:
+            assert binding.cart_suffix_len(lw.ctx, lw.reqs[b], layers[-1]) == int(lw.suffix[b]) + steps
+    finally:
+        lw.close()
+        torch.cuda.empty_cache()
+
+
+def test_config2_full_size_sampled_outputs():
+    run_steps(synth.config2(), steps=1, check_steps=[1], layers=[0, 13, 27], requests=[0, 21, 63])
+
+
+def test_config3_full_size_64_decode_steps_with_append():
+    run_steps(synth.config3(), steps=64, check_steps=[1, 32, 64], layers=[0, 31], requests=[0, 77, 127])
+
+
+def test_config4_full_size_composed_pairs():
+    run_steps(synth.config4(), steps=1, check_steps=[1], layers=[0, 31], requests=[0, 50, 95])
+
+
+def test_config5_cartridge_side_full_size():
+    run_steps(synth.config5_cartridge(), steps=1, check_steps=[1], layers=[0, 31], requests=[0, 255])
+
+
+def test_config5_full_context_side_full_size():
+    # 8 private 100 000-token prefixes over 32 layers: 105 GB, rows addressed beyond 2^28
+    run_steps(synth.config5_full(), steps=1, check_steps=[1], layers=[0, 31], requests=[0, 7])
