@@ -145,6 +145,14 @@ CART_API cart_status cart_decode_attention(cart_ctx *ctx, int32_t layer, const c
                                   int32_t n_reqs, const void *q /*device*/, void *out /*device*/,
                                   float *lse /*device or NULL*/, void *stream);
 
+/* Sharing policy.  When at least min_readers requests of a decode batch attend to the same stored
+ * Cartridge (one Cartridge serving many users, Sec. 1 and Sec. 3.3; pool members composed by many
+ * requests, Sec. 5.4), cart_decode_attention reads each of its K/V tiles once for up to 128 query
+ * rows (all heads of up to 128 / G readers) and multiplies them on the tensor cores, instead of once
+ * per request; the result is the same up to fp32 rounding.  Default 4; 0 switches sharing off (every
+ * request streams its whole cache).  Errors: INVALID_ARG. */
+CART_API cart_status cart_set_share_min_readers(cart_ctx *ctx, int32_t min_readers);
+
 /* Current suffix length of a request in a layer (host-side mirror). */
 CART_API cart_status cart_suffix_len(cart_ctx *ctx, cart_req req, int32_t layer, int32_t *out_len /*host*/);
 
@@ -159,8 +167,8 @@ CART_API cart_status cart_kv_bytes(cart_ctx *ctx, cart_req req, uint64_t *logica
 CART_API cart_status cart_sync_status(cart_ctx *ctx, void *stream);
 
 /* Kernel timing for the benchmark's roofline line.  With timing enabled, every decode-attention
- * kernel launch (not the append) is bracketed by a pair of CUDA events on
- * its stream.  cart_get_timing synchronises the recorded events, returns the summed kernel time in
+ * call's kernels (the shared-segment kernel, if the batch shares a Cartridge, and the stream kernel; not
+ * the append) are bracketed by one pair of CUDA events on their stream.  cart_get_timing synchronises the recorded events, returns the summed kernel time in
  * milliseconds and the number of launches since the last call, and forgets them.  At most 8192
  * launches are remembered between two reads; later ones go untimed.  Errors: INVALID_ARG, CUDA. */
 CART_API cart_status cart_set_timing(cart_ctx *ctx, int32_t enable);

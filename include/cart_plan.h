@@ -79,6 +79,70 @@ CART_API cart_status cart_plan_build(const cart_plan_seg *segs, const int32_t *s
                             int32_t *n_merges, int32_t *n_cta_used, int32_t *n_slots,
                             int64_t *total_tiles);
 
+/*
+ * Shared segments.  When several requests of a batch attend to the same stored Cartridge (one
+ * Cartridge serving many users, Sec. 1 and Sec. 3.3; members of a pool composed by many requests,
+ * Sec. 5.4), its K/V tiles need not be streamed once per request: the query heads of all its readers
+ * form the rows of one dense product per tile.  cart_plan_build_shared takes such segments out of the
+ * per-request stream and describes them as "shared units" for a tensor-core kernel:
+ *   - a segment is shared when at least share_min_readers requests of the batch hold it (same k_row,
+ *     v_row and length) and it has at least one full tile of share_tile_tokens tokens;
+ *   - its readers, in batch order, are cut into M-tiles of at most 128 / group requests (128 query
+ *     rows: row i * group + h is head h of the M-tile's i-th reader);
+ *   - only the full share_tile_tokens-token tiles are shared; the ragged tail (fewer tokens than one
+ *     tile) stays in each reader's stream as a short segment;
+ *   - the (segment, M-tile, KV head) tile runs, laid end to end, are divided into contiguous ranges,
+ *     one per block, as the stream is; a range boundary inside a run cuts it into "chunks".
+ * Every unit writes one partial (o, lse) per reader row group; the partial slots of a row group are
+ * contiguous: first its shared chunks (segments in cache order, chunks in order), then its stream
+ * pieces.  A row group with a shared part is never written directly: its cart_merge_item counts all
+ * of its partials and whichever block delivers the last one merges them.
+ */
+typedef struct {
+    uint32_t k_row;        /* first row of the run for layer 0 (KV head and token offset applied) */
+    uint32_t v_row;
+    uint32_t layer_stride; /* add layer * layer_stride to both rows */
+    uint32_t n_tiles;      /* full tiles of share_tile_tokens tokens in the run (> 0) */
+    uint32_t reader_begin; /* first entry of the M-tile in readers[] */
+    uint32_t n_readers;    /* entries of the M-tile (1 .. 128 / group) */
+    uint32_t kv_head;
+    uint32_t chunk;        /* ordinal of the run among the runs of its (segment, M-tile, KV head) */
+} cart_shared_unit;
+
+/* Capacities (in) and results (out) of cart_plan_build_shared; all arrays are host memory. */
+typedef struct {
+    /* stream part, as in cart_plan_build */
+    cart_work_item *items;     int32_t items_cap;    int32_t n_items;
+    uint32_t *cta_begin;       /* [n_cta + 1] */
+    cart_merge_item *merges;   int32_t merges_cap;   int32_t n_merges;
+    int32_t n_cta_used;        /* blocks of the stream kernel that received work (may be 0) */
+    int32_t slots_cap;         /* partial slots available */
+    int32_t n_slots;           /* partial slots used (shared + stream) */
+    int64_t total_tiles;       /* stream tiles */
+    /* shared part */
+    cart_shared_unit *units;   int32_t units_cap;    int32_t n_units;
+    uint32_t *unit_cta_begin;  /* [n_cta + 1]: block c of the shared kernel owns units[unit_cta_begin[c] ..] */
+    int32_t n_unit_cta_used;   /* blocks of the shared kernel that received work (0 = nothing shared) */
+    uint32_t *readers;         int32_t readers_cap;  int32_t n_readers;  /* batch index per reader entry */
+    uint32_t *reader_slot;     /* [readers_cap * n_kv_heads]: first slot of (entry, KV head); + unit.chunk */
+    uint32_t *reader_merge;    /* [readers_cap * n_kv_heads]: merge item of (entry, KV head) */
+    int64_t shared_tiles;      /* tile runs handed to the shared kernel, in share_tile_tokens tiles */
+} cart_plan_out;
+
+/*
+ * Builds the stream plan and the shared units.  segs / seg_begin / n_reqs / n_kv_heads / n_cta /
+ * tile_tokens as in cart_plan_build; group = query heads per KV head (1..8);
+ * share_min_readers = 0 disables sharing (the result then equals cart_plan_build's);
+ * share_tile_tokens is a multiple of tile_tokens.
+ * If the partial slots the shared chunks need exceed slots_cap, the shared ranges are made longer
+ * (fewer blocks, fewer chunks) until they fit; if they cannot fit, nothing is shared.
+ * Errors: INVALID_ARG, EMPTY, CAPACITY (an output array is too small).
+ */
+CART_API cart_status cart_plan_build_shared(const cart_plan_seg *segs, const int32_t *seg_begin, int32_t n_reqs,
+                                            int32_t n_kv_heads, int32_t group, int32_t n_cta, int32_t tile_tokens,
+                                            int32_t share_min_readers, int32_t share_tile_tokens,
+                                            cart_plan_out *out);
+
 #ifdef __cplusplus
 }
 #endif

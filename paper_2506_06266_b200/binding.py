@@ -29,6 +29,7 @@ EXPORTS = ["cart_scratch_bytes", "cart_create", "cart_destroy", "cart_register_c
            "cart_compose", "cart_release_cartridge", "cart_request_open", "cart_request_close",
            "cart_append_kv", "cart_extend_kv", "cart_decode_attention", "cart_suffix_len",
            "cart_kv_bytes", "cart_sync_status", "cart_set_timing", "cart_get_timing",
+           "cart_set_share_min_readers", "cart_plan_build_shared",
            "cart_decode_attention_static", "cart_launch_count", "cart_status_string",
            "cart_last_error", "cart_plan_build"]
 
@@ -58,6 +59,30 @@ class cart_work_item(ctypes.Structure):
 class cart_merge_item(ctypes.Structure):
     _fields_ = [("row_group", ctypes.c_uint32), ("slot_begin", ctypes.c_uint32),
                 ("slot_end", ctypes.c_uint32), ("reserved", ctypes.c_uint32)]
+
+
+class cart_shared_unit(ctypes.Structure):
+    _fields_ = [("k_row", ctypes.c_uint32), ("v_row", ctypes.c_uint32),
+                ("layer_stride", ctypes.c_uint32), ("n_tiles", ctypes.c_uint32),
+                ("reader_begin", ctypes.c_uint32), ("n_readers", ctypes.c_uint32),
+                ("kv_head", ctypes.c_uint32), ("chunk", ctypes.c_uint32)]
+
+
+class cart_plan_out(ctypes.Structure):
+    _fields_ = [("items", ctypes.POINTER(cart_work_item)), ("items_cap", ctypes.c_int32), ("n_items", ctypes.c_int32),
+                ("cta_begin", ctypes.POINTER(ctypes.c_uint32)),
+                ("merges", ctypes.POINTER(cart_merge_item)), ("merges_cap", ctypes.c_int32),
+                ("n_merges", ctypes.c_int32),
+                ("n_cta_used", ctypes.c_int32), ("slots_cap", ctypes.c_int32), ("n_slots", ctypes.c_int32),
+                ("total_tiles", ctypes.c_int64),
+                ("units", ctypes.POINTER(cart_shared_unit)), ("units_cap", ctypes.c_int32),
+                ("n_units", ctypes.c_int32),
+                ("unit_cta_begin", ctypes.POINTER(ctypes.c_uint32)), ("n_unit_cta_used", ctypes.c_int32),
+                ("readers", ctypes.POINTER(ctypes.c_uint32)), ("readers_cap", ctypes.c_int32),
+                ("n_readers", ctypes.c_int32),
+                ("reader_slot", ctypes.POINTER(ctypes.c_uint32)),
+                ("reader_merge", ctypes.POINTER(ctypes.c_uint32)),
+                ("shared_tiles", ctypes.c_int64)]
 
 
 CART_ITEM_BEGIN, CART_ITEM_END, CART_ITEM_DIRECT = 1, 2, 4
@@ -100,6 +125,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.cart_kv_bytes.argtypes = [vp, i32, u64p, u64p]
     lib.cart_sync_status.argtypes = [vp, vp]
     lib.cart_set_timing.argtypes = [vp, i32]
+    lib.cart_set_share_min_readers.argtypes = [vp, i32]
     lib.cart_get_timing.argtypes = [vp, ctypes.POINTER(ctypes.c_double), u64p]
     lib.cart_decode_attention_static.argtypes = [vp, vp, i32, i32, i32, i32, ctypes.c_float, vp, vp, i32, vp]
     lib.cart_launch_count.argtypes = [vp]
@@ -112,6 +138,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
         ctypes.POINTER(cart_plan_seg), i32p, i32, i32, i32, i32, ctypes.POINTER(cart_work_item), i32,
         i32p, ctypes.POINTER(ctypes.c_uint32), ctypes.POINTER(cart_merge_item), i32, i32p, i32p, i32p,
         ctypes.POINTER(ctypes.c_int64)]
+    lib.cart_plan_build_shared.argtypes = [ctypes.POINTER(cart_plan_seg), i32p, i32, i32, i32, i32, i32, i32, i32,
+                                           ctypes.POINTER(cart_plan_out)]
     for name in EXPORTS:
         fn = getattr(lib, name)
         if name not in ("cart_launch_count", "cart_status_string", "cart_last_error"):
@@ -252,6 +280,10 @@ def cart_set_timing(ctx: int, enable: bool) -> None:
     _check(load_library().cart_set_timing(ctx, 1 if enable else 0), "cart_set_timing", ctx)
 
 
+def cart_set_share_min_readers(ctx: int, min_readers: int) -> None:
+    _check(load_library().cart_set_share_min_readers(ctx, int(min_readers)), "cart_set_share_min_readers", ctx)
+
+
 def cart_get_timing(ctx: int) -> Tuple[float, int]:
     ms, n = ctypes.c_double(0.0), ctypes.c_uint64(0)
     _check(load_library().cart_get_timing(ctx, ctypes.byref(ms), ctypes.byref(n)), "cart_get_timing", ctx)
@@ -299,3 +331,48 @@ def cart_plan_build(segs: Sequence[Sequence[Tuple[int, int, int, int, int]]], n_
     return {"items": [items[i] for i in range(n_items.value)], "cta_begin": list(cta_begin),
             "merges": [merges[i] for i in range(n_merges.value)], "n_cta_used": n_used.value,
             "n_slots": n_slots.value, "total_tiles": total.value}
+
+
+def cart_plan_build_shared(segs: Sequence[Sequence[Tuple[int, int, int, int, int]]], n_kv_heads: int, group: int,
+                           n_cta: int, tile_tokens: int, share_min_readers: int, share_tile_tokens: int,
+                           slots_cap: int = 1 << 20):
+    """Host-only planner with shared segments (see include/cart_plan.h).  Returns a dict with the
+    stream plan (items, cta_begin, merges, ...) and the shared part (units, unit_cta_begin, readers,
+    reader_slot[entry][head], reader_merge[entry][head])."""
+    lib = load_library()
+    flat = [s for r in segs for s in r]
+    seg_arr = (cart_plan_seg * max(len(flat), 1))(*[cart_plan_seg(*s) for s in flat])
+    begins = [0]
+    for r in segs:
+        begins.append(begins[-1] + len(r))
+    sb = (ctypes.c_int32 * len(begins))(*begins)
+    n_rg = len(segs) * n_kv_heads
+    items_cap = 2 * len(flat) * n_kv_heads + n_cta + 8
+    merges_cap = n_rg + n_cta
+    readers_cap = max(len(flat), 1)
+    units_cap = readers_cap * n_kv_heads + n_cta
+    o = cart_plan_out()
+    items = (cart_work_item * items_cap)()
+    cta_begin = (ctypes.c_uint32 * (n_cta + 1))()
+    merges = (cart_merge_item * merges_cap)()
+    units = (cart_shared_unit * units_cap)()
+    unit_cta_begin = (ctypes.c_uint32 * (n_cta + 1))()
+    readers = (ctypes.c_uint32 * readers_cap)()
+    reader_slot = (ctypes.c_uint32 * (readers_cap * n_kv_heads))()
+    reader_merge = (ctypes.c_uint32 * (readers_cap * n_kv_heads))()
+    o.items, o.items_cap, o.cta_begin = items, items_cap, cta_begin
+    o.merges, o.merges_cap, o.slots_cap = merges, merges_cap, slots_cap
+    o.units, o.units_cap, o.unit_cta_begin = units, units_cap, unit_cta_begin
+    o.readers, o.readers_cap, o.reader_slot, o.reader_merge = readers, readers_cap, reader_slot, reader_merge
+    st = lib.cart_plan_build_shared(seg_arr, sb, len(segs), n_kv_heads, group, n_cta, tile_tokens,
+                                    share_min_readers, share_tile_tokens, ctypes.byref(o))
+    _check(st, "cart_plan_build_shared")
+    nr = o.n_readers
+    return {"items": [items[i] for i in range(o.n_items)], "cta_begin": list(cta_begin),
+            "merges": [merges[i] for i in range(o.n_merges)], "n_cta_used": o.n_cta_used,
+            "n_slots": o.n_slots, "total_tiles": o.total_tiles,
+            "units": [units[i] for i in range(o.n_units)], "unit_cta_begin": list(unit_cta_begin),
+            "n_unit_cta_used": o.n_unit_cta_used, "readers": [readers[i] for i in range(nr)],
+            "reader_slot": [[reader_slot[e * n_kv_heads + g] for g in range(n_kv_heads)] for e in range(nr)],
+            "reader_merge": [[reader_merge[e * n_kv_heads + g] for g in range(n_kv_heads)] for e in range(nr)],
+            "shared_tiles": o.shared_tiles}

@@ -23,10 +23,16 @@ constexpr size_t kMaxTimedLaunches = 8192;
 
 uint64_t round_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
 
+// A Cartridge is handed to the shared-segment kernel when at least this many requests of the batch
+// hold it (and it has at least one full 128-token tile); below that its readers stream it one by one.
+constexpr int kShareMinReaders = 4;
+
 struct ScratchLayout {
     uint64_t status_off, tickets_off, plan_off, plan_slot_bytes, cta_begin_off, merges_off, items_off;
+    // shared-segment part of a plan slot
+    uint64_t shared_off, unit_cta_begin_off, readers_off, reader_slot_off, reader_merge_off, units_off;
     uint64_t part_o_off, part_lse_off, total;
-    int items_cap, slots_cap;
+    int items_cap, slots_cap, merges_cap, units_cap, readers_cap;
 };
 
 ScratchLayout scratch_layout(const cart_config &c)
@@ -34,16 +40,29 @@ ScratchLayout scratch_layout(const cart_config &c)
     ScratchLayout s{};
     const int parts = c.max_parts > 0 ? c.max_parts : 8;
     const int group = c.n_q_heads / c.n_kv_heads;
-    s.items_cap = c.max_requests * c.n_kv_heads * (parts + 1) + kMaxCta;
-    s.slots_cap = 2 * kMaxCta;
+    const int row_groups = c.max_requests * c.n_kv_heads;
+    s.items_cap = row_groups * (parts + 1) + kMaxCta;
+    // a row group with a shared part is always merged; the others only when a block boundary splits them
+    s.merges_cap = row_groups + kMaxCta;
+    // partial slots: stream pieces (one per row group with a shared part, two per block boundary) plus
+    // the chunks of shared segments (the planner keeps them within what is left)
+    s.slots_cap = 10 * row_groups + 2 * kMaxCta;
+    s.readers_cap = c.max_requests * parts;
+    s.units_cap = s.readers_cap * c.n_kv_heads + kMaxCta;
     s.status_off = 0;
-    s.tickets_off = kAlign;  // one arrival counter per split row group, zero between launches
-    s.plan_off = s.tickets_off + round_up((uint64_t)kMaxCta * 4, kAlign);
-    // one plan slot: [cta_begin][merges][items]
+    s.tickets_off = kAlign;  // one arrival counter per merge item, zero between launches
+    s.plan_off = s.tickets_off + round_up((uint64_t)s.merges_cap * 4, kAlign);
+    // one plan slot: [cta_begin][merges][items] [unit_cta_begin][readers][reader_slot][reader_merge][units]
     s.cta_begin_off = 0;
     s.merges_off = round_up((uint64_t)(kMaxCta + 1) * 4, kAlign);
-    s.items_off = s.merges_off + round_up((uint64_t)kMaxCta * sizeof(cart_merge_item), kAlign);
-    s.plan_slot_bytes = s.items_off + round_up((uint64_t)s.items_cap * sizeof(cart_work_item), kAlign);
+    s.items_off = s.merges_off + round_up((uint64_t)s.merges_cap * sizeof(cart_merge_item), kAlign);
+    s.shared_off = s.items_off + round_up((uint64_t)s.items_cap * sizeof(cart_work_item), kAlign);
+    s.unit_cta_begin_off = s.shared_off;
+    s.readers_off = s.unit_cta_begin_off + round_up((uint64_t)(kMaxCta + 1) * 4, kAlign);
+    s.reader_slot_off = s.readers_off + round_up((uint64_t)s.readers_cap * 4, kAlign);
+    s.reader_merge_off = s.reader_slot_off + round_up((uint64_t)s.readers_cap * c.n_kv_heads * 4, kAlign);
+    s.units_off = s.reader_merge_off + round_up((uint64_t)s.readers_cap * c.n_kv_heads * 4, kAlign);
+    s.plan_slot_bytes = s.units_off + round_up((uint64_t)s.units_cap * sizeof(cart_shared_unit), kAlign);
     s.part_o_off = s.plan_off + (uint64_t)kPlanSlots * s.plan_slot_bytes;
     s.part_lse_off = s.part_o_off + round_up((uint64_t)s.slots_cap * group * kHeadDim * 4, kAlign);
     s.total = s.part_lse_off + round_up((uint64_t)s.slots_cap * kMaxGroup * 4, kAlign);
@@ -94,6 +113,7 @@ struct PlanSlot {
     std::vector<uint32_t> key;
     uint64_t epoch = 0;
     int32_t n_items = 0, n_merges = 0, n_cta_used = 0, n_slots = 0;
+    int32_t n_units = 0, n_unit_cta_used = 0;
 };
 
 }  // namespace
@@ -104,6 +124,7 @@ struct cart_ctx {
     int group = 1;
     float scale = 0.f;
     int n_cta = 0;
+    int share_min_readers = kShareMinReaders;
     uint64_t n_rows = 0;
     alignas(64) CUtensorMap tmap;
     std::vector<FreeBlock> free_list;
@@ -284,7 +305,7 @@ cart_status cart_create(const cart_config *cfg, cart_ctx **out)
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, cfg->device);
     if (e != cudaSuccess || sms < 1) return bail(CART_ERR_CUDA);
     ctx->n_cta = std::min(sms, kMaxCta);
-    if (prepare_kernels() != cudaSuccess) return bail(CART_ERR_CUDA);
+    if (prepare_kernels() != cudaSuccess || prepare_shared_kernel() != cudaSuccess) return bail(CART_ERR_CUDA);
     if (encode_tensor_map(ctx) != CART_OK) return bail(CART_ERR_CUDA);
     for (int i = 0; i < kPlanSlots; ++i) {
         PlanSlot &sl = ctx->slots[i];
@@ -322,6 +343,15 @@ cart_status cart_set_timing(cart_ctx *ctx, int32_t enable)
 {
     if (!ctx) return CART_ERR_INVALID_ARG;
     ctx->timing = enable != 0;
+    return CART_OK;
+}
+
+cart_status cart_set_share_min_readers(cart_ctx *ctx, int32_t min_readers)
+{
+    if (!ctx) return CART_ERR_INVALID_ARG;
+    if (min_readers < 0) return fail(ctx, CART_ERR_INVALID_ARG, "share_min_readers: negative");
+    ctx->share_min_readers = min_readers;
+    ++ctx->epoch;  // cached plans were built under the old policy
     return CART_OK;
 }
 
@@ -612,17 +642,36 @@ cart_status cart_decode_attention(cart_ctx *ctx, int32_t layer, const cart_req *
             sb.push_back((int32_t)segs.size());
         }
         const ScratchLayout &lay = ctx->lay;
-        int64_t total_tiles = 0;
-        cart_status st = cart_plan_build(
-            segs.data(), sb.data(), n_reqs, Hkv, ctx->n_cta, kTileTokens,
-            reinterpret_cast<cart_work_item *>(ns.host + lay.items_off), lay.items_cap, &ns.n_items,
-            reinterpret_cast<uint32_t *>(ns.host + lay.cta_begin_off),
-            reinterpret_cast<cart_merge_item *>(ns.host + lay.merges_off), kMaxCta, &ns.n_merges, &ns.n_cta_used,
-            &ns.n_slots, &total_tiles);
+        cart_plan_out po{};
+        po.items = reinterpret_cast<cart_work_item *>(ns.host + lay.items_off);
+        po.items_cap = lay.items_cap;
+        po.cta_begin = reinterpret_cast<uint32_t *>(ns.host + lay.cta_begin_off);
+        po.merges = reinterpret_cast<cart_merge_item *>(ns.host + lay.merges_off);
+        po.merges_cap = lay.merges_cap;
+        po.slots_cap = lay.slots_cap;
+        po.units = reinterpret_cast<cart_shared_unit *>(ns.host + lay.units_off);
+        po.units_cap = lay.units_cap;
+        po.unit_cta_begin = reinterpret_cast<uint32_t *>(ns.host + lay.unit_cta_begin_off);
+        po.readers = reinterpret_cast<uint32_t *>(ns.host + lay.readers_off);
+        po.readers_cap = lay.readers_cap;
+        po.reader_slot = reinterpret_cast<uint32_t *>(ns.host + lay.reader_slot_off);
+        po.reader_merge = reinterpret_cast<uint32_t *>(ns.host + lay.reader_merge_off);
+        cart_status st = cart_plan_build_shared(segs.data(), sb.data(), n_reqs, Hkv, ctx->group, ctx->n_cta,
+                                                kTileTokens, ctx->share_min_readers, kShareTileTokens, &po);
         if (st != CART_OK) return fail(ctx, st, "decode: planning failed (%s)", cart_status_string(st));
-        if (ns.n_slots > lay.slots_cap) return fail(ctx, CART_ERR_CAPACITY, "decode: too many partial slots");
+        ns.n_items = po.n_items;
+        ns.n_merges = po.n_merges;
+        ns.n_cta_used = po.n_cta_used;
+        ns.n_slots = po.n_slots;
+        ns.n_units = po.n_units;
+        ns.n_unit_cta_used = po.n_unit_cta_used;
         const uint64_t bytes = lay.items_off + (uint64_t)ns.n_items * sizeof(cart_work_item);
         CART_CUDA(ctx, cudaMemcpyAsync(ns.dev, ns.host, bytes, cudaMemcpyHostToDevice, s));
+        if (ns.n_units > 0) {
+            const uint64_t sh_bytes = lay.units_off + (uint64_t)ns.n_units * sizeof(cart_shared_unit) - lay.shared_off;
+            CART_CUDA(ctx, cudaMemcpyAsync(ns.dev + lay.shared_off, ns.host + lay.shared_off, sh_bytes,
+                                           cudaMemcpyHostToDevice, s));
+        }
         ns.key = key;
         ns.epoch = ctx->epoch;
         ns.valid = true;
@@ -641,7 +690,10 @@ cart_status cart_decode_attention(cart_ctx *ctx, int32_t layer, const cart_req *
     dp.part_o = reinterpret_cast<float *>(arena + ctx->lay.part_o_off);
     dp.part_lse2 = reinterpret_cast<float *>(arena + ctx->lay.part_lse_off);
     dp.merges = reinterpret_cast<const cart_merge_item *>(sl->dev + ctx->lay.merges_off);
-    dp.tickets = reinterpret_cast<uint32_t *>(arena + ctx->lay.tickets_off);
+    // Few split row groups: the block that delivers the last partial merges (arrival tickets, no extra
+    // launch).  Many (every reader of a shared Cartridge is one): a merge kernel over all of them.
+    const bool merge_after = sl->n_merges > ctx->n_cta;
+    dp.tickets = merge_after ? nullptr : reinterpret_cast<uint32_t *>(arena + ctx->lay.tickets_off);
     dp.status = reinterpret_cast<uint32_t *>(arena + ctx->lay.status_off);
     dp.layer = layer;
     dp.group = ctx->group;
@@ -655,8 +707,44 @@ cart_status cart_decode_attention(cart_ctx *ctx, int32_t layer, const cart_req *
         }
         CART_CUDA(ctx, cudaEventRecord(ctx->ev_pool[ctx->ev_used], s));
     }
-    CART_CUDA(ctx, launch_decode(ctx->tmap, dp, sl->n_cta_used, s));
-    ++ctx->launches;
+    if (sl->n_units > 0) {
+        SharedParams sp;
+        sp.unit_cta_begin = reinterpret_cast<const uint32_t *>(sl->dev + ctx->lay.unit_cta_begin_off);
+        sp.units = reinterpret_cast<const cart_shared_unit *>(sl->dev + ctx->lay.units_off);
+        sp.readers = reinterpret_cast<const uint32_t *>(sl->dev + ctx->lay.readers_off);
+        sp.reader_slot = reinterpret_cast<const uint32_t *>(sl->dev + ctx->lay.reader_slot_off);
+        sp.reader_merge = reinterpret_cast<const uint32_t *>(sl->dev + ctx->lay.reader_merge_off);
+        sp.merges = dp.merges;
+        sp.q = q;
+        sp.out = out;
+        sp.lse = lse;
+        sp.part_o = dp.part_o;
+        sp.part_lse2 = dp.part_lse2;
+        sp.tickets = dp.tickets;
+        sp.status = dp.status;
+        sp.layer = layer;
+        sp.group = ctx->group;
+        sp.n_kv_heads = Hkv;
+        sp.n_q_heads = ctx->cfg.n_q_heads;
+        sp.scale_log2 = dp.scale_log2;
+        CART_CUDA(ctx, launch_shared(ctx->tmap, sp, sl->n_unit_cta_used, s));
+        ++ctx->launches;
+    }
+    if (sl->n_items > 0) {
+        CART_CUDA(ctx, launch_decode(ctx->tmap, dp, sl->n_cta_used, s));
+        ++ctx->launches;
+    }
+    if (merge_after) {
+        MergeParams mp;
+        mp.merges = dp.merges;
+        mp.part_o = dp.part_o;
+        mp.part_lse2 = dp.part_lse2;
+        mp.out = out;
+        mp.lse = lse;
+        mp.group = ctx->group;
+        CART_CUDA(ctx, launch_merge(mp, sl->n_merges, s));
+        ++ctx->launches;
+    }
     if (timed) {
         CART_CUDA(ctx, cudaEventRecord(ctx->ev_pool[ctx->ev_used + 1], s));
         ctx->ev_used += 2;

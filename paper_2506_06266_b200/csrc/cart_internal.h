@@ -14,11 +14,13 @@ constexpr int kHeadDim = 128;
 constexpr int kRowBytes = kHeadDim * 2;  // one token of one KV head: 128 bf16
 constexpr int kTileTokens = 64;          // tokens per shared-memory stage
 constexpr int kMaxGroup = 8;             // query heads per KV head the kernels support
+constexpr int kShareTileTokens = 128;    // tokens per tile of the shared-segment kernel
 constexpr int kAppendBatch = 256;        // requests one append launch takes (kernel-parameter budget)
 
 // bits of the device status word
 constexpr uint32_t kStatusTimeoutProducer = 1u;
 constexpr uint32_t kStatusTimeoutConsumer = 2u;
+constexpr uint32_t kStatusTimeoutMma = 4u;
 
 struct DecodeParams {
     const uint32_t *cta_begin;   // [grid + 1]
@@ -29,11 +31,43 @@ struct DecodeParams {
     float *part_o;               // fp32 [slot][G][128], normalised partial outputs
     float *part_lse2;            // fp32 [slot][kMaxGroup], base-2 log-sum-exp of a partial
     const cart_merge_item *merges;  // split row groups (which slots belong together)
-    uint32_t *tickets;           // one arrival counter per merge item; zero between launches
+    uint32_t *tickets;           // one arrival counter per merge item, zero between launches; null: the
+                                 // merge kernel runs afterwards and nobody takes tickets
     uint32_t *status;
     int32_t layer;
     int32_t group;               // G
     float scale_log2;            // softmax scale * log2(e)
+};
+
+// Parameters of the shared-segment kernel (units and reader tables as the planner lays them out).
+struct SharedParams {
+    const uint32_t *unit_cta_begin;  // [grid + 1]
+    const cart_shared_unit *units;
+    const uint32_t *readers;         // batch index per reader entry
+    const uint32_t *reader_slot;     // [entry * Hkv + KV head]: first partial slot; + unit.chunk
+    const uint32_t *reader_merge;    // [entry * Hkv + KV head]: merge item
+    const cart_merge_item *merges;
+    const void *q;                   // bf16 [n_reqs][Hq][128]
+    void *out;
+    float *lse;
+    float *part_o;
+    float *part_lse2;
+    uint32_t *tickets;
+    uint32_t *status;
+    int32_t layer;
+    int32_t group;
+    int32_t n_kv_heads;
+    int32_t n_q_heads;
+    float scale_log2;
+};
+
+struct MergeParams {
+    const cart_merge_item *merges;
+    const float *part_o;
+    const float *part_lse2;
+    void *out;
+    float *lse;
+    int32_t group;
 };
 
 struct AppendEntry {
@@ -67,6 +101,9 @@ size_t decode_smem_bytes();
 int decode_threads();
 cudaError_t prepare_kernels();  // sets the dynamic shared-memory attribute; call once per device
 cudaError_t launch_decode(const CUtensorMap &tmap, const DecodeParams &p, int grid, cudaStream_t s);
+cudaError_t prepare_shared_kernel();
+cudaError_t launch_shared(const CUtensorMap &tmap, const SharedParams &p, int grid, cudaStream_t s);
+cudaError_t launch_merge(const MergeParams &p, int n_merges, cudaStream_t s);
 cudaError_t launch_append(const AppendParams &p, cudaStream_t s);
 cudaError_t launch_extend(const ExtendParams &p, cudaStream_t s);
 

@@ -16,6 +16,7 @@
 #include <cuda_bf16.h>
 
 #include "cart_internal.h"
+#include "cart_device.cuh"
 
 namespace cart {
 namespace {
@@ -39,73 +40,6 @@ constexpr uint32_t kSmemUsed = kStages * kStageBytes + kScratchOBytes + kScratch
 constexpr uint32_t kSmemBytes = kSmemUsed + 1024;     // slack to align the stages to 1024 bytes
 static_assert(kSmemBytes <= 232448, "shared memory budget of one sm_100 block exceeded");
 
-constexpr uint64_t kWaitLimitNs = 2000000000ull;      // a wait gives up after about two seconds
-
-// ---- small PTX wrappers ---------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void *p)
-{
-    return (uint32_t)__cvta_generic_to_shared(p);
-}
-__device__ __forceinline__ uint64_t global_timer_ns()
-{
-    uint64_t t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n"
-        ".reg .pred p;\n"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-        "selp.u32 %0, 1, 0, p;\n"
-        "}\n"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// Bounded wait.  Returns false if the block has given up (this wait ran out, or another warp's did).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag,
-                                          uint32_t *status, uint32_t code)
-{
-    if (mbar_try_wait(bar, parity)) return true;
-    if (*abort_flag) return false;
-    const uint64_t t0 = global_timer_ns();
-    uint32_t spins = 0;
-    for (;;) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((++spins & 0xFFu) == 0) {
-            if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > kWaitLimitNs) {
-                *abort_flag = 1;
-                atomicOr(status, code);
-                return false;
-            }
-        }
-    }
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tmap, int32_t x, int32_t y,
-                                            uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(bar)
-        : "memory");
-}
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3)
 {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
@@ -127,17 +61,6 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a2
         "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
         : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ float fast_exp2(float x)
-{
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
-{
-    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<uint32_t *>(&v);
 }
 __device__ __forceinline__ void consumer_bar()
 {
@@ -429,10 +352,11 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeParams 
                     }
                 }
             }
-            if (!(w.flags & CART_ITEM_DIRECT)) __threadfence();  // publish the partial before the ticket
+            const bool ticketed = !(w.flags & CART_ITEM_DIRECT) && p.tickets != nullptr;
+            if (ticketed) __threadfence();  // publish the partial before the ticket
             consumer_bar();  // the scratch may be overwritten by the next piece from here on
 
-            if (!(w.flags & CART_ITEM_DIRECT)) {
+            if (ticketed) {
                 // Split row group: the block whose piece arrives last merges all pieces.  Nobody waits.
                 const cart_merge_item mi = p.merges[w.merge];
                 if (threadIdx.x == 0) {
@@ -446,32 +370,20 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeParams 
                 consumer_bar();
                 if (*last_flag) {
                     __threadfence();
-                    for (int idx = threadIdx.x; idx < G * 64; idx += kConsumerThreads) {
-                        const int r = idx >> 6, dpair = idx & 63;
-                        float M = -INFINITY;
-                        for (uint32_t c = mi.slot_begin; c < mi.slot_end; ++c)
-                            M = fmaxf(M, __ldcg(p.part_lse2 + (size_t)c * kMaxGroup + r));
-                        float L = 0.f, a0 = 0.f, a1 = 0.f;
-                        for (uint32_t c = mi.slot_begin; c < mi.slot_end; ++c) {
-                            const float wgt = fast_exp2(__ldcg(p.part_lse2 + (size_t)c * kMaxGroup + r) - M);
-                            const float2 v = __ldcg(reinterpret_cast<const float2 *>(
-                                p.part_o + ((size_t)c * G + r) * kHeadDim + 2 * dpair));
-                            L += wgt;
-                            a0 += wgt * v.x;
-                            a1 += wgt * v.y;
-                        }
-                        const float inv = 1.f / L;
-                        const size_t orow = (size_t)mi.row_group * G + r;
-                        __nv_bfloat162 *op = reinterpret_cast<__nv_bfloat162 *>(
-                            reinterpret_cast<__nv_bfloat16 *>(p.out) + orow * kHeadDim + 2 * dpair);
-                        *op = __floats2bfloat162_rn(a0 * inv, a1 * inv);
-                        if (dpair == 0 && p.lse) p.lse[orow] = (M + log2f(L)) * 0.6931471805599453f;
-                    }
+                    merge_row_group(mi, G, p.part_o, p.part_lse2, p.out, p.lse, (int)threadIdx.x, kConsumerThreads);
                     if (threadIdx.x == 0) p.tickets[w.merge] = 0;  // ready for the next launch
                 }
             }
         }
     }
+}
+
+// Merges split row groups after the decode kernels, one block per row group.  Used instead of the
+// in-kernel arrival tickets when a batch has more split row groups than blocks (every reader of a
+// shared Cartridge is one).
+__global__ void __launch_bounds__(128) cart_merge_kernel(const MergeParams p)
+{
+    merge_row_group(p.merges[blockIdx.x], p.group, p.part_o, p.part_lse2, p.out, p.lse, (int)threadIdx.x, 128);
 }
 
 // One block per request: copy the new token's K and V rows (Hkv x 256 bytes each) to the suffix end.
@@ -524,6 +436,12 @@ cudaError_t prepare_kernels()
 cudaError_t launch_decode(const CUtensorMap &tmap, const DecodeParams &p, int grid, cudaStream_t s)
 {
     cart_decode_kernel<<<grid, kThreads, kSmemBytes, s>>>(tmap, p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_merge(const MergeParams &p, int n_merges, cudaStream_t s)
+{
+    cart_merge_kernel<<<n_merges, 128, 0, s>>>(p);
     return cudaGetLastError();
 }
 

@@ -1,69 +1,280 @@
 // Host-side work planner: see include/cart_plan.h for the contract.
 #include <algorithm>
 #include <cstdint>
+#include <tuple>
 #include <vector>
 
 #include "cart_plan.h"
 
-extern "C" cart_status cart_plan_build(const cart_plan_seg *segs, const int32_t *seg_begin,
-                                       int32_t n_reqs, int32_t n_kv_heads, int32_t n_cta,
-                                       int32_t tile_tokens, cart_work_item *items, int32_t items_cap,
-                                       int32_t *n_items, uint32_t *cta_begin, cart_merge_item *merges,
-                                       int32_t merges_cap, int32_t *n_merges, int32_t *n_cta_used,
-                                       int32_t *n_slots, int64_t *total_tiles)
+namespace {
+
+// One (shared segment, M-tile, KV head) run of full shared tiles.
+struct Combo {
+    int32_t cls;           // shared segment class
+    uint32_t reader_begin; // first reader entry of the M-tile
+    uint32_t n_readers;
+    uint32_t kv_head;
+    uint64_t n_tiles;
+    uint32_t n_chunks;     // filled by the partition
+};
+
+struct SharedClass {
+    cart_plan_seg seg;      // the stored segment (row of token 0, KV head 0, layer 0)
+    uint32_t reader_begin;  // entries of this class are contiguous in readers[]
+    uint32_t n_readers;
+    uint32_t first_combo;   // combos of this class: (m * n_kv_heads + g) from here
+};
+
+bool same_storage(const cart_plan_seg &a, const cart_plan_seg &b)
 {
-    if (!segs || !seg_begin || !items || !n_items || !cta_begin || !merges || !n_merges ||
-        !n_cta_used || !n_slots || !total_tiles)
+    return a.k_row == b.k_row && a.v_row == b.v_row && a.n_tok == b.n_tok && a.head_stride == b.head_stride &&
+           a.layer_stride == b.layer_stride;
+}
+
+}  // namespace
+
+extern "C" cart_status cart_plan_build_shared(const cart_plan_seg *segs, const int32_t *seg_begin, int32_t n_reqs,
+                                              int32_t n_kv_heads, int32_t group, int32_t n_cta,
+                                              int32_t tile_tokens, int32_t share_min_readers,
+                                              int32_t share_tile_tokens, cart_plan_out *o)
+{
+    if (!segs || !seg_begin || !o || !o->items || !o->cta_begin || !o->merges) return CART_ERR_INVALID_ARG;
+    if (n_reqs < 1 || n_kv_heads < 1 || n_cta < 1 || tile_tokens < 1 || group < 1 || group > 128 ||
+        share_min_readers < 0)
         return CART_ERR_INVALID_ARG;
-    if (n_reqs < 1 || n_kv_heads < 1 || n_cta < 1 || tile_tokens < 1) return CART_ERR_INVALID_ARG;
+    const bool want_share = share_min_readers > 0;
+    if (want_share && (share_tile_tokens < tile_tokens || share_tile_tokens % tile_tokens != 0 || !o->units ||
+                       !o->unit_cta_begin || !o->readers || !o->reader_slot || !o->reader_merge))
+        return CART_ERR_INVALID_ARG;
 
     const uint64_t T = (uint64_t)tile_tokens;
-    uint64_t tiles_per_head = 0; // tiles of one KV head summed over the batch
+    const uint64_t TS = want_share ? (uint64_t)share_tile_tokens : 0;
+    const int32_t n_segs = seg_begin[n_reqs];
     for (int32_t i = 0; i < n_reqs; ++i) {
         uint64_t toks = 0;
         for (int32_t s = seg_begin[i]; s < seg_begin[i + 1]; ++s) {
             if (segs[s].n_tok == 0) return CART_ERR_INVALID_ARG;
             toks += segs[s].n_tok;
-            tiles_per_head += (segs[s].n_tok + T - 1) / T;
         }
         if (toks == 0) return CART_ERR_EMPTY;
+    }
+
+    // ---- 1. which segments are shared, and by whom ------------------------------------------------
+    std::vector<int32_t> seg_entry((size_t)n_segs, -1);  // reader entry of a shared segment occurrence
+    std::vector<int32_t> seg_cls((size_t)n_segs, -1);
+    std::vector<SharedClass> classes;
+    std::vector<Combo> combos;
+    int32_t n_entries = 0;
+    const uint32_t R = (uint32_t)(128 / group);  // readers per M-tile
+    if (want_share) {
+        // order the candidate occurrences by storage, then by position in the batch
+        std::vector<int32_t> order;
+        for (int32_t s = 0; s < n_segs; ++s)
+            if (segs[s].n_tok >= TS) order.push_back(s);
+        auto key = [&](int32_t s) {
+            return std::make_tuple(segs[s].k_row, segs[s].v_row, segs[s].n_tok, segs[s].head_stride,
+                                   segs[s].layer_stride, s);
+        };
+        std::sort(order.begin(), order.end(), [&](int32_t a, int32_t b) { return key(a) < key(b); });
+        std::vector<std::pair<int32_t, int32_t>> groups;  // (first index in order, count), shared ones only
+        for (size_t a = 0; a < order.size();) {
+            size_t b = a + 1;
+            while (b < order.size() && same_storage(segs[order[a]], segs[order[b]])) ++b;
+            if ((int64_t)(b - a) >= share_min_readers) groups.emplace_back((int32_t)a, (int32_t)(b - a));
+            a = b;
+        }
+        // classes in order of first appearance in the batch (a deterministic, input-order layout)
+        std::sort(groups.begin(), groups.end(), [&](const std::pair<int32_t, int32_t> &x,
+                                                    const std::pair<int32_t, int32_t> &y) {
+            return order[(size_t)x.first] < order[(size_t)y.first];
+        });
+        for (const auto &gr : groups) {
+            if (n_entries + gr.second > o->readers_cap) return CART_ERR_CAPACITY;
+            SharedClass c;
+            c.seg = segs[order[(size_t)gr.first]];
+            c.reader_begin = (uint32_t)n_entries;
+            c.n_readers = (uint32_t)gr.second;
+            c.first_combo = (uint32_t)combos.size();
+            for (int32_t j = 0; j < gr.second; ++j) {
+                const int32_t s = order[(size_t)(gr.first + j)];
+                seg_entry[(size_t)s] = n_entries;
+                seg_cls[(size_t)s] = (int32_t)classes.size();
+                // batch index of the request that owns occurrence s
+                const int32_t req = (int32_t)(std::upper_bound(seg_begin, seg_begin + n_reqs + 1, s) - seg_begin) - 1;
+                o->readers[n_entries++] = (uint32_t)req;
+            }
+            const uint32_t m_tiles = (c.n_readers + R - 1) / R;
+            for (uint32_t m = 0; m < m_tiles; ++m)
+                for (int32_t g = 0; g < n_kv_heads; ++g) {
+                    Combo cb;
+                    cb.cls = (int32_t)classes.size();
+                    cb.reader_begin = c.reader_begin + m * R;
+                    cb.n_readers = std::min(R, c.n_readers - m * R);
+                    cb.kv_head = (uint32_t)g;
+                    cb.n_tiles = c.seg.n_tok / TS;
+                    cb.n_chunks = 0;
+                    combos.push_back(cb);
+                }
+            classes.push_back(c);
+        }
+    }
+
+    // ---- 2. divide the shared runs over blocks; shrink the block count until the partials fit ------
+    uint64_t W_sh = 0;
+    for (const Combo &cb : combos) W_sh += cb.n_tiles;
+    uint64_t C_sh = 0;
+    if (W_sh > 0) {
+        // a block should get at least two tiles: every unit pays for loading its queries and writing
+        // its partials
+        C_sh = std::min<uint64_t>((uint64_t)n_cta, std::max<uint64_t>(1, W_sh / 2));
+        // every stream piece of a row group with a shared part takes a slot, and so does every split
+        const int64_t stream_reserve = (int64_t)n_reqs * n_kv_heads + 2 * (int64_t)n_cta;
+        for (;;) {
+            uint64_t pos = 0, c = 0;
+            int64_t need = 0;
+            for (Combo &cb : combos) {
+                uint32_t chunks = 0;
+                uint64_t end = pos + cb.n_tiles;
+                while (pos < end) {
+                    const uint64_t re = ((c + 1) * W_sh) / C_sh;
+                    pos = std::min(end, re);
+                    ++chunks;
+                    if (pos == re) ++c;
+                }
+                cb.n_chunks = chunks;
+                need += (int64_t)chunks * cb.n_readers;
+            }
+            if (need + stream_reserve <= (int64_t)o->slots_cap) break;
+            C_sh /= 2;
+            if (C_sh == 0) break;
+        }
+        if (C_sh == 0) {  // cannot fit: share nothing
+            combos.clear();
+            classes.clear();
+            std::fill(seg_entry.begin(), seg_entry.end(), -1);
+            std::fill(seg_cls.begin(), seg_cls.end(), -1);
+            n_entries = 0;
+            W_sh = 0;
+        }
+    }
+
+    // ---- 3. emit the shared units ------------------------------------------------------------------
+    int32_t nu = 0;
+    if (want_share) {
+        o->unit_cta_begin[0] = 0;
+        uint64_t pos = 0, c = 0;
+        for (const Combo &cb : combos) {
+            const cart_plan_seg &sg = classes[(size_t)cb.cls].seg;
+            uint64_t done = 0;  // tiles of this run already handed out
+            uint32_t chunk = 0;
+            const uint64_t end = pos + cb.n_tiles;
+            while (pos < end) {
+                const uint64_t re = ((c + 1) * W_sh) / C_sh;
+                const uint64_t take = std::min(end, re) - pos;
+                if (nu >= o->units_cap) return CART_ERR_CAPACITY;
+                cart_shared_unit &u = o->units[nu++];
+                const uint32_t tok0 = (uint32_t)(done * TS);
+                u.k_row = sg.k_row + cb.kv_head * sg.head_stride + tok0;
+                u.v_row = sg.v_row + cb.kv_head * sg.head_stride + tok0;
+                u.layer_stride = sg.layer_stride;
+                u.n_tiles = (uint32_t)take;
+                u.reader_begin = cb.reader_begin;
+                u.n_readers = cb.n_readers;
+                u.kv_head = cb.kv_head;
+                u.chunk = chunk++;
+                done += take;
+                pos += take;
+                if (pos == re) { ++c; o->unit_cta_begin[c] = (uint32_t)nu; }
+            }
+        }
+        for (uint64_t b = c; b < (uint64_t)n_cta; ++b) o->unit_cta_begin[b + 1] = (uint32_t)nu;
+    }
+    o->n_units = nu;
+    o->n_unit_cta_used = (int32_t)C_sh;
+    o->n_readers = n_entries;
+    o->shared_tiles = (int64_t)W_sh;
+
+    // ---- 4. the stream: what is left of every request, laid end to end -------------------------------
+    // A shared segment leaves its ragged tail (n_tok mod TS tokens) in its readers' streams.
+    auto stream_part = [&](int32_t s, uint32_t *tok0, uint32_t *ntok) {
+        if (seg_cls[(size_t)s] < 0) { *tok0 = 0; *ntok = segs[s].n_tok; return; }
+        const uint32_t full = (uint32_t)((segs[s].n_tok / TS) * TS);
+        *tok0 = full;
+        *ntok = segs[s].n_tok - full;
+    };
+    uint64_t tiles_per_head = 0;
+    for (int32_t s = 0; s < n_segs; ++s) {
+        uint32_t t0, nt;
+        stream_part(s, &t0, &nt);
+        tiles_per_head += (nt + T - 1) / T;
     }
     const uint64_t W = tiles_per_head * (uint64_t)n_kv_heads;
     const uint64_t C = std::min<uint64_t>((uint64_t)n_cta, W);
 
     int32_t ni = 0, nm = 0;
     uint32_t next_slot = 0;
-    uint64_t pos = 0; // tiles handed out so far
-    uint64_t c = 0;   // block being filled
-    auto range_end = [&](uint64_t blk) { return ((blk + 1) * W) / C; };
-    cta_begin[0] = 0;
+    uint64_t pos = 0;  // tiles handed out so far
+    uint64_t c = 0;    // block being filled
+    auto range_end = [&](uint64_t blk) { return C ? ((blk + 1) * W) / C : 0; };
+    o->cta_begin[0] = 0;
 
     for (int32_t i = 0; i < n_reqs; ++i) {
         const int32_t s0 = seg_begin[i], s1 = seg_begin[i + 1];
         uint64_t rg_tiles = 0;
-        for (int32_t s = s0; s < s1; ++s) rg_tiles += (segs[s].n_tok + T - 1) / T;
+        bool has_shared = false;
+        for (int32_t s = s0; s < s1; ++s) {
+            uint32_t t0, nt;
+            stream_part(s, &t0, &nt);
+            rg_tiles += (nt + T - 1) / T;
+            has_shared = has_shared || seg_cls[(size_t)s] >= 0;
+        }
         for (int32_t g = 0; g < n_kv_heads; ++g) {
             const uint32_t rg = (uint32_t)i * (uint32_t)n_kv_heads + (uint32_t)g;
             const uint64_t rg_start = pos, rg_end = pos + rg_tiles;
-            int32_t s = s0;        // segment under the cursor
-            uint64_t seg_tile = 0; // tiles of segment s already handed out
             const uint32_t slot_first = next_slot;
             bool split = false;
             int32_t my_merge = -1;
+            if (has_shared) {
+                if (nm >= o->merges_cap) return CART_ERR_CAPACITY;
+                my_merge = nm++;
+                split = true;
+                for (int32_t s = s0; s < s1; ++s) {
+                    if (seg_cls[(size_t)s] < 0) continue;
+                    const SharedClass &cl = classes[(size_t)seg_cls[(size_t)s]];
+                    const uint32_t e = (uint32_t)seg_entry[(size_t)s];
+                    const uint32_t m = (e - cl.reader_begin) / R;
+                    const Combo &cb = combos[cl.first_combo + m * (uint32_t)n_kv_heads + (uint32_t)g];
+                    o->reader_slot[(size_t)e * n_kv_heads + g] = next_slot;
+                    o->reader_merge[(size_t)e * n_kv_heads + g] = (uint32_t)my_merge;
+                    next_slot += cb.n_chunks;
+                }
+            }
+            // skip segments that leave nothing in the stream
+            int32_t s = s0;
+            uint32_t seg_tok0 = 0, seg_ntok = 0;
+            auto settle = [&]() {
+                while (s < s1) {
+                    stream_part(s, &seg_tok0, &seg_ntok);
+                    if (seg_ntok > 0) break;
+                    ++s;
+                }
+            };
+            settle();
+            uint64_t seg_tile = 0;  // tiles of segment s already handed out
             while (pos < rg_end) {
                 const uint64_t piece_end = std::min(rg_end, range_end(c));
-                const bool direct = (pos == rg_start && piece_end == rg_end);
+                const bool direct = !has_shared && pos == rg_start && piece_end == rg_end;
                 uint64_t want = piece_end - pos;
                 bool first = true;
                 while (want > 0) {
-                    const uint64_t seg_tiles = (segs[s].n_tok + T - 1) / T;
+                    const uint64_t seg_tiles = (seg_ntok + T - 1) / T;
                     const uint64_t take = std::min(want, seg_tiles - seg_tile);
-                    if (ni >= items_cap) return CART_ERR_CAPACITY;
-                    cart_work_item &it = items[ni++];
+                    if (ni >= o->items_cap) return CART_ERR_CAPACITY;
+                    cart_work_item &it = o->items[ni++];
                     const uint64_t tok0 = seg_tile * T;
-                    const uint64_t tok1 = std::min<uint64_t>(segs[s].n_tok, (seg_tile + take) * T);
-                    it.k_row = segs[s].k_row + (uint32_t)g * segs[s].head_stride + (uint32_t)tok0;
-                    it.v_row = segs[s].v_row + (uint32_t)g * segs[s].head_stride + (uint32_t)tok0;
+                    const uint64_t tok1 = std::min<uint64_t>(seg_ntok, (seg_tile + take) * T);
+                    it.k_row = segs[s].k_row + (uint32_t)g * segs[s].head_stride + seg_tok0 + (uint32_t)tok0;
+                    it.v_row = segs[s].v_row + (uint32_t)g * segs[s].head_stride + seg_tok0 + (uint32_t)tok0;
                     it.layer_stride = segs[s].layer_stride;
                     it.n_tok = (uint32_t)(tok1 - tok0);
                     it.row_group = rg;
@@ -73,15 +284,15 @@ extern "C" cart_status cart_plan_build(const cart_plan_seg *segs, const int32_t 
                     first = false;
                     want -= take;
                     seg_tile += take;
-                    if (seg_tile == seg_tiles) { ++s; seg_tile = 0; }
+                    if (seg_tile == seg_tiles) { ++s; seg_tile = 0; settle(); }
                 }
-                cart_work_item &last = items[ni - 1];
+                cart_work_item &last = o->items[ni - 1];
                 last.flags |= CART_ITEM_END;
                 if (direct) {
                     last.flags |= CART_ITEM_DIRECT;
                 } else {
                     if (!split) {
-                        if (nm >= merges_cap) return CART_ERR_CAPACITY;
+                        if (nm >= o->merges_cap) return CART_ERR_CAPACITY;
                         my_merge = nm++;
                         split = true;
                     }
@@ -89,21 +300,47 @@ extern "C" cart_status cart_plan_build(const cart_plan_seg *segs, const int32_t 
                     last.merge = (uint32_t)my_merge;
                 }
                 pos = piece_end;
-                if (pos == range_end(c)) { ++c; cta_begin[c] = (uint32_t)ni; }
+                if (pos == range_end(c)) { ++c; o->cta_begin[c] = (uint32_t)ni; }
             }
             if (split) {
-                merges[my_merge].row_group = rg;
-                merges[my_merge].slot_begin = slot_first;
-                merges[my_merge].slot_end = next_slot;
-                merges[my_merge].reserved = 0;
+                o->merges[my_merge].row_group = rg;
+                o->merges[my_merge].slot_begin = slot_first;
+                o->merges[my_merge].slot_end = next_slot;
+                o->merges[my_merge].reserved = 0;
             }
         }
     }
-    for (uint64_t b = c; b < (uint64_t)n_cta; ++b) cta_begin[b + 1] = (uint32_t)ni;
-    *n_items = ni;
-    *n_merges = nm;
-    *n_cta_used = (int32_t)C;
-    *n_slots = (int32_t)next_slot;
-    *total_tiles = (int64_t)W;
+    for (uint64_t b = c; b < (uint64_t)n_cta; ++b) o->cta_begin[b + 1] = (uint32_t)ni;
+    if ((int64_t)next_slot > (int64_t)o->slots_cap) return CART_ERR_CAPACITY;
+    o->n_items = ni;
+    o->n_merges = nm;
+    o->n_cta_used = (int32_t)C;
+    o->n_slots = (int32_t)next_slot;
+    o->total_tiles = (int64_t)W;
+    return CART_OK;
+}
+
+extern "C" cart_status cart_plan_build(const cart_plan_seg *segs, const int32_t *seg_begin,
+                                       int32_t n_reqs, int32_t n_kv_heads, int32_t n_cta,
+                                       int32_t tile_tokens, cart_work_item *items, int32_t items_cap,
+                                       int32_t *n_items, uint32_t *cta_begin, cart_merge_item *merges,
+                                       int32_t merges_cap, int32_t *n_merges, int32_t *n_cta_used,
+                                       int32_t *n_slots, int64_t *total_tiles)
+{
+    if (!n_items || !n_merges || !n_cta_used || !n_slots || !total_tiles) return CART_ERR_INVALID_ARG;
+    cart_plan_out o{};
+    o.items = items;
+    o.items_cap = items_cap;
+    o.cta_begin = cta_begin;
+    o.merges = merges;
+    o.merges_cap = merges_cap;
+    o.slots_cap = INT32_MAX;
+    const cart_status st = cart_plan_build_shared(segs, seg_begin, n_reqs, n_kv_heads, 1, n_cta, tile_tokens, 0, 0, &o);
+    if (st != CART_OK) return st;
+    *n_items = o.n_items;
+    *n_merges = o.n_merges;
+    *n_cta_used = o.n_cta_used;
+    *n_slots = o.n_slots;
+    *total_tiles = o.total_tiles;
     return CART_OK;
 }

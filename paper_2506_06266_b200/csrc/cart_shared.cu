@@ -1,0 +1,530 @@
+// Shared-segment decode attention for sm_100a: the dense part of the path.
+//
+// When many requests of a batch attend to the same stored Cartridge (one Cartridge serving many
+// users, Sec. 1 / Sec. 3.3 of the paper; pool members composed by many requests, Sec. 5.4), the scores
+// of all their query heads against one K tile are one matrix product, and so is the weighted sum of
+// the V tile.  This kernel evaluates Eq. 1 restricted to a run of 128-token tiles of such a segment
+// for up to 128 query rows at once (row i * G + h = head h of the M-tile's i-th reader) on the
+// tcgen05 tensor cores, so the tile is fetched once per 128 rows instead of once per request:
+//
+//   producer warp   TMA loads of K and V tiles (128 tokens x 128 dims, 128-byte swizzle) into a
+//                   two-stage ring, completion on mbarriers
+//   MMA warp        one thread issues  S = Q K^T  (128 x 128 x 128, accumulator in tensor memory)
+//                   and  O_t = P V  (fresh accumulator per tile); tcgen05.commit signals mbarriers
+//   2 x 4 softmax  two warpgroups take alternate tiles (warpgroup w owns S, P and O buffer w).  Thread r
+//   warps           of a warpgroup owns query row r: reads S from tensor memory, keeps the running
+//                   maximum and sum of an online softmax over its warpgroup's tiles in fp32, writes
+//                   P = 2^(s - m) as bf16 into shared memory (the A operand of the second product),
+//                   then adds the finished O_t of its previous tile to its fp32 register accumulator,
+//                   rescaled to the new maximum.  At the end of a unit the two warpgroups' states are
+//                   combined through shared memory.
+//
+// S and O_t are double-buffered in tensor memory (4 x 128 columns), so the products of tile t+1 run
+// while the softmax of tile t does.  At the end of a unit every row is written as a normalised fp32
+// partial (o, lse); the partials of a (request, KV head) row group are merged by log-sum-exp either by
+// the block that delivers the last one -- this kernel's or the stream kernel's -- or, when the batch
+// has more split row groups than blocks, by a merge kernel that runs afterwards.
+//
+// Every wait is bounded; on expiry the block raises a flag in the device status word, stops issuing
+// work, waits (bounded) for what is in flight, frees its tensor memory and returns.
+#include <cuda_bf16.h>
+
+#include "cart_device.cuh"
+#include "cart_internal.h"
+
+namespace cart {
+namespace {
+
+constexpr int kShTile = kShareTileTokens;             // tokens per tile = N of the score product
+constexpr uint32_t kShBlock = 128u * 128u;            // 128 rows x 128 bytes: one swizzled block (64 bf16 wide)
+constexpr uint32_t kShTileBytes = 2u * kShBlock;      // 128 x 128 bf16
+constexpr int kShStages = 2;
+constexpr int kShThreads = 384;                       // utility warpgroup (producer, MMA, 2 idle) + 2 softmax warpgroups
+// Registers per thread after the warpgroups have re-divided the block's allocation (384 x 168): the
+// utility warps need few, the softmax threads hold a 128-float accumulator.  4 x 32 x 40 + 8 x 32 x 232
+// = 64512 registers, and per SM sub-partition 1 utility + 2 softmax warps = 16128 of its 16384.
+constexpr int kRegsUtility = 40;
+constexpr int kRegsSoftmax = 232;
+constexpr int kSoftmaxThreads = 128;                  // one softmax warpgroup
+constexpr uint32_t kTmemCols = 512;                   // S0 S1 O0 O1, 128 fp32 columns each
+
+// shared-memory layout (offsets from a 1024-byte aligned base)
+constexpr uint32_t kOffQ = 0;
+constexpr uint32_t kOffK = kOffQ + kShTileBytes;
+constexpr uint32_t kOffV = kOffK + kShStages * kShTileBytes;
+constexpr uint32_t kOffP = kOffV + kShStages * kShTileBytes;
+constexpr uint32_t kOffBar = kOffP + 2 * kShTileBytes;
+constexpr uint32_t kOffMisc = kOffBar + 32 * 8;        // room for 32 barriers (22 used); then: tmem address, abort flag, unit flag
+constexpr uint32_t kOffFlags = kOffMisc + 16;          // one word per reader: "merge this row group"
+constexpr uint32_t kOffComb = kOffFlags + 128 * 4;     // running maximum and sum of the second warpgroup's rows
+constexpr uint32_t kShSmemUsed = kOffComb + 2 * 128 * 4;
+constexpr uint32_t kShSmemBytes = kShSmemUsed + 1024;  // slack to align the base
+static_assert(kShSmemBytes <= 232448, "shared memory budget of one sm_100 block exceeded");
+
+enum Bar : int {
+    kBarKFull = 0,   // [2] TMA -> MMA
+    kBarKEmpty = 2,  // [2] MMA (commit) -> TMA
+    kBarVFull = 4,
+    kBarVEmpty = 6,
+    kBarSFull = 8,   // [2] MMA (commit) -> softmax
+    kBarSFree = 10,  // [2] softmax -> MMA          (4 arrivals: one per softmax warp)
+    kBarPReady = 12, // [2] softmax -> MMA          (4 arrivals)
+    kBarPFree = 14,  // [2] MMA (commit) -> softmax
+    kBarOFull = 16,  // [2] MMA (commit) -> softmax
+    kBarOFree = 18,  // [2] softmax -> MMA          (4 arrivals)
+    kBarQReady = 20, // softmax -> MMA              (8 arrivals: every softmax warp)
+    kBarDrain = 21,  // MMA (commit) -> MMA, on the way out
+};
+
+// ---- tcgen05 wrappers ---------------------------------------------------------------------------
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle.  lbo / sbo in bytes.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, uint32_t lbo, uint32_t sbo)
+{
+    uint64_t d = (uint64_t)((saddr >> 4) & 0x3FFFu);
+    d |= (uint64_t)((lbo >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((sbo >> 4) & 0x3FFFu) << 32;
+    d |= 1ull << 46;  // descriptor version of this architecture
+    d |= 2ull << 61;  // layout type: 128-byte swizzle
+    return d;
+}
+// Instruction descriptor, kind::f16: fp32 accumulator, bf16 A and B, M = 128, N = 128.
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+constexpr uint32_t kIdescS = kIdesc;                  // A (Q) and B (K tile) both K-major
+constexpr uint32_t kIdescPV = kIdesc | (1u << 16);    // B (V tile) is MN-major: dims contiguous
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate)
+{
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+        "}\n" ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 32 consecutive fp32 columns of this thread's tensor-memory lane; waits for the data.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32])
+{
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,"
+        "%29,%30,%31}, [%32];\n"
+        "tcgen05.wait::ld.sync.aligned;"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void softmax_bar()  // the first softmax warpgroup
+{
+    asm volatile("bar.sync 2, %0;" ::"n"(kSoftmaxThreads) : "memory");
+}
+__device__ __forceinline__ void softmax_bar_both()  // both softmax warpgroups
+{
+    asm volatile("bar.sync 3, %0;" ::"n"(2 * kSoftmaxThreads) : "memory");
+}
+
+__global__ void __launch_bounds__(kShThreads, 1)
+cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams p)
+{
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t *smem = smem_raw + (base - raw);
+    auto bar = [&](int i) { return base + kOffBar + (uint32_t)i * 8u; };
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + kOffMisc);
+    volatile uint32_t *abort_flag = tmem_slot + 1;
+    volatile uint32_t *unit_ok = tmem_slot + 2;
+    volatile uint32_t *flags = reinterpret_cast<volatile uint32_t *>(smem + kOffFlags);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bar(kBarKFull + i), 1);
+            mbar_init(bar(kBarKEmpty + i), 1);
+            mbar_init(bar(kBarVFull + i), 1);
+            mbar_init(bar(kBarVEmpty + i), 1);
+            mbar_init(bar(kBarSFull + i), 1);
+            mbar_init(bar(kBarSFree + i), 4);
+            mbar_init(bar(kBarPReady + i), 4);
+            mbar_init(bar(kBarPFree + i), 1);
+            mbar_init(bar(kBarOFull + i), 1);
+            mbar_init(bar(kBarOFree + i), 4);
+        }
+        mbar_init(bar(kBarQReady), 8);
+        mbar_init(bar(kBarDrain), 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        // the whole tensor memory of the SM: one block per SM runs this kernel (shared memory sees to that)
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(base + kOffMisc),
+                     "r"(kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    const uint32_t unit_begin = p.unit_cta_begin[blockIdx.x];
+    const uint32_t unit_end = p.unit_cta_begin[blockIdx.x + 1];
+
+    if (warp < 4) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsUtility));
+        if (warp == 0) {
+            // ================= producer ===================================================================
+            if (lane == 0) {
+                asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap)) : "memory");
+                uint32_t tt = 0;
+                bool ok = true;
+                for (uint32_t ui = unit_begin; ui < unit_end && ok; ++ui) {
+                    const cart_shared_unit u = p.units[ui];
+                    const uint32_t k_row = u.k_row + (uint32_t)p.layer * u.layer_stride;
+                    const uint32_t v_row = u.v_row + (uint32_t)p.layer * u.layer_stride;
+                    for (uint32_t t = 0; t < u.n_tiles; ++t, ++tt) {
+                        const int st = (int)(tt & 1u);
+                        const uint32_t par = (tt >> 1) & 1u;
+                        const int32_t yk = (int32_t)(k_row + t * kShTile), yv = (int32_t)(v_row + t * kShTile);
+                        ok = mbar_wait(bar(kBarKEmpty + st), par ^ 1u, abort_flag, p.status, kStatusTimeoutProducer);
+                        if (!ok) break;
+                        const uint32_t kdst = base + kOffK + (uint32_t)st * kShTileBytes;
+                        mbar_expect_tx(bar(kBarKFull + st), kShTileBytes);
+                        // a block of the tile = 128 rows x 64 dims = two boxes of 64 rows
+                        tma_load_2d(kdst, &tmap, 0, yk, bar(kBarKFull + st));
+                        tma_load_2d(kdst + kShBlock / 2, &tmap, 0, yk + 64, bar(kBarKFull + st));
+                        tma_load_2d(kdst + kShBlock, &tmap, 64, yk, bar(kBarKFull + st));
+                        tma_load_2d(kdst + kShBlock + kShBlock / 2, &tmap, 64, yk + 64, bar(kBarKFull + st));
+                        ok = mbar_wait(bar(kBarVEmpty + st), par ^ 1u, abort_flag, p.status, kStatusTimeoutProducer);
+                        if (!ok) break;
+                        const uint32_t vdst = base + kOffV + (uint32_t)st * kShTileBytes;
+                        mbar_expect_tx(bar(kBarVFull + st), kShTileBytes);
+                        tma_load_2d(vdst, &tmap, 0, yv, bar(kBarVFull + st));
+                        tma_load_2d(vdst + kShBlock / 2, &tmap, 0, yv + 64, bar(kBarVFull + st));
+                        tma_load_2d(vdst + kShBlock, &tmap, 64, yv, bar(kBarVFull + st));
+                        tma_load_2d(vdst + kShBlock + kShBlock / 2, &tmap, 64, yv + 64, bar(kBarVFull + st));
+                    }
+                }
+                if (!ok) {
+                    // gave up: wait (bounded) for the copies still in flight before the block leaves
+                    for (uint32_t u2 = (tt > 2u ? tt - 2u : 0u); u2 <= tt; ++u2) {
+                        const int st = (int)(u2 & 1u);
+                        const uint32_t par = (u2 >> 1) & 1u;
+                        const uint64_t t0 = global_timer_ns();
+                        while (!mbar_try_wait(bar(kBarKFull + st), par) && global_timer_ns() - t0 < kWaitLimitNs) {}
+                        while (!mbar_try_wait(bar(kBarVFull + st), par) && global_timer_ns() - t0 < kWaitLimitNs) {}
+                    }
+                }
+            }
+            __syncwarp();
+        } else if (warp == 1) {
+            // ================= MMA issuer ===================================================================
+            if (lane == 0) {
+                const uint32_t q_lo = base + kOffQ;
+                uint32_t tt0 = 0;   // tiles of earlier units
+                uint32_t nunit = 0;
+                bool ok = true;
+                // S(tt) = Q K^T into S buffer tt & 1
+                auto issue_s = [&](uint32_t tt) -> bool {
+                    const int st = (int)(tt & 1u);
+                    const uint32_t par = (tt >> 1) & 1u;
+                    if (!mbar_wait(bar(kBarKFull + st), par, abort_flag, p.status, kStatusTimeoutMma)) return false;
+                    if (!mbar_wait(bar(kBarSFree + st), par ^ 1u, abort_flag, p.status, kStatusTimeoutMma)) return false;
+                    tc_fence_after();
+                    const uint32_t k_lo = base + kOffK + (uint32_t)st * kShTileBytes;
+    #pragma unroll
+                    for (uint32_t k = 0; k < 8; ++k) {  // 16 dims per instruction
+                        const uint32_t off = (k >> 2) * kShBlock + (k & 3u) * 32u;
+                        umma_bf16(tmem + (uint32_t)st * 128u, umma_desc(q_lo + off, 16, 1024), umma_desc(k_lo + off, 16, 1024),
+                                  kIdescS, k);
+                    }
+                    umma_commit(bar(kBarSFull + st));
+                    umma_commit(bar(kBarKEmpty + st));
+                    return true;
+                };
+                // O(tt) = P V into O buffer tt & 1
+                auto issue_pv = [&](uint32_t tt) -> bool {
+                    const int st = (int)(tt & 1u);
+                    const uint32_t par = (tt >> 1) & 1u;
+                    if (!mbar_wait(bar(kBarVFull + st), par, abort_flag, p.status, kStatusTimeoutMma)) return false;
+                    if (!mbar_wait(bar(kBarOFree + st), par ^ 1u, abort_flag, p.status, kStatusTimeoutMma)) return false;
+                    if (!mbar_wait(bar(kBarPReady + st), par, abort_flag, p.status, kStatusTimeoutMma)) return false;
+                    tc_fence_after();
+                    const uint32_t p_lo = base + kOffP + (uint32_t)st * kShTileBytes;
+                    const uint32_t v_lo = base + kOffV + (uint32_t)st * kShTileBytes;
+    #pragma unroll
+                    for (uint32_t k = 0; k < 8; ++k) {  // 16 tokens per instruction
+                        const uint64_t a = umma_desc(p_lo + (k >> 2) * kShBlock + (k & 3u) * 32u, 16, 1024);
+                        // V: tokens are rows of 128 bytes (8-token groups 1024 bytes apart); the two 64-dim
+                        // blocks of the tile are kShBlock bytes apart
+                        const uint64_t b = umma_desc(v_lo + k * 16u * 128u, kShBlock, 1024);
+                        umma_bf16(tmem + 256u + (uint32_t)st * 128u, a, b, kIdescPV, k);
+                    }
+                    umma_commit(bar(kBarOFull + st));
+                    umma_commit(bar(kBarVEmpty + st));
+                    umma_commit(bar(kBarPFree + st));
+                    return true;
+                };
+                for (uint32_t ui = unit_begin; ui < unit_end && ok; ++ui, ++nunit) {
+                    const uint32_t n = p.units[ui].n_tiles;
+                    ok = mbar_wait(bar(kBarQReady), nunit & 1u, abort_flag, p.status, kStatusTimeoutMma);
+                    if (!ok) break;
+                    tc_fence_after();
+                    ok = issue_s(tt0);
+                    for (uint32_t t = 0; t < n && ok; ++t) {
+                        if (t + 1 < n) ok = issue_s(tt0 + t + 1);
+                        if (ok) ok = issue_pv(tt0 + t);
+                    }
+                    tt0 += n;
+                }
+                // products still in flight must finish before the tensor memory is given back
+                umma_commit(bar(kBarDrain));
+                const uint64_t t0 = global_timer_ns();
+                while (!mbar_try_wait(bar(kBarDrain), 0) && global_timer_ns() - t0 < kWaitLimitNs) {}
+            }
+            __syncwarp();
+        }
+    } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
+        // ================= softmax / epilogue warps ====================================================
+        const int G = p.group;
+        const int wg = (warp - 4) >> 2;       // softmax warpgroup 0 or 1: owns the tiles with (index & 1) == wg
+        const int sw = warp & 3;              // the tensor-memory lanes this warp may read: 32 sw .. 32 sw + 31
+        const int row = 32 * sw + lane;       // query row of the M-tile = tensor-memory lane
+        const int tid = row;                  // index among the 128 threads of the warpgroup
+        const uint32_t lane_addr = tmem + ((uint32_t)(32 * sw) << 16);
+        const __nv_bfloat16 *q = reinterpret_cast<const __nv_bfloat16 *>(p.q);
+        const uint32_t swz = (uint32_t)(row & 7);
+        float *comb_o = reinterpret_cast<float *>(smem + kOffP);     // [128 dims][128 rows], unit end only
+        float *comb_ml = reinterpret_cast<float *>(smem + kOffComb); // [2][128 rows]
+        uint32_t tt0 = 0;
+        bool alive = true;
+        float o_acc[128];
+        // the warp's lanes must stay together (the tensor-memory loads are warp-wide): a wait fails for
+        // all of them or for none
+        auto warp_wait = [&](uint32_t b, uint32_t parity) -> bool {
+            return __all_sync(0xffffffffu, mbar_wait(b, parity, abort_flag, p.status, kStatusTimeoutConsumer));
+        };
+        const uint32_t s_addr = lane_addr + (uint32_t)wg * 128u;
+        const uint32_t o_addr = lane_addr + 256u + (uint32_t)wg * 128u;
+        const uint32_t prow = base + kOffP + (uint32_t)wg * kShTileBytes + (uint32_t)row * 128u;
+
+        for (uint32_t ui = unit_begin; ui < unit_end && alive; ++ui) {
+            const cart_shared_unit u = p.units[ui];
+            const int i_reader = row / G, h = row - i_reader * G;
+            const bool valid = (uint32_t)i_reader < u.n_readers;
+            uint32_t entry = 0, batch = 0;
+            if (valid) {
+                entry = u.reader_begin + (uint32_t)i_reader;
+                batch = p.readers[entry];
+            }
+            // ---- this row's query into shared memory, in the swizzled K-major operand layout; each
+            //      warpgroup copies one 64-dim half -------------------------------------------------
+            {
+                const uint4 *src = reinterpret_cast<const uint4 *>(
+                    q + ((size_t)batch * p.n_q_heads + (size_t)u.kv_head * G + h) * kHeadDim) + 8 * wg;
+                const uint32_t qrow = base + kOffQ + (uint32_t)wg * kShBlock + (uint32_t)row * 128u;
+#pragma unroll
+                for (uint32_t c = 0; c < 8; ++c) {
+                    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                    if (valid) v = __ldg(src + c);
+                    const uint32_t a = qrow + ((c ^ swz) << 4);
+                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+                                 : "memory");
+                }
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(kBarQReady));
+            }
+            float m_run = -INFINITY, l_run = 0.f, alpha_prev = 0.f;
+#pragma unroll
+            for (int d = 0; d < 128; ++d) o_acc[d] = 0.f;
+
+            // adds the finished O of tile tt (relative to the running maximum after tile tt) to o_acc
+            auto take_o = [&](uint32_t tt, float alpha) -> bool {
+                const uint32_t par = (tt >> 1) & 1u;
+                if (!warp_wait(bar(kBarOFull + wg), par)) return false;
+                tc_fence_after();
+#pragma unroll
+                for (int c4 = 0; c4 < 4; ++c4) {
+                    float v[32];
+                    tmem_ld32(o_addr + (uint32_t)c4 * 32u, v);
+#pragma unroll
+                    for (int k = 0; k < 32; ++k) o_acc[c4 * 32 + k] = fmaf(o_acc[c4 * 32 + k], alpha, v[k]);
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(kBarOFree + wg));
+                return true;
+            };
+
+            // this warpgroup's tiles of the unit: those whose block-wide index is congruent to wg mod 2
+            bool have_prev = false;
+            uint32_t prev_tt = 0;
+            for (uint32_t t = ((uint32_t)wg ^ tt0) & 1u; t < u.n_tiles; t += 2) {
+                const uint32_t tt = tt0 + t;
+                const uint32_t par = (tt >> 1) & 1u;
+                alive = warp_wait(bar(kBarSFull + wg), par);
+                if (!alive) break;
+                tc_fence_after();
+                // pass 1: the row's maximum over the tile
+                float mx = -INFINITY;
+#pragma unroll
+                for (int c4 = 0; c4 < 4; ++c4) {
+                    float v[32];
+                    tmem_ld32(s_addr + (uint32_t)c4 * 32u, v);
+#pragma unroll
+                    for (int k = 0; k < 32; ++k) mx = fmaxf(mx, v[k]);
+                }
+                const float m_new = fmaxf(m_run, mx * p.scale_log2);
+                const float alpha = fast_exp2(m_run - m_new);  // 0 on the first tile
+                m_run = m_new;
+                // pass 2: probabilities, as bf16, into the P buffer (free once this warpgroup's previous
+                // tile has been multiplied)
+                alive = warp_wait(bar(kBarPFree + wg), par ^ 1u);
+                if (!alive) break;
+                float psum = 0.f;
+#pragma unroll
+                for (int c4 = 0; c4 < 4; ++c4) {
+                    float v[32];
+                    tmem_ld32(s_addr + (uint32_t)c4 * 32u, v);
+#pragma unroll
+                    for (int k8 = 0; k8 < 4; ++k8) {  // 8 tokens = one 16-byte chunk
+                        uint32_t w[4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const float p0 = fast_exp2(fmaf(v[8 * k8 + 2 * j], p.scale_log2, -m_new));
+                            const float p1 = fast_exp2(fmaf(v[8 * k8 + 2 * j + 1], p.scale_log2, -m_new));
+                            psum += p0 + p1;
+                            w[j] = pack_bf16(p0, p1);
+                        }
+                        const uint32_t chunk = (uint32_t)((c4 & 1) * 4 + k8);
+                        const uint32_t a = prow + (uint32_t)(c4 >> 1) * kShBlock + ((chunk ^ swz) << 4);
+                        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(w[0]), "r"(w[1]), "r"(w[2]),
+                                     "r"(w[3])
+                                     : "memory");
+                    }
+                }
+                l_run = fmaf(l_run, alpha, psum);
+                tc_fence_before();
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(bar(kBarSFree + wg));
+                    mbar_arrive(bar(kBarPReady + wg));
+                }
+                // this warpgroup's previous tile has long been multiplied: fold its O in
+                if (have_prev) {
+                    alive = take_o(prev_tt, alpha_prev);
+                    if (!alive) break;
+                }
+                alpha_prev = alpha;
+                prev_tt = tt;
+                have_prev = true;
+            }
+            if (alive && have_prev) alive = take_o(prev_tt, alpha_prev);
+            tt0 += u.n_tiles;
+
+            // ---- combine the two warpgroups' states of each row (all products of the unit are complete
+            //      once both have taken their last O, so the P buffers can serve as scratch) -----------------
+            softmax_bar_both();
+            if (wg == 1) {
+#pragma unroll
+                for (int d = 0; d < 128; ++d) comb_o[d * 128 + row] = o_acc[d];
+                comb_ml[row] = m_run;
+                comb_ml[128 + row] = l_run;
+            }
+            softmax_bar_both();
+            if (wg == 0) {
+                const float m1 = comb_ml[row], l1 = comb_ml[128 + row];
+                const float M = fmaxf(m_run, m1);   // finite: the unit has at least one tile
+                const float w0 = fast_exp2(m_run - M), w1 = fast_exp2(m1 - M);
+                l_run = l_run * w0 + l1 * w1;
+                m_run = M;
+#pragma unroll
+                for (int d = 0; d < 128; ++d) o_acc[d] = o_acc[d] * w0 + comb_o[d * 128 + row] * w1;
+            }
+
+            // ---- epilogue: normalised fp32 partial of every valid row, then the arrival tickets ---------
+            if (wg == 0) {
+                if (alive && valid) {
+                    const uint32_t slot = p.reader_slot[(size_t)entry * p.n_kv_heads + u.kv_head] + u.chunk;
+                    const float inv = 1.f / l_run;
+                    float4 *dst = reinterpret_cast<float4 *>(p.part_o + ((size_t)slot * G + h) * kHeadDim);
+#pragma unroll
+                    for (int d = 0; d < 32; ++d)
+                        dst[d] = make_float4(o_acc[4 * d] * inv, o_acc[4 * d + 1] * inv, o_acc[4 * d + 2] * inv,
+                                             o_acc[4 * d + 3] * inv);
+                    p.part_lse2[(size_t)slot * kMaxGroup + h] = m_run + log2f(l_run);
+                    if (p.tickets) __threadfence();  // publish the partial before the ticket
+                }
+                softmax_bar();
+                // one thread decides for all whether the block is still in business, so that all softmax
+                // threads leave the unit loop together
+                if (tid == 0) *unit_ok = (*abort_flag == 0u) ? 1u : 0u;
+                if (p.tickets && tid < 128 / G) {
+                    uint32_t mine = 0;
+                    if (*abort_flag == 0u && (uint32_t)tid < u.n_readers) {
+                        // thread tid speaks for reader tid (rows tid * G .. tid * G + G - 1): the block that
+                        // delivers the last partial of the reader's row group merges it
+                        const uint32_t e2 = u.reader_begin + (uint32_t)tid;
+                        const uint32_t mg = p.reader_merge[(size_t)e2 * p.n_kv_heads + u.kv_head];
+                        const cart_merge_item mi = p.merges[mg];
+                        const uint32_t seen = atomicAdd(&p.tickets[mg], 1u);
+                        if (seen + 1u == mi.slot_end - mi.slot_begin) mine = mg + 1u;
+                    }
+                    flags[tid] = mine;
+                }
+                softmax_bar();
+                for (uint32_t r = 0; p.tickets && *unit_ok != 0u && r < u.n_readers; ++r) {
+                    const uint32_t f = flags[r];
+                    if (f == 0) continue;
+                    __threadfence();
+                    merge_row_group(p.merges[f - 1u], G, p.part_o, p.part_lse2, p.out, p.lse, tid, kSoftmaxThreads);
+                    if (tid == 0) p.tickets[f - 1u] = 0;  // ready for the next launch
+                }
+            }
+            softmax_bar_both();  // scratch, flags and unit_ok may be rewritten by the next unit from here on
+            alive = *unit_ok != 0u;
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
+}  // namespace
+
+cudaError_t prepare_shared_kernel()
+{
+    return cudaFuncSetAttribute(cart_shared_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kShSmemBytes);
+}
+
+cudaError_t launch_shared(const CUtensorMap &tmap, const SharedParams &p, int grid, cudaStream_t s)
+{
+    cart_shared_kernel<<<grid, kShThreads, kShSmemBytes, s>>>(tmap, p);
+    return cudaGetLastError();
+}
+
+}  // namespace cart
