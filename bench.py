@@ -152,7 +152,7 @@ def run_ours(args):
 
     # ---- device-resident timing ------------------------------------------------------------
     for _ in range(args.warmup):
-        lw.step(q, k_new, v_new, out, lse)
+        lw.step(q, k_new, v_new, out, lse, fused=not args.unfused)
     binding.cart_sync_status(ctx, stream)
     replicas.barrier(world)
     torch.cuda.synchronize(dev)
@@ -165,7 +165,7 @@ def run_ours(args):
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
     for _ in range(args.steps):
-        lw.step(q, k_new, v_new, out, lse)
+        lw.step(q, k_new, v_new, out, lse, fused=not args.unfused)
         bytes_layer_sum += lw.algorithmic_bytes_per_layer()
     e1.record(stream)
     torch.cuda.synchronize(dev)
@@ -208,8 +208,12 @@ def run_ours(args):
                 dq[layer].copy_(hq[layer], non_blocking=True)
                 dk[layer].copy_(hk[layer], non_blocking=True)
                 dv[layer].copy_(hv[layer], non_blocking=True)
-                binding.cart_append_kv(ctx, layer, lw.req_list, dk[layer], dv[layer], stream)
-                binding.cart_decode_attention(ctx, layer, lw.req_list, dq[layer], out[layer], lse[layer], stream)
+                if args.unfused:
+                    binding.cart_append_kv(ctx, layer, lw.req_list, dk[layer], dv[layer], stream)
+                    binding.cart_decode_attention(ctx, layer, lw.req_list, dq[layer], out[layer], lse[layer], stream)
+                else:
+                    binding.cart_decode_step(ctx, layer, lw.req_list, dk[layer], dv[layer], dq[layer], out[layer],
+                                             lse[layer], stream)
                 hout[layer].copy_(out[layer], non_blocking=True)
                 hlse[layer].copy_(lse[layer], non_blocking=True)
             lw.appended += 1
@@ -255,7 +259,8 @@ def run_ours(args):
                    "kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "cartridge_tokens": w.p,
                    "cartridges": w.cartridges, "suffix": "uniform[%d,%d]" % (w.suffix_lo, w.suffix_hi),
                    "mean_kv_tokens": round(float(kv_tokens.mean()), 1),
-                   "step": "per layer: append 1 KV token per request, then decode attention",
+                   "step": ("per layer: cart_append_kv, then cart_decode_attention" if args.unfused else
+                            "per layer: cart_decode_step (append 1 KV token per request and attend, one call)"),
                    "l2": "inputs larger than L2 (%.0f MB of KV per layer, %.1f GB per step)"
                          % (bytes_per_launch / 1e6, bytes_per_launch * L / 1e9),
                    "parallelism": "replicas only" if world > 1 else "single GPU",
@@ -333,6 +338,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--unfused", action="store_true",
+                    help="append and attend with two calls per layer instead of cart_decode_step")
     ap.add_argument("--no-kernel-events", action="store_true",
                     help="do not bracket each decode kernel with CUDA events (to see what the events cost)")
     ap.add_argument("--cpu-layers", type=int, default=4, help="layers the CPU oracle sample covers")

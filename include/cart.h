@@ -145,6 +145,18 @@ CART_API cart_status cart_decode_attention(cart_ctx *ctx, int32_t layer, const c
                                   int32_t n_reqs, const void *q /*device*/, void *out /*device*/,
                                   float *lse /*device or NULL*/, void *stream);
 
+/* Sec. 2.3, one decode step of a layer in one call: what cart_append_kv followed by
+ * cart_decode_attention computes, with the append done inside the attention kernel (the block that
+ * reads the last tile of a request's suffix first writes the new token's K and V rows there), so a
+ * step costs one kernel launch less per layer.  k_new / v_new: device bf16 [n_reqs][n_kv_heads][128];
+ * q, out, lse as in cart_decode_attention.  A handle may appear at most once in reqs.  On success every
+ * request's suffix in `layer` is one token longer and that token has been attended to (Eq. 1 sums
+ * over j <= i: the query sees its own position).
+ * Errors: those of cart_append_kv and cart_decode_attention; on an error nothing is appended. */
+CART_API cart_status cart_decode_step(cart_ctx *ctx, int32_t layer, const cart_req *reqs /*host*/, int32_t n_reqs,
+                             const void *k_new /*device*/, const void *v_new /*device*/, const void *q /*device*/,
+                             void *out /*device*/, float *lse /*device or NULL*/, void *stream);
+
 /* Sharing policy.  When at least min_readers requests of a decode batch attend to the same stored
  * Cartridge (one Cartridge serving many users, Sec. 1 and Sec. 3.3; pool members composed by many
  * requests, Sec. 5.4), cart_decode_attention reads each of its K/V tiles once for up to 128 query

@@ -37,6 +37,8 @@ typedef struct {
 #define CART_ITEM_BEGIN 1u  /* first item of a row-group piece in this block: load q, reset state */
 #define CART_ITEM_END 2u    /* last item of the piece: combine the warps' states and write */
 #define CART_ITEM_DIRECT 4u /* the piece is the whole row group: write out / lse, not a partial */
+#define CART_ITEM_TAIL 8u   /* the item ends with the last token of the request's cache (the token a fused
+                               append + decode call writes before it attends) */
 
 /* A run of consecutive tiles of one segment of one row group, processed by one block. */
 typedef struct {

@@ -568,10 +568,15 @@ cart_status cart_extend_kv(cart_ctx *ctx, int32_t layer, cart_req req, const voi
     return CART_OK;
 }
 
-cart_status cart_decode_attention(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int32_t n_reqs, const void *q,
-                                  void *out, float *lse, void *stream)
+}  // extern "C"
+
+namespace {
+
+// Decode attention for a batch; with k_new / v_new non-null the stream kernel first writes each
+// request's new token at position len - 1 of its suffix (the host lengths already count it).
+cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int32_t n_reqs, const void *q,
+                        void *out, float *lse, const void *k_new, const void *v_new, void *stream)
 {
-    if (!ctx) return CART_ERR_INVALID_ARG;
     if (!reqs || n_reqs < 1 || !aligned16(q) || !aligned16(out) || (lse && (reinterpret_cast<uintptr_t>(lse) & 3u)))
         return fail(ctx, CART_ERR_INVALID_ARG, "decode: null/misaligned pointer or empty batch");
     if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, CART_ERR_BAD_HANDLE, "decode: layer out of range");
@@ -685,6 +690,9 @@ cart_status cart_decode_attention(cart_ctx *ctx, int32_t layer, const cart_req *
     dp.cta_begin = reinterpret_cast<const uint32_t *>(sl->dev + ctx->lay.cta_begin_off);
     dp.items = reinterpret_cast<const cart_work_item *>(sl->dev + ctx->lay.items_off);
     dp.q = q;
+    dp.k_new = k_new;
+    dp.v_new = v_new;
+    dp.arena = ctx->cfg.arena;
     dp.out = out;
     dp.lse = lse;
     dp.part_o = reinterpret_cast<float *>(arena + ctx->lay.part_o_off);
@@ -750,6 +758,42 @@ cart_status cart_decode_attention(cart_ctx *ctx, int32_t layer, const cart_req *
         ctx->ev_used += 2;
     }
     return CART_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+cart_status cart_decode_attention(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int32_t n_reqs, const void *q,
+                                  void *out, float *lse, void *stream)
+{
+    if (!ctx) return CART_ERR_INVALID_ARG;
+    return decode_impl(ctx, layer, reqs, n_reqs, q, out, lse, nullptr, nullptr, stream);
+}
+
+cart_status cart_decode_step(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int32_t n_reqs, const void *k_new,
+                             const void *v_new, const void *q, void *out, float *lse, void *stream)
+{
+    if (!ctx) return CART_ERR_INVALID_ARG;
+    if (!reqs || n_reqs < 1 || !aligned16(k_new) || !aligned16(v_new))
+        return fail(ctx, CART_ERR_INVALID_ARG, "decode_step: null/misaligned pointer or empty batch");
+    if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, CART_ERR_BAD_HANDLE, "decode_step: layer out of range");
+    const uint64_t stamp = ++ctx->stamp;
+    for (int32_t i = 0; i < n_reqs; ++i) {
+        Request *r = get_req(ctx, reqs[i]);
+        if (!r) return fail(ctx, CART_ERR_BAD_HANDLE, "decode_step: reqs[%d] is not an open request", i);
+        if (r->stamp == stamp) return fail(ctx, CART_ERR_INVALID_ARG, "decode_step: reqs[%d] appears twice", i);
+        r->stamp = stamp;
+        if (r->len[(size_t)layer] >= r->cap)
+            return fail(ctx, CART_ERR_CAPACITY, "decode_step: suffix of reqs[%d] is full (%d tokens)", i, r->cap);
+    }
+    // The plan must see the new token: count it first, take it back if nothing was launched.
+    for (int32_t i = 0; i < n_reqs; ++i) ++ctx->reqs[(size_t)reqs[i]].len[(size_t)layer];
+    const uint64_t launches_before = ctx->launches;
+    const cart_status st = decode_impl(ctx, layer, reqs, n_reqs, q, out, lse, k_new, v_new, stream);
+    if (st != CART_OK && ctx->launches == launches_before)
+        for (int32_t i = 0; i < n_reqs; ++i) --ctx->reqs[(size_t)reqs[i]].len[(size_t)layer];
+    return st;
 }
 
 cart_status cart_suffix_len(cart_ctx *ctx, cart_req req, int32_t layer, int32_t *out_len)

@@ -26,6 +26,9 @@ struct DecodeParams {
     const uint32_t *cta_begin;   // [grid + 1]
     const cart_work_item *items;
     const void *q;               // bf16 [n_reqs][Hq][128]
+    const void *k_new = nullptr; // fused append: bf16 [n_reqs][Hkv][128] written to the suffix ends; else null
+    const void *v_new = nullptr;
+    void *arena = nullptr;                 // base of the row heap (row r is at arena + 256 r)
     void *out;                   // bf16 [n_reqs][Hq][128]
     float *lse;                  // fp32 [n_reqs][Hq] or null
     float *part_o;               // fp32 [slot][G][128], normalised partial outputs

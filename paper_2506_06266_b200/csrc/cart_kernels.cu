@@ -212,21 +212,36 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeParams 
     const uint32_t item_end = p.cta_begin[blockIdx.x + 1];
 
     if (warp == kConsumerWarps) {
-        // ================= producer: one thread feeds the ring ====================================
-        if (lane == 0) {
-            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap)) : "memory");
-            uint32_t t = 0;  // tiles issued by this block so far
-            bool ok = true;
-            for (uint32_t it = item_begin; it < item_end && ok; ++it) {
-                const cart_work_item w = p.items[it];
-                const uint32_t k_row = w.k_row + (uint32_t)p.layer * w.layer_stride;
-                const uint32_t v_row = w.v_row + (uint32_t)p.layer * w.layer_stride;
-                const uint32_t ntiles = (w.n_tok + kTileTokens - 1) / kTileTokens;
-                for (uint32_t j = 0; j < ntiles; ++j, ++t) {
-                    const int s = (int)(t % kStages);
-                    const uint32_t round = t / kStages;
-                    ok = mbar_wait(empty(s), (round & 1u) ^ 1u, abort_flag, p.status, kStatusTimeoutProducer);
-                    if (!ok) break;
+        // ================= producer: the warp walks the items together, lane 0 feeds the ring =========
+        if (lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap)) : "memory");
+        uint32_t t = 0;  // tiles issued by this block so far
+        bool ok = true;
+        for (uint32_t it = item_begin; it < item_end && ok; ++it) {
+            const cart_work_item w = p.items[it];
+            const uint32_t k_row = w.k_row + (uint32_t)p.layer * w.layer_stride;
+            const uint32_t v_row = w.v_row + (uint32_t)p.layer * w.layer_stride;
+            const uint32_t ntiles = (w.n_tok + kTileTokens - 1) / kTileTokens;
+            for (uint32_t j = 0; j < ntiles; ++j, ++t) {
+                const int s = (int)(t % kStages);
+                const uint32_t round = t / kStages;
+                bool ok0 = true;
+                if (lane == 0) ok0 = mbar_wait(empty(s), (round & 1u) ^ 1u, abort_flag, p.status, kStatusTimeoutProducer);
+                ok = __shfl_sync(0xffffffffu, (int)ok0, 0) != 0;
+                if (!ok) break;
+                if (p.k_new != nullptr && (w.flags & CART_ITEM_TAIL) && j + 1 == ntiles) {
+                    // Fused append (decode phase of Sec. 2.3): this tile ends with the request's new token.
+                    // Write its K row (lanes 0-15) and V row (lanes 16-31) into the suffix before the tile
+                    // is fetched; no other block reads these rows in this launch.
+                    const uint32_t c = (uint32_t)lane & 15u;
+                    const uint4 *src = reinterpret_cast<const uint4 *>(lane < 16 ? p.k_new : p.v_new) +
+                                       (size_t)w.row_group * 16 + c;
+                    const size_t dst_row = (size_t)(lane < 16 ? k_row : v_row) + (w.n_tok - 1);
+                    reinterpret_cast<uint4 *>(p.arena)[dst_row * 16 + c] = __ldg(src);
+                    __threadfence();
+                    asm volatile("fence.proxy.async;" ::: "memory");  // generic-proxy stores before the TMA read
+                    __syncwarp();
+                }
+                if (lane == 0) {
                     const uint32_t kdst = stages + (uint32_t)s * kStageBytes;
                     const uint32_t vdst = kdst + kTileBytes;
                     const int32_t yk = (int32_t)(k_row + j * kTileTokens);
@@ -239,17 +254,17 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeParams 
                     tma_load_2d(vdst + kHalfBytes, &tmap, 64, yv, full_v(s));
                 }
             }
-            if (!ok) {
-                // Gave up: no new copies are issued; wait (bounded) for those still in flight so that
-                // none lands in shared memory after the block has gone.
-                const uint32_t issued = t;
-                for (uint32_t u = (issued > (uint32_t)kStages ? issued - kStages : 0u); u < issued; ++u) {
-                    const int s = (int)(u % kStages);
-                    const uint32_t par = (u / kStages) & 1u;
-                    const uint64_t t0 = global_timer_ns();
-                    while (!mbar_try_wait(full_k(s), par) && global_timer_ns() - t0 < kWaitLimitNs) {}
-                    while (!mbar_try_wait(full_v(s), par) && global_timer_ns() - t0 < kWaitLimitNs) {}
-                }
+        }
+        if (!ok && lane == 0) {
+            // Gave up: no new copies are issued; wait (bounded) for those still in flight so that
+            // none lands in shared memory after the block has gone.
+            const uint32_t issued = t;
+            for (uint32_t u = (issued > (uint32_t)kStages ? issued - kStages : 0u); u < issued; ++u) {
+                const int s = (int)(u % kStages);
+                const uint32_t par = (u / kStages) & 1u;
+                const uint64_t t0 = global_timer_ns();
+                while (!mbar_try_wait(full_k(s), par) && global_timer_ns() - t0 < kWaitLimitNs) {}
+                while (!mbar_try_wait(full_v(s), par) && global_timer_ns() - t0 < kWaitLimitNs) {}
             }
         }
         return;

@@ -279,6 +279,7 @@ extern "C" cart_status cart_plan_build_shared(const cart_plan_seg *segs, const i
                     it.n_tok = (uint32_t)(tok1 - tok0);
                     it.row_group = rg;
                     it.flags = first ? CART_ITEM_BEGIN : 0u;
+                    if (s == s1 - 1 && tok1 == seg_ntok) it.flags |= CART_ITEM_TAIL;
                     it.slot = 0;
                     it.merge = 0;
                     first = false;

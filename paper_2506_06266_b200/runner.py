@@ -107,14 +107,18 @@ class LoadedWorkload:
         return kv + io
 
     def step(self, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor, out: torch.Tensor,
-             lse: Optional[torch.Tensor], layers: Optional[Iterable[int]] = None) -> None:
-        """One decode step: per layer, append every request's new token, then attend.
+             lse: Optional[torch.Tensor], layers: Optional[Iterable[int]] = None, fused: bool = True) -> None:
+        """One decode step: per layer, append every request's new token, then attend -- in one call
+        (cart_decode_step) or, with fused=False, as cart_append_kv followed by cart_decode_attention.
         q, out: [L][B][Hq][D]; k_new, v_new: [L][B][Hkv][D]; lse: [L][B][Hq] or None."""
         ctx, rl, s = self.ctx, self.req_list, self.stream
         for layer in (range(self.w.n_layers) if layers is None else layers):
-            binding.cart_append_kv(ctx, layer, rl, k_new[layer], v_new[layer], s)
-            binding.cart_decode_attention(ctx, layer, rl, q[layer], out[layer],
-                                          None if lse is None else lse[layer], s)
+            ls = None if lse is None else lse[layer]
+            if fused:
+                binding.cart_decode_step(ctx, layer, rl, k_new[layer], v_new[layer], q[layer], out[layer], ls, s)
+            else:
+                binding.cart_append_kv(ctx, layer, rl, k_new[layer], v_new[layer], s)
+                binding.cart_decode_attention(ctx, layer, rl, q[layer], out[layer], ls, s)
         self.appended += 1
 
     def close(self) -> None:

@@ -120,6 +120,18 @@ class Session:
         binding.cart_sync_status(self.ctx)
         return out, lse
 
+    def decode_step(self, layer: int, reqs: Sequence[int], k_new: torch.Tensor, v_new: torch.Tensor,
+                    q: torch.Tensor):
+        """Fused append + decode on the GPU; the oracle's bookkeeping gets the same append."""
+        k_new, v_new, q = k_new.to(self.dev).contiguous(), v_new.to(self.dev).contiguous(), q.to(self.dev).contiguous()
+        out = torch.full_like(q, float("nan"))
+        lse = torch.full(q.shape[:2], float("nan"), dtype=torch.float32, device=self.dev)
+        binding.cart_decode_step(self.ctx, layer, reqs, k_new, v_new, q, out, lse)
+        binding.cart_sync_status(self.ctx)
+        if self.oc is not None:
+            self.oc.append(layer, [self.req_map[r] for r in reqs], synth.bits(k_new), synth.bits(v_new))
+        return out, lse
+
     def oracle_decode(self, layer: int, reqs: Sequence[int], q: torch.Tensor):
         return self.oc.decode(layer, [self.req_map[r] for r in reqs], synth.bits(q))
 

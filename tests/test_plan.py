@@ -6,6 +6,7 @@ import pytest
 from paper_2506_06266_b200 import binding, buildlib, synth
 
 B_, E_, D_ = binding.CART_ITEM_BEGIN, binding.CART_ITEM_END, binding.CART_ITEM_DIRECT
+T_ = binding.CART_ITEM_TAIL
 
 
 @pytest.fixture(scope="module", autouse=True)
@@ -87,6 +88,10 @@ def check_plan(segs, Hkv, n_cta, tile):
                     got += nt
                     pos += 1
             assert pos == len(runs)
+            # exactly one item carries the tail mark: the one that ends with the cache's last token
+            (k, v, hs, ls, n) = r[-1]
+            tails = [it for it in items if it.row_group == rg and it.flags & T_]
+            assert len(tails) == 1 and tails[0].k_row + tails[0].n_tok == k + g * hs + n
             ps = pieces[rg]
             if len(ps) == 1 and ps[0][0]:
                 assert rg not in merges
