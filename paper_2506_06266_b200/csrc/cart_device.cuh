@@ -78,6 +78,18 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tma
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(bar)
         : "memory");
 }
+// Programmatic dependent launch.  The decode kernels are launched so that the next kernel on the
+// stream may become resident while this one drains: every block says at once that dependents may be
+// scheduled, and a dependent thread waits for the full completion (and memory visibility) of the
+// kernels before it only when it first needs what they may have written.
+__device__ __forceinline__ void pdl_launch_dependents()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void pdl_wait()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
 __device__ __forceinline__ float fast_exp2(float x)
 {
     float y;

@@ -99,6 +99,23 @@ struct ExtendParams {
     int32_t n_kv_heads;
 };
 
+// Launch configuration shared by the decode kernels: the kernel may start (become resident, run its
+// prologue) before the kernel before it on the stream has finished; it orders itself with
+// griddepcontrol.wait.
+inline cudaLaunchConfig_t pdl_config(int grid, int block, size_t smem, cudaStream_t s, cudaLaunchAttribute *attr)
+{
+    attr->id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr->val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t c{};
+    c.gridDim = dim3((unsigned)grid);
+    c.blockDim = dim3((unsigned)block);
+    c.dynamicSmemBytes = smem;
+    c.stream = s;
+    c.attrs = attr;
+    c.numAttrs = 1;
+    return c;
+}
+
 // Launchers (defined in cart_kernels.cu).  Each returns the cudaError_t of the launch.
 size_t decode_smem_bytes();
 int decode_threads();

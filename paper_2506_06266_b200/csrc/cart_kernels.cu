@@ -196,6 +196,7 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeParams 
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+    pdl_launch_dependents();
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -216,6 +217,11 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeParams 
         if (lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap)) : "memory");
         uint32_t t = 0;  // tiles issued by this block so far
         bool ok = true;
+        // Until the kernels before this one on the stream are known to be complete, only tiles that
+        // they cannot have written are fetched: a fused append writes a request's last token, which
+        // lies in the last tile of an item marked CART_ITEM_TAIL.  Everything else in the arena is
+        // written by copies or by kernels that complete before this one may start.
+        bool waited = false;
         for (uint32_t it = item_begin; it < item_end && ok; ++it) {
             const cart_work_item w = p.items[it];
             const uint32_t k_row = w.k_row + (uint32_t)p.layer * w.layer_stride;
@@ -228,6 +234,10 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeParams 
                 if (lane == 0) ok0 = mbar_wait(empty(s), (round & 1u) ^ 1u, abort_flag, p.status, kStatusTimeoutProducer);
                 ok = __shfl_sync(0xffffffffu, (int)ok0, 0) != 0;
                 if (!ok) break;
+                if (!waited && (w.flags & CART_ITEM_TAIL) && j + 1 == ntiles) {
+                    pdl_wait();
+                    waited = true;
+                }
                 if (p.k_new != nullptr && (w.flags & CART_ITEM_TAIL) && j + 1 == ntiles) {
                     // Fused append (decode phase of Sec. 2.3): this tile ends with the request's new token.
                     // Write its K row (lanes 0-15) and V row (lanes 16-31) into the suffix before the tile
@@ -271,6 +281,7 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeParams 
     }
 
     // ===================== consumers ==============================================================
+    pdl_wait();  // q, the partial slots and the tickets belong to the kernels before until they are done
     const int G = p.group;
     const int row = lane >> 2;  // query head inside the group that this thread's c0/c1 belong to
     const __nv_bfloat16 *q = reinterpret_cast<const __nv_bfloat16 *>(p.q);
@@ -398,6 +409,8 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeParams 
 // shared Cartridge is one).
 __global__ void __launch_bounds__(128) cart_merge_kernel(const MergeParams p)
 {
+    pdl_launch_dependents();
+    pdl_wait();  // the partials come from the kernels before
     merge_row_group(p.merges[blockIdx.x], p.group, p.part_o, p.part_lse2, p.out, p.lse, (int)threadIdx.x, 128);
 }
 
@@ -450,14 +463,16 @@ cudaError_t prepare_kernels()
 
 cudaError_t launch_decode(const CUtensorMap &tmap, const DecodeParams &p, int grid, cudaStream_t s)
 {
-    cart_decode_kernel<<<grid, kThreads, kSmemBytes, s>>>(tmap, p);
-    return cudaGetLastError();
+    cudaLaunchAttribute attr;
+    const cudaLaunchConfig_t cfg = pdl_config(grid, kThreads, kSmemBytes, s, &attr);
+    return cudaLaunchKernelEx(&cfg, cart_decode_kernel, tmap, p);
 }
 
 cudaError_t launch_merge(const MergeParams &p, int n_merges, cudaStream_t s)
 {
-    cart_merge_kernel<<<n_merges, 128, 0, s>>>(p);
-    return cudaGetLastError();
+    cudaLaunchAttribute attr;
+    const cudaLaunchConfig_t cfg = pdl_config(n_merges, 128, 0, s, &attr);
+    return cudaLaunchKernelEx(&cfg, cart_merge_kernel, p);
 }
 
 cudaError_t launch_append(const AppendParams &p, cudaStream_t s)

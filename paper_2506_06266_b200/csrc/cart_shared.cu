@@ -153,6 +153,7 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+    pdl_launch_dependents();
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < 2; ++i) {
@@ -184,6 +185,9 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
+    // Shared tiles are whole tiles of stored Cartridges, which no kernel writes; the queries, the
+    // partial slots and the tickets may still be in use by the kernels before this one.
+    if (warp >= 4) pdl_wait();
     const uint32_t unit_begin = p.unit_cta_begin[blockIdx.x];
     const uint32_t unit_end = p.unit_cta_begin[blockIdx.x + 1];
 
@@ -523,8 +527,9 @@ cudaError_t prepare_shared_kernel()
 
 cudaError_t launch_shared(const CUtensorMap &tmap, const SharedParams &p, int grid, cudaStream_t s)
 {
-    cart_shared_kernel<<<grid, kShThreads, kShSmemBytes, s>>>(tmap, p);
-    return cudaGetLastError();
+    cudaLaunchAttribute attr;
+    const cudaLaunchConfig_t cfg = pdl_config(grid, kShThreads, kShSmemBytes, s, &attr);
+    return cudaLaunchKernelEx(&cfg, cart_shared_kernel, tmap, p);
 }
 
 }  // namespace cart
