@@ -40,7 +40,7 @@ WORKLOADS = {
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the decode kernel, from the ncu capture
 # summarised under profiles/ (a smaller case of the same kernel, scaled by KV bytes); None = not captured.
-NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = {"c2": 622.56 / 608.27}   # profiles/decode_kernel_c2.md
+NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = {"c2": 622.38 / 608.27}   # profiles/decode_kernel_c2.md
 
 
 def measured_peak_gbs():
@@ -207,31 +207,57 @@ def run_ours(args):
         hk, hv = k_new.cpu().pin_memory(), v_new.cpu().pin_memory()
         hout = torch.empty(out.shape, dtype=out.dtype).pin_memory()
         hlse = torch.empty(lse.shape, dtype=lse.dtype).pin_memory()
-        dq, dk, dv = torch.empty_like(q), torch.empty_like(k_new), torch.empty_like(v_new)
+        # Double-buffered, as a server would run it: the inputs of step i+1 cross PCIe on a copy stream
+        # while step i computes, and the result of step i goes back while step i+1 computes.  Every
+        # step's host-to-device and device-to-host copies are inside the timed region.
+        cs_in, cs_out = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+        dq = [torch.empty_like(q) for _ in range(2)]
+        dk = [torch.empty_like(k_new) for _ in range(2)]
+        dv = [torch.empty_like(v_new) for _ in range(2)]
+        dout = [torch.empty_like(out) for _ in range(2)]
+        dlse = [torch.empty_like(lse) for _ in range(2)]
+        ev_in = [torch.cuda.Event() for _ in range(2)]
+        ev_done = [torch.cuda.Event() for _ in range(2)]
+        ev_out = [torch.cuda.Event() for _ in range(2)]
 
-        def e2e_step():
-            for layer in range(L):
-                dq[layer].copy_(hq[layer], non_blocking=True)
-                dk[layer].copy_(hk[layer], non_blocking=True)
-                dv[layer].copy_(hv[layer], non_blocking=True)
-                if args.unfused:
-                    binding.cart_append_kv(ctx, layer, lw.req_list, dk[layer], dv[layer], stream)
-                    binding.cart_decode_attention(ctx, layer, lw.req_list, dq[layer], out[layer], lse[layer], stream)
-                else:
-                    binding.cart_decode_step(ctx, layer, lw.req_list, dk[layer], dv[layer], dq[layer], out[layer],
-                                             lse[layer], stream)
-                hout[layer].copy_(out[layer], non_blocking=True)
-                hlse[layer].copy_(lse[layer], non_blocking=True)
-            lw.appended += 1
+        def e2e_steps(n, start_ev):
+            for i in range(n):
+                b = i & 1
+                with torch.cuda.stream(cs_in):
+                    cs_in.wait_event(ev_done[b] if i >= 2 else start_ev)   # step i-2 has consumed buffer b
+                    dq[b].copy_(hq, non_blocking=True)
+                    dk[b].copy_(hk, non_blocking=True)
+                    dv[b].copy_(hv, non_blocking=True)
+                    ev_in[b].record(cs_in)
+                stream.wait_event(ev_in[b])
+                if i >= 2:
+                    stream.wait_event(ev_out[b])                           # step i-2's result has left buffer b
+                for layer in range(L):
+                    if args.unfused:
+                        binding.cart_append_kv(ctx, layer, lw.req_list, dk[b][layer], dv[b][layer], stream)
+                        binding.cart_decode_attention(ctx, layer, lw.req_list, dq[b][layer], dout[b][layer],
+                                                      dlse[b][layer], stream)
+                    else:
+                        binding.cart_decode_step(ctx, layer, lw.req_list, dk[b][layer], dv[b][layer], dq[b][layer],
+                                                 dout[b][layer], dlse[b][layer], stream)
+                ev_done[b].record(stream)
+                with torch.cuda.stream(cs_out):
+                    cs_out.wait_event(ev_done[b])
+                    hout.copy_(dout[b], non_blocking=True)
+                    hlse.copy_(dlse[b], non_blocking=True)
+                    ev_out[b].record(cs_out)
+                lw.appended += 1
+            for b in range(min(n, 2)):
+                stream.wait_event(ev_out[b])                               # the region ends when the results are home
 
-        for _ in range(args.warmup):
-            e2e_step()
+        w0 = torch.cuda.Event()
+        w0.record(stream)
+        e2e_steps(args.warmup, w0)
         torch.cuda.synchronize(dev)
         replicas.barrier(world)
         f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         f0.record(stream)
-        for _ in range(args.e2e_steps):
-            e2e_step()
+        e2e_steps(args.e2e_steps, f0)
         f1.record(stream)
         torch.cuda.synchronize(dev)
         replicas.barrier(world)
@@ -240,6 +266,7 @@ def run_ours(args):
         d2h = L * (hout[0].numel() * 2 + hlse[0].numel() * 4)
         e2e = {"value": round(e2e_value, 1), "unit": UNIT,
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": args.e2e_steps,
+               "pipeline": "double-buffered: copies of neighbouring steps overlap the kernels on two copy streams",
                "ms_per_step": round(ems / args.e2e_steps, 4)}
         binding.cart_sync_status(ctx, stream)
 
@@ -336,12 +363,12 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2", choices=sorted(WORKLOADS))
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling small cases)")
-    ap.add_argument("--e2e-steps", type=int, default=10)
+    ap.add_argument("--e2e-steps", type=int, default=50)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--unfused", action="store_true",
