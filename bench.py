@@ -143,6 +143,8 @@ def run_ours(args):
     stream = torch.cuda.current_stream(dev)
     lw = runner.LoadedWorkload(w, dev, extra_capacity=total_steps, keep_layers=sample_layers, stream=stream)
     ctx = lw.ctx
+    if args.piece_cost >= 0:
+        binding.cart_set_piece_cost(ctx, args.piece_cost)
 
     q = w.queries(0, dev)
     k_new, v_new = w.appended_kv(0, dev)
@@ -373,6 +375,8 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--unfused", action="store_true",
                     help="append and attend with two calls per layer instead of cart_decode_step")
+    ap.add_argument("--piece-cost", type=int, default=-1,
+                    help="planner tuning (cart_set_piece_cost); -1 keeps the library's default")
     ap.add_argument("--kernel-events", action="store_true",
                     help="bracket every decode call's kernels with a pair of CUDA events and report their mean "
                          "duration; the events sit between the kernels, so a kernel can then no longer start "

@@ -165,6 +165,13 @@ CART_API cart_status cart_decode_step(cart_ctx *ctx, int32_t layer, const cart_r
  * request streams its whole cache).  Errors: INVALID_ARG. */
 CART_API cart_status cart_set_share_min_readers(cart_ctx *ctx, int32_t min_readers);
 
+/* Planner tuning.  The stream kernel's blocks are given equal shares of tiles + tiles_per_piece * pieces,
+ * a piece being the part of a (request, KV head) cache that one block handles; the constant stands
+ * for what finishing a piece (combining the warps' states, writing the result) costs a block, in
+ * units of the time a 64-token tile takes.  Default 3; 0 balances by tiles alone; at most 64.  The
+ * results do not depend on it beyond fp32 rounding.  Errors: INVALID_ARG. */
+CART_API cart_status cart_set_piece_cost(cart_ctx *ctx, int32_t tiles_per_piece);
+
 /* Current suffix length of a request in a layer (host-side mirror). */
 CART_API cart_status cart_suffix_len(cart_ctx *ctx, cart_req req, int32_t layer, int32_t *out_len /*host*/);
 

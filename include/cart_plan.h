@@ -121,6 +121,8 @@ typedef struct {
     int32_t slots_cap;         /* partial slots available */
     int32_t n_slots;           /* partial slots used (shared + stream) */
     int64_t total_tiles;       /* stream tiles */
+    int32_t piece_cost;        /* in: what starting a row-group piece costs a block, in tile times; the stream
+                                  blocks are balanced by tiles + piece_cost * pieces (0: by tiles alone) */
     /* shared part */
     cart_shared_unit *units;   int32_t units_cap;    int32_t n_units;
     uint32_t *unit_cta_begin;  /* [n_cta + 1]: block c of the shared kernel owns units[unit_cta_begin[c] ..] */

@@ -29,7 +29,7 @@ EXPORTS = ["cart_scratch_bytes", "cart_create", "cart_destroy", "cart_register_c
            "cart_compose", "cart_release_cartridge", "cart_request_open", "cart_request_close",
            "cart_append_kv", "cart_extend_kv", "cart_decode_attention", "cart_decode_step", "cart_suffix_len",
            "cart_kv_bytes", "cart_sync_status", "cart_set_timing", "cart_get_timing",
-           "cart_set_share_min_readers", "cart_plan_build_shared",
+           "cart_set_share_min_readers", "cart_set_piece_cost", "cart_plan_build_shared",
            "cart_decode_attention_static", "cart_launch_count", "cart_status_string",
            "cart_last_error", "cart_plan_build"]
 
@@ -74,7 +74,7 @@ class cart_plan_out(ctypes.Structure):
                 ("merges", ctypes.POINTER(cart_merge_item)), ("merges_cap", ctypes.c_int32),
                 ("n_merges", ctypes.c_int32),
                 ("n_cta_used", ctypes.c_int32), ("slots_cap", ctypes.c_int32), ("n_slots", ctypes.c_int32),
-                ("total_tiles", ctypes.c_int64),
+                ("total_tiles", ctypes.c_int64), ("piece_cost", ctypes.c_int32),
                 ("units", ctypes.POINTER(cart_shared_unit)), ("units_cap", ctypes.c_int32),
                 ("n_units", ctypes.c_int32),
                 ("unit_cta_begin", ctypes.POINTER(ctypes.c_uint32)), ("n_unit_cta_used", ctypes.c_int32),
@@ -127,6 +127,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.cart_sync_status.argtypes = [vp, vp]
     lib.cart_set_timing.argtypes = [vp, i32]
     lib.cart_set_share_min_readers.argtypes = [vp, i32]
+    lib.cart_set_piece_cost.argtypes = [vp, i32]
     lib.cart_get_timing.argtypes = [vp, ctypes.POINTER(ctypes.c_double), u64p]
     lib.cart_decode_attention_static.argtypes = [vp, vp, i32, i32, i32, i32, ctypes.c_float, vp, vp, i32, vp]
     lib.cart_launch_count.argtypes = [vp]
@@ -291,6 +292,10 @@ def cart_set_share_min_readers(ctx: int, min_readers: int) -> None:
     _check(load_library().cart_set_share_min_readers(ctx, int(min_readers)), "cart_set_share_min_readers", ctx)
 
 
+def cart_set_piece_cost(ctx: int, tiles_per_piece: int) -> None:
+    _check(load_library().cart_set_piece_cost(ctx, int(tiles_per_piece)), "cart_set_piece_cost", ctx)
+
+
 def cart_get_timing(ctx: int) -> Tuple[float, int]:
     ms, n = ctypes.c_double(0.0), ctypes.c_uint64(0)
     _check(load_library().cart_get_timing(ctx, ctypes.byref(ms), ctypes.byref(n)), "cart_get_timing", ctx)
@@ -342,7 +347,7 @@ def cart_plan_build(segs: Sequence[Sequence[Tuple[int, int, int, int, int]]], n_
 
 def cart_plan_build_shared(segs: Sequence[Sequence[Tuple[int, int, int, int, int]]], n_kv_heads: int, group: int,
                            n_cta: int, tile_tokens: int, share_min_readers: int, share_tile_tokens: int,
-                           slots_cap: int = 1 << 20):
+                           slots_cap: int = 1 << 20, piece_cost: int = 0):
     """Host-only planner with shared segments (see include/cart_plan.h).  Returns a dict with the
     stream plan (items, cta_begin, merges, ...) and the shared part (units, unit_cta_begin, readers,
     reader_slot[entry][head], reader_merge[entry][head])."""
@@ -369,6 +374,7 @@ def cart_plan_build_shared(segs: Sequence[Sequence[Tuple[int, int, int, int, int
     reader_merge = (ctypes.c_uint32 * (readers_cap * n_kv_heads))()
     o.items, o.items_cap, o.cta_begin = items, items_cap, cta_begin
     o.merges, o.merges_cap, o.slots_cap = merges, merges_cap, slots_cap
+    o.piece_cost = piece_cost
     o.units, o.units_cap, o.unit_cta_begin = units, units_cap, unit_cta_begin
     o.readers, o.readers_cap, o.reader_slot, o.reader_merge = readers, readers_cap, reader_slot, reader_merge
     st = lib.cart_plan_build_shared(seg_arr, sb, len(segs), n_kv_heads, group, n_cta, tile_tokens,

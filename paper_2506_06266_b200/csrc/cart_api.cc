@@ -26,6 +26,8 @@ uint64_t round_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
 // A Cartridge is handed to the shared-segment kernel when at least this many requests of the batch
 // hold it (and it has at least one full 128-token tile); below that its readers stream it one by one.
 constexpr int kShareMinReaders = 4;
+// What the planner charges a stream block for starting a row-group piece, in 64-token tile times.
+constexpr int kPieceCostTiles = 3;
 
 struct ScratchLayout {
     uint64_t status_off, tickets_off, plan_off, plan_slot_bytes, cta_begin_off, merges_off, items_off;
@@ -125,6 +127,7 @@ struct cart_ctx {
     float scale = 0.f;
     int n_cta = 0;
     int share_min_readers = kShareMinReaders;
+    int piece_cost = kPieceCostTiles;
     uint64_t n_rows = 0;
     alignas(64) CUtensorMap tmap;
     std::vector<FreeBlock> free_list;
@@ -352,6 +355,15 @@ cart_status cart_set_share_min_readers(cart_ctx *ctx, int32_t min_readers)
     if (min_readers < 0) return fail(ctx, CART_ERR_INVALID_ARG, "share_min_readers: negative");
     ctx->share_min_readers = min_readers;
     ++ctx->epoch;  // cached plans were built under the old policy
+    return CART_OK;
+}
+
+cart_status cart_set_piece_cost(cart_ctx *ctx, int32_t tiles)
+{
+    if (!ctx) return CART_ERR_INVALID_ARG;
+    if (tiles < 0 || tiles > 64) return fail(ctx, CART_ERR_INVALID_ARG, "piece_cost: out of range");
+    ctx->piece_cost = tiles;
+    ++ctx->epoch;
     return CART_OK;
 }
 
@@ -654,6 +666,7 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
         po.merges = reinterpret_cast<cart_merge_item *>(ns.host + lay.merges_off);
         po.merges_cap = lay.merges_cap;
         po.slots_cap = lay.slots_cap;
+        po.piece_cost = ctx->piece_cost;
         po.units = reinterpret_cast<cart_shared_unit *>(ns.host + lay.units_off);
         po.units_cap = lay.units_cap;
         po.unit_cta_begin = reinterpret_cast<uint32_t *>(ns.host + lay.unit_cta_begin_off);

@@ -104,29 +104,76 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 // Log-sum-exp merge of the partials of one split row group (softmax over a union of token sets is
 // the lse-weighted mix of the softmaxes over the sets, from Eq. 1): slots mi.slot_begin .. slot_end-1
 // hold normalised fp32 outputs [slot][G][128] and base-2 lse values [slot][kMaxGroup].  Called by
-// `nthreads` threads of one block with tid = 0 .. nthreads-1; the caller has fenced.
+// `nthreads` threads of one block with tid = 0 .. nthreads-1; the caller has fenced.  An item is one
+// query row times four output dims; a thread works on up to four items at once and on two slots at
+// a time, so that a lone warp has 8 independent 16-byte loads in flight.
 __device__ __forceinline__ void merge_row_group(const cart_merge_item mi, int G, const float *part_o,
                                                 const float *part_lse2, void *out, float *lse, int tid,
                                                 int nthreads)
 {
-    for (int idx = tid; idx < G * 64; idx += nthreads) {
-        const int r = idx >> 6, dpair = idx & 63;
-        float M = -INFINITY;
-        for (uint32_t c = mi.slot_begin; c < mi.slot_end; ++c)
-            M = fmaxf(M, __ldcg(part_lse2 + (size_t)c * kMaxGroup + r));
-        float L = 0.f, a0 = 0.f, a1 = 0.f;
-        for (uint32_t c = mi.slot_begin; c < mi.slot_end; ++c) {
-            const float wgt = fast_exp2(__ldcg(part_lse2 + (size_t)c * kMaxGroup + r) - M);
-            const float2 v = __ldcg(reinterpret_cast<const float2 *>(part_o + ((size_t)c * G + r) * kHeadDim + 2 * dpair));
-            L += wgt;
-            a0 += wgt * v.x;
-            a1 += wgt * v.y;
+    constexpr int kItems = 4;
+    const uint32_t n = mi.slot_end - mi.slot_begin;
+    const int total = G * 32;
+    for (int base = tid; base < total; base += kItems * nthreads) {
+        const float *lp[kItems];
+        const float4 *op4[kItems];
+        float M[kItems], L[kItems];
+        float4 a[kItems];
+        bool on[kItems];
+#pragma unroll
+        for (int k = 0; k < kItems; ++k) {
+            const int idx = base + k * nthreads;
+            on[k] = idx < total;
+            const int r = on[k] ? idx >> 5 : 0, quad = idx & 31;
+            lp[k] = part_lse2 + (size_t)mi.slot_begin * kMaxGroup + r;
+            op4[k] = reinterpret_cast<const float4 *>(part_o + ((size_t)mi.slot_begin * G + r) * kHeadDim) + quad;
+            M[k] = -INFINITY;
+            L[k] = 0.f;
+            a[k] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        const float inv = 1.f / L;
-        const size_t orow = (size_t)mi.row_group * G + r;
-        __nv_bfloat162 *op = reinterpret_cast<__nv_bfloat162 *>(reinterpret_cast<__nv_bfloat16 *>(out) + orow * kHeadDim + 2 * dpair);
-        *op = __floats2bfloat162_rn(a0 * inv, a1 * inv);
-        if (dpair == 0 && lse) lse[orow] = (M + log2f(L)) * 0.6931471805599453f;
+        for (uint32_t c = 0; c < n; ++c) {
+#pragma unroll
+            for (int k = 0; k < kItems; ++k)
+                if (on[k]) M[k] = fmaxf(M[k], __ldcg(lp[k] + (size_t)c * kMaxGroup));
+        }
+        for (uint32_t c0 = 0; c0 < n; c0 += 2) {
+            float lv[kItems][2];
+            float4 v[kItems][2];
+#pragma unroll
+            for (int k = 0; k < kItems; ++k) {
+#pragma unroll
+                for (uint32_t j = 0; j < 2; ++j) {
+                    const bool in = on[k] && c0 + j < n;
+                    lv[k][j] = in ? __ldcg(lp[k] + (size_t)(c0 + j) * kMaxGroup) : -INFINITY;
+                    v[k][j] = in ? __ldcg(op4[k] + (size_t)(c0 + j) * G * (kHeadDim / 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < kItems; ++k) {
+#pragma unroll
+                for (uint32_t j = 0; j < 2; ++j) {
+                    const float wgt = on[k] ? fast_exp2(lv[k][j] - M[k]) : 0.f;  // 0 for the slots past the end
+                    L[k] += wgt;
+                    a[k].x += wgt * v[k][j].x;
+                    a[k].y += wgt * v[k][j].y;
+                    a[k].z += wgt * v[k][j].z;
+                    a[k].w += wgt * v[k][j].w;
+                }
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < kItems; ++k) {
+            const int idx = base + k * nthreads;
+            if (!on[k]) continue;
+            const int r = idx >> 5, quad = idx & 31;
+            const float inv = 1.f / L[k];
+            const size_t orow = (size_t)mi.row_group * G + r;
+            uint2 packed;
+            packed.x = pack_bf16(a[k].x * inv, a[k].y * inv);
+            packed.y = pack_bf16(a[k].z * inv, a[k].w * inv);
+            *reinterpret_cast<uint2 *>(reinterpret_cast<__nv_bfloat16 *>(out) + orow * kHeadDim + 4 * quad) = packed;
+            if (quad == 0 && lse) lse[orow] = (M[k] + log2f(L[k])) * 0.6931471805599453f;
+        }
     }
 }
 

@@ -8,9 +8,10 @@
 // consumer multiplies the group's G query heads (padded to the 16 rows of an m16n8k16 bf16 MMA, so
 // a K/V tile is read once per group) with the tile, keeps an fp32 online softmax (running max, sum,
 // rescaled output) in registers, and multiplies the probabilities with V.  At the end of a row-group
-// piece the warps' states are combined through shared memory and written either as the final bf16
-// output + lse (piece = whole row group) or as an fp32 partial; the block that delivers the last
-// partial of a split row group merges them (an arrival ticket per split row group, no waiting).
+// piece every warp deposits its state in shared memory and moves on; the warp that deposits last
+// combines the six states and writes either the final bf16 output + lse (piece = whole row group) or
+// an fp32 partial; the block that delivers the last partial of a split row group merges them (an
+// arrival ticket per split row group, no waiting), unless a merge kernel follows.
 // Arithmetic follows Eq. 1 of the paper evaluated at the last position; the split and the merge use
 // that a softmax over a union of token sets is the lse-weighted mix of the softmaxes over the sets.
 #include <cuda_bf16.h>
@@ -34,8 +35,8 @@ constexpr uint32_t kTileBytes = 2 * kHalfBytes;       // K or V tile: 64 tokens 
 constexpr uint32_t kStageBytes = 2 * kTileBytes;      // K tile then V tile
 constexpr int kScratchStride = 132;                   // floats per scratch row (128 + pad)
 constexpr uint32_t kScratchOBytes = kConsumerWarps * kMaxGroup * kScratchStride * 4;
-constexpr uint32_t kScratchMLBytes = kConsumerWarps * kMaxGroup * 2 * 4;
-constexpr uint32_t kBarrierBytes = 3 * kStages * 8;
+constexpr uint32_t kScratchMLBytes = 2 * kConsumerWarps * kMaxGroup * 2 * 4;  // two buffers
+constexpr uint32_t kBarrierBytes = (3 * kStages + 2) * 8;
 constexpr uint32_t kSmemUsed = kStages * kStageBytes + kScratchOBytes + kScratchMLBytes + kBarrierBytes + 16;  // + flags
 constexpr uint32_t kSmemBytes = kSmemUsed + 1024;     // slack to align the stages to 1024 bytes
 static_assert(kSmemBytes <= 232448, "shared memory budget of one sm_100 block exceeded");
@@ -61,10 +62,6 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a2
         "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
         : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ void consumer_bar()
-{
-    asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory");
 }
 
 // Online-softmax state of one warp for one row-group piece.  Thread (lane) owns query row lane/4
@@ -189,10 +186,11 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeParams 
     const uint32_t bars = base + kStages * kStageBytes + kScratchOBytes + kScratchMLBytes;
     volatile uint32_t *abort_flag =
         reinterpret_cast<volatile uint32_t *>(smem + kStages * kStageBytes + kScratchOBytes + kScratchMLBytes + kBarrierBytes);
-    volatile uint32_t *last_flag = abort_flag + 1;  // "this block merges the split row group"
+    volatile uint32_t *arrivals = abort_flag + 1;   // [2] warps that have deposited their state of a piece
     auto full_k = [&](int s) { return bars + (uint32_t)s * 8u; };
     auto full_v = [&](int s) { return bars + (uint32_t)(kStages + s) * 8u; };
     auto empty = [&](int s) { return bars + (uint32_t)(2 * kStages + s) * 8u; };
+    auto scratch_free = [&](uint32_t b) { return bars + (uint32_t)(3 * kStages) * 8u + b * 8u; };
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -204,7 +202,11 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeParams 
             mbar_init(full_v(s), 1);
             mbar_init(empty(s), 1);
         }
+        mbar_init(scratch_free(0), 1);
+        mbar_init(scratch_free(1), 1);
         *abort_flag = 0;
+        arrivals[0] = 0;
+        arrivals[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -289,6 +291,11 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeParams 
     uint32_t qa0[8], qa2[8];
     uint32_t t = 0;       // tiles seen by this block so far (same count as the producer's)
     bool alive = true;    // false once the block has given up
+    // The combine scratch holds the six warps' states of a piece.  With G <= 4 it fits twice, and
+    // consecutive pieces alternate between the halves; larger groups use it as one buffer.
+    const uint32_t nbuf = G <= kMaxGroup / 2 ? 2u : 1u;
+    const int rows_buf = G <= kMaxGroup / 2 ? kMaxGroup / 2 : kMaxGroup;
+    uint32_t piece = 0;   // pieces this block has finished
 
     for (uint32_t it = item_begin; it < item_end; ++it) {
         const cart_work_item w = p.items[it];
@@ -330,74 +337,99 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeParams 
         t += ntiles;
 
         if (w.flags & CART_ITEM_END) {
-            // ---- combine the consumer warps' states ---------------------------------------------
+            // ---- hand this warp's state of the piece to whichever warp arrives last ----------------
+            // No block-wide barrier: a warp that has deposited goes straight on to its tiles of the next
+            // piece.  Pieces alternate between the scratch buffers; a buffer is free again once the
+            // combine of the piece that used it before is done.
+            const uint32_t b = piece % nbuf, use = piece / nbuf;
+            ++piece;
+            if (alive && use > 0)
+                alive = __all_sync(0xffffffffu, mbar_wait(scratch_free(b), (use - 1u) & 1u, abort_flag, p.status,
+                                                          kStatusTimeoutConsumer));
+            if (!alive) continue;
             float lsum = st.l;
             lsum += __shfl_xor_sync(0xffffffffu, lsum, 1);
             lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);
+            float *buf_o = scratch_o + (size_t)b * kConsumerWarps * rows_buf * kScratchStride;
+            float *buf_ml = scratch_ml + (size_t)b * kConsumerWarps * kMaxGroup * 2;
             if (row < G) {
-                float *so = scratch_o + ((size_t)warp * kMaxGroup + row) * kScratchStride + 2 * (lane & 3);
+                float *so = buf_o + ((size_t)warp * rows_buf + row) * kScratchStride + 2 * (lane & 3);
 #pragma unroll
                 for (int d = 0; d < 16; ++d)
                     *reinterpret_cast<float2 *>(so + 8 * d) = make_float2(st.o[d][0], st.o[d][1]);
                 if ((lane & 3) == 0) {
-                    scratch_ml[(warp * kMaxGroup + row) * 2 + 0] = st.m;
-                    scratch_ml[(warp * kMaxGroup + row) * 2 + 1] = lsum;
+                    buf_ml[(warp * kMaxGroup + row) * 2 + 0] = st.m;   // -inf if the warp had no tile of the piece
+                    buf_ml[(warp * kMaxGroup + row) * 2 + 1] = lsum;
                 }
             }
-            consumer_bar();
-            if (*abort_flag) alive = false;
-            for (int idx = threadIdx.x; idx < G * 64; idx += kConsumerThreads) {
-                const int r = idx >> 6, dpair = idx & 63;
+            __syncwarp();
+            uint32_t last = 0;
+            if (lane == 0) {
+                __threadfence_block();
+                last = (atomicAdd(const_cast<uint32_t *>(&arrivals[b]), 1u) == (uint32_t)kConsumerWarps - 1u) ? 1u : 0u;
+                __threadfence_block();
+            }
+            last = __shfl_sync(0xffffffffu, last, 0);
+            __syncwarp();
+            if (!last) continue;
+
+            // ---- this warp arrived last: combine the six states and write the piece -------------------
+            for (int idx = lane; idx < G * 32; idx += 32) {  // one query row, four output dims
+                const int r = idx >> 5, quad = idx & 31;
+                float mw[kConsumerWarps];
                 float M = -INFINITY;
 #pragma unroll
-                for (int wv = 0; wv < kConsumerWarps; ++wv) M = fmaxf(M, scratch_ml[(wv * kMaxGroup + r) * 2]);
-                float L = 0.f, a0 = 0.f, a1 = 0.f;
+                for (int wv = 0; wv < kConsumerWarps; ++wv) {
+                    mw[wv] = buf_ml[(wv * kMaxGroup + r) * 2];
+                    M = fmaxf(M, mw[wv]);
+                }
+                float L = 0.f;
+                float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
                 for (int wv = 0; wv < kConsumerWarps; ++wv) {
-                    const float wgt = fast_exp2(scratch_ml[(wv * kMaxGroup + r) * 2] - M);
-                    L += wgt * scratch_ml[(wv * kMaxGroup + r) * 2 + 1];
-                    const float2 v = *reinterpret_cast<const float2 *>(
-                        scratch_o + ((size_t)wv * kMaxGroup + r) * kScratchStride + 2 * dpair);
-                    a0 += wgt * v.x;
-                    a1 += wgt * v.y;
+                    if (mw[wv] == -INFINITY) continue;  // that warp had no tile of the piece
+                    const float wgt = fast_exp2(mw[wv] - M);
+                    L += wgt * buf_ml[(wv * kMaxGroup + r) * 2 + 1];
+                    const float4 v = *reinterpret_cast<const float4 *>(
+                        buf_o + ((size_t)wv * rows_buf + r) * kScratchStride + 4 * quad);
+                    a.x += wgt * v.x;
+                    a.y += wgt * v.y;
+                    a.z += wgt * v.z;
+                    a.w += wgt * v.w;
                 }
                 const float inv = 1.f / L;
                 const float lse2 = M + log2f(L);
-                if (alive) {
-                    if (w.flags & CART_ITEM_DIRECT) {
-                        const size_t orow = (size_t)w.row_group * G + r;
-                        __nv_bfloat162 *op = reinterpret_cast<__nv_bfloat162 *>(
-                            reinterpret_cast<__nv_bfloat16 *>(p.out) + orow * kHeadDim + 2 * dpair);
-                        *op = __floats2bfloat162_rn(a0 * inv, a1 * inv);
-                        if (dpair == 0 && p.lse) p.lse[orow] = lse2 * 0.6931471805599453f;
-                    } else {
-                        float2 *pp = reinterpret_cast<float2 *>(
-                            p.part_o + ((size_t)w.slot * G + r) * kHeadDim + 2 * dpair);
-                        *pp = make_float2(a0 * inv, a1 * inv);
-                        if (dpair == 0) p.part_lse2[(size_t)w.slot * kMaxGroup + r] = lse2;
-                    }
+                if (w.flags & CART_ITEM_DIRECT) {
+                    const size_t orow = (size_t)w.row_group * G + r;
+                    uint2 packed;
+                    packed.x = pack_bf16(a.x * inv, a.y * inv);
+                    packed.y = pack_bf16(a.z * inv, a.w * inv);
+                    *reinterpret_cast<uint2 *>(reinterpret_cast<__nv_bfloat16 *>(p.out) + orow * kHeadDim + 4 * quad) = packed;
+                    if (quad == 0 && p.lse) p.lse[orow] = lse2 * 0.6931471805599453f;
+                } else {
+                    float4 *pp = reinterpret_cast<float4 *>(p.part_o + ((size_t)w.slot * G + r) * kHeadDim) + quad;
+                    *pp = make_float4(a.x * inv, a.y * inv, a.z * inv, a.w * inv);
+                    if (quad == 0) p.part_lse2[(size_t)w.slot * kMaxGroup + r] = lse2;
                 }
             }
-            const bool ticketed = !(w.flags & CART_ITEM_DIRECT) && p.tickets != nullptr;
-            if (ticketed) __threadfence();  // publish the partial before the ticket
-            consumer_bar();  // the scratch may be overwritten by the next piece from here on
-
-            if (ticketed) {
+            __syncwarp();
+            if (lane == 0) {
+                arrivals[b] = 0;
+                mbar_arrive(scratch_free(b));  // the buffer may be refilled from here on
+            }
+            if (!(w.flags & CART_ITEM_DIRECT) && p.tickets != nullptr) {
                 // Split row group: the block whose piece arrives last merges all pieces.  Nobody waits.
+                __threadfence();  // publish the partial before the ticket
+                __syncwarp();
                 const cart_merge_item mi = p.merges[w.merge];
-                if (threadIdx.x == 0) {
-                    uint32_t last = 0;
-                    if (alive) {
-                        const uint32_t seen = atomicAdd(&p.tickets[w.merge], 1u);
-                        last = (seen + 1u == mi.slot_end - mi.slot_begin) ? 1u : 0u;
-                    }
-                    *last_flag = last;
-                }
-                consumer_bar();
-                if (*last_flag) {
+                uint32_t mine = 0;
+                if (lane == 0) mine = (atomicAdd(&p.tickets[w.merge], 1u) + 1u == mi.slot_end - mi.slot_begin) ? 1u : 0u;
+                mine = __shfl_sync(0xffffffffu, mine, 0);
+                if (mine) {
                     __threadfence();
-                    merge_row_group(mi, G, p.part_o, p.part_lse2, p.out, p.lse, (int)threadIdx.x, kConsumerThreads);
-                    if (threadIdx.x == 0) p.tickets[w.merge] = 0;  // ready for the next launch
+                    merge_row_group(mi, G, p.part_o, p.part_lse2, p.out, p.lse, lane, 32);
+                    __syncwarp();
+                    if (lane == 0) p.tickets[w.merge] = 0;  // ready for the next launch
                 }
             }
         }

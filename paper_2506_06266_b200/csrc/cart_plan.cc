@@ -215,7 +215,24 @@ extern "C" cart_status cart_plan_build_shared(const cart_plan_seg *segs, const i
     uint32_t next_slot = 0;
     uint64_t pos = 0;  // tiles handed out so far
     uint64_t c = 0;    // block being filled
-    auto range_end = [&](uint64_t blk) { return C ? ((blk + 1) * W) / C : 0; };
+    // Blocks are balanced by weight: a tile weighs 1, starting a piece weighs piece_cost (what its
+    // epilogue costs a block, in tile times).  Every block boundary is assumed to cut a row group
+    // and so to start one more piece.
+    const uint64_t A = o->piece_cost > 0 ? (uint64_t)o->piece_cost : 0;
+    uint64_t rgs_with_tiles = 0;
+    for (int32_t i = 0; i < n_reqs; ++i) {
+        bool any = false;
+        for (int32_t s = seg_begin[i]; s < seg_begin[i + 1] && !any; ++s) {
+            uint32_t t0, nt;
+            stream_part(s, &t0, &nt);
+            any = nt > 0;
+        }
+        if (any) rgs_with_tiles += (uint64_t)n_kv_heads;
+    }
+    const uint64_t Wt = W + A * (rgs_with_tiles + (C > 0 ? C - 1 : 0));
+    auto target = [&](uint64_t blk) { return C ? ((blk + 1) * Wt) / C : 0; };
+    uint64_t wpos = 0;          // weight handed out so far
+    bool block_has_work = false;
     o->cta_begin[0] = 0;
 
     for (int32_t i = 0; i < n_reqs; ++i) {
@@ -262,7 +279,18 @@ extern "C" cart_status cart_plan_build_shared(const cart_plan_seg *segs, const i
             settle();
             uint64_t seg_tile = 0;  // tiles of segment s already handed out
             while (pos < rg_end) {
-                const uint64_t piece_end = std::min(rg_end, range_end(c));
+                // tiles of this row group that fit in block c after paying for the piece
+                const uint64_t paid = wpos + A;
+                uint64_t room = target(c) > paid ? target(c) - paid : 0;
+                if (room == 0 && block_has_work && c + 1 < C) {  // block c is full: go on in the next one
+                    ++c;
+                    o->cta_begin[c] = (uint32_t)ni;
+                    block_has_work = false;
+                    continue;
+                }
+                if (room == 0) room = 1;
+                if (c + 1 == C) room = rg_end - pos;  // the last block takes what is left
+                const uint64_t piece_end = std::min(rg_end, pos + room);
                 const bool direct = !has_shared && pos == rg_start && piece_end == rg_end;
                 uint64_t want = piece_end - pos;
                 bool first = true;
@@ -300,8 +328,14 @@ extern "C" cart_status cart_plan_build_shared(const cart_plan_seg *segs, const i
                     last.slot = next_slot++;
                     last.merge = (uint32_t)my_merge;
                 }
+                wpos += A + (piece_end - pos);
                 pos = piece_end;
-                if (pos == range_end(c)) { ++c; o->cta_begin[c] = (uint32_t)ni; }
+                block_has_work = true;
+                if (wpos >= target(c) && c + 1 < C) {
+                    ++c;
+                    o->cta_begin[c] = (uint32_t)ni;
+                    block_has_work = false;
+                }
             }
             if (split) {
                 o->merges[my_merge].row_group = rg;
@@ -311,11 +345,12 @@ extern "C" cart_status cart_plan_build_shared(const cart_plan_seg *segs, const i
             }
         }
     }
+    const uint64_t used = C ? (block_has_work ? c + 1 : c) : 0;
     for (uint64_t b = c; b < (uint64_t)n_cta; ++b) o->cta_begin[b + 1] = (uint32_t)ni;
     if ((int64_t)next_slot > (int64_t)o->slots_cap) return CART_ERR_CAPACITY;
     o->n_items = ni;
     o->n_merges = nm;
-    o->n_cta_used = (int32_t)C;
+    o->n_cta_used = (int32_t)used;
     o->n_slots = (int32_t)next_slot;
     o->total_tiles = (int64_t)W;
     return CART_OK;

@@ -31,8 +31,8 @@ class Arena:
         return (k, v, hs, self.Hkv * hs, n)
 
 
-def check(segs, Hkv, G, n_cta, tile=64, share_min=4, share_tile=128, slots_cap=1 << 20):
-    plan = binding.cart_plan_build_shared(segs, Hkv, G, n_cta, tile, share_min, share_tile, slots_cap)
+def check(segs, Hkv, G, n_cta, tile=64, share_min=4, share_tile=128, slots_cap=1 << 20, piece_cost=0):
+    plan = binding.cart_plan_build_shared(segs, Hkv, G, n_cta, tile, share_min, share_tile, slots_cap, piece_cost)
     items, cta_begin, units = plan["items"], plan["cta_begin"], plan["units"]
     R = 128 // G
 
@@ -45,6 +45,7 @@ def check(segs, Hkv, G, n_cta, tile=64, share_min=4, share_tile=128, slots_cap=1
     # ---- stream items ---------------------------------------------------------------------------
     pieces = {}
     per_cta = []
+    per_cta_pieces = []
     for c in range(n_cta):
         tiles, open_rg = 0, None
         for it in items[cta_begin[c]:cta_begin[c + 1]]:
@@ -60,10 +61,17 @@ def check(segs, Hkv, G, n_cta, tile=64, share_min=4, share_tile=128, slots_cap=1
                 open_rg = None
         assert open_rg is None
         per_cta.append(tiles)
+        per_cta_pieces.append(sum(1 for it in items[cta_begin[c]:cta_begin[c + 1]] if it.flags & E_))
     used = plan["n_cta_used"]
     assert sum(per_cta) == plan["total_tiles"] and all(t == 0 for t in per_cta[used:])
-    if used:
+    if used and piece_cost == 0:
         assert max(per_cta[:used]) - min(per_cta[:used]) <= 1 and min(per_cta[:used]) >= 1
+    elif used:
+        # balanced by weight = tiles + piece_cost * pieces: no block is more than one piece and one tile
+        # above the even share (the last block takes what is left and may be lighter)
+        weight = [t + piece_cost * n for t, n in zip(per_cta[:used], per_cta_pieces[:used])]
+        assert min(per_cta[:used]) >= 1
+        assert max(weight) <= -(-sum(weight) // used) + piece_cost + 1
     assert cta_begin[n_cta] == len(items)
 
     # ---- shared units -----------------------------------------------------------------------------
@@ -213,3 +221,16 @@ def test_benchmark_shapes_with_sharing(w):
     assert plan["n_unit_cta_used"] == 148 and plan["n_cta_used"] == 148
     per_rg = plan["n_slots"] / (w.batch * w.n_kv_heads)
     assert per_rg < 10          # what the library's scratch is sized for
+
+
+@pytest.mark.parametrize("piece_cost", [1, 3, 8])
+def test_blocks_balanced_by_tiles_and_pieces(piece_cost):
+    # many short suffixes next to a few long ones: by tiles alone some blocks would hold 20 pieces, others 4
+    a = Arena(8)
+    cart = a.store(4096)
+    rng = np.random.default_rng(11)
+    segs = [[cart, a.store(int(n))] for n in rng.integers(1, 1025, size=128)]
+    plan = check(segs, 8, 4, 148, piece_cost=piece_cost)
+    assert plan["n_cta_used"] >= 140
+    flat = check([[a.store(int(n))] for n in rng.integers(1, 300, size=40)], 2, 4, 37, share_min=0, piece_cost=piece_cost)
+    assert flat["n_cta_used"] >= 25      # a boundary that falls between row groups saves the piece it was charged for
