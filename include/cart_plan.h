@@ -131,6 +131,8 @@ typedef struct {
     uint32_t *reader_slot;     /* [readers_cap * n_kv_heads]: first slot of (entry, KV head); + unit.chunk */
     uint32_t *reader_merge;    /* [readers_cap * n_kv_heads]: merge item of (entry, KV head) */
     int64_t shared_tiles;      /* tile runs handed to the shared kernel, in share_tile_tokens tiles */
+    int32_t unit_cost;         /* in: what a shared unit costs a block on top of its tiles, in tile times; the
+                                  shared blocks are balanced by tiles + unit_cost * units (0: by tiles alone) */
 } cart_plan_out;
 
 /*

@@ -82,7 +82,7 @@ class cart_plan_out(ctypes.Structure):
                 ("n_readers", ctypes.c_int32),
                 ("reader_slot", ctypes.POINTER(ctypes.c_uint32)),
                 ("reader_merge", ctypes.POINTER(ctypes.c_uint32)),
-                ("shared_tiles", ctypes.c_int64)]
+                ("shared_tiles", ctypes.c_int64), ("unit_cost", ctypes.c_int32)]
 
 
 CART_ITEM_BEGIN, CART_ITEM_END, CART_ITEM_DIRECT, CART_ITEM_TAIL = 1, 2, 4, 8
@@ -347,7 +347,7 @@ def cart_plan_build(segs: Sequence[Sequence[Tuple[int, int, int, int, int]]], n_
 
 def cart_plan_build_shared(segs: Sequence[Sequence[Tuple[int, int, int, int, int]]], n_kv_heads: int, group: int,
                            n_cta: int, tile_tokens: int, share_min_readers: int, share_tile_tokens: int,
-                           slots_cap: int = 1 << 20, piece_cost: int = 0):
+                           slots_cap: int = 1 << 20, piece_cost: int = 0, unit_cost: int = 0):
     """Host-only planner with shared segments (see include/cart_plan.h).  Returns a dict with the
     stream plan (items, cta_begin, merges, ...) and the shared part (units, unit_cta_begin, readers,
     reader_slot[entry][head], reader_merge[entry][head])."""
@@ -375,6 +375,7 @@ def cart_plan_build_shared(segs: Sequence[Sequence[Tuple[int, int, int, int, int
     o.items, o.items_cap, o.cta_begin = items, items_cap, cta_begin
     o.merges, o.merges_cap, o.slots_cap = merges, merges_cap, slots_cap
     o.piece_cost = piece_cost
+    o.unit_cost = unit_cost
     o.units, o.units_cap, o.unit_cta_begin = units, units_cap, unit_cta_begin
     o.readers, o.readers_cap, o.reader_slot, o.reader_merge = readers, readers_cap, reader_slot, reader_merge
     st = lib.cart_plan_build_shared(seg_arr, sb, len(segs), n_kv_heads, group, n_cta, tile_tokens,

@@ -28,6 +28,8 @@ uint64_t round_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
 constexpr int kShareMinReaders = 4;
 // What the planner charges a stream block for starting a row-group piece, in 64-token tile times.
 constexpr int kPieceCostTiles = 3;
+// What the planner charges a shared-segment block per unit on top of its tiles, in 128-token tile times.
+constexpr int kUnitCostTiles = 4;
 
 struct ScratchLayout {
     uint64_t status_off, tickets_off, plan_off, plan_slot_bytes, cta_begin_off, merges_off, items_off;
@@ -667,6 +669,7 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
         po.merges_cap = lay.merges_cap;
         po.slots_cap = lay.slots_cap;
         po.piece_cost = ctx->piece_cost;
+        po.unit_cost = kUnitCostTiles;
         po.units = reinterpret_cast<cart_shared_unit *>(ns.host + lay.units_off);
         po.units_cap = lay.units_cap;
         po.unit_cta_begin = reinterpret_cast<uint32_t *>(ns.host + lay.unit_cta_begin_off);

@@ -131,10 +131,16 @@ __device__ __forceinline__ void merge_row_group(const cart_merge_item mi, int G,
             L[k] = 0.f;
             a[k] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        for (uint32_t c = 0; c < n; ++c) {
+        for (uint32_t c0 = 0; c0 < n; c0 += 4) {  // four slots' lse values in flight per item
+            float lv[kItems][4];
 #pragma unroll
             for (int k = 0; k < kItems; ++k)
-                if (on[k]) M[k] = fmaxf(M[k], __ldcg(lp[k] + (size_t)c * kMaxGroup));
+#pragma unroll
+                for (uint32_t j = 0; j < 4; ++j)
+                    lv[k][j] = (on[k] && c0 + j < n) ? __ldcg(lp[k] + (size_t)(c0 + j) * kMaxGroup) : -INFINITY;
+#pragma unroll
+            for (int k = 0; k < kItems; ++k)
+                M[k] = fmaxf(fmaxf(M[k], fmaxf(lv[k][0], lv[k][1])), fmaxf(lv[k][2], lv[k][3]));
         }
         for (uint32_t c0 = 0; c0 < n; c0 += 2) {
             float lv[kItems][2];

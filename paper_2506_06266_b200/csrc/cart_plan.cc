@@ -25,6 +25,54 @@ struct SharedClass {
     uint32_t first_combo;   // combos of this class: (m * n_kv_heads + g) from here
 };
 
+// Hands out tiles of consecutive groups (row groups of the stream, tile runs of the shared part) to
+// `C` blocks in order.  A tile weighs 1, every part of a group that a block takes ("unit") weighs
+// `A` on top.  When a block is opened it is given an equal share of the weight that is left, counting
+// one unit per group still to come and one more per block boundary still to come (a boundary is
+// assumed to cut a group); the share is recomputed for every block, so an error in that assumption
+// does not pile up on the last block.  With A = 0 the blocks' tile counts differ by at most one.
+struct Balancer {
+    uint64_t C, A;
+    uint64_t tiles_left;   // tiles not handed out yet
+    uint64_t groups_left;  // groups of which nothing has been handed out yet
+    uint64_t c = 0;        // block being filled
+    uint64_t acc = 0;      // weight block c holds
+    uint64_t budget = 0;
+
+    Balancer(uint64_t blocks, uint64_t unit_cost, uint64_t tiles, uint64_t groups)
+        : C(blocks), A(unit_cost), tiles_left(tiles), groups_left(groups) { open(false); }
+
+    void open(bool mid_group)
+    {
+        const uint64_t blocks = C > c ? C - c : 1;
+        const uint64_t wt = tiles_left + A * (groups_left + (mid_group ? 1 : 0) + (blocks - 1));
+        budget = (wt + blocks - 1) / blocks;
+        acc = 0;
+    }
+    // Tiles the current block takes from a group with `rem` tiles left (>= 1); moves on to the next block
+    // first if the current one cannot pay for another unit.  `fresh`: nothing of the group was taken yet.
+    uint64_t take(uint64_t rem, bool fresh)
+    {
+        for (;;) {
+            const uint64_t paid = acc + A;
+            uint64_t room = budget > paid ? budget - paid : 0;
+            if (room == 0 && acc > 0 && c + 1 < C) { ++c; open(!fresh); continue; }
+            if (room == 0) room = 1;
+            if (c + 1 >= C) room = rem;  // the last block takes what is left
+            return rem < room ? rem : room;
+        }
+    }
+    // Books `t` tiles of a group on block c; `more`: the group still has tiles after them.
+    void commit(uint64_t t, bool fresh, bool more)
+    {
+        acc += A + t;
+        tiles_left -= t;
+        if (fresh) --groups_left;
+        if (acc >= budget && c + 1 < C) { ++c; open(more); }
+    }
+    bool block_has_work() const { return acc > 0; }
+};
+
 bool same_storage(const cart_plan_seg &a, const cart_plan_seg &b)
 {
     return a.k_row == b.k_row && a.v_row == b.v_row && a.n_tok == b.n_tok && a.head_stride == b.head_stride &&
@@ -120,30 +168,42 @@ extern "C" cart_status cart_plan_build_shared(const cart_plan_seg *segs, const i
     }
 
     // ---- 2. divide the shared runs over blocks; shrink the block count until the partials fit ------
+    // Blocks are balanced by weight: a tile weighs 1, a unit weighs unit_cost on top (its queries are
+    // loaded, its partials written).
     uint64_t W_sh = 0;
     for (const Combo &cb : combos) W_sh += cb.n_tiles;
+    const uint64_t Au = o->unit_cost > 0 ? (uint64_t)o->unit_cost : 0;
+    // walks the runs; calls emit(combo index, tiles done before, tiles taken, chunk, block) per unit and
+    // returns the number of blocks that received work
+    auto walk = [&](uint64_t C, auto &&emit) -> uint64_t {
+        Balancer bal(C, Au, W_sh, (uint64_t)combos.size());
+        for (size_t ci = 0; ci < combos.size(); ++ci) {
+            uint64_t rem = combos[ci].n_tiles, done = 0;
+            uint32_t chunk = 0;
+            while (rem > 0) {
+                const bool fresh = done == 0;
+                const uint64_t t = bal.take(rem, fresh);
+                emit(ci, done, t, chunk++, bal.c);
+                rem -= t;
+                done += t;
+                bal.commit(t, fresh, rem > 0);
+            }
+        }
+        return bal.block_has_work() ? bal.c + 1 : bal.c;
+    };
     uint64_t C_sh = 0;
     if (W_sh > 0) {
-        // a block should get at least two tiles: every unit pays for loading its queries and writing
-        // its partials
+        // a block should get at least two tiles
         C_sh = std::min<uint64_t>((uint64_t)n_cta, std::max<uint64_t>(1, W_sh / 2));
         // every stream piece of a row group with a shared part takes a slot, and so does every split
         const int64_t stream_reserve = (int64_t)n_reqs * n_kv_heads + 2 * (int64_t)n_cta;
         for (;;) {
-            uint64_t pos = 0, c = 0;
             int64_t need = 0;
-            for (Combo &cb : combos) {
-                uint32_t chunks = 0;
-                uint64_t end = pos + cb.n_tiles;
-                while (pos < end) {
-                    const uint64_t re = ((c + 1) * W_sh) / C_sh;
-                    pos = std::min(end, re);
-                    ++chunks;
-                    if (pos == re) ++c;
-                }
-                cb.n_chunks = chunks;
-                need += (int64_t)chunks * cb.n_readers;
-            }
+            for (Combo &cb : combos) cb.n_chunks = 0;
+            walk(C_sh, [&](size_t ci, uint64_t, uint64_t, uint32_t, uint64_t) {
+                ++combos[ci].n_chunks;
+                need += combos[ci].n_readers;
+            });
             if (need + stream_reserve <= (int64_t)o->slots_cap) break;
             C_sh /= 2;
             if (C_sh == 0) break;
@@ -160,18 +220,17 @@ extern "C" cart_status cart_plan_build_shared(const cart_plan_seg *segs, const i
 
     // ---- 3. emit the shared units ------------------------------------------------------------------
     int32_t nu = 0;
+    uint64_t used_sh = 0;
     if (want_share) {
         o->unit_cta_begin[0] = 0;
-        uint64_t pos = 0, c = 0;
-        for (const Combo &cb : combos) {
-            const cart_plan_seg &sg = classes[(size_t)cb.cls].seg;
-            uint64_t done = 0;  // tiles of this run already handed out
-            uint32_t chunk = 0;
-            const uint64_t end = pos + cb.n_tiles;
-            while (pos < end) {
-                const uint64_t re = ((c + 1) * W_sh) / C_sh;
-                const uint64_t take = std::min(end, re) - pos;
-                if (nu >= o->units_cap) return CART_ERR_CAPACITY;
+        uint64_t cur = 0;  // block whose units are being written
+        bool overflow = false;
+        if (C_sh > 0)
+            used_sh = walk(C_sh, [&](size_t ci, uint64_t done, uint64_t take, uint32_t chunk, uint64_t c) {
+                if (nu >= o->units_cap) { overflow = true; return; }
+                while (cur < c) o->unit_cta_begin[++cur] = (uint32_t)nu;
+                const Combo &cb = combos[ci];
+                const cart_plan_seg &sg = classes[(size_t)cb.cls].seg;
                 cart_shared_unit &u = o->units[nu++];
                 const uint32_t tok0 = (uint32_t)(done * TS);
                 u.k_row = sg.k_row + cb.kv_head * sg.head_stride + tok0;
@@ -181,16 +240,13 @@ extern "C" cart_status cart_plan_build_shared(const cart_plan_seg *segs, const i
                 u.reader_begin = cb.reader_begin;
                 u.n_readers = cb.n_readers;
                 u.kv_head = cb.kv_head;
-                u.chunk = chunk++;
-                done += take;
-                pos += take;
-                if (pos == re) { ++c; o->unit_cta_begin[c] = (uint32_t)nu; }
-            }
-        }
-        for (uint64_t b = c; b < (uint64_t)n_cta; ++b) o->unit_cta_begin[b + 1] = (uint32_t)nu;
+                u.chunk = chunk;
+            });
+        if (overflow) return CART_ERR_CAPACITY;
+        for (uint64_t b = cur; b < (uint64_t)n_cta; ++b) o->unit_cta_begin[b + 1] = (uint32_t)nu;
     }
     o->n_units = nu;
-    o->n_unit_cta_used = (int32_t)C_sh;
+    o->n_unit_cta_used = (int32_t)used_sh;
     o->n_readers = n_entries;
     o->shared_tiles = (int64_t)W_sh;
 
@@ -216,8 +272,7 @@ extern "C" cart_status cart_plan_build_shared(const cart_plan_seg *segs, const i
     uint64_t pos = 0;  // tiles handed out so far
     uint64_t c = 0;    // block being filled
     // Blocks are balanced by weight: a tile weighs 1, starting a piece weighs piece_cost (what its
-    // epilogue costs a block, in tile times).  Every block boundary is assumed to cut a row group
-    // and so to start one more piece.
+    // epilogue costs a block, in tile times).
     const uint64_t A = o->piece_cost > 0 ? (uint64_t)o->piece_cost : 0;
     uint64_t rgs_with_tiles = 0;
     for (int32_t i = 0; i < n_reqs; ++i) {
@@ -229,10 +284,7 @@ extern "C" cart_status cart_plan_build_shared(const cart_plan_seg *segs, const i
         }
         if (any) rgs_with_tiles += (uint64_t)n_kv_heads;
     }
-    const uint64_t Wt = W + A * (rgs_with_tiles + (C > 0 ? C - 1 : 0));
-    auto target = [&](uint64_t blk) { return C ? ((blk + 1) * Wt) / C : 0; };
-    uint64_t wpos = 0;          // weight handed out so far
-    bool block_has_work = false;
+    Balancer bal(C ? C : 1, A, W, rgs_with_tiles);
     o->cta_begin[0] = 0;
 
     for (int32_t i = 0; i < n_reqs; ++i) {
@@ -279,18 +331,11 @@ extern "C" cart_status cart_plan_build_shared(const cart_plan_seg *segs, const i
             settle();
             uint64_t seg_tile = 0;  // tiles of segment s already handed out
             while (pos < rg_end) {
-                // tiles of this row group that fit in block c after paying for the piece
-                const uint64_t paid = wpos + A;
-                uint64_t room = target(c) > paid ? target(c) - paid : 0;
-                if (room == 0 && block_has_work && c + 1 < C) {  // block c is full: go on in the next one
-                    ++c;
-                    o->cta_begin[c] = (uint32_t)ni;
-                    block_has_work = false;
-                    continue;
-                }
-                if (room == 0) room = 1;
-                if (c + 1 == C) room = rg_end - pos;  // the last block takes what is left
-                const uint64_t piece_end = std::min(rg_end, pos + room);
+                // tiles of this row group that the block takes (the balancer may close the block first)
+                const bool fresh = pos == rg_start;
+                const uint64_t piece_tiles = bal.take(rg_end - pos, fresh);
+                while (c < bal.c) o->cta_begin[++c] = (uint32_t)ni;
+                const uint64_t piece_end = pos + piece_tiles;
                 const bool direct = !has_shared && pos == rg_start && piece_end == rg_end;
                 uint64_t want = piece_end - pos;
                 bool first = true;
@@ -328,14 +373,9 @@ extern "C" cart_status cart_plan_build_shared(const cart_plan_seg *segs, const i
                     last.slot = next_slot++;
                     last.merge = (uint32_t)my_merge;
                 }
-                wpos += A + (piece_end - pos);
                 pos = piece_end;
-                block_has_work = true;
-                if (wpos >= target(c) && c + 1 < C) {
-                    ++c;
-                    o->cta_begin[c] = (uint32_t)ni;
-                    block_has_work = false;
-                }
+                bal.commit(piece_tiles, fresh, pos < rg_end);
+                while (c < bal.c) o->cta_begin[++c] = (uint32_t)ni;
             }
             if (split) {
                 o->merges[my_merge].row_group = rg;
@@ -345,7 +385,7 @@ extern "C" cart_status cart_plan_build_shared(const cart_plan_seg *segs, const i
             }
         }
     }
-    const uint64_t used = C ? (block_has_work ? c + 1 : c) : 0;
+    const uint64_t used = C ? (bal.block_has_work() ? bal.c + 1 : bal.c) : 0;
     for (uint64_t b = c; b < (uint64_t)n_cta; ++b) o->cta_begin[b + 1] = (uint32_t)ni;
     if ((int64_t)next_slot > (int64_t)o->slots_cap) return CART_ERR_CAPACITY;
     o->n_items = ni;

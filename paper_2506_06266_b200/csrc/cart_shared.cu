@@ -316,7 +316,6 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
         const uint32_t lane_addr = tmem + ((uint32_t)(32 * sw) << 16);
         const __nv_bfloat16 *q = reinterpret_cast<const __nv_bfloat16 *>(p.q);
         const uint32_t swz = (uint32_t)(row & 7);
-        float *comb_o = reinterpret_cast<float *>(smem + kOffP);     // [128 dims][128 rows], unit end only
         float *comb_ml = reinterpret_cast<float *>(smem + kOffComb); // [2][128 rows]
         uint32_t tt0 = 0;
         bool alive = true;
@@ -446,12 +445,19 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
             if (alive && have_prev) alive = take_o(prev_tt, alpha_prev);
             tt0 += u.n_tiles;
 
-            // ---- combine the two warpgroups' states of each row (all products of the unit are complete
-            //      once both have taken their last O, so the P buffers can serve as scratch) -----------------
+            // ---- combine the two warpgroups' states of each row and write the partials ------------------
+            // All products of the unit are complete once both warpgroups have taken their last O, so the P
+            // buffers can serve as scratch: row r lives at r * 512 bytes, its 16-byte quad q at position
+            // q ^ (r & 31), which keeps both the row-per-lane and the quad-per-lane accesses free of bank
+            // conflicts.
             softmax_bar_both();
+            uint8_t *comb = smem + kOffP;
+            const uint32_t rsw = (uint32_t)(row & 31);
             if (wg == 1) {
 #pragma unroll
-                for (int d = 0; d < 128; ++d) comb_o[d * 128 + row] = o_acc[d];
+                for (uint32_t q4 = 0; q4 < 32; ++q4)
+                    *reinterpret_cast<float4 *>(comb + (size_t)row * 512 + ((q4 ^ rsw) << 4)) =
+                        make_float4(o_acc[4 * q4], o_acc[4 * q4 + 1], o_acc[4 * q4 + 2], o_acc[4 * q4 + 3]);
                 comb_ml[row] = m_run;
                 comb_ml[128 + row] = l_run;
             }
@@ -460,26 +466,38 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                 const float m1 = comb_ml[row], l1 = comb_ml[128 + row];
                 const float M = fmaxf(m_run, m1);   // finite: the unit has at least one tile
                 const float w0 = fast_exp2(m_run - M), w1 = fast_exp2(m1 - M);
-                l_run = l_run * w0 + l1 * w1;
-                m_run = M;
+                const float l = l_run * w0 + l1 * w1;
+                const float inv = 1.f / l;
+                const float c0 = w0 * inv, c1 = w1 * inv;
 #pragma unroll
-                for (int d = 0; d < 128; ++d) o_acc[d] = o_acc[d] * w0 + comb_o[d * 128 + row] * w1;
-            }
-
-            // ---- epilogue: normalised fp32 partial of every valid row, then the arrival tickets ---------
-            if (wg == 0) {
+                for (uint32_t q4 = 0; q4 < 32; ++q4) {
+                    float4 *cell = reinterpret_cast<float4 *>(comb + (size_t)row * 512 + ((q4 ^ rsw) << 4));
+                    const float4 v = *cell;
+                    *cell = make_float4(o_acc[4 * q4] * c0 + v.x * c1, o_acc[4 * q4 + 1] * c0 + v.y * c1,
+                                        o_acc[4 * q4 + 2] * c0 + v.z * c1, o_acc[4 * q4 + 3] * c0 + v.w * c1);
+                }
+                uint32_t dst_row = 0xFFFFFFFFu;  // row of part_o ([slot][G] flattened) this query row goes to
                 if (alive && valid) {
                     const uint32_t slot = p.reader_slot[(size_t)entry * p.n_kv_heads + u.kv_head] + u.chunk;
-                    const float inv = 1.f / l_run;
-                    float4 *dst = reinterpret_cast<float4 *>(p.part_o + ((size_t)slot * G + h) * kHeadDim);
-#pragma unroll
-                    for (int d = 0; d < 32; ++d)
-                        dst[d] = make_float4(o_acc[4 * d] * inv, o_acc[4 * d + 1] * inv, o_acc[4 * d + 2] * inv,
-                                             o_acc[4 * d + 3] * inv);
-                    p.part_lse2[(size_t)slot * kMaxGroup + h] = m_run + log2f(l_run);
-                    if (p.tickets) __threadfence();  // publish the partial before the ticket
+                    dst_row = slot * (uint32_t)G + (uint32_t)h;
+                    p.part_lse2[(size_t)slot * kMaxGroup + h] = M + log2f(l);
                 }
-                softmax_bar();
+                flags[row] = dst_row;
+            }
+            softmax_bar_both();
+            // both warpgroups copy the normalised rows out, a warp writing one 512-byte row per instruction
+            for (uint32_t item = (uint32_t)(wg * kSoftmaxThreads + tid); item < 128u * 32u; item += 2u * kSoftmaxThreads) {
+                const uint32_t r = item >> 5, q4 = item & 31u;
+                const uint32_t dst_row = flags[r];
+                if (dst_row == 0xFFFFFFFFu) continue;
+                const float4 v = *reinterpret_cast<const float4 *>(comb + (size_t)r * 512 + ((q4 ^ (r & 31u)) << 4));
+                reinterpret_cast<float4 *>(p.part_o + (size_t)dst_row * kHeadDim)[q4] = v;
+            }
+            if (p.tickets) __threadfence();  // publish the partials before the tickets
+            softmax_bar_both();
+
+            // ---- arrival tickets (when no merge kernel follows) -------------------------------------------
+            if (wg == 0) {
                 // one thread decides for all whether the block is still in business, so that all softmax
                 // threads leave the unit loop together
                 if (tid == 0) *unit_ok = (*abort_flag == 0u) ? 1u : 0u;

@@ -31,8 +31,10 @@ class Arena:
         return (k, v, hs, self.Hkv * hs, n)
 
 
-def check(segs, Hkv, G, n_cta, tile=64, share_min=4, share_tile=128, slots_cap=1 << 20, piece_cost=0):
-    plan = binding.cart_plan_build_shared(segs, Hkv, G, n_cta, tile, share_min, share_tile, slots_cap, piece_cost)
+def check(segs, Hkv, G, n_cta, tile=64, share_min=4, share_tile=128, slots_cap=1 << 20, piece_cost=0,
+          unit_cost=0):
+    plan = binding.cart_plan_build_shared(segs, Hkv, G, n_cta, tile, share_min, share_tile, slots_cap, piece_cost,
+                                          unit_cost)
     items, cta_begin, units = plan["items"], plan["cta_begin"], plan["units"]
     R = 128 // G
 
@@ -78,6 +80,7 @@ def check(segs, Hkv, G, n_cta, tile=64, share_min=4, share_tile=128, slots_cap=1
     ucb = plan["unit_cta_begin"]
     uused = plan["n_unit_cta_used"]
     per_ucta = []
+    per_ucta_units = []
     shared_slots = {}   # row group -> list of slots its shared chunks write
     for c in range(n_cta):
         t = 0
@@ -92,9 +95,14 @@ def check(segs, Hkv, G, n_cta, tile=64, share_min=4, share_tile=128, slots_cap=1
                 shared_slots.setdefault(rg, []).append(
                     (plan["reader_slot"][e][u.kv_head] + u.chunk, plan["reader_merge"][e][u.kv_head]))
         per_ucta.append(t)
+        per_ucta_units.append(ucb[c + 1] - ucb[c])
     assert sum(per_ucta) == plan["shared_tiles"] and all(t == 0 for t in per_ucta[uused:])
-    if uused:
+    if uused and unit_cost == 0:
         assert max(per_ucta[:uused]) - min(per_ucta[:uused]) <= 1 and min(per_ucta[:uused]) >= 1
+    elif uused:
+        weight = [t + unit_cost * n for t, n in zip(per_ucta[:uused], per_ucta_units[:uused])]
+        assert min(per_ucta[:uused]) >= 1
+        assert max(weight) <= -(-sum(weight) // uused) + unit_cost + 1
     assert ucb[n_cta] == len(units)
 
     # ---- coverage: exactly the tokens of the request's segments, each once ---------------------------
@@ -234,3 +242,17 @@ def test_blocks_balanced_by_tiles_and_pieces(piece_cost):
     assert plan["n_cta_used"] >= 140
     flat = check([[a.store(int(n))] for n in rng.integers(1, 300, size=40)], 2, 4, 37, share_min=0, piece_cost=piece_cost)
     assert flat["n_cta_used"] >= 25      # a boundary that falls between row groups saves the piece it was charged for
+
+
+@pytest.mark.parametrize("w", [synth.config3(), synth.config4()])
+def test_shared_blocks_balanced_by_tiles_and_units(w):
+    a = Arena(w.n_kv_heads)
+    carts = [a.store(w.p) for _ in range(w.n_cartridges)]
+    suffix = w.suffix_lengths()
+    segs = [[carts[c] for c in parts] + [a.store(int(suffix[b]) + 64)] for b, parts in enumerate(w.request_parts())]
+    G = w.n_q_heads // w.n_kv_heads
+    flat = check(segs, w.n_kv_heads, G, 148)
+    plan = check(segs, w.n_kv_heads, G, 148, piece_cost=3, unit_cost=4)
+    assert plan["n_unit_cta_used"] >= 140
+    # charging for units makes the planner cut fewer runs in two
+    assert len(plan["units"]) <= len(flat["units"])
