@@ -105,13 +105,14 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 // the lse-weighted mix of the softmaxes over the sets, from Eq. 1): slots mi.slot_begin .. slot_end-1
 // hold normalised fp32 outputs [slot][G][128] and base-2 lse values [slot][kMaxGroup].  Called by
 // `nthreads` threads of one block with tid = 0 .. nthreads-1; the caller has fenced.  An item is one
-// query row times four output dims; a thread works on up to four items at once and on two slots at
-// a time, so that a lone warp has 8 independent 16-byte loads in flight.
+// query row times four output dims; a thread works on up to kItems items at once and on kSlots slots
+// at a time, so that kItems * kSlots independent 16-byte loads are in flight (a lone warp: 4 x 2; a
+// block with a thread per item: 1 x 8).
+template <int kItems, int kSlots>
 __device__ __forceinline__ void merge_row_group(const cart_merge_item mi, int G, const float *part_o,
                                                 const float *part_lse2, void *out, float *lse, int tid,
                                                 int nthreads)
 {
-    constexpr int kItems = 4;
     const uint32_t n = mi.slot_end - mi.slot_begin;
     const int total = G * 32;
     for (int base = tid; base < total; base += kItems * nthreads) {
@@ -131,24 +132,25 @@ __device__ __forceinline__ void merge_row_group(const cart_merge_item mi, int G,
             L[k] = 0.f;
             a[k] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        for (uint32_t c0 = 0; c0 < n; c0 += 4) {  // four slots' lse values in flight per item
-            float lv[kItems][4];
+        for (uint32_t c0 = 0; c0 < n; c0 += 8) {  // eight slots' lse values in flight per item
+            float lv[kItems][8];
 #pragma unroll
             for (int k = 0; k < kItems; ++k)
 #pragma unroll
-                for (uint32_t j = 0; j < 4; ++j)
+                for (uint32_t j = 0; j < 8; ++j)
                     lv[k][j] = (on[k] && c0 + j < n) ? __ldcg(lp[k] + (size_t)(c0 + j) * kMaxGroup) : -INFINITY;
 #pragma unroll
             for (int k = 0; k < kItems; ++k)
-                M[k] = fmaxf(fmaxf(M[k], fmaxf(lv[k][0], lv[k][1])), fmaxf(lv[k][2], lv[k][3]));
+#pragma unroll
+                for (uint32_t j = 0; j < 8; ++j) M[k] = fmaxf(M[k], lv[k][j]);
         }
-        for (uint32_t c0 = 0; c0 < n; c0 += 2) {
-            float lv[kItems][2];
-            float4 v[kItems][2];
+        for (uint32_t c0 = 0; c0 < n; c0 += kSlots) {
+            float lv[kItems][kSlots];
+            float4 v[kItems][kSlots];
 #pragma unroll
             for (int k = 0; k < kItems; ++k) {
 #pragma unroll
-                for (uint32_t j = 0; j < 2; ++j) {
+                for (uint32_t j = 0; j < kSlots; ++j) {
                     const bool in = on[k] && c0 + j < n;
                     lv[k][j] = in ? __ldcg(lp[k] + (size_t)(c0 + j) * kMaxGroup) : -INFINITY;
                     v[k][j] = in ? __ldcg(op4[k] + (size_t)(c0 + j) * G * (kHeadDim / 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
@@ -157,7 +159,7 @@ __device__ __forceinline__ void merge_row_group(const cart_merge_item mi, int G,
 #pragma unroll
             for (int k = 0; k < kItems; ++k) {
 #pragma unroll
-                for (uint32_t j = 0; j < 2; ++j) {
+                for (uint32_t j = 0; j < kSlots; ++j) {
                     const float wgt = on[k] ? fast_exp2(lv[k][j] - M[k]) : 0.f;  // 0 for the slots past the end
                     L[k] += wgt;
                     a[k].x += wgt * v[k][j].x;

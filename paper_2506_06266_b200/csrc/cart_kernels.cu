@@ -427,7 +427,7 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeParams 
                 mine = __shfl_sync(0xffffffffu, mine, 0);
                 if (mine) {
                     __threadfence();
-                    merge_row_group(mi, G, p.part_o, p.part_lse2, p.out, p.lse, lane, 32);
+                    merge_row_group<4, 2>(mi, G, p.part_o, p.part_lse2, p.out, p.lse, lane, 32);
                     __syncwarp();
                     if (lane == 0) p.tickets[w.merge] = 0;  // ready for the next launch
                 }
@@ -443,7 +443,7 @@ __global__ void __launch_bounds__(128) cart_merge_kernel(const MergeParams p)
 {
     pdl_launch_dependents();
     pdl_wait();  // the partials come from the kernels before
-    merge_row_group(p.merges[blockIdx.x], p.group, p.part_o, p.part_lse2, p.out, p.lse, (int)threadIdx.x, 128);
+    merge_row_group<1, 8>(p.merges[blockIdx.x], p.group, p.part_o, p.part_lse2, p.out, p.lse, (int)threadIdx.x, 128);
 }
 
 // One block per request: copy the new token's K and V rows (Hkv x 256 bytes each) to the suffix end.

@@ -7,8 +7,8 @@
 // for up to 128 query rows at once (row i * G + h = head h of the M-tile's i-th reader) on the
 // tcgen05 tensor cores, so the tile is fetched once per 128 rows instead of once per request:
 //
-//   producer warp   TMA loads of K and V tiles (128 tokens x 128 dims, 128-byte swizzle) into a
-//                   two-stage ring, completion on mbarriers
+//   producer warps  TMA loads of K tiles (warp 0) and V tiles (warp 2), 128 tokens x 128 dims, 128-byte
+//                   swizzle, each into its own two-stage ring, completion on mbarriers
 //   MMA warp        one thread issues  S = Q K^T  (128 x 128 x 128, accumulator in tensor memory)
 //                   and  O_t = P V  (fresh accumulator per tile); tcgen05.commit signals mbarriers
 //   2 x 4 softmax  two warpgroups take alternate tiles (warpgroup w owns S, P and O buffer w).  Thread r
@@ -38,8 +38,9 @@ namespace {
 constexpr int kShTile = kShareTileTokens;             // tokens per tile = N of the score product
 constexpr uint32_t kShBlock = 128u * 128u;            // 128 rows x 128 bytes: one swizzled block (64 bf16 wide)
 constexpr uint32_t kShTileBytes = 2u * kShBlock;      // 128 x 128 bf16
-constexpr int kShStages = 2;
-constexpr int kShThreads = 384;                       // utility warpgroup (producer, MMA, 2 idle) + 2 softmax warpgroups
+constexpr int kKStages = 2;                           // K tiles in flight (each ring has its own producer warp)
+constexpr int kVStages = 2;
+constexpr int kShThreads = 384;                       // utility warpgroup (K producer, MMA, V producer, 1 idle) + 2 softmax warpgroups
 // Registers per thread after the warpgroups have re-divided the block's allocation (384 x 168): the
 // utility warps need few, the softmax threads hold a 128-float accumulator.  4 x 32 x 40 + 8 x 32 x 232
 // = 64512 registers, and per SM sub-partition 1 utility + 2 softmax warps = 16128 of its 16384.
@@ -50,10 +51,10 @@ constexpr uint32_t kTmemCols = 512;                   // S0 S1 O0 O1, 128 fp32 c
 
 // shared-memory layout (offsets from a 1024-byte aligned base)
 constexpr uint32_t kOffQ = 0;
-constexpr uint32_t kOffK = kOffQ + kShTileBytes;
-constexpr uint32_t kOffV = kOffK + kShStages * kShTileBytes;
-constexpr uint32_t kOffP = kOffV + kShStages * kShTileBytes;
-constexpr uint32_t kOffBar = kOffP + 2 * kShTileBytes;
+constexpr uint32_t kOffP = kOffQ + kShTileBytes;       // two P buffers, one per softmax warpgroup; 64 KB scratch at a unit's end
+constexpr uint32_t kOffK = kOffP + 2 * kShTileBytes;
+constexpr uint32_t kOffV = kOffK + kKStages * kShTileBytes;
+constexpr uint32_t kOffBar = kOffV + kVStages * kShTileBytes;
 constexpr uint32_t kOffMisc = kOffBar + 32 * 8;        // room for 32 barriers (22 used); then: tmem address, abort flag, unit flag
 constexpr uint32_t kOffFlags = kOffMisc + 16;          // one word per reader: "merge this row group"
 constexpr uint32_t kOffComb = kOffFlags + 128 * 4;     // running maximum and sum of the second warpgroup's rows
@@ -64,10 +65,10 @@ static_assert(kShSmemBytes <= 232448, "shared memory budget of one sm_100 block 
 enum Bar : int {
     kBarKFull = 0,   // [2] TMA -> MMA
     kBarKEmpty = 2,  // [2] MMA (commit) -> TMA
-    kBarVFull = 4,
-    kBarVEmpty = 6,
+    kBarVFull = 4,   // [2]
+    kBarVEmpty = 6,  // [2]
     kBarSFull = 8,   // [2] MMA (commit) -> softmax
-    kBarSFree = 10,  // [2] softmax -> MMA          (4 arrivals: one per softmax warp)
+    kBarSFree = 10,  // [2] softmax -> MMA          (4 arrivals: one per warp of the warpgroup)
     kBarPReady = 12, // [2] softmax -> MMA          (4 arrivals)
     kBarPFree = 14,  // [2] MMA (commit) -> softmax
     kBarOFull = 16,  // [2] MMA (commit) -> softmax
@@ -156,17 +157,19 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
     pdl_launch_dependents();
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < kKStages; ++i) {
             mbar_init(bar(kBarKFull + i), 1);
             mbar_init(bar(kBarKEmpty + i), 1);
+        }
+        for (int i = 0; i < 2; ++i) {
             mbar_init(bar(kBarVFull + i), 1);
             mbar_init(bar(kBarVEmpty + i), 1);
             mbar_init(bar(kBarSFull + i), 1);
             mbar_init(bar(kBarSFree + i), 4);
-            mbar_init(bar(kBarPReady + i), 4);
-            mbar_init(bar(kBarPFree + i), 1);
             mbar_init(bar(kBarOFull + i), 1);
             mbar_init(bar(kBarOFree + i), 4);
+            mbar_init(bar(kBarPReady + i), 4);
+            mbar_init(bar(kBarPFree + i), 1);
         }
         mbar_init(bar(kBarQReady), 8);
         mbar_init(bar(kBarDrain), 1);
@@ -185,55 +188,51 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
-    // Shared tiles are whole tiles of stored Cartridges, which no kernel writes; the queries, the
-    // partial slots and the tickets may still be in use by the kernels before this one.
-    if (warp >= 4) pdl_wait();
+    // Shared tiles are whole tiles of stored Cartridges, which no kernel writes, and the plan is in place
+    // before any of these kernels starts; the queries, the partial slots and the tickets may still be in
+    // use by the kernels before this one: the softmax warps wait for those before they read a query.
     const uint32_t unit_begin = p.unit_cta_begin[blockIdx.x];
     const uint32_t unit_end = p.unit_cta_begin[blockIdx.x + 1];
 
     if (warp < 4) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsUtility));
-        if (warp == 0) {
-            // ================= producer ===================================================================
+        if (warp == 0 || warp == 2) {
+            // ================= producers: warp 0 feeds the K ring, warp 2 the V ring ========================
+            // (separate threads, so that a K tile is requested the moment its stage is free, whatever the
+            //  V ring is waiting for)
             if (lane == 0) {
+                const bool is_v = warp == 2;
+                const int full0 = is_v ? kBarVFull : kBarKFull, empty0 = is_v ? kBarVEmpty : kBarKEmpty;
+                const uint32_t ring = base + (is_v ? kOffV : kOffK);
+                const uint32_t nst = is_v ? (uint32_t)kVStages : (uint32_t)kKStages;
                 asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap)) : "memory");
                 uint32_t tt = 0;
                 bool ok = true;
                 for (uint32_t ui = unit_begin; ui < unit_end && ok; ++ui) {
                     const cart_shared_unit u = p.units[ui];
-                    const uint32_t k_row = u.k_row + (uint32_t)p.layer * u.layer_stride;
-                    const uint32_t v_row = u.v_row + (uint32_t)p.layer * u.layer_stride;
+                    const uint32_t row0 = (is_v ? u.v_row : u.k_row) + (uint32_t)p.layer * u.layer_stride;
                     for (uint32_t t = 0; t < u.n_tiles; ++t, ++tt) {
-                        const int st = (int)(tt & 1u);
-                        const uint32_t par = (tt >> 1) & 1u;
-                        const int32_t yk = (int32_t)(k_row + t * kShTile), yv = (int32_t)(v_row + t * kShTile);
-                        ok = mbar_wait(bar(kBarKEmpty + st), par ^ 1u, abort_flag, p.status, kStatusTimeoutProducer);
+                        const int st = (int)(tt % nst);
+                        const uint32_t par = (tt / nst) & 1u;
+                        const int32_t y = (int32_t)(row0 + t * kShTile);
+                        ok = mbar_wait(bar(empty0 + st), par ^ 1u, abort_flag, p.status, kStatusTimeoutProducer);
                         if (!ok) break;
-                        const uint32_t kdst = base + kOffK + (uint32_t)st * kShTileBytes;
-                        mbar_expect_tx(bar(kBarKFull + st), kShTileBytes);
+                        const uint32_t dst = ring + (uint32_t)st * kShTileBytes;
+                        mbar_expect_tx(bar(full0 + st), kShTileBytes);
                         // a block of the tile = 128 rows x 64 dims = two boxes of 64 rows
-                        tma_load_2d(kdst, &tmap, 0, yk, bar(kBarKFull + st));
-                        tma_load_2d(kdst + kShBlock / 2, &tmap, 0, yk + 64, bar(kBarKFull + st));
-                        tma_load_2d(kdst + kShBlock, &tmap, 64, yk, bar(kBarKFull + st));
-                        tma_load_2d(kdst + kShBlock + kShBlock / 2, &tmap, 64, yk + 64, bar(kBarKFull + st));
-                        ok = mbar_wait(bar(kBarVEmpty + st), par ^ 1u, abort_flag, p.status, kStatusTimeoutProducer);
-                        if (!ok) break;
-                        const uint32_t vdst = base + kOffV + (uint32_t)st * kShTileBytes;
-                        mbar_expect_tx(bar(kBarVFull + st), kShTileBytes);
-                        tma_load_2d(vdst, &tmap, 0, yv, bar(kBarVFull + st));
-                        tma_load_2d(vdst + kShBlock / 2, &tmap, 0, yv + 64, bar(kBarVFull + st));
-                        tma_load_2d(vdst + kShBlock, &tmap, 64, yv, bar(kBarVFull + st));
-                        tma_load_2d(vdst + kShBlock + kShBlock / 2, &tmap, 64, yv + 64, bar(kBarVFull + st));
+                        tma_load_2d(dst, &tmap, 0, y, bar(full0 + st));
+                        tma_load_2d(dst + kShBlock / 2, &tmap, 0, y + 64, bar(full0 + st));
+                        tma_load_2d(dst + kShBlock, &tmap, 64, y, bar(full0 + st));
+                        tma_load_2d(dst + kShBlock + kShBlock / 2, &tmap, 64, y + 64, bar(full0 + st));
                     }
                 }
                 if (!ok) {
                     // gave up: wait (bounded) for the copies still in flight before the block leaves
-                    for (uint32_t u2 = (tt > 2u ? tt - 2u : 0u); u2 <= tt; ++u2) {
-                        const int st = (int)(u2 & 1u);
-                        const uint32_t par = (u2 >> 1) & 1u;
+                    for (uint32_t u2 = (tt > nst ? tt - nst : 0u); u2 <= tt; ++u2) {
+                        const int st = (int)(u2 % nst);
+                        const uint32_t par = (u2 / nst) & 1u;
                         const uint64_t t0 = global_timer_ns();
-                        while (!mbar_try_wait(bar(kBarKFull + st), par) && global_timer_ns() - t0 < kWaitLimitNs) {}
-                        while (!mbar_try_wait(bar(kBarVFull + st), par) && global_timer_ns() - t0 < kWaitLimitNs) {}
+                        while (!mbar_try_wait(bar(full0 + st), par) && global_timer_ns() - t0 < kWaitLimitNs) {}
                     }
                 }
             }
@@ -249,10 +248,11 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                 auto issue_s = [&](uint32_t tt) -> bool {
                     const int st = (int)(tt & 1u);
                     const uint32_t par = (tt >> 1) & 1u;
-                    if (!mbar_wait(bar(kBarKFull + st), par, abort_flag, p.status, kStatusTimeoutMma)) return false;
+                    const uint32_t kst = tt % (uint32_t)kKStages, kpar = (tt / (uint32_t)kKStages) & 1u;
+                    if (!mbar_wait(bar(kBarKFull + (int)kst), kpar, abort_flag, p.status, kStatusTimeoutMma)) return false;
                     if (!mbar_wait(bar(kBarSFree + st), par ^ 1u, abort_flag, p.status, kStatusTimeoutMma)) return false;
                     tc_fence_after();
-                    const uint32_t k_lo = base + kOffK + (uint32_t)st * kShTileBytes;
+                    const uint32_t k_lo = base + kOffK + kst * kShTileBytes;
     #pragma unroll
                     for (uint32_t k = 0; k < 8; ++k) {  // 16 dims per instruction
                         const uint32_t off = (k >> 2) * kShBlock + (k & 3u) * 32u;
@@ -260,7 +260,7 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                                   kIdescS, k);
                     }
                     umma_commit(bar(kBarSFull + st));
-                    umma_commit(bar(kBarKEmpty + st));
+                    umma_commit(bar(kBarKEmpty + (int)kst));
                     return true;
                 };
                 // O(tt) = P V into O buffer tt & 1
@@ -319,6 +319,7 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
         float *comb_ml = reinterpret_cast<float *>(smem + kOffComb); // [2][128 rows]
         uint32_t tt0 = 0;
         bool alive = true;
+        bool waited = false;  // for the kernels before this one on the stream
         float o_acc[128];
         // the warp's lanes must stay together (the tensor-memory loads are warp-wide): a wait fails for
         // all of them or for none
@@ -333,23 +334,30 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
             const cart_shared_unit u = p.units[ui];
             const int i_reader = row / G, h = row - i_reader * G;
             const bool valid = (uint32_t)i_reader < u.n_readers;
-            uint32_t entry = 0, batch = 0;
+            uint32_t entry = 0, batch = 0, slot = 0;
             if (valid) {
                 entry = u.reader_begin + (uint32_t)i_reader;
                 batch = p.readers[entry];
+                slot = p.reader_slot[(size_t)entry * p.n_kv_heads + u.kv_head] + u.chunk;  // where this row's partial goes
             }
             // ---- this row's query into shared memory, in the swizzled K-major operand layout; each
             //      warpgroup copies one 64-dim half -------------------------------------------------
+            if (!waited) {
+                pdl_wait();
+                waited = true;
+            }
             {
                 const uint4 *src = reinterpret_cast<const uint4 *>(
                     q + ((size_t)batch * p.n_q_heads + (size_t)u.kv_head * G + h) * kHeadDim) + 8 * wg;
                 const uint32_t qrow = base + kOffQ + (uint32_t)wg * kShBlock + (uint32_t)row * 128u;
+                uint4 v[8];
+#pragma unroll
+                for (uint32_t c = 0; c < 8; ++c) v[c] = valid ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);  // all in flight
 #pragma unroll
                 for (uint32_t c = 0; c < 8; ++c) {
-                    uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                    if (valid) v = __ldg(src + c);
                     const uint32_t a = qrow + ((c ^ swz) << 4);
-                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(v[c].x), "r"(v[c].y), "r"(v[c].z),
+                                 "r"(v[c].w)
                                  : "memory");
                 }
                 fence_async_smem();
@@ -399,6 +407,12 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                 const float m_new = fmaxf(m_run, mx * p.scale_log2);
                 const float alpha = fast_exp2(m_run - m_new);  // 0 on the first tile
                 m_run = m_new;
+                // this warpgroup's previous tile has been multiplied by now: fold its O in, which also frees
+                // the O buffer for the product of this tile
+                if (have_prev) {
+                    alive = take_o(prev_tt, alpha_prev);
+                    if (!alive) break;
+                }
                 // pass 2: probabilities, as bf16, into the P buffer (free once this warpgroup's previous
                 // tile has been multiplied)
                 alive = warp_wait(bar(kBarPFree + wg), par ^ 1u);
@@ -433,11 +447,6 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                     mbar_arrive(bar(kBarSFree + wg));
                     mbar_arrive(bar(kBarPReady + wg));
                 }
-                // this warpgroup's previous tile has long been multiplied: fold its O in
-                if (have_prev) {
-                    alive = take_o(prev_tt, alpha_prev);
-                    if (!alive) break;
-                }
                 alpha_prev = alpha;
                 prev_tt = tt;
                 have_prev = true;
@@ -451,7 +460,7 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
             // q ^ (r & 31), which keeps both the row-per-lane and the quad-per-lane accesses free of bank
             // conflicts.
             softmax_bar_both();
-            uint8_t *comb = smem + kOffP;
+            uint8_t *comb = smem + kOffP;   // the two P buffers: 64 KB
             const uint32_t rsw = (uint32_t)(row & 31);
             if (wg == 1) {
 #pragma unroll
@@ -478,7 +487,6 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                 }
                 uint32_t dst_row = 0xFFFFFFFFu;  // row of part_o ([slot][G] flattened) this query row goes to
                 if (alive && valid) {
-                    const uint32_t slot = p.reader_slot[(size_t)entry * p.n_kv_heads + u.kv_head] + u.chunk;
                     dst_row = slot * (uint32_t)G + (uint32_t)h;
                     p.part_lse2[(size_t)slot * kMaxGroup + h] = M + log2f(l);
                 }
@@ -486,12 +494,17 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
             }
             softmax_bar_both();
             // both warpgroups copy the normalised rows out, a warp writing one 512-byte row per instruction
-            for (uint32_t item = (uint32_t)(wg * kSoftmaxThreads + tid); item < 128u * 32u; item += 2u * kSoftmaxThreads) {
-                const uint32_t r = item >> 5, q4 = item & 31u;
-                const uint32_t dst_row = flags[r];
-                if (dst_row == 0xFFFFFFFFu) continue;
-                const float4 v = *reinterpret_cast<const float4 *>(comb + (size_t)r * 512 + ((q4 ^ (r & 31u)) << 4));
-                reinterpret_cast<float4 *>(p.part_o + (size_t)dst_row * kHeadDim)[q4] = v;
+            {
+                const uint32_t *dst_rows = reinterpret_cast<const uint32_t *>(smem + kOffFlags);
+                const uint32_t q4 = (uint32_t)lane;                       // a warp = one row per pass
+                const uint32_t r0 = (uint32_t)(wg * 4 + (warp & 3));      // 8 softmax warps, 16 rows each
+#pragma unroll 4
+                for (uint32_t r = r0; r < 128u; r += 8u) {
+                    const uint32_t dst_row = dst_rows[r];
+                    if (dst_row == 0xFFFFFFFFu) continue;
+                    const float4 v = *reinterpret_cast<const float4 *>(comb + (size_t)r * 512 + ((q4 ^ (r & 31u)) << 4));
+                    reinterpret_cast<float4 *>(p.part_o + (size_t)dst_row * kHeadDim)[q4] = v;
+                }
             }
             if (p.tickets) __threadfence();  // publish the partials before the tickets
             softmax_bar_both();
@@ -519,7 +532,7 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                     const uint32_t f = flags[r];
                     if (f == 0) continue;
                     __threadfence();
-                    merge_row_group(p.merges[f - 1u], G, p.part_o, p.part_lse2, p.out, p.lse, tid, kSoftmaxThreads);
+                    merge_row_group<1, 4>(p.merges[f - 1u], G, p.part_o, p.part_lse2, p.out, p.lse, tid, kSoftmaxThreads);
                     if (tid == 0) p.tickets[f - 1u] = 0;  // ready for the next launch
                 }
             }
