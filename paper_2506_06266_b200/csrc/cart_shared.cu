@@ -253,11 +253,14 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                     if (!mbar_wait(bar(kBarSFree + st), par ^ 1u, abort_flag, p.status, kStatusTimeoutMma)) return false;
                     tc_fence_after();
                     const uint32_t k_lo = base + kOffK + kst * kShTileBytes;
+                    // the operands' descriptors differ from step to step only in the start address field
+                    // (units of 16 bytes): the next 16 dims are 32 bytes on, the second 64-dim block kShBlock on
+                    const uint64_t a0 = umma_desc(q_lo, 16, 1024), b0 = umma_desc(k_lo, 16, 1024);
+                    const uint32_t d_s = tmem + (uint32_t)st * 128u;
     #pragma unroll
                     for (uint32_t k = 0; k < 8; ++k) {  // 16 dims per instruction
-                        const uint32_t off = (k >> 2) * kShBlock + (k & 3u) * 32u;
-                        umma_bf16(tmem + (uint32_t)st * 128u, umma_desc(q_lo + off, 16, 1024), umma_desc(k_lo + off, 16, 1024),
-                                  kIdescS, k);
+                        const uint64_t off16 = (uint64_t)(((k >> 2) * kShBlock + (k & 3u) * 32u) >> 4);
+                        umma_bf16(d_s, a0 + off16, b0 + off16, kIdescS, k);
                     }
                     umma_commit(bar(kBarSFull + st));
                     umma_commit(bar(kBarKEmpty + (int)kst));
@@ -273,13 +276,14 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                     tc_fence_after();
                     const uint32_t p_lo = base + kOffP + (uint32_t)st * kShTileBytes;
                     const uint32_t v_lo = base + kOffV + (uint32_t)st * kShTileBytes;
+                    // P: K-major, as Q above.  V: tokens are rows of 128 bytes (8-token groups 1024 bytes apart,
+                    // 16 tokens = 2048 bytes per step); the two 64-dim blocks of the tile are kShBlock bytes apart
+                    const uint64_t a0 = umma_desc(p_lo, 16, 1024), b0 = umma_desc(v_lo, kShBlock, 1024);
+                    const uint32_t d_o = tmem + 256u + (uint32_t)st * 128u;
     #pragma unroll
                     for (uint32_t k = 0; k < 8; ++k) {  // 16 tokens per instruction
-                        const uint64_t a = umma_desc(p_lo + (k >> 2) * kShBlock + (k & 3u) * 32u, 16, 1024);
-                        // V: tokens are rows of 128 bytes (8-token groups 1024 bytes apart); the two 64-dim
-                        // blocks of the tile are kShBlock bytes apart
-                        const uint64_t b = umma_desc(v_lo + k * 16u * 128u, kShBlock, 1024);
-                        umma_bf16(tmem + 256u + (uint32_t)st * 128u, a, b, kIdescPV, k);
+                        const uint64_t a_off16 = (uint64_t)(((k >> 2) * kShBlock + (k & 3u) * 32u) >> 4);
+                        umma_bf16(d_o, a0 + a_off16, b0 + (uint64_t)(k * 128u), kIdescPV, k);
                     }
                     umma_commit(bar(kBarOFull + st));
                     umma_commit(bar(kBarVEmpty + st));
