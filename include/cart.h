@@ -157,6 +157,18 @@ CART_API cart_status cart_decode_step(cart_ctx *ctx, int32_t layer, const cart_r
                              const void *k_new /*device*/, const void *v_new /*device*/, const void *q /*device*/,
                              void *out /*device*/, float *lse /*device or NULL*/, void *stream);
 
+/* Sec. 2.3, prefill of the user's message over a Cartridge: attention for the LAST n_new tokens of
+ * request req's suffix in `layer` (append them first with cart_extend_kv).  Row i of q (device bf16
+ * [n_new][n_q_heads][128], token-major as the projection produces it) is the query of the i-th new
+ * token and attends, per Eq. 1 with its causal sum over j <= i, to the request's Cartridge(s), the
+ * suffix tokens before the new ones and the new tokens 0 .. i.  out, lse as in cart_decode_attention,
+ * with n_new rows.  The Cartridge(s) and the old part of the suffix are read once for all rows
+ * (tensor-core kernel) when n_new reaches the sharing threshold.  n_new <= max_requests.
+ * Errors: INVALID_ARG (also: the suffix holds fewer than n_new tokens), BAD_HANDLE, CAPACITY, CUDA. */
+CART_API cart_status cart_prefill_attention(cart_ctx *ctx, int32_t layer, cart_req req, const void *q /*device*/,
+                                   int32_t n_new, void *out /*device*/, float *lse /*device or NULL*/,
+                                   void *stream);
+
 /* Sharing policy.  When at least min_readers requests of a decode batch attend to the same stored
  * Cartridge (one Cartridge serving many users, Sec. 1 and Sec. 3.3; pool members composed by many
  * requests, Sec. 5.4), cart_decode_attention reads each of its K/V tiles once for up to 128 query

@@ -27,7 +27,7 @@ STATUS_NAMES = ["CART_OK", "CART_ERR_INVALID_ARG", "CART_ERR_SHAPE", "CART_ERR_B
 # every symbol include/cart.h and include/cart_plan.h declare
 EXPORTS = ["cart_scratch_bytes", "cart_create", "cart_destroy", "cart_register_cartridge",
            "cart_compose", "cart_release_cartridge", "cart_request_open", "cart_request_close",
-           "cart_append_kv", "cart_extend_kv", "cart_decode_attention", "cart_decode_step", "cart_suffix_len",
+           "cart_append_kv", "cart_extend_kv", "cart_decode_attention", "cart_decode_step", "cart_prefill_attention", "cart_suffix_len",
            "cart_kv_bytes", "cart_sync_status", "cart_set_timing", "cart_get_timing",
            "cart_set_share_min_readers", "cart_set_piece_cost", "cart_plan_build_shared",
            "cart_decode_attention_static", "cart_launch_count", "cart_status_string",
@@ -122,6 +122,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.cart_extend_kv.argtypes = [vp, i32, i32, vp, vp, i32, vp]
     lib.cart_decode_attention.argtypes = [vp, i32, i32p, i32, vp, vp, vp, vp]
     lib.cart_decode_step.argtypes = [vp, i32, i32p, i32, vp, vp, vp, vp, vp, vp]
+    lib.cart_prefill_attention.argtypes = [vp, i32, i32, vp, i32, vp, vp, vp]
     lib.cart_suffix_len.argtypes = [vp, i32, i32, i32p]
     lib.cart_kv_bytes.argtypes = [vp, i32, u64p, u64p]
     lib.cart_sync_status.argtypes = [vp, vp]
@@ -266,6 +267,11 @@ def cart_decode_step(ctx: int, layer: int, reqs, k_new, v_new, q, out, lse=None,
     arr, n = _reqs(reqs)
     _check(load_library().cart_decode_step(ctx, int(layer), arr, n, _ptr(k_new), _ptr(v_new), _ptr(q), _ptr(out),
                                            _ptr(lse), _stream(stream)), "cart_decode_step", ctx)
+
+
+def cart_prefill_attention(ctx: int, layer: int, req: int, q, n_new: int, out, lse=None, stream=None) -> None:
+    _check(load_library().cart_prefill_attention(ctx, int(layer), int(req), _ptr(q), int(n_new), _ptr(out), _ptr(lse),
+                                                 _stream(stream)), "cart_prefill_attention", ctx)
 
 
 def cart_suffix_len(ctx: int, req: int, layer: int) -> int:

@@ -51,7 +51,7 @@ ScratchLayout scratch_layout(const cart_config &c)
     // partial slots: stream pieces (one per row group with a shared part, two per block boundary) plus
     // the chunks of shared segments (the planner keeps them within what is left)
     s.slots_cap = 10 * row_groups + 2 * kMaxCta;
-    s.readers_cap = c.max_requests * parts;
+    s.readers_cap = c.max_requests * (parts + 1);  // + 1: the shared head of a suffix during prefill
     s.units_cap = s.readers_cap * c.n_kv_heads + kMaxCta;
     s.status_off = 0;
     s.tickets_off = kAlign;  // one arrival counter per merge item, zero between launches
@@ -588,9 +588,15 @@ namespace {
 
 // Decode attention for a batch; with k_new / v_new non-null the stream kernel first writes each
 // request's new token at position len - 1 of its suffix (the host lengths already count it).
+// Prefill mode (n_new > 0): reqs[0] is one request, and the batch is its last n_new suffix tokens as
+// n_new query rows; row i attends over the Cartridge(s) and the suffix up to and including its own
+// token (Eq. 1 for the rows of the new block).  The rows are planned like n_new requests that share the
+// Cartridge(s) and the head of the suffix, so those go through the shared-segment kernel.
 cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int32_t n_reqs, const void *q,
-                        void *out, float *lse, const void *k_new, const void *v_new, void *stream)
+                        void *out, float *lse, const void *k_new, const void *v_new, void *stream, int32_t n_new = 0)
 {
+    const bool prefill = n_new > 0;
+    if (prefill) n_reqs = n_new;
     if (!reqs || n_reqs < 1 || !aligned16(q) || !aligned16(out) || (lse && (reinterpret_cast<uintptr_t>(lse) & 3u)))
         return fail(ctx, CART_ERR_INVALID_ARG, "decode: null/misaligned pointer or empty batch");
     if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, CART_ERR_BAD_HANDLE, "decode: layer out of range");
@@ -603,7 +609,17 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
     std::vector<uint32_t> &key = ctx->key_tmp;
     key.clear();
     key.push_back((uint32_t)n_reqs);
-    for (int32_t i = 0; i < n_reqs; ++i) {
+    if (prefill) {
+        Request *r = get_req(ctx, reqs[0]);
+        if (!r) return fail(ctx, CART_ERR_BAD_HANDLE, "prefill: not an open request");
+        if (r->len[(size_t)layer] < n_new)
+            return fail(ctx, CART_ERR_INVALID_ARG, "prefill: the suffix holds %d tokens, fewer than n_new = %d",
+                        r->len[(size_t)layer], n_new);
+        key.push_back(0xFFFFFFFFu);  // no batch of requests starts like this
+        key.push_back((uint32_t)reqs[0]);
+        key.push_back((uint32_t)r->len[(size_t)layer]);
+    }
+    for (int32_t i = 0; i < n_reqs && !prefill; ++i) {
         Request *r = get_req(ctx, reqs[i]);
         if (!r) return fail(ctx, CART_ERR_BAD_HANDLE, "decode: reqs[%d] is not an open request", i);
         const int32_t len = r->len[(size_t)layer];
@@ -633,7 +649,7 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
         sb.clear();
         sb.push_back(0);
         for (int32_t i = 0; i < n_reqs; ++i) {
-            const Request &r = ctx->reqs[(size_t)reqs[i]];
+            const Request &r = ctx->reqs[(size_t)reqs[prefill ? 0 : i]];
             auto push_cart = [&](const Cartridge &c) {
                 cart_plan_seg sg;
                 sg.k_row = (uint32_t)c.k_row;
@@ -648,14 +664,32 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
                 if (c.composed) for (int32_t b : c.parts) push_cart(ctx->carts[(size_t)b]);
                 else push_cart(c);
             }
-            const int32_t len = r.len[(size_t)layer];
-            if (len > 0) {
+            int32_t len = r.len[(size_t)layer];
+            uint32_t first = 0;  // first suffix token of the segment
+            if (prefill) {
+                // row i sees the suffix up to its own token; the part before the new tokens, rounded down
+                // to whole shared tiles, is the same block for every row: a segment of its own
+                const int32_t s_old = len - n_new;
+                len = s_old + i + 1;
+                const int32_t head = s_old / kShareTileTokens * kShareTileTokens;
+                if (head > 0 && ctx->share_min_readers > 0 && n_new >= ctx->share_min_readers) {
+                    cart_plan_seg sg;
+                    sg.k_row = (uint32_t)r.k_row;
+                    sg.v_row = (uint32_t)r.v_row;
+                    sg.head_stride = (uint32_t)r.cap;
+                    sg.layer_stride = (uint32_t)((uint64_t)Hkv * r.cap);
+                    sg.n_tok = (uint32_t)head;
+                    segs.push_back(sg);
+                    first = (uint32_t)head;
+                }
+            }
+            if (len > (int32_t)first) {
                 cart_plan_seg sg;
-                sg.k_row = (uint32_t)r.k_row;
-                sg.v_row = (uint32_t)r.v_row;
+                sg.k_row = (uint32_t)r.k_row + first;
+                sg.v_row = (uint32_t)r.v_row + first;
                 sg.head_stride = (uint32_t)r.cap;
                 sg.layer_stride = (uint32_t)((uint64_t)Hkv * r.cap);
-                sg.n_tok = (uint32_t)len;
+                sg.n_tok = (uint32_t)len - first;
                 segs.push_back(sg);
             }
             sb.push_back((int32_t)segs.size());
@@ -785,6 +819,14 @@ cart_status cart_decode_attention(cart_ctx *ctx, int32_t layer, const cart_req *
 {
     if (!ctx) return CART_ERR_INVALID_ARG;
     return decode_impl(ctx, layer, reqs, n_reqs, q, out, lse, nullptr, nullptr, stream);
+}
+
+cart_status cart_prefill_attention(cart_ctx *ctx, int32_t layer, cart_req req, const void *q, int32_t n_new, void *out,
+                                   float *lse, void *stream)
+{
+    if (!ctx) return CART_ERR_INVALID_ARG;
+    if (n_new < 1) return fail(ctx, CART_ERR_INVALID_ARG, "prefill: n_new < 1");
+    return decode_impl(ctx, layer, &req, 1, q, out, lse, nullptr, nullptr, stream, n_new);
 }
 
 cart_status cart_decode_step(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int32_t n_reqs, const void *k_new,

@@ -1,0 +1,108 @@
+"""GPU parity of cart_prefill_attention: the last n_new suffix tokens of a request as query rows, each
+attending over [Cartridge(s) ; suffix up to its own token].  The oracle computes every row by itself from
+the explicitly truncated cache."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2506_06266_b200 import binding, synth
+
+import cart_harness as H
+
+pytestmark = pytest.mark.gpu
+
+
+def oracle_rows(sess, layer, req, q, n_new):
+    """Eq. 1 for each new token: its own query against the cache truncated after that token."""
+    segs = sess.oc.segments(layer, sess.req_map[req])
+    cart, (ks, vs) = segs[:-1], segs[-1]
+    total = ks.shape[1]
+    per_row = []
+    for i in range(n_new):
+        n = total - n_new + i + 1
+        per_row.append(list(cart) + [(np.ascontiguousarray(ks[:, :n]), np.ascontiguousarray(vs[:, :n]))])
+    return oracle.decode_layer(synth.bits(q), per_row, sess.oc.scale)
+
+
+def prefill(sess, layer, req, q, n_new):
+    out = torch.full_like(q, float("nan"))
+    lse = torch.full(q.shape[:2], float("nan"), dtype=torch.float32, device=q.device)
+    binding.cart_prefill_attention(sess.ctx, layer, req, q, n_new, out, lse)
+    binding.cart_sync_status(sess.ctx)
+    return out, lse
+
+
+def run(Hq, Hkv, p, s_old, n_new, parts=1, layers=2, seed=0):
+    w = synth.Workload("prefill", 600 + seed + p + s_old + n_new, layers, Hq, Hkv, 1, max(p, 1), s_old, s_old,
+                       cartridges="pool" if parts > 1 else ("none" if p == 0 else "private"), pool=parts, compose=parts)
+    sess = H.Session(layers, Hq, Hkv, 64 << 20, max_requests=max(n_new, 4))
+    try:
+        if p == 0:
+            cart = binding.CART_NONE
+        else:
+            cids = [sess.register(*w.cartridge_kv(c, "cuda:0")) for c in range(parts)]
+            cart = cids[0] if parts == 1 else sess.compose(cids)
+        req = sess.open(cart, s_old + n_new)
+        if s_old:
+            sess.extend(req, *w.suffix_kv(0, s_old, "cuda:0"))
+        k_new, v_new = w.suffix_kv(1, n_new, "cuda:0")          # the message's tokens, [L][n_new][Hkv][D]
+        sess.extend(req, k_new, v_new)
+        for layer in range(layers):
+            q = synth.normal_bf16((n_new, Hq, 128), 700 + seed + layer, "cuda:0")
+            out, lse = prefill(sess, layer, req, q, n_new)
+            ro, rl = oracle_rows(sess, layer, req, q, n_new)
+            H.assert_close(out, lse, ro, rl, "prefill p=%d s_old=%d n_new=%d layer %d" % (p, s_old, n_new, layer))
+            # the last row is what a decode call computes for the request
+            o1, l1 = sess.decode(layer, [req], q[-1:])
+            assert float((o1.float() - out[-1:].float()).abs().max()) < 4e-3
+            assert float((l1 - lse[-1:]).abs().max()) < 2e-4
+    finally:
+        sess.close()
+
+
+@pytest.mark.parametrize("s_old,n_new", [(0, 1), (0, 3), (5, 4), (130, 37), (260, 64), (127, 129), (300, 5)])
+def test_prefill_over_a_private_cartridge(s_old, n_new):
+    run(32, 8, 300, s_old, n_new, seed=1)
+
+
+@pytest.mark.parametrize("Hq,Hkv", [(24, 8), (8, 8), (8, 1)])
+def test_prefill_group_sizes(Hq, Hkv):
+    run(Hq, Hkv, 520, 140, 33, seed=2)
+
+
+def test_prefill_without_a_cartridge_is_causal_self_attention():
+    run(32, 8, 0, 0, 70, layers=1, seed=3)
+
+
+def test_prefill_over_composed_cartridges():
+    run(32, 8, 256, 64, 48, parts=3, seed=4)
+
+
+def test_prefill_many_rows_long_cartridge():
+    run(32, 8, 4096, 0, 256, layers=1, seed=5)
+
+
+def test_prefill_errors():
+    sess = H.Session(1, 32, 8, 8 << 20, max_requests=8)
+    try:
+        w = synth.Workload("pe", 801, 1, 32, 8, 1, 64, 6, 6)
+        req = sess.open(sess.register(*w.cartridge_kv(0, "cuda:0")), 64)
+        sess.extend(req, *w.suffix_kv(0, 6, "cuda:0"))
+        q = torch.zeros(16, 32, 128, dtype=torch.bfloat16, device="cuda:0")
+        out = torch.empty_like(q)
+        for n_new, status in [(7, binding.CART_ERR_INVALID_ARG), (0, binding.CART_ERR_INVALID_ARG)]:
+            with pytest.raises(binding.CartError) as ei:
+                binding.cart_prefill_attention(sess.ctx, 0, req, q, n_new, out)
+            assert ei.value.status == status
+        big = torch.zeros(10, 8, 128, dtype=torch.bfloat16, device="cuda:0")
+        binding.cart_extend_kv(sess.ctx, 0, req, big, big, 10)
+        with pytest.raises(binding.CartError) as ei:
+            binding.cart_prefill_attention(sess.ctx, 0, req, q, 9, out)       # more rows than max_requests
+        assert ei.value.status == binding.CART_ERR_CAPACITY
+        with pytest.raises(binding.CartError) as ei:
+            binding.cart_prefill_attention(sess.ctx, 0, req + 1, q, 2, out)
+        assert ei.value.status == binding.CART_ERR_BAD_HANDLE
+        binding.cart_sync_status(sess.ctx)
+    finally:
+        sess.close()
