@@ -7,23 +7,24 @@
 // for up to 128 query rows at once (row i * G + h = head h of the M-tile's i-th reader) on the
 // tcgen05 tensor cores, so the tile is fetched once per 128 rows instead of once per request:
 //
-//   producer warps  TMA loads of K tiles (warp 0) and V tiles (warp 2), 128 tokens x 128 dims, 128-byte
-//                   swizzle, each into its own two-stage ring, completion on mbarriers
-//   MMA warp        one thread issues  S = Q K^T  (128 x 128 x 128, accumulator in tensor memory)
-//                   and  O_t = P V  (fresh accumulator per tile); tcgen05.commit signals mbarriers
-//   2 x 4 softmax  two warpgroups take alternate tiles (warpgroup w owns S, P and O buffer w).  Thread r
-//   warps           of a warpgroup owns query row r: reads S from tensor memory, keeps the running
-//                   maximum and sum of an online softmax over its warpgroup's tiles in fp32, writes
-//                   P = 2^(s - m) as bf16 into shared memory (the A operand of the second product),
-//                   then adds the finished O_t of its previous tile to its fp32 register accumulator,
-//                   rescaled to the new maximum.  At the end of a unit the two warpgroups' states are
-//                   combined through shared memory.
+//   producer warps  TMA loads of K tiles (warp 0, three stages) and V tiles (warp 2, two stages), 128 tokens
+//                   x 128 dims, 128-byte swizzle, completion on mbarriers
+//   MMA warp        one thread issues  S = Q K^T  (128 x 128 x 128, both operands from shared memory,
+//                   accumulator in tensor memory) and  O_t = P V  (A operand P from tensor memory, V from
+//                   shared memory, fresh accumulator per tile); tcgen05.commit signals mbarriers
+//   2 x 4 softmax  two warpgroups take alternate tiles (warpgroup w owns S and O buffer w).  Thread r of a
+//   warps           warpgroup owns query row r: reads S from tensor memory (two loads in flight), keeps the
+//                   running maximum and sum of an online softmax over its warpgroup's tiles in fp32,
+//                   writes P = 2^(s - m) as bf16 pairs back over the first half of the S buffer
+//                   (tcgen05.st), and adds the finished O_t of its previous tile to its fp32 register
+//                   accumulator, rescaled to the new maximum.  At the end of a unit the two warpgroups'
+//                   states are combined through shared memory.
 //
-// S and O_t are double-buffered in tensor memory (4 x 128 columns), so the products of tile t+1 run
-// while the softmax of tile t does.  At the end of a unit every row is written as a normalised fp32
-// partial (o, lse); the partials of a (request, KV head) row group are merged by log-sum-exp either by
-// the block that delivers the last one -- this kernel's or the stream kernel's -- or, when the batch
-// has more split row groups than blocks, by a merge kernel that runs afterwards.
+// S (with P in it) and O_t are double-buffered in tensor memory (4 x 128 columns), so the products of
+// tile t+1 run while the softmax of tile t does.  At the end of a unit every row is written as a
+// normalised fp32 partial (o, lse); the partials of a (request, KV head) row group are merged by
+// log-sum-exp either by the block that delivers the last one -- this kernel's or the stream kernel's --
+// or, when the batch has more split row groups than blocks, by a merge kernel that runs afterwards.
 //
 // Every wait is bounded; on expiry the block raises a flag in the device status word, stops issuing
 // work, waits (bounded) for what is in flight, frees its tensor memory and returns.
@@ -38,7 +39,7 @@ namespace {
 constexpr int kShTile = kShareTileTokens;             // tokens per tile = N of the score product
 constexpr uint32_t kShBlock = 128u * 128u;            // 128 rows x 128 bytes: one swizzled block (64 bf16 wide)
 constexpr uint32_t kShTileBytes = 2u * kShBlock;      // 128 x 128 bf16
-constexpr int kKStages = 2;                           // K tiles in flight (each ring has its own producer warp)
+constexpr int kKStages = 3;                           // K tiles in flight (each ring has its own producer warp)
 constexpr int kVStages = 2;
 constexpr int kShThreads = 384;                       // utility warpgroup (K producer, MMA, V producer, 1 idle) + 2 softmax warpgroups
 // Registers per thread after the warpgroups have re-divided the block's allocation (384 x 168): the
@@ -51,8 +52,8 @@ constexpr uint32_t kTmemCols = 512;                   // S0 S1 O0 O1, 128 fp32 c
 
 // shared-memory layout (offsets from a 1024-byte aligned base)
 constexpr uint32_t kOffQ = 0;
-constexpr uint32_t kOffP = kOffQ + kShTileBytes;       // two P buffers, one per softmax warpgroup; 64 KB scratch at a unit's end
-constexpr uint32_t kOffK = kOffP + 2 * kShTileBytes;
+constexpr uint32_t kOffX = kOffQ + kShTileBytes;       // with Q: the 64 KB scratch of a unit's end
+constexpr uint32_t kOffK = kOffX + kShTileBytes;
 constexpr uint32_t kOffV = kOffK + kKStages * kShTileBytes;
 constexpr uint32_t kOffBar = kOffV + kVStages * kShTileBytes;
 constexpr uint32_t kOffMisc = kOffBar + 32 * 8;        // room for 32 barriers (22 used); then: tmem address, abort flag, unit flag
@@ -63,19 +64,20 @@ constexpr uint32_t kShSmemBytes = kShSmemUsed + 1024;  // slack to align the bas
 static_assert(kShSmemBytes <= 232448, "shared memory budget of one sm_100 block exceeded");
 
 enum Bar : int {
-    kBarKFull = 0,   // [2] TMA -> MMA
-    kBarKEmpty = 2,  // [2] MMA (commit) -> TMA
-    kBarVFull = 4,   // [2]
-    kBarVEmpty = 6,  // [2]
-    kBarSFull = 8,   // [2] MMA (commit) -> softmax
-    kBarSFree = 10,  // [2] softmax -> MMA          (4 arrivals: one per warp of the warpgroup)
-    kBarPReady = 12, // [2] softmax -> MMA          (4 arrivals)
-    kBarPFree = 14,  // [2] MMA (commit) -> softmax
+    kBarKFull = 0,   // [kKStages] TMA -> MMA
+    kBarKEmpty = 3,  // [kKStages] MMA (commit) -> TMA
+    kBarVFull = 6,   // [kVStages]
+    kBarVEmpty = 8,  // [kVStages]
+    kBarSFull = 10,  // [2] MMA (commit) -> softmax
+    kBarSFree = 12,  // [2] MMA (commit of P V: the probabilities live in the S buffer) -> MMA
+    kBarPReady = 14, // [2] softmax -> MMA          (4 arrivals: one per warp of the warpgroup)
     kBarOFull = 16,  // [2] MMA (commit) -> softmax
     kBarOFree = 18,  // [2] softmax -> MMA          (4 arrivals)
     kBarQReady = 20, // softmax -> MMA              (8 arrivals: every softmax warp)
     kBarDrain = 21,  // MMA (commit) -> MMA, on the way out
 };
+static_assert(kBarKEmpty - kBarKFull >= kKStages && kBarVFull - kBarKEmpty >= kKStages &&
+              kBarVEmpty - kBarVFull >= kVStages && kBarSFull - kBarVEmpty >= kVStages, "barrier indices overlap");
 
 // ---- tcgen05 wrappers ---------------------------------------------------------------------------
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -108,27 +110,58 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint
         "}\n" ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// The same with the A operand in tensor memory (lane = row, 8 columns of bf16 pairs per 16-wide step).
+__device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                             uint32_t accumulate)
+{
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n"
+        "}\n" ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
 __device__ __forceinline__ void umma_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-// 32 consecutive fp32 columns of this thread's tensor-memory lane; waits for the data.
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32])
+// Writes 16 consecutive 32-bit columns of this thread's tensor-memory lane.
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&w)[16])
 {
-    uint32_t r[32];
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(taddr),
+        "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]), "r"(w[8]), "r"(w[9]),
+        "r"(w[10]), "r"(w[11]), "r"(w[12]), "r"(w[13]), "r"(w[14]), "r"(w[15])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// 32 consecutive 32-bit columns of this thread's tensor-memory lane, in two steps, so that several
+// loads can be in flight and arithmetic can run under them: tmem_ld32_issue starts a load, tmem_ld_wait waits for all loads issued so far; the registers named
+// in the wait are only then valid (naming them keeps the compiler from reading them earlier).
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32])
+{
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
         "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,"
-        "%29,%30,%31}, [%32];\n"
-        "tcgen05.wait::ld.sync.aligned;"
+        "%29,%30,%31}, [%32];"
         : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
           "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
           "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
           "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr)
         : "memory");
-#pragma unroll
-    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32])
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                   "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+                   "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+                   "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+                 :
+                 : "memory");
 }
 __device__ __forceinline__ void softmax_bar()  // the first softmax warpgroup
 {
@@ -165,11 +198,10 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
             mbar_init(bar(kBarVFull + i), 1);
             mbar_init(bar(kBarVEmpty + i), 1);
             mbar_init(bar(kBarSFull + i), 1);
-            mbar_init(bar(kBarSFree + i), 4);
+            mbar_init(bar(kBarSFree + i), 1);
             mbar_init(bar(kBarOFull + i), 1);
             mbar_init(bar(kBarOFree + i), 4);
             mbar_init(bar(kBarPReady + i), 4);
-            mbar_init(bar(kBarPFree + i), 1);
         }
         mbar_init(bar(kBarQReady), 8);
         mbar_init(bar(kBarDrain), 1);
@@ -274,20 +306,20 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                     if (!mbar_wait(bar(kBarOFree + st), par ^ 1u, abort_flag, p.status, kStatusTimeoutMma)) return false;
                     if (!mbar_wait(bar(kBarPReady + st), par, abort_flag, p.status, kStatusTimeoutMma)) return false;
                     tc_fence_after();
-                    const uint32_t p_lo = base + kOffP + (uint32_t)st * kShTileBytes;
                     const uint32_t v_lo = base + kOffV + (uint32_t)st * kShTileBytes;
-                    // P: K-major, as Q above.  V: tokens are rows of 128 bytes (8-token groups 1024 bytes apart,
-                    // 16 tokens = 2048 bytes per step); the two 64-dim blocks of the tile are kShBlock bytes apart
-                    const uint64_t a0 = umma_desc(p_lo, 16, 1024), b0 = umma_desc(v_lo, kShBlock, 1024);
+                    // P: the A operand comes from tensor memory, where the softmax warps left it in the first
+                    // 64 columns of the S buffer (two bf16 per column, 16 tokens = 8 columns per step).
+                    // V: tokens are rows of 128 bytes (8-token groups 1024 bytes apart, 16 tokens = 2048 bytes
+                    // per step); the two 64-dim blocks of the tile are kShBlock bytes apart.
+                    const uint64_t b0 = umma_desc(v_lo, kShBlock, 1024);
+                    const uint32_t p_tm = tmem + (uint32_t)st * 128u;
                     const uint32_t d_o = tmem + 256u + (uint32_t)st * 128u;
     #pragma unroll
-                    for (uint32_t k = 0; k < 8; ++k) {  // 16 tokens per instruction
-                        const uint64_t a_off16 = (uint64_t)(((k >> 2) * kShBlock + (k & 3u) * 32u) >> 4);
-                        umma_bf16(d_o, a0 + a_off16, b0 + (uint64_t)(k * 128u), kIdescPV, k);
-                    }
+                    for (uint32_t k = 0; k < 8; ++k)  // 16 tokens per instruction
+                        umma_bf16_ts(d_o, p_tm + 8u * k, b0 + (uint64_t)(k * 128u), kIdescPV, k);
                     umma_commit(bar(kBarOFull + st));
                     umma_commit(bar(kBarVEmpty + st));
-                    umma_commit(bar(kBarPFree + st));
+                    umma_commit(bar(kBarSFree + st));  // the S buffer (and the P in it) may be overwritten
                     return true;
                 };
                 for (uint32_t ui = unit_begin; ui < unit_end && ok; ++ui, ++nunit) {
@@ -332,7 +364,6 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
         };
         const uint32_t s_addr = lane_addr + (uint32_t)wg * 128u;
         const uint32_t o_addr = lane_addr + 256u + (uint32_t)wg * 128u;
-        const uint32_t prow = base + kOffP + (uint32_t)wg * kShTileBytes + (uint32_t)row * 128u;
 
         for (uint32_t ui = unit_begin; ui < unit_end && alive; ++ui) {
             const cart_shared_unit u = p.units[ui];
@@ -378,11 +409,17 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                 if (!warp_wait(bar(kBarOFull + wg), par)) return false;
                 tc_fence_after();
 #pragma unroll
-                for (int c4 = 0; c4 < 4; ++c4) {
-                    float v[32];
-                    tmem_ld32(o_addr + (uint32_t)c4 * 32u, v);
+                for (int c2 = 0; c2 < 2; ++c2) {  // two loads of 32 columns in flight
+                    uint32_t a[32], b[32];
+                    tmem_ld32_issue(o_addr + (uint32_t)c2 * 64u, a);
+                    tmem_ld32_issue(o_addr + (uint32_t)c2 * 64u + 32u, b);
+                    tmem_ld_wait(a);
+                    tmem_ld_wait(b);
 #pragma unroll
-                    for (int k = 0; k < 32; ++k) o_acc[c4 * 32 + k] = fmaf(o_acc[c4 * 32 + k], alpha, v[k]);
+                    for (int k = 0; k < 32; ++k) {
+                        o_acc[c2 * 64 + k] = fmaf(o_acc[c2 * 64 + k], alpha, __uint_as_float(a[k]));
+                        o_acc[c2 * 64 + 32 + k] = fmaf(o_acc[c2 * 64 + 32 + k], alpha, __uint_as_float(b[k]));
+                    }
                 }
                 tc_fence_before();
                 __syncwarp();
@@ -402,11 +439,14 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                 // pass 1: the row's maximum over the tile
                 float mx = -INFINITY;
 #pragma unroll
-                for (int c4 = 0; c4 < 4; ++c4) {
-                    float v[32];
-                    tmem_ld32(s_addr + (uint32_t)c4 * 32u, v);
+                for (int c2 = 0; c2 < 2; ++c2) {  // two loads of 32 columns in flight
+                    uint32_t a[32], b[32];
+                    tmem_ld32_issue(s_addr + (uint32_t)c2 * 64u, a);
+                    tmem_ld32_issue(s_addr + (uint32_t)c2 * 64u + 32u, b);
+                    tmem_ld_wait(a);
+                    tmem_ld_wait(b);
 #pragma unroll
-                    for (int k = 0; k < 32; ++k) mx = fmaxf(mx, v[k]);
+                    for (int k = 0; k < 32; ++k) mx = fmaxf(mx, fmaxf(__uint_as_float(a[k]), __uint_as_float(b[k])));
                 }
                 const float m_new = fmaxf(m_run, mx * p.scale_log2);
                 const float alpha = fast_exp2(m_run - m_new);  // 0 on the first tile
@@ -417,40 +457,35 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                     alive = take_o(prev_tt, alpha_prev);
                     if (!alive) break;
                 }
-                // pass 2: probabilities, as bf16, into the P buffer (free once this warpgroup's previous
-                // tile has been multiplied)
-                alive = warp_wait(bar(kBarPFree + wg), par ^ 1u);
-                if (!alive) break;
+                // pass 2: probabilities, as bf16 pairs, back into tensor memory over the first half of the
+                // scores they came from (32 scores are read, then 16 columns behind the read position are
+                // written): the A operand of the second product
                 float psum = 0.f;
+                {
+                    uint32_t buf[2][32];  // the load of the next 32 scores runs under the arithmetic on these
+                    tmem_ld32_issue(s_addr, buf[0]);
+                    tmem_ld_wait(buf[0]);
 #pragma unroll
-                for (int c4 = 0; c4 < 4; ++c4) {
-                    float v[32];
-                    tmem_ld32(s_addr + (uint32_t)c4 * 32u, v);
+                    for (int c4 = 0; c4 < 4; ++c4) {
+                        uint32_t(&v)[32] = buf[c4 & 1];
+                        if (c4 < 3) tmem_ld32_issue(s_addr + (uint32_t)(c4 + 1) * 32u, buf[(c4 + 1) & 1]);
+                        uint32_t w[16];
 #pragma unroll
-                    for (int k8 = 0; k8 < 4; ++k8) {  // 8 tokens = one 16-byte chunk
-                        uint32_t w[4];
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const float p0 = fast_exp2(fmaf(v[8 * k8 + 2 * j], p.scale_log2, -m_new));
-                            const float p1 = fast_exp2(fmaf(v[8 * k8 + 2 * j + 1], p.scale_log2, -m_new));
+                        for (int j = 0; j < 16; ++j) {
+                            const float p0 = fast_exp2(fmaf(__uint_as_float(v[2 * j]), p.scale_log2, -m_new));
+                            const float p1 = fast_exp2(fmaf(__uint_as_float(v[2 * j + 1]), p.scale_log2, -m_new));
                             psum += p0 + p1;
-                            w[j] = pack_bf16(p0, p1);
+                            w[j] = pack_bf16(p0, p1);  // the even token in the low half
                         }
-                        const uint32_t chunk = (uint32_t)((c4 & 1) * 4 + k8);
-                        const uint32_t a = prow + (uint32_t)(c4 >> 1) * kShBlock + ((chunk ^ swz) << 4);
-                        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(w[0]), "r"(w[1]), "r"(w[2]),
-                                     "r"(w[3])
-                                     : "memory");
+                        tmem_st16(s_addr + (uint32_t)c4 * 16u, w);
+                        if (c4 < 3) tmem_ld_wait(buf[(c4 + 1) & 1]);
                     }
                 }
                 l_run = fmaf(l_run, alpha, psum);
+                tmem_st_wait();
                 tc_fence_before();
-                fence_async_smem();
                 __syncwarp();
-                if (lane == 0) {
-                    mbar_arrive(bar(kBarSFree + wg));
-                    mbar_arrive(bar(kBarPReady + wg));
-                }
+                if (lane == 0) mbar_arrive(bar(kBarPReady + wg));
                 alpha_prev = alpha;
                 prev_tt = tt;
                 have_prev = true;
@@ -464,7 +499,7 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
             // q ^ (r & 31), which keeps both the row-per-lane and the quad-per-lane accesses free of bank
             // conflicts.
             softmax_bar_both();
-            uint8_t *comb = smem + kOffP;   // the two P buffers: 64 KB
+            uint8_t *comb = smem + kOffQ;   // the query buffer and the block behind it: 64 KB
             const uint32_t rsw = (uint32_t)(row & 31);
             if (wg == 1) {
 #pragma unroll
