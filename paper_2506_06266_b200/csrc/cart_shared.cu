@@ -518,11 +518,18 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                 const float inv = 1.f / l;
                 const float c0 = w0 * inv, c1 = w1 * inv;
 #pragma unroll
-                for (uint32_t q4 = 0; q4 < 32; ++q4) {
-                    float4 *cell = reinterpret_cast<float4 *>(comb + (size_t)row * 512 + ((q4 ^ rsw) << 4));
-                    const float4 v = *cell;
-                    *cell = make_float4(o_acc[4 * q4] * c0 + v.x * c1, o_acc[4 * q4 + 1] * c0 + v.y * c1,
-                                        o_acc[4 * q4 + 2] * c0 + v.z * c1, o_acc[4 * q4 + 3] * c0 + v.w * c1);
+                for (uint32_t q0 = 0; q0 < 32; q0 += 8) {  // eight loads in flight, then eight stores
+                    float4 v[8];
+#pragma unroll
+                    for (uint32_t j = 0; j < 8; ++j)
+                        v[j] = *reinterpret_cast<const float4 *>(comb + (size_t)row * 512 + (((q0 + j) ^ rsw) << 4));
+#pragma unroll
+                    for (uint32_t j = 0; j < 8; ++j) {
+                        const uint32_t q4 = q0 + j;
+                        *reinterpret_cast<float4 *>(comb + (size_t)row * 512 + ((q4 ^ rsw) << 4)) =
+                            make_float4(o_acc[4 * q4] * c0 + v[j].x * c1, o_acc[4 * q4 + 1] * c0 + v[j].y * c1,
+                                        o_acc[4 * q4 + 2] * c0 + v[j].z * c1, o_acc[4 * q4 + 3] * c0 + v[j].w * c1);
+                    }
                 }
                 uint32_t dst_row = 0xFFFFFFFFu;  // row of part_o ([slot][G] flattened) this query row goes to
                 if (alive && valid) {
@@ -537,12 +544,20 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                 const uint32_t *dst_rows = reinterpret_cast<const uint32_t *>(smem + kOffFlags);
                 const uint32_t q4 = (uint32_t)lane;                       // a warp = one row per pass
                 const uint32_t r0 = (uint32_t)(wg * 4 + (warp & 3));      // 8 softmax warps, 16 rows each
-#pragma unroll 4
-                for (uint32_t r = r0; r < 128u; r += 8u) {
-                    const uint32_t dst_row = dst_rows[r];
-                    if (dst_row == 0xFFFFFFFFu) continue;
-                    const float4 v = *reinterpret_cast<const float4 *>(comb + (size_t)r * 512 + ((q4 ^ (r & 31u)) << 4));
-                    reinterpret_cast<float4 *>(p.part_o + (size_t)dst_row * kHeadDim)[q4] = v;
+#pragma unroll
+                for (uint32_t rb = 0; rb < 16; rb += 8) {  // eight rows' loads in flight, then their stores
+                    uint32_t dst[8];
+                    float4 v[8];
+#pragma unroll
+                    for (uint32_t j = 0; j < 8; ++j) {
+                        const uint32_t r = r0 + 8u * (rb + j);
+                        dst[j] = dst_rows[r];
+                        v[j] = *reinterpret_cast<const float4 *>(comb + (size_t)r * 512 + ((q4 ^ (r & 31u)) << 4));
+                    }
+#pragma unroll
+                    for (uint32_t j = 0; j < 8; ++j)
+                        if (dst[j] != 0xFFFFFFFFu)
+                            reinterpret_cast<float4 *>(p.part_o + (size_t)dst[j] * kHeadDim)[q4] = v[j];
                 }
             }
             if (p.tickets) __threadfence();  // publish the partials before the tickets
