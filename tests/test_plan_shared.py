@@ -256,3 +256,27 @@ def test_shared_blocks_balanced_by_tiles_and_units(w):
     assert plan["n_unit_cta_used"] >= 140
     # charging for units makes the planner cut fewer runs in two
     assert len(plan["units"]) <= len(flat["units"])
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_random_batches_keep_every_invariant(seed):
+    """Random pools, compositions, suffix lengths, block counts and cost constants: coverage, slot
+    bookkeeping and balance must hold for all of them."""
+    rng = np.random.default_rng(1000 + seed)
+    Hkv = int(rng.choice([1, 2, 8]))
+    G = int(rng.choice([1, 3, 4, 8]))
+    a = Arena(Hkv)
+    pool = [a.store(int(rng.choice([1, 63, 64, 127, 128, 129, 300, 513, 1024, 2048]))) for _ in range(int(rng.integers(1, 5)))]
+    n_reqs = int(rng.integers(1, 40))
+    segs = []
+    for _ in range(n_reqs):
+        k = int(rng.integers(0, min(3, len(pool)) + 1))
+        parts = [pool[int(i)] for i in rng.choice(len(pool), k, replace=bool(rng.integers(0, 2)) or k > len(pool))] if k else []
+        n_suffix = int(rng.choice([0, 1, 5, 64, 65, 200, 700]))
+        r = list(parts)
+        if n_suffix or not r:
+            r.append(a.store(max(n_suffix, 1), cap_pad=int(rng.integers(0, 70))))
+        segs.append(r)
+    n_cta = int(rng.choice([1, 2, 7, 37, 148]))
+    check(segs, Hkv, G, n_cta, share_min=int(rng.choice([0, 2, 4])), piece_cost=int(rng.choice([0, 1, 3, 9])),
+          unit_cost=int(rng.choice([0, 2, 4])))
