@@ -163,13 +163,17 @@ def run_ours(args):
         sampler.start()
     binding.cart_set_timing(ctx, args.kernel_events)
     launches0 = binding.cart_launch_count(ctx)
-    bytes_layer_sum = 0
+    bytes_before = lw.algorithmic_bytes_per_layer()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
     for _ in range(args.steps):
         lw.step(q, k_new, v_new, out, lse, fused=not args.unfused)
-        bytes_layer_sum += lw.algorithmic_bytes_per_layer()
     e1.record(stream)
+    # every step appends one token per request, so the bytes per layer grow linearly over the steps: the sum
+    # over the steps (each counted with its own token already appended) follows from the two end points
+    bytes_after = lw.algorithmic_bytes_per_layer()
+    per_step = (bytes_after - bytes_before) / args.steps
+    bytes_layer_sum = args.steps * ((bytes_before + per_step) + bytes_after) / 2
     torch.cuda.synchronize(dev)
     replicas.barrier(world)
     clocks = sampler.stop() if rank == 0 else None
