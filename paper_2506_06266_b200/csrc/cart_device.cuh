@@ -12,6 +12,7 @@ namespace cart {
 namespace {
 
 constexpr uint64_t kWaitLimitNs = 2000000000ull;      // a wait gives up after about two seconds
+constexpr long long kWaitLimitCycles = 4000000000ll;   // the same in SM cycles (2 s at 2 GHz, 3 s at 1.3 GHz)
 
 // ---- small PTX wrappers ---------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void *p)
@@ -51,18 +52,22 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 // Bounded wait.  Returns false if the block has given up (this wait ran out, or another warp's did).
+// The limit is kept with the SM's cycle counter, which costs a few cycles to read and is first read
+// after a thousand polls: a wait that is about to succeed never pays for time keeping.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag,
                                           uint32_t *status, uint32_t code)
 {
     if (mbar_try_wait(bar, parity)) return true;
-    if (*abort_flag) return false;
-    const uint64_t t0 = global_timer_ns();
     uint32_t spins = 0;
+    long long t0 = 0;
     for (;;) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((++spins & 0xFFu) == 0) {
+        if ((++spins & 0x3FFu) == 0) {
             if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > kWaitLimitNs) {
+            const long long now = clock64();
+            if (t0 == 0) {
+                t0 = now | 1;
+            } else if (now - t0 > kWaitLimitCycles) {
                 *abort_flag = 1;
                 atomicOr(status, code);
                 return false;
