@@ -88,11 +88,13 @@ CART_API cart_status cart_create(const cart_config *cfg /*host*/, cart_ctx **out
 CART_API cart_status cart_destroy(cart_ctx *ctx);
 
 /* Sec. 3.2 / Sec. 3.3: make a trained Cartridge resident ("loaded into the KV cache slots") and
- * addressable by handle.  k and v are device bf16 [n_layers][n_kv_heads][p][128]; they are copied
- * into the arena on `stream` (the caller may free them once the stream has passed this point).
- * p >= 1, the same in every layer.  A Cartridge is stored once however many requests open on it.
+ * addressable by handle.  k and v are bf16 [n_layers][n_kv_heads][p][128], in device memory or in host
+ * memory (a Cartridge loaded from disk and swapped in while other requests decode: page-locked host
+ * memory makes the copy asynchronous); they are copied into the arena on `stream` (the caller may free
+ * or reuse them once the stream has passed this point).  p >= 1, the same in every layer.  A Cartridge
+ * is stored once however many requests open on it; cart_release_cartridge gives its space back.
  * Errors: INVALID_ARG, CAPACITY (table full), OOM, CUDA. */
-CART_API cart_status cart_register_cartridge(cart_ctx *ctx, const void *k /*device*/, const void *v /*device*/,
+CART_API cart_status cart_register_cartridge(cart_ctx *ctx, const void *k /*device or host*/, const void *v /*device or host*/,
                                     int32_t p, void *stream /*cudaStream_t*/, cart_id *out /*host*/);
 
 /* Sec. 3.1 ("capable of composition"), Sec. 5.4: the handle returned stands for the concatenation

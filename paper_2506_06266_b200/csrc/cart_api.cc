@@ -402,9 +402,9 @@ cart_status cart_register_cartridge(cart_ctx *ctx, const void *k, const void *v,
         return fail(ctx, CART_ERR_OOM, "register: arena has no room for %llu bytes",
                     (unsigned long long)(2 * rows_one * kRowBytes));
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    cudaError_t e = cudaMemcpyAsync(arena_ptr(ctx, start), k, rows_one * kRowBytes, cudaMemcpyDeviceToDevice, s);
+    cudaError_t e = cudaMemcpyAsync(arena_ptr(ctx, start), k, rows_one * kRowBytes, cudaMemcpyDefault, s);
     if (e == cudaSuccess)
-        e = cudaMemcpyAsync(arena_ptr(ctx, start + rows_one), v, rows_one * kRowBytes, cudaMemcpyDeviceToDevice, s);
+        e = cudaMemcpyAsync(arena_ptr(ctx, start + rows_one), v, rows_one * kRowBytes, cudaMemcpyDefault, s);
     if (e != cudaSuccess) {
         arena_free(ctx, start, 2 * rows_one);
         return fail(ctx, CART_ERR_CUDA, "register: copy failed: %s", cudaGetErrorString(e));

@@ -289,3 +289,40 @@ def test_plan_is_rebuilt_when_lengths_or_batch_change():
         assert launches > 0
     finally:
         sess.close()
+
+
+def test_cartridge_swapped_in_from_pinned_host_memory_while_others_stay():
+    # hot swap: one Cartridge is released and another registered from page-locked host memory in its place
+    wa = synth.Workload("swap_a", 71, 2, 24, 8, 1, 300, 4, 4)
+    wb = synth.Workload("swap_b", 72, 2, 24, 8, 1, 300, 6, 6)
+    sess = H.Session(2, 24, 8, 16 << 20, max_requests=4, max_cartridges=4)
+    try:
+        ca = sess.register(*wa.cartridge_kv(0, "cuda:0"))
+        ra = sess.open(ca, 8)
+        sess.extend(ra, *wa.suffix_kv(0, 4, "cuda:0"))
+        kb, vb = wb.cartridge_kv(0, "cpu")
+        kb_h, vb_h = kb.pin_memory(), vb.pin_memory()
+        stream = torch.cuda.current_stream()
+        cb = binding.cart_register_cartridge(sess.ctx, kb_h, vb_h, 300, stream)
+        torch.cuda.synchronize()
+        sess.cart_map[cb] = sess.oc.register(synth.bits(kb), synth.bits(vb))
+        rb = sess.open(cb, 8)
+        sess.extend(rb, *wb.suffix_kv(0, 6, "cuda:0"))
+        q = synth.normal_bf16((2, 24, 128), 73, "cuda:0")
+        for layer in range(2):
+            sess.decode_and_check(layer, [ra, rb], q)
+        # swap A out, a third one in (from host again), B untouched
+        binding.cart_request_close(sess.ctx, ra)
+        binding.cart_release_cartridge(sess.ctx, ca)
+        wc = synth.Workload("swap_c", 74, 2, 24, 8, 1, 280, 3, 3)
+        kc, vc = wc.cartridge_kv(0, "cpu")
+        kc_h, vc_h = kc.pin_memory(), vc.pin_memory()
+        cc = binding.cart_register_cartridge(sess.ctx, kc_h, vc_h, 280, stream)
+        torch.cuda.synchronize()
+        sess.cart_map[cc] = sess.oc.register(synth.bits(kc), synth.bits(vc))
+        rc = sess.open(cc, 8)
+        sess.extend(rc, *wc.suffix_kv(0, 3, "cuda:0"))
+        for layer in range(2):
+            sess.decode_and_check(layer, [rb, rc], q)
+    finally:
+        sess.close()
