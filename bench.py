@@ -311,6 +311,71 @@ def run_ours(args):
     print(json.dumps(line))
 
 
+def run_prefill(args):
+    """Side measurement (its own JSON line, not the headline): prefill attention of a T-token message over a
+    Cartridge of the chosen workload's shape -- cart_extend_kv of the message's KV, then
+    cart_prefill_attention, per layer."""
+    from paper_2506_06266_b200 import binding, runner
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    w0 = WORKLOADS[args.workload]()
+    T, s_old = args.prefill, 256
+    w = synth.shrink(w0, batch=1, suffix_lo=s_old, suffix_hi=s_old, cartridges="private" if w0.p else "none")
+    if args.layers:
+        w = synth.shrink(w, n_layers=args.layers)
+    L = w.n_layers
+    stream = torch.cuda.current_stream(dev)
+    reps = args.warmup + args.steps
+    cfg = binding.make_config(L, w.n_q_heads, w.n_kv_heads, max(T, 4), 4, device=0, softmax_scale=w.scale)
+    per_tok = L * w.kv_bytes_per_token_layer()
+    arena_bytes = binding.cart_scratch_bytes(cfg) + (w.p + s_old + reps * T + 128) * per_tok + 4096
+    arena = torch.empty(arena_bytes, dtype=torch.uint8, device=dev)
+    cfg.arena, cfg.arena_bytes = arena.data_ptr(), arena_bytes
+    ctx = binding.cart_create(cfg)
+    k, v = w.cartridge_kv(0, dev)
+    cart = binding.cart_register_cartridge(ctx, k, v, w.p, stream)
+    req = binding.cart_request_open(ctx, cart, s_old + reps * T)
+    ks, vs = w.suffix_kv(0, s_old, dev)
+    for layer in range(L):
+        binding.cart_extend_kv(ctx, layer, req, ks[layer], vs[layer], s_old, stream)
+    km, vm = w.suffix_kv(1, T, dev)                                   # the message's K and V, [L][T][Hkv][D]
+    q = synth.normal_bf16((L, T, w.n_q_heads, 128), w.seed + 77, dev)
+    out = torch.empty_like(q)
+
+    def step():
+        for layer in range(L):
+            binding.cart_extend_kv(ctx, layer, req, km[layer], vm[layer], T, stream)
+            binding.cart_prefill_attention(ctx, layer, req, q[layer], T, out[layer], None, stream)
+
+    for _ in range(args.warmup):
+        step()
+    binding.cart_sync_status(ctx, stream)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n0 = binding.cart_launch_count(ctx)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize(dev)
+    binding.cart_sync_status(ctx, stream)
+    ms = e0.elapsed_time(e1)
+    launches = binding.cart_launch_count(ctx) - n0
+    # the message grows the suffix by T per step: mean context of a row over the timed steps
+    mean_ctx = w.p + s_old + (args.warmup + (args.steps - 1) / 2.0) * T + (T + 1) / 2.0
+    flops = 4.0 * w.n_q_heads * 128 * mean_ctx * T                    # per layer
+    us_layer = ms * 1e3 / args.steps / L
+    binding.cart_destroy(ctx)
+    print(json.dumps({"metric": "prefill_attention_tokens_per_s", "value": round(T * args.steps / (ms * 1e-3), 1),
+                      "unit": "tokens/s", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
+                      "ms_per_step": round(ms / args.steps, 4), "higher_is_better": True, "dtype": "bf16",
+                      "data": "synthetic",
+                      "config": {"workload": "prefill of %d tokens over %s shapes" % (T, w0.name), "layers": L,
+                                 "cartridge_tokens": w.p, "suffix_before": s_old, "mean_context": round(mean_ctx, 1),
+                                 "attention_us_per_layer": round(us_layer, 2),
+                                 "tflops": round(flops / (us_layer * 1e-6) / 1e12, 2)},
+                      "gpu_launches": int(launches)}))
+
+
 def run_reference(args):
     """The reference arm is the CPU oracle, as it stands, timed on the host cores."""
     rank = int(os.environ.get("RANK", "0"))
@@ -377,6 +442,9 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=50)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--prefill", type=int, default=0,
+                    help="side measurement: prefill attention of a message of this many tokens over one Cartridge "
+                         "of the workload's shape (prints its own JSON line)")
     ap.add_argument("--unfused", action="store_true",
                     help="append and attend with two calls per layer instead of cart_decode_step")
     ap.add_argument("--piece-cost", type=int, default=-1,
@@ -390,7 +458,9 @@ def main():
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
-    if args.impl == "reference":
+    if args.prefill > 0:
+        run_prefill(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

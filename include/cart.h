@@ -164,8 +164,10 @@ CART_API cart_status cart_decode_step(cart_ctx *ctx, int32_t layer, const cart_r
  * [n_new][n_q_heads][128], token-major as the projection produces it) is the query of the i-th new
  * token and attends, per Eq. 1 with its causal sum over j <= i, to the request's Cartridge(s), the
  * suffix tokens before the new ones and the new tokens 0 .. i.  out, lse as in cart_decode_attention,
- * with n_new rows.  The Cartridge(s) and the old part of the suffix are read once for all rows
- * (tensor-core kernel) when n_new reaches the sharing threshold.  n_new <= max_requests.
+ * with n_new rows.  When n_new reaches the sharing threshold, the Cartridge(s) are read once for all
+ * rows and the suffix before each group of 128 / (n_q_heads / n_kv_heads) consecutive new tokens once
+ * for that group (tensor-core kernel); a row reads by itself only the fewer than 128 + 128 / G tokens
+ * around the causal diagonal.  n_new <= max_requests.
  * Errors: INVALID_ARG (also: the suffix holds fewer than n_new tokens), BAD_HANDLE, CAPACITY, CUDA. */
 CART_API cart_status cart_prefill_attention(cart_ctx *ctx, int32_t layer, cart_req req, const void *q /*device*/,
                                    int32_t n_new, void *out /*device*/, float *lse /*device or NULL*/,

@@ -141,6 +141,7 @@ struct cart_ctx {
     uint64_t stamp = 0;
     uint64_t launches = 0;
     std::vector<cart_plan_seg> seg_tmp;
+    std::vector<int32_t> head_tmp;
     std::vector<int32_t> seg_begin_tmp;
     std::vector<uint32_t> key_tmp;
     bool timing = false;
@@ -591,7 +592,8 @@ namespace {
 // Prefill mode (n_new > 0): reqs[0] is one request, and the batch is its last n_new suffix tokens as
 // n_new query rows; row i attends over the Cartridge(s) and the suffix up to and including its own
 // token (Eq. 1 for the rows of the new block).  The rows are planned like n_new requests that share the
-// Cartridge(s) and the head of the suffix, so those go through the shared-segment kernel.
+// Cartridge(s) and, group by group, the part of the suffix before the group's first token, so those go
+// through the shared-segment kernel.
 cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int32_t n_reqs, const void *q,
                         void *out, float *lse, const void *k_new, const void *v_new, void *stream, int32_t n_new = 0)
 {
@@ -648,6 +650,30 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
         segs.clear();
         sb.clear();
         sb.push_back(0);
+        // Prefill: the rows are cut into groups of 128 / G consecutive tokens (the rows one tensor-core
+        // tile holds per KV head).  Everything before a group's first token, rounded down to whole shared
+        // tiles, is visible to all of its rows: that is the group's shared head of the suffix, a
+        // staircase that follows the causal diagonal, so a row streams fewer than 128 + 128 / G tokens
+        // by itself.  A step is only taken if enough rows stand on it to be shared.
+        std::vector<int32_t> &head_of_group = ctx->head_tmp;
+        head_of_group.clear();
+        const int32_t rows_per_tile = 128 / ctx->group;
+        if (prefill && ctx->share_min_readers > 0 && n_new >= ctx->share_min_readers) {
+            const int32_t s_old = ctx->reqs[(size_t)reqs[0]].len[(size_t)layer] - n_new;
+            const int32_t n_groups = (n_new + rows_per_tile - 1) / rows_per_tile;
+            auto natural = [&](int32_t g) { return (s_old + g * rows_per_tile) / kShareTileTokens * kShareTileTokens; };
+            int32_t cur = natural(0);
+            for (int32_t g = 0; g < n_groups; ++g) {
+                const int32_t nat = natural(g);
+                if (nat != cur) {
+                    int32_t g2 = g;
+                    while (g2 < n_groups && natural(g2) == nat) ++g2;
+                    const int32_t rows = std::min(n_new, g2 * rows_per_tile) - g * rows_per_tile;
+                    if (rows >= ctx->share_min_readers) cur = nat;
+                }
+                head_of_group.push_back(cur);
+            }
+        }
         for (int32_t i = 0; i < n_reqs; ++i) {
             const Request &r = ctx->reqs[(size_t)reqs[prefill ? 0 : i]];
             auto push_cart = [&](const Cartridge &c) {
@@ -667,12 +693,11 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
             int32_t len = r.len[(size_t)layer];
             uint32_t first = 0;  // first suffix token of the segment
             if (prefill) {
-                // row i sees the suffix up to its own token; the part before the new tokens, rounded down
-                // to whole shared tiles, is the same block for every row: a segment of its own
+                // row i sees the suffix up to its own token; its group's shared head is a segment of its own
                 const int32_t s_old = len - n_new;
                 len = s_old + i + 1;
-                const int32_t head = s_old / kShareTileTokens * kShareTileTokens;
-                if (head > 0 && ctx->share_min_readers > 0 && n_new >= ctx->share_min_readers) {
+                const int32_t head = head_of_group.empty() ? 0 : head_of_group[(size_t)(i / rows_per_tile)];
+                if (head > 0) {
                     cart_plan_seg sg;
                     sg.k_row = (uint32_t)r.k_row;
                     sg.v_row = (uint32_t)r.v_row;

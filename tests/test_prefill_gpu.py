@@ -83,6 +83,14 @@ def test_prefill_many_rows_long_cartridge():
     run(32, 8, 4096, 0, 256, layers=1, seed=5)
 
 
+@pytest.mark.parametrize("Hq,Hkv,s_old,n_new", [(32, 8, 100, 300), (24, 8, 77, 200), (64, 8, 0, 150), (8, 1, 250, 140),
+                                                (32, 8, 0, 130), (32, 8, 126, 35)])
+def test_prefill_of_a_long_message_shares_the_suffix_in_causal_steps(Hq, Hkv, s_old, n_new):
+    # the message spans several shared tiles: groups of 128 / G rows share the suffix before their first
+    # token (a staircase along the diagonal); (0, 130) leaves 2 rows on the last step, too few to share it
+    run(Hq, Hkv, 200, s_old, n_new, layers=1, seed=6)
+
+
 def test_prefill_errors():
     sess = H.Session(1, 32, 8, 8 << 20, max_requests=8)
     try:
