@@ -10,18 +10,22 @@
 //   producer warps  TMA loads of K tiles (warp 0, three stages) and V tiles (warp 2, two stages), 128 tokens
 //                   x 128 dims, 128-byte swizzle, completion on mbarriers
 //   MMA warp        one thread issues  S = Q K^T  (128 x 128 x 128, both operands from shared memory,
-//                   accumulator in tensor memory) and  O_t = P V  (A operand P from tensor memory, V from
-//                   shared memory, fresh accumulator per tile); tcgen05.commit signals mbarriers
-//   2 x 4 softmax  two warpgroups take alternate tiles (warpgroup w owns S and O buffer w).  Thread r of a
-//   warps           warpgroup owns query row r: reads S from tensor memory (two loads in flight), keeps the
-//                   running maximum and sum of an online softmax over its warpgroup's tiles in fp32,
-//                   writes P = 2^(s - m) as bf16 pairs back over the first half of the S buffer
-//                   (tcgen05.st), and adds the finished O_t of its previous tile to its fp32 register
-//                   accumulator, rescaled to the new maximum.  At the end of a unit the two warpgroups'
-//                   states are combined through shared memory.
+//                   accumulator in tensor memory) and  O += P V  (A operand P from tensor memory, V from
+//                   shared memory, accumulating in tensor memory over the warpgroup's tiles of the unit);
+//                   tcgen05.commit signals mbarriers
+//   2 x 4 softmax  two warpgroups take alternate tiles (warpgroup w owns S buffer w and accumulator w).
+//   warps           Thread r of a warpgroup owns query row r: reads S from tensor memory (two loads in
+//                   flight), keeps a reference maximum and the sum of an online softmax over its
+//                   warpgroup's tiles in fp32, and writes P = 2^(s - m) as bf16 pairs back over the first
+//                   half of the S buffer (tcgen05.st).  The reference maximum only moves when a row's
+//                   maximum has grown by more than 2^8 (then the warp rescales its lanes of the accumulator
+//                   in tensor memory); sum and accumulator always refer to the same reference, so the
+//                   result is exact.  At the end of a unit the warpgroups read their accumulators and
+//                   combine their states through shared memory.
 //
-// S (with P in it) and O_t are double-buffered in tensor memory (4 x 128 columns), so the products of
-// tile t+1 run while the softmax of tile t does.  At the end of a unit every row is written as a
+// S (with P in it) is double-buffered in tensor memory and each warpgroup has its own accumulator
+// (4 x 128 columns), so the products of tile t+1 run while the softmax of tile t does.  At the end of a
+// unit every row is written as a
 // normalised fp32 partial (o, lse); the partials of a (request, KV head) row group are merged by
 // log-sum-exp either by the block that delivers the last one -- this kernel's or the stream kernel's --
 // or, when the batch has more split row groups than blocks, by a merge kernel that runs afterwards.
@@ -43,12 +47,13 @@ constexpr int kKStages = 3;                           // K tiles in flight (each
 constexpr int kVStages = 2;
 constexpr int kShThreads = 384;                       // utility warpgroup (K producer, MMA, V producer, 1 idle) + 2 softmax warpgroups
 // Registers per thread after the warpgroups have re-divided the block's allocation (384 x 168): the
-// utility warps need few, the softmax threads hold a 128-float accumulator.  4 x 32 x 40 + 8 x 32 x 232
+// utility warps need few, the softmax threads hold a 128-float accumulator at the end of a unit.  4 x 32 x 40 + 8 x 32 x 232
 // = 64512 registers, and per SM sub-partition 1 utility + 2 softmax warps = 16128 of its 16384.
 constexpr int kRegsUtility = 40;
 constexpr int kRegsSoftmax = 232;
 constexpr int kSoftmaxThreads = 128;                  // one softmax warpgroup
-constexpr uint32_t kTmemCols = 512;                   // S0 S1 O0 O1, 128 fp32 columns each
+constexpr uint32_t kTmemCols = 512;                   // S0 S1 (scores, then P), O0 O1 (accumulators): 128 fp32 columns each
+constexpr float kRescaleStep = 8.f;                   // how far a row's maximum may outgrow its reference (base-2 units)
 
 // shared-memory layout (offsets from a 1024-byte aligned base)
 constexpr uint32_t kOffQ = 0;
@@ -71,8 +76,7 @@ enum Bar : int {
     kBarSFull = 10,  // [2] MMA (commit) -> softmax
     kBarSFree = 12,  // [2] MMA (commit of P V: the probabilities live in the S buffer) -> MMA
     kBarPReady = 14, // [2] softmax -> MMA          (4 arrivals: one per warp of the warpgroup)
-    kBarOFull = 16,  // [2] MMA (commit) -> softmax
-    kBarOFree = 18,  // [2] softmax -> MMA          (4 arrivals)
+    kBarOFull = 16,  // [2] MMA (commit of P V) -> softmax: the accumulator holds the product
     kBarQReady = 20, // softmax -> MMA              (8 arrivals: every softmax warp)
     kBarDrain = 21,  // MMA (commit) -> MMA, on the way out
 };
@@ -200,7 +204,6 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
             mbar_init(bar(kBarSFull + i), 1);
             mbar_init(bar(kBarSFree + i), 1);
             mbar_init(bar(kBarOFull + i), 1);
-            mbar_init(bar(kBarOFree + i), 4);
             mbar_init(bar(kBarPReady + i), 4);
         }
         mbar_init(bar(kBarQReady), 8);
@@ -298,12 +301,11 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                     umma_commit(bar(kBarKEmpty + (int)kst));
                     return true;
                 };
-                // O(tt) = P V into O buffer tt & 1
-                auto issue_pv = [&](uint32_t tt) -> bool {
+                // O += P V into the accumulator of warpgroup tt & 1; `first`: the warpgroup's first tile of the unit
+                auto issue_pv = [&](uint32_t tt, bool first) -> bool {
                     const int st = (int)(tt & 1u);
                     const uint32_t par = (tt >> 1) & 1u;
                     if (!mbar_wait(bar(kBarVFull + st), par, abort_flag, p.status, kStatusTimeoutMma)) return false;
-                    if (!mbar_wait(bar(kBarOFree + st), par ^ 1u, abort_flag, p.status, kStatusTimeoutMma)) return false;
                     if (!mbar_wait(bar(kBarPReady + st), par, abort_flag, p.status, kStatusTimeoutMma)) return false;
                     tc_fence_after();
                     const uint32_t v_lo = base + kOffV + (uint32_t)st * kShTileBytes;
@@ -316,7 +318,7 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                     const uint32_t d_o = tmem + 256u + (uint32_t)st * 128u;
     #pragma unroll
                     for (uint32_t k = 0; k < 8; ++k)  // 16 tokens per instruction
-                        umma_bf16_ts(d_o, p_tm + 8u * k, b0 + (uint64_t)(k * 128u), kIdescPV, k);
+                        umma_bf16_ts(d_o, p_tm + 8u * k, b0 + (uint64_t)(k * 128u), kIdescPV, (first && k == 0u) ? 0u : 1u);
                     umma_commit(bar(kBarOFull + st));
                     umma_commit(bar(kBarVEmpty + st));
                     umma_commit(bar(kBarSFree + st));  // the S buffer (and the P in it) may be overwritten
@@ -330,7 +332,7 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                     ok = issue_s(tt0);
                     for (uint32_t t = 0; t < n && ok; ++t) {
                         if (t + 1 < n) ok = issue_s(tt0 + t + 1);
-                        if (ok) ok = issue_pv(tt0 + t);
+                        if (ok) ok = issue_pv(tt0 + t, t < 2u);
                     }
                     tt0 += n;
                 }
@@ -399,33 +401,10 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(kBarQReady));
             }
-            float m_run = -INFINITY, l_run = 0.f, alpha_prev = 0.f;
-#pragma unroll
-            for (int d = 0; d < 128; ++d) o_acc[d] = 0.f;
-
-            // adds the finished O of tile tt (relative to the running maximum after tile tt) to o_acc
-            auto take_o = [&](uint32_t tt, float alpha) -> bool {
-                const uint32_t par = (tt >> 1) & 1u;
-                if (!warp_wait(bar(kBarOFull + wg), par)) return false;
-                tc_fence_after();
-#pragma unroll
-                for (int c2 = 0; c2 < 2; ++c2) {  // two loads of 32 columns in flight
-                    uint32_t a[32], b[32];
-                    tmem_ld32_issue(o_addr + (uint32_t)c2 * 64u, a);
-                    tmem_ld32_issue(o_addr + (uint32_t)c2 * 64u + 32u, b);
-                    tmem_ld_wait(a);
-                    tmem_ld_wait(b);
-#pragma unroll
-                    for (int k = 0; k < 32; ++k) {
-                        o_acc[c2 * 64 + k] = fmaf(o_acc[c2 * 64 + k], alpha, __uint_as_float(a[k]));
-                        o_acc[c2 * 64 + 32 + k] = fmaf(o_acc[c2 * 64 + 32 + k], alpha, __uint_as_float(b[k]));
-                    }
-                }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(kBarOFree + wg));
-                return true;
-            };
+            // m_run: the reference maximum that l_run and the warpgroup's accumulator in tensor memory refer to.
+            // It only moves when a row's maximum has outgrown it by more than kRescaleStep (base 2); until then
+            // probabilities may exceed 1 (by at most that factor), which bf16 and the fp32 sums hold easily.
+            float m_run = -INFINITY, l_run = 0.f;
 
             // this warpgroup's tiles of the unit: those whose block-wide index is congruent to wg mod 2
             bool have_prev = false;
@@ -448,15 +427,34 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
 #pragma unroll
                     for (int k = 0; k < 32; ++k) mx = fmaxf(mx, fmaxf(__uint_as_float(a[k]), __uint_as_float(b[k])));
                 }
-                const float m_new = fmaxf(m_run, mx * p.scale_log2);
-                const float alpha = fast_exp2(m_run - m_new);  // 0 on the first tile
-                m_run = m_new;
-                // this warpgroup's previous tile has been multiplied by now: fold its O in, which also frees
-                // the O buffer for the product of this tile
-                if (have_prev) {
-                    alive = take_o(prev_tt, alpha_prev);
+                mx *= p.scale_log2;
+                if (!have_prev) {
+                    m_run = mx;
+                } else if (__any_sync(0xffffffffu, mx > m_run + kRescaleStep)) {
+                    // a row of this warp has outgrown its reference: every row moves up to its maximum and the
+                    // warp rescales its lanes of the accumulator (tensor-memory accesses are warp-wide, so the
+                    // warp decides together; the other rows' factors are 1 or close to it)
+                    const float m_new = fmaxf(m_run, mx);
+                    const float f = fast_exp2(m_run - m_new);
+                    m_run = m_new;
+                    l_run *= f;
+                    // the product of this warpgroup's previous tile must have landed first
+                    alive = warp_wait(bar(kBarOFull + wg), (prev_tt >> 1) & 1u);
                     if (!alive) break;
+                    tc_fence_after();
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t o[32];
+                        tmem_ld32_issue(o_addr + (uint32_t)c * 32u, o);
+                        tmem_ld_wait(o);
+#pragma unroll
+                        for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * f);
+                        tmem_st16(o_addr + (uint32_t)c * 32u, reinterpret_cast<const uint32_t(&)[16]>(o[0]));
+                        tmem_st16(o_addr + (uint32_t)c * 32u + 16u, reinterpret_cast<const uint32_t(&)[16]>(o[16]));
+                    }
+                    // (these stores are waited for with those of P below, before the MMA warp hears of the tile)
                 }
+                const float m_new = m_run;
                 // pass 2: probabilities, as bf16 pairs, back into tensor memory over the first half of the
                 // scores they came from (32 scores are read, then 16 columns behind the read position are
                 // written): the A operand of the second product
@@ -481,16 +479,38 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                         if (c4 < 3) tmem_ld_wait(buf[(c4 + 1) & 1]);
                     }
                 }
-                l_run = fmaf(l_run, alpha, psum);
+                l_run += psum;
                 tmem_st_wait();
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(kBarPReady + wg));
-                alpha_prev = alpha;
                 prev_tt = tt;
                 have_prev = true;
             }
-            if (alive && have_prev) alive = take_o(prev_tt, alpha_prev);
+            // the warpgroup's share of the unit's output, out of tensor memory
+            if (alive && have_prev) {
+                alive = warp_wait(bar(kBarOFull + wg), (prev_tt >> 1) & 1u);
+                if (alive) {
+                    tc_fence_after();
+#pragma unroll
+                    for (int c2 = 0; c2 < 2; ++c2) {  // two loads of 32 columns in flight
+                        uint32_t a[32], b[32];
+                        tmem_ld32_issue(o_addr + (uint32_t)c2 * 64u, a);
+                        tmem_ld32_issue(o_addr + (uint32_t)c2 * 64u + 32u, b);
+                        tmem_ld_wait(a);
+                        tmem_ld_wait(b);
+#pragma unroll
+                        for (int k = 0; k < 32; ++k) {
+                            o_acc[c2 * 64 + k] = __uint_as_float(a[k]);
+                            o_acc[c2 * 64 + 32 + k] = __uint_as_float(b[k]);
+                        }
+                    }
+                    tc_fence_before();
+                }
+            } else {
+#pragma unroll
+                for (int d = 0; d < 128; ++d) o_acc[d] = 0.f;
+            }
             tt0 += u.n_tiles;
 
             // ---- combine the two warpgroups' states of each row and write the partials ------------------
