@@ -141,3 +141,40 @@ def test_shared_path_with_decode_appends_is_bitwise_reproducible():
             assert torch.equal(o1, o2) and torch.equal(l1, l2)
     finally:
         sess.close()
+
+
+@pytest.mark.parametrize("growth", [(1.0, 6.0, 30.0), (30.0, 1.0, 1.0, 12.0), (1.0, 1.0, 8.0, 8.0, 40.0, 40.0, 1.0, 1.0) * 12])
+def test_row_maxima_that_outgrow_the_reference_rescale_the_accumulator(growth):
+    """The tensor-core kernel keeps its sums relative to a reference maximum that only moves once a row's
+    maximum has outgrown it by more than 2^8.  Keys that get larger from one 128-token tile to the next make
+    that happen (per-tile key scales `growth`; a scale of 30 moves the scores' spread from a few units to
+    dozens), for some rows and not for others; rows whose scores shrink again keep their old reference.  A
+    block is given at least two tiles of a segment when there are blocks to spare, so only the long case (96
+    tiles per KV head, five or so per block) puts several tiles of one block in front of the same warpgroup,
+    which is what moves a reference.  The oracle knows nothing of tiles or references."""
+    Hq, Hkv, n_req = 32, 8, 9
+    p = 128 * len(growth) + 40                        # the 40-token tail is streamed per request
+    w = synth.Workload("sh_grow", 470 + len(growth), 1, Hq, Hkv, n_req, p, 1, 50, cartridges="shared")
+    sess = H.Session(1, Hq, Hkv, 160 << 20, max_requests=n_req)
+    try:
+        k, v = w.cartridge_kv(0, "cuda:0")
+        kf = k.float()
+        for t, g in enumerate(growth):
+            kf[:, :, 128 * t:128 * (t + 1), :] *= g
+        c = sess.register(kf.to(torch.bfloat16), v)
+        reqs = []
+        suffix = w.suffix_lengths()
+        for b in range(n_req):
+            r = sess.open(c, int(suffix[b]) + 1)
+            sess.extend(r, *w.suffix_kv(b, int(suffix[b]), "cuda:0"))
+            reqs.append(r)
+        q = w.queries(0, "cuda:0")[0]
+        (o1, l1), (o0, l0), launches = decode_both_ways(sess, 0, reqs, q)
+        assert launches in (2, 3)
+        ro, rl = sess.oracle_decode(0, reqs, q)
+        H.assert_close(o1, l1, ro, rl, "shared, growth %s" % (growth,))
+        H.assert_close(o0, l0, ro, rl, "streamed, growth %s" % (growth,))
+        # the scores really do outgrow the step: the spread of lse over rows is far beyond 8 base-2 units
+        assert float(l1.max() - l1.min()) > 8 * 0.6931
+    finally:
+        sess.close()
