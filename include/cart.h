@@ -117,6 +117,16 @@ CART_API cart_status cart_release_cartridge(cart_ctx *ctx, cart_id id);
 CART_API cart_status cart_request_open(cart_ctx *ctx, cart_id cartridge, int32_t suffix_capacity,
                               cart_req *out /*host*/);
 
+/* Grows the suffix buffer of an open request to at least suffix_capacity tokens per layer (rounded up
+ * to a multiple of 64), for conversations that outlive the capacity they were opened with (Sec. 3.3:
+ * per-user KV caches of any length next to the shared prefix).  A new buffer is taken from the arena,
+ * the tokens stored so far are copied into it on `stream` (device to device, one strided copy for K and
+ * one for V), and the old buffer returns to the arena; decode calls enqueued on the same stream before
+ * the call still read the old buffer, later ones the new.  A capacity not above the current one
+ * changes nothing.  The arena must have room for the new buffer while the old one is still held.
+ * Errors: BAD_HANDLE, INVALID_ARG, OOM (nothing has changed), CUDA. */
+CART_API cart_status cart_request_reserve(cart_ctx *ctx, cart_req req, int32_t suffix_capacity, void *stream);
+
 /* Closes a request and returns its suffix buffer to the arena.  Errors: BAD_HANDLE. */
 CART_API cart_status cart_request_close(cart_ctx *ctx, cart_req req);
 

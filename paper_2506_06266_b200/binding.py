@@ -26,7 +26,7 @@ STATUS_NAMES = ["CART_OK", "CART_ERR_INVALID_ARG", "CART_ERR_SHAPE", "CART_ERR_B
 
 # every symbol include/cart.h and include/cart_plan.h declare
 EXPORTS = ["cart_scratch_bytes", "cart_create", "cart_destroy", "cart_register_cartridge",
-           "cart_compose", "cart_release_cartridge", "cart_request_open", "cart_request_close",
+           "cart_compose", "cart_release_cartridge", "cart_request_open", "cart_request_reserve", "cart_request_close",
            "cart_append_kv", "cart_extend_kv", "cart_decode_attention", "cart_decode_step", "cart_prefill_attention", "cart_suffix_len",
            "cart_kv_bytes", "cart_sync_status", "cart_set_timing", "cart_get_timing",
            "cart_set_share_min_readers", "cart_set_piece_cost", "cart_plan_build_shared",
@@ -118,6 +118,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.cart_release_cartridge.argtypes = [vp, i32]
     lib.cart_request_open.argtypes = [vp, i32, i32, i32p]
     lib.cart_request_close.argtypes = [vp, i32]
+    lib.cart_request_reserve.argtypes = [vp, i32, i32, vp]
     lib.cart_append_kv.argtypes = [vp, i32, i32p, i32, vp, vp, vp]
     lib.cart_extend_kv.argtypes = [vp, i32, i32, vp, vp, i32, vp]
     lib.cart_decode_attention.argtypes = [vp, i32, i32p, i32, vp, vp, vp, vp]
@@ -227,6 +228,11 @@ def cart_request_open(ctx: int, cartridge: int, suffix_capacity: int) -> int:
     _check(load_library().cart_request_open(ctx, int(cartridge), int(suffix_capacity), ctypes.byref(out)),
            "cart_request_open", ctx)
     return int(out.value)
+
+
+def cart_request_reserve(ctx: int, req: int, suffix_capacity: int, stream=None) -> None:
+    _check(load_library().cart_request_reserve(ctx, int(req), int(suffix_capacity), _stream(stream)),
+           "cart_request_reserve", ctx)
 
 
 def cart_request_close(ctx: int, req: int) -> None:

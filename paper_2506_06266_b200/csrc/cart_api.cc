@@ -502,6 +502,46 @@ cart_status cart_request_open(cart_ctx *ctx, cart_id cartridge, int32_t suffix_c
     return CART_OK;
 }
 
+cart_status cart_request_reserve(cart_ctx *ctx, cart_req req, int32_t suffix_capacity, void *stream)
+{
+    if (!ctx) return CART_ERR_INVALID_ARG;
+    Request *r = get_req(ctx, req);
+    if (!r) return fail(ctx, CART_ERR_BAD_HANDLE, "reserve: not an open request");
+    if (suffix_capacity < 0) return fail(ctx, CART_ERR_INVALID_ARG, "reserve: negative capacity");
+    const int64_t cap = ((int64_t)suffix_capacity + kTileTokens - 1) / kTileTokens * kTileTokens;
+    if (cap <= r->cap) return CART_OK;  // a buffer never shrinks
+    const uint64_t heads = (uint64_t)ctx->cfg.n_layers * ctx->cfg.n_kv_heads;
+    const uint64_t rows_one = heads * (uint64_t)cap;
+    uint64_t start = 0;
+    if (!arena_alloc(ctx, 2 * rows_one, &start))
+        return fail(ctx, CART_ERR_OOM, "reserve: arena has no room for a suffix of %lld tokens", (long long)cap);
+    int32_t longest = 0;
+    for (int32_t l : r->len) longest = std::max(longest, l);
+    if (longest > 0) {
+        // every (layer, KV head) keeps its tokens in one run: old runs are r->cap rows apart, new ones cap rows
+        cudaStream_t s = static_cast<cudaStream_t>(stream);
+        cudaError_t e = cudaMemcpy2DAsync(arena_ptr(ctx, start), (size_t)cap * kRowBytes, arena_ptr(ctx, r->k_row),
+                                          (size_t)r->cap * kRowBytes, (size_t)longest * kRowBytes, heads,
+                                          cudaMemcpyDeviceToDevice, s);
+        if (e == cudaSuccess)
+            e = cudaMemcpy2DAsync(arena_ptr(ctx, start + rows_one), (size_t)cap * kRowBytes, arena_ptr(ctx, r->v_row),
+                                  (size_t)r->cap * kRowBytes, (size_t)longest * kRowBytes, heads,
+                                  cudaMemcpyDeviceToDevice, s);
+        if (e != cudaSuccess) {
+            arena_free(ctx, start, 2 * rows_one);
+            return fail(ctx, CART_ERR_CUDA, "reserve: copy failed: %s", cudaGetErrorString(e));
+        }
+    }
+    if (r->alloc_rows > 0) arena_free(ctx, r->alloc_start, r->alloc_rows);
+    r->cap = (int32_t)cap;
+    r->k_row = start;
+    r->v_row = start + rows_one;
+    r->alloc_start = start;
+    r->alloc_rows = 2 * rows_one;
+    ++ctx->epoch;  // cached plans address the old buffer
+    return CART_OK;
+}
+
 cart_status cart_request_close(cart_ctx *ctx, cart_req req)
 {
     if (!ctx) return CART_ERR_INVALID_ARG;
