@@ -219,6 +219,7 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeParams 
         if (lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap)) : "memory");
         uint32_t t = 0;  // tiles issued by this block so far
         bool ok = true;
+        const uint64_t stream_once = l2_evict_first_policy();  // a tile is read once per launch: let it leave L2 first
         // Until the kernels before this one on the stream are known to be complete, only tiles that
         // they cannot have written are fetched: a fused append writes a request's last token, which
         // lies in the last tile of an item marked CART_ITEM_TAIL.  Everything else in the arena is
@@ -259,11 +260,11 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeParams 
                     const int32_t yk = (int32_t)(k_row + j * kTileTokens);
                     const int32_t yv = (int32_t)(v_row + j * kTileTokens);
                     mbar_expect_tx(full_k(s), kTileBytes);
-                    tma_load_2d(kdst, &tmap, 0, yk, full_k(s));
-                    tma_load_2d(kdst + kHalfBytes, &tmap, 64, yk, full_k(s));
+                    tma_load_2d_hint(kdst, &tmap, 0, yk, full_k(s), stream_once);
+                    tma_load_2d_hint(kdst + kHalfBytes, &tmap, 64, yk, full_k(s), stream_once);
                     mbar_expect_tx(full_v(s), kTileBytes);
-                    tma_load_2d(vdst, &tmap, 0, yv, full_v(s));
-                    tma_load_2d(vdst + kHalfBytes, &tmap, 64, yv, full_v(s));
+                    tma_load_2d_hint(vdst, &tmap, 0, yv, full_v(s), stream_once);
+                    tma_load_2d_hint(vdst + kHalfBytes, &tmap, 64, yv, full_v(s), stream_once);
                 }
             }
         }
