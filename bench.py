@@ -184,6 +184,33 @@ def run_ours(args):
     binding.cart_sync_status(ctx, stream)
     value, ms_max = replicas.whole_job_tokens_per_s(B * args.steps, ms, world, dev)
 
+    # ---- the single-layer workload: one decode call by itself, L2 warm and L2 cold ----------------
+    single_call = None
+    if L == 1 and world == 1:
+        ca, cb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+        def one_call_us(flush):
+            if flush is not None:
+                flush.fill_(1)                       # 256 MB written: nothing of the KV is left in L2
+            else:
+                torch.cuda._sleep(200000)            # keeps the GPU busy while the host enqueues the call, as the
+                                                     # fill does in the cold case: the events then bracket GPU time
+            ca.record(stream)
+            binding.cart_decode_attention(ctx, 0, lw.req_list, q[0], out[0], lse[0], stream)
+            cb.record(stream)
+            cb.synchronize()
+            return ca.elapsed_time(cb) * 1e3
+
+        one_call_us(None)                            # the plan for the current lengths is built here
+        warm = [one_call_us(None) for _ in range(20)]
+        flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+        cold = [one_call_us(flush_buf) for _ in range(5)]
+        del flush_buf
+        single_call = {"what": "one cart_decode_attention call, plan cached, CUDA events around the call",
+                       "warm_us_mean": round(sum(warm) / len(warm), 2), "warm_us_min": round(min(warm), 2),
+                       "cold_us_mean": round(sum(cold) / len(cold), 2), "cold_us_min": round(min(cold), 2)}
+        binding.cart_sync_status(ctx, stream)
+
     # ---- roofline of the dominant kernel (split-KV decode attention) -------------------------
     peak, peak_kind = measured_peak_gbs()
     bytes_per_launch = bytes_layer_sum / args.steps          # one launch = one layer of one step
@@ -306,7 +333,7 @@ def run_ours(args):
                    "attention_us_per_layer": round(ms_max * 1e3 / args.steps / L, 2),
                    "kv_bytes_per_request": int(logical), "kv_bytes_private_per_request": int(private)},
         "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
-        "clocks": clocks,
+        "clocks": clocks, **({"single_call": single_call} if single_call else {}),
     }
     print(json.dumps(line))
 
