@@ -132,6 +132,7 @@ struct cart_ctx {
     int piece_cost = kPieceCostTiles;
     uint64_t n_rows = 0;
     alignas(64) CUtensorMap tmap;
+    alignas(64) CUtensorMap tmap_edge;
     std::vector<FreeBlock> free_list;
     std::vector<Cartridge> carts;
     std::vector<Request> reqs;
@@ -240,6 +241,13 @@ cart_status encode_tensor_map(cart_ctx *ctx)
                                                 CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                                                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(ctx, CART_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+    // The same matrix in smaller boxes: a ragged last tile of a segment is fetched only as far as it has tokens.
+    const cuuint32_t edge_box[2] = {64u, (cuuint32_t)kEdgeBoxRows};
+    r = reinterpret_cast<EncodeFn>(fn)(&ctx->tmap_edge, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ctx->cfg.arena, gdim,
+                                       gstride, edge_box, estride, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                       CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(ctx, CART_ERR_CUDA, "cuTensorMapEncodeTiled (edge) failed with code %d", (int)r);
     return CART_OK;
 }
 
@@ -821,6 +829,7 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
     dp.layer = layer;
     dp.group = ctx->group;
     dp.scale_log2 = ctx->scale * 1.4426950408889634f;
+    dp.edge_boxes = 1u;
     const bool timed = ctx->timing && ctx->ev_used + 2 <= kMaxTimedLaunches * 2;
     if (timed) {
         while (ctx->ev_pool.size() < ctx->ev_used + 2) {
@@ -854,7 +863,7 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
         ++ctx->launches;
     }
     if (sl->n_items > 0) {
-        CART_CUDA(ctx, launch_decode(ctx->tmap, dp, sl->n_cta_used, s));
+        CART_CUDA(ctx, launch_decode(ctx->tmap, ctx->tmap_edge, dp, sl->n_cta_used, s));
         ++ctx->launches;
     }
     if (merge_after) {

@@ -13,6 +13,7 @@ namespace cart {
 constexpr int kHeadDim = 128;
 constexpr int kRowBytes = kHeadDim * 2;  // one token of one KV head: 128 bf16
 constexpr int kTileTokens = 64;          // tokens per shared-memory stage
+constexpr int kEdgeBoxRows = 32;         // tokens per box when a ragged last tile is fetched piecewise
 constexpr int kMaxGroup = 8;             // query heads per KV head the kernels support
 constexpr int kShareTileTokens = 128;    // tokens per tile of the shared-segment kernel
 constexpr int kAppendBatch = 256;        // requests one append launch takes (kernel-parameter budget)
@@ -40,6 +41,8 @@ struct DecodeParams {
     int32_t layer;
     int32_t group;               // G
     float scale_log2;            // softmax scale * log2(e)
+    uint32_t edge_boxes = 0;     // 1: ragged last tiles are fetched in boxes of kEdgeBoxRows rows through the second
+                                 // tensor map; 0: every tile is fetched whole
 };
 
 // Parameters of the shared-segment kernel (units and reader tables as the planner lays them out).
@@ -120,7 +123,10 @@ inline cudaLaunchConfig_t pdl_config(int grid, int block, size_t smem, cudaStrea
 size_t decode_smem_bytes();
 int decode_threads();
 cudaError_t prepare_kernels();  // sets the dynamic shared-memory attribute; call once per device
-cudaError_t launch_decode(const CUtensorMap &tmap, const DecodeParams &p, int grid, cudaStream_t s);
+// tmap: boxes of kTileTokens rows x 64 elements; tmap_edge: the same matrix in boxes of kEdgeBoxRows rows (only read
+// when p.edge_boxes is set; otherwise pass tmap twice)
+cudaError_t launch_decode(const CUtensorMap &tmap, const CUtensorMap &tmap_edge, const DecodeParams &p, int grid,
+                          cudaStream_t s);
 cudaError_t prepare_shared_kernel();
 cudaError_t launch_shared(const CUtensorMap &tmap, const SharedParams &p, int grid, cudaStream_t s);
 cudaError_t launch_merge(const MergeParams &p, int n_merges, cudaStream_t s);

@@ -33,6 +33,10 @@ constexpr int kThreads = kConsumerThreads + 32;
 constexpr uint32_t kHalfBytes = kTileTokens * 128;    // 64 tokens x 64 dims of bf16
 constexpr uint32_t kTileBytes = 2 * kHalfBytes;       // K or V tile: 64 tokens x 128 dims
 constexpr uint32_t kStageBytes = 2 * kTileBytes;      // K tile then V tile
+constexpr uint32_t kEdgeRows = kEdgeBoxRows;           // rows of the small box that ragged tiles are fetched in
+constexpr uint32_t kEdgeBoxBytes = kEdgeRows * 128;    // kEdgeRows tokens x 64 dims of bf16
+static_assert(kEdgeRows % 16 == 0 && kTileTokens % kEdgeRows == 0,
+              "an edge box must hold whole 8-row swizzle groups and whole 16-token steps of the P V product");
 constexpr int kScratchStride = 132;                   // floats per scratch row (128 + pad)
 constexpr uint32_t kScratchOBytes = kConsumerWarps * kMaxGroup * kScratchStride * 4;
 constexpr uint32_t kScratchMLBytes = 2 * kConsumerWarps * kMaxGroup * 2 * 4;  // two buffers
@@ -174,7 +178,8 @@ __device__ __forceinline__ void process_tile(WarpState &st, const uint32_t (&qa0
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
-cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeParams p)
+cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ CUtensorMap tmap_edge,
+                   const DecodeParams p)
 {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -216,7 +221,10 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeParams 
 
     if (warp == kConsumerWarps) {
         // ================= producer: the warp walks the items together, lane 0 feeds the ring =========
-        if (lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap)) : "memory");
+        if (lane == 0) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap)) : "memory");
+            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap_edge)) : "memory");
+        }
         uint32_t t = 0;  // tiles issued by this block so far
         bool ok = true;
         const uint64_t stream_once = l2_evict_first_policy();  // a tile is read once per launch: let it leave L2 first
@@ -259,12 +267,37 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeParams 
                     const uint32_t vdst = kdst + kTileBytes;
                     const int32_t yk = (int32_t)(k_row + j * kTileTokens);
                     const int32_t yv = (int32_t)(v_row + j * kTileTokens);
-                    mbar_expect_tx(full_k(s), kTileBytes);
-                    tma_load_2d_hint(kdst, &tmap, 0, yk, full_k(s), stream_once);
-                    tma_load_2d_hint(kdst + kHalfBytes, &tmap, 64, yk, full_k(s), stream_once);
-                    mbar_expect_tx(full_v(s), kTileBytes);
-                    tma_load_2d_hint(vdst, &tmap, 0, yv, full_v(s), stream_once);
-                    tma_load_2d_hint(vdst + kHalfBytes, &tmap, 64, yv, full_v(s), stream_once);
+                    const uint32_t valid = min((uint32_t)kTileTokens, w.n_tok - j * kTileTokens);
+                    if (p.edge_boxes != 0u && valid + kEdgeRows <= (uint32_t)kTileTokens) {
+                        // Ragged last tile of a segment that leaves at least one small box empty: only the boxes
+                        // that hold tokens are fetched (the consumers read no row past the 16-row step that
+                        // holds the last token), not the rows that follow the segment in memory.  A small box
+                        // is a whole number of 8-row swizzle groups, so the tile's layout is unchanged.  (Boxes
+                        // of 16 rows save more bytes but cost up to three times the copy instructions, which
+                        // made batches of many short segments slower.)
+                        const uint32_t nb = (valid + kEdgeRows - 1u) / kEdgeRows;
+                        mbar_expect_tx(full_k(s), nb * 2u * kEdgeBoxBytes);
+                        for (uint32_t b = 0; b < nb; ++b) {
+                            tma_load_2d_hint(kdst + b * kEdgeBoxBytes, &tmap_edge, 0, yk + (int32_t)(b * kEdgeRows),
+                                             full_k(s), stream_once);
+                            tma_load_2d_hint(kdst + kHalfBytes + b * kEdgeBoxBytes, &tmap_edge, 64,
+                                             yk + (int32_t)(b * kEdgeRows), full_k(s), stream_once);
+                        }
+                        mbar_expect_tx(full_v(s), nb * 2u * kEdgeBoxBytes);
+                        for (uint32_t b = 0; b < nb; ++b) {
+                            tma_load_2d_hint(vdst + b * kEdgeBoxBytes, &tmap_edge, 0, yv + (int32_t)(b * kEdgeRows),
+                                             full_v(s), stream_once);
+                            tma_load_2d_hint(vdst + kHalfBytes + b * kEdgeBoxBytes, &tmap_edge, 64,
+                                             yv + (int32_t)(b * kEdgeRows), full_v(s), stream_once);
+                        }
+                    } else {
+                        mbar_expect_tx(full_k(s), kTileBytes);
+                        tma_load_2d_hint(kdst, &tmap, 0, yk, full_k(s), stream_once);
+                        tma_load_2d_hint(kdst + kHalfBytes, &tmap, 64, yk, full_k(s), stream_once);
+                        mbar_expect_tx(full_v(s), kTileBytes);
+                        tma_load_2d_hint(vdst, &tmap, 0, yv, full_v(s), stream_once);
+                        tma_load_2d_hint(vdst + kHalfBytes, &tmap, 64, yv, full_v(s), stream_once);
+                    }
                 }
             }
         }
@@ -494,11 +527,12 @@ cudaError_t prepare_kernels()
     return cudaFuncSetAttribute(cart_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
 }
 
-cudaError_t launch_decode(const CUtensorMap &tmap, const DecodeParams &p, int grid, cudaStream_t s)
+cudaError_t launch_decode(const CUtensorMap &tmap, const CUtensorMap &tmap_edge, const DecodeParams &p, int grid,
+                          cudaStream_t s)
 {
     cudaLaunchAttribute attr;
     const cudaLaunchConfig_t cfg = pdl_config(grid, kThreads, kSmemBytes, s, &attr);
-    return cudaLaunchKernelEx(&cfg, cart_decode_kernel, tmap, p);
+    return cudaLaunchKernelEx(&cfg, cart_decode_kernel, tmap, tmap_edge, p);
 }
 
 cudaError_t launch_merge(const MergeParams &p, int n_merges, cudaStream_t s)

@@ -159,6 +159,6 @@ extern "C" cart_status cart_decode_attention_static(const void *q, const void *k
     dp.group = n_q_heads / n_kv_heads;
     const float scale = softmax_scale > 0.f ? softmax_scale : 0.08838834764831845f;  // 1/sqrt(128)
     dp.scale_log2 = scale * 1.4426950408889634f;
-    if (launch_decode(tmap, dp, n_cta_used, s) != cudaSuccess) return CART_ERR_CUDA;
+    if (launch_decode(tmap, tmap, dp, n_cta_used, s) != cudaSuccess) return CART_ERR_CUDA;  // whole tiles only
     return CART_OK;
 }
