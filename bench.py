@@ -40,7 +40,7 @@ WORKLOADS = {
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the decode kernel, from the ncu capture
 # summarised under profiles/ (a smaller case of the same kernel, scaled by KV bytes); None = not captured.
-NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = {"c2": 615.87 / 608.27}   # profiles/decode_kernel_c2.md
+NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = {"c2": 617.90 / 608.27}   # profiles/decode_kernel_c2.md
 
 
 def measured_peak_gbs():

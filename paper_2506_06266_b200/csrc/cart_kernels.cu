@@ -4,7 +4,9 @@
 // Decode kernel in one paragraph.  One persistent block per SM walks its list of work items (runs
 // of 64-token tiles of one KV segment of one (request, KV head) row group).  A producer warp streams
 // K and V tiles from HBM into a ring of shared-memory stages with TMA (cp.async.bulk.tensor, 128-byte
-// swizzle, completion on mbarriers); each stage has its own consumer warp, which takes whole tiles.  A
+// swizzle, completion on mbarriers); each stage has its own consumer warp, which takes whole tiles.  In a
+// fused decode step one more warp writes the requests' new tokens into their suffixes and tells the
+// producer, which fetches a tile that ends with such a token only afterwards.  A
 // consumer multiplies the group's G query heads (padded to the 16 rows of an m16n8k16 bf16 MMA, so
 // a K/V tile is read once per group) with the tile, keeps an fp32 online softmax (running max, sum,
 // rescaled output) in registers, and multiplies the probabilities with V.  At the end of a row-group
@@ -29,7 +31,7 @@ constexpr int kStages = 6;
 // current phase from the one before.)
 constexpr int kConsumerWarps = kStages;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
-constexpr int kThreads = kConsumerThreads + 32;
+constexpr int kThreads = kConsumerThreads + 64;      // + the producer warp + the append warp
 constexpr uint32_t kHalfBytes = kTileTokens * 128;    // 64 tokens x 64 dims of bf16
 constexpr uint32_t kTileBytes = 2 * kHalfBytes;       // K or V tile: 64 tokens x 128 dims
 constexpr uint32_t kStageBytes = 2 * kTileBytes;      // K tile then V tile
@@ -191,11 +193,13 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
     const uint32_t bars = base + kStages * kStageBytes + kScratchOBytes + kScratchMLBytes;
     volatile uint32_t *abort_flag =
         reinterpret_cast<volatile uint32_t *>(smem + kStages * kStageBytes + kScratchOBytes + kScratchMLBytes + kBarrierBytes);
-    volatile uint32_t *arrivals = abort_flag + 1;   // [2] warps that have deposited their state of a piece
+    volatile uint32_t *arrivals = abort_flag + 1;   // [0], [1]: warps that have deposited their state of a piece; [2]: see append_count
     auto full_k = [&](int s) { return bars + (uint32_t)s * 8u; };
     auto full_v = [&](int s) { return bars + (uint32_t)(kStages + s) * 8u; };
     auto empty = [&](int s) { return bars + (uint32_t)(2 * kStages + s) * 8u; };
     auto scratch_free = [&](uint32_t b) { return bars + (uint32_t)(3 * kStages) * 8u + b * 8u; };
+    // [1] how many of the block's new tokens (in work-list order) are in the arena: append warp -> producer
+    const uint32_t append_count = smem_u32(const_cast<uint32_t *>(arrivals + 2));
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -212,6 +216,7 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
         *abort_flag = 0;
         arrivals[0] = 0;
         arrivals[1] = 0;
+        arrivals[2] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -233,6 +238,7 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
         // lies in the last tile of an item marked CART_ITEM_TAIL.  Everything else in the arena is
         // written by copies or by kernels that complete before this one may start.
         bool waited = false;
+        uint32_t tails_seen = 0;  // tiles met so far that end with a new token
         for (uint32_t it = item_begin; it < item_end && ok; ++it) {
             const cart_work_item w = p.items[it];
             const uint32_t k_row = w.k_row + (uint32_t)p.layer * w.layer_stride;
@@ -250,17 +256,34 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
                     waited = true;
                 }
                 if (p.k_new != nullptr && (w.flags & CART_ITEM_TAIL) && j + 1 == ntiles) {
-                    // Fused append (decode phase of Sec. 2.3): this tile ends with the request's new token.
-                    // Write its K row (lanes 0-15) and V row (lanes 16-31) into the suffix before the tile
-                    // is fetched; no other block reads these rows in this launch.
-                    const uint32_t c = (uint32_t)lane & 15u;
-                    const uint4 *src = reinterpret_cast<const uint4 *>(lane < 16 ? p.k_new : p.v_new) +
-                                       (size_t)w.row_group * 16 + c;
-                    const size_t dst_row = (size_t)(lane < 16 ? k_row : v_row) + (w.n_tok - 1);
-                    reinterpret_cast<uint4 *>(p.arena)[dst_row * 16 + c] = __ldg(src);
-                    __threadfence();
-                    asm volatile("fence.proxy.async;" ::: "memory");  // generic-proxy stores before the TMA read
-                    __syncwarp();
+                    // Fused append: this tile ends with the request's new token, which the append warp writes.
+                    // It works through the block's list far ahead of the producer.
+                    ++tails_seen;
+                    bool ok1 = true;
+                    if (lane == 0) {
+                        uint32_t spins = 0;
+                        long long t0 = 0;
+                        for (;;) {
+                            uint32_t done;
+                            asm volatile("ld.acquire.cta.shared.u32 %0, [%1];" : "=r"(done) : "r"(append_count) : "memory");
+                            if (done >= tails_seen) break;
+                            if ((++spins & 0x3FFu) == 0) {  // bounded like every other wait of the kernel
+                                if (*abort_flag) { ok1 = false; break; }
+                                const long long now = clock64();
+                                if (t0 == 0) {
+                                    t0 = now | 1;
+                                } else if (now - t0 > kWaitLimitCycles) {
+                                    *abort_flag = 1;
+                                    atomicOr(p.status, kStatusTimeoutProducer);
+                                    ok1 = false;
+                                    break;
+                                }
+                            }
+                        }
+                        asm volatile("fence.proxy.async;" ::: "memory");  // those generic-proxy stores before this TMA read
+                    }
+                    ok = __shfl_sync(0xffffffffu, (int)ok1, 0) != 0;
+                    if (!ok) break;
                 }
                 if (lane == 0) {
                     const uint32_t kdst = stages + (uint32_t)s * kStageBytes;
@@ -311,6 +334,63 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
                 const uint64_t t0 = global_timer_ns();
                 while (!mbar_try_wait(full_k(s), par) && global_timer_ns() - t0 < kWaitLimitNs) {}
                 while (!mbar_try_wait(full_v(s), par) && global_timer_ns() - t0 < kWaitLimitNs) {}
+            }
+        }
+        return;
+    }
+
+    if (warp == kConsumerWarps + 1) {
+        // ================= append warp (decode phase of Sec. 2.3, fused) ===============================
+        // Writes the new token of every request whose cache ends in this block's work list to the end of
+        // its suffix -- K row by lanes 0-15, V row by lanes 16-31, 256 bytes each -- and then tells the
+        // producer, which fetches the tiles that hold these rows only afterwards.  No other block reads
+        // them in this launch.  Doing this on a warp of its own keeps the producer issuing copies.
+        if (p.k_new != nullptr) {
+            const uint32_t c = (uint32_t)lane & 15u;
+            bool waited = false;
+            const uint4 *new_rows = reinterpret_cast<const uint4 *>(lane < 16 ? p.k_new : p.v_new);
+            uint32_t n_done = 0;
+            for (uint32_t base_it = item_begin; base_it < item_end; base_it += 32u) {
+                const uint32_t mine = base_it + (uint32_t)lane;
+                cart_work_item a{};
+                if (mine < item_end) a = p.items[mine];
+                uint32_t tails = __ballot_sync(0xffffffffu, (a.flags & CART_ITEM_TAIL) != 0u);
+                if (!waited) {
+                    pdl_wait();  // k_new and v_new come from the kernels before (the plan does not: it is read above)
+                    waited = true;
+                }
+                while (tails) {
+                    // up to four requests at a time, their loads in flight together; the very first one alone,
+                    // so that the producer does not wait long for it at the start of a launch
+                    uint4 val[4];
+                    size_t dst[4];
+                    int n = 0;
+                    const int batch = n_done == 0u ? 1 : 4;
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        if (tails && u < batch) {
+                            const int src_lane = __ffs((int)tails) - 1;
+                            tails &= tails - 1u;
+                            const uint32_t a_k = __shfl_sync(0xffffffffu, a.k_row, src_lane);
+                            const uint32_t a_v = __shfl_sync(0xffffffffu, a.v_row, src_lane);
+                            const uint32_t row0 = lane < 16 ? a_k : a_v;
+                            const uint32_t a_ls = __shfl_sync(0xffffffffu, a.layer_stride, src_lane);
+                            const uint32_t a_n = __shfl_sync(0xffffffffu, a.n_tok, src_lane);
+                            const uint32_t a_rg = __shfl_sync(0xffffffffu, a.row_group, src_lane);
+                            val[u] = __ldg(new_rows + (size_t)a_rg * 16 + c);
+                            dst[u] = ((size_t)row0 + (size_t)p.layer * a_ls + (a_n - 1u)) * 16 + c;
+                            n = u + 1;
+                        }
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        if (u < n) reinterpret_cast<uint4 *>(p.arena)[dst[u]] = val[u];
+                    __threadfence();  // the rows are in memory before the producer hears of them
+                    __syncwarp();
+                    n_done += (uint32_t)n;
+                    if (lane == 0)
+                        asm volatile("st.release.cta.shared.u32 [%0], %1;" ::"r"(append_count), "r"(n_done) : "memory");
+                }
             }
         }
         return;
