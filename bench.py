@@ -145,6 +145,8 @@ def run_ours(args):
     ctx = lw.ctx
     if args.piece_cost >= 0:
         binding.cart_set_piece_cost(ctx, args.piece_cost)
+    if args.side_by_side >= 0:
+        binding.cart_set_side_by_side(ctx, args.side_by_side)
 
     q = w.queries(0, dev)
     k_new, v_new = w.appended_kv(0, dev)
@@ -476,6 +478,10 @@ def main():
                     help="append and attend with two calls per layer instead of cart_decode_step")
     ap.add_argument("--piece-cost", type=int, default=-1,
                     help="planner tuning (cart_set_piece_cost); -1 keeps the library's default")
+    ap.add_argument("--side-by-side", type=int, default=-1,
+                    help="planner tuning (cart_set_side_by_side): 0 = shared and stream kernel one after the other, "
+                         "1 = side by side with the planner's division, N > 1 = N blocks for the shared kernel; "
+                         "-1 keeps the library's default")
     ap.add_argument("--kernel-events", action="store_true",
                     help="bracket every decode call's kernels with a pair of CUDA events and report their mean "
                          "duration; the events sit between the kernels, so a kernel can then no longer start "

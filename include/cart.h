@@ -4,8 +4,8 @@
  * The library serves the attention part of decoding with Cartridges (arXiv 2506.06266): every
  * request attends over a trained, compact KV cache (a Cartridge of p key/value tokens per layer,
  * Sec. 3.2; possibly several Cartridges concatenated, Sec. 3.1 / Sec. 5.4; possibly shared by many
- * requests and stored once) followed by the request's own growing suffix KV (Sec. 2.3), exactly as
- * "a request with a prefix of length p" (Sec. 3.3).
+ * requests and stored once) followed by the request's own growing suffix KV (Sec. 2.3): a Cartridge is
+ * served like a cached prefix of p tokens (Sec. 3.3).
  *
  * Conventions that hold for every entry point
  *   - Returns a cart_status.  Out-parameters are written only on CART_OK.  Nothing throws, aborts
@@ -17,9 +17,14 @@
  *   - All device memory comes from the caller: the arena handed to cart_create and the q / k / v /
  *     out tensors passed per call.  The library itself never allocates device memory.  The arena
  *     stays owned by the caller and must outlive the context.
- *   - Calls that take a stream enqueue work on it and return without synchronising.  A context is
+ *   - Calls that take a stream enqueue work on it and return without synchronising the stream or the
+ *     device, with one bounded exception: the attention calls keep their work lists (plans) in a ring of
+ *     four device buffers, and a call that has to build a new plan first waits on the host until the
+ *     kernels that used the buffer three plans back have finished (back-pressure; in a decode loop a
+ *     plan is kept for many steps, so this wait is rare and normally already satisfied).  A context is
  *     meant to be driven from one host thread on one stream at a time; to switch streams the caller
- *     orders them (event or synchronise).
+ *     orders them (event or synchronise).  Capturing calls into a CUDA graph is not supported: lengths and
+ *     plans live on the host and change from call to call.
  *   - Tensors are bf16 (upper half of IEEE binary32), head_dim = 128, dense row-major in the stated
  *     index order.  Device tensor pointers must be 16-byte aligned.
  *   - Query head h reads KV head h / (n_q_heads / n_kv_heads) (contiguous groups).
@@ -87,8 +92,7 @@ CART_API cart_status cart_create(const cart_config *cfg /*host*/, cart_ctx **out
 /* Synchronises the device, frees host-side state.  The arena is untouched.  NULL is accepted. */
 CART_API cart_status cart_destroy(cart_ctx *ctx);
 
-/* Sec. 3.2 / Sec. 3.3: make a trained Cartridge resident ("loaded into the KV cache slots") and
- * addressable by handle.  k and v are bf16 [n_layers][n_kv_heads][p][128], in device memory or in host
+/* Sec. 3.2 / Sec. 3.3: make a trained Cartridge resident in the KV cache and addressable by handle.  k and v are bf16 [n_layers][n_kv_heads][p][128], in device memory or in host
  * memory (a Cartridge loaded from disk and swapped in while other requests decode: page-locked host
  * memory makes the copy asynchronous); they are copied into the arena on `stream` (the caller may free
  * or reuse them once the stream has passed this point).  p >= 1, the same in every layer.  A Cartridge
@@ -97,7 +101,7 @@ CART_API cart_status cart_destroy(cart_ctx *ctx);
 CART_API cart_status cart_register_cartridge(cart_ctx *ctx, const void *k /*device or host*/, const void *v /*device or host*/,
                                     int32_t p, void *stream /*cudaStream_t*/, cart_id *out /*host*/);
 
-/* Sec. 3.1 ("capable of composition"), Sec. 5.4: the handle returned stands for the concatenation
+/* Composition (Sec. 3.1, Sec. 5.4): the handle returned stands for the concatenation
  * [Z_1, Z_2, ...] of the parts along the token axis, in list order, with no retraining, no copy and
  * no re-encoding of positions.  Parts may themselves be compositions (flattened).  The parts stay
  * referenced until the composition is released.  parts is a host array.
@@ -130,7 +134,7 @@ CART_API cart_status cart_request_reserve(cart_ctx *ctx, cart_req req, int32_t s
 /* Closes a request and returns its suffix buffer to the arena.  Errors: BAD_HANDLE. */
 CART_API cart_status cart_request_close(cart_ctx *ctx, cart_req req);
 
-/* Sec. 2.3, decode phase ("append to the KV cache"): for i < n_reqs, writes token i of k_new / v_new
+/* Sec. 2.3, decode phase (the new token's key and value join the KV cache): for i < n_reqs, writes token i of k_new / v_new
  * (device bf16 [n_reqs][n_kv_heads][128]) at the end of request reqs[i]'s suffix in `layer`, and
  * advances that length by one.  reqs is a host array; a handle may appear at most once.
  * Errors: INVALID_ARG, BAD_HANDLE, CAPACITY (some suffix is full; nothing is appended), CUDA. */
@@ -151,7 +155,8 @@ CART_API cart_status cart_extend_kv(cart_ctx *ctx, int32_t layer, cart_req req, 
  * [n_reqs][n_q_heads][128]; lse is device fp32 [n_reqs][n_q_heads] or NULL.  Products and sums are
  * accumulated in fp32; out is rounded to nearest-even bf16.  reqs is a host array (duplicates
  * allowed).  The result does not depend on how the library splits the cache across thread blocks
- * beyond fp32 rounding, and is bitwise reproducible for the same batch and lengths.
+ * beyond fp32 rounding, and is bitwise reproducible for the same sequence of calls (the split is a
+ * function of the batch, its lengths and the plan that was kept, see cart_set_plan_reuse).
  * Errors: INVALID_ARG, BAD_HANDLE, EMPTY, CAPACITY (batch larger than max_requests), CUDA. */
 CART_API cart_status cart_decode_attention(cart_ctx *ctx, int32_t layer, const cart_req *reqs /*host*/,
                                   int32_t n_reqs, const void *q /*device*/, void *out /*device*/,
@@ -191,12 +196,32 @@ CART_API cart_status cart_prefill_attention(cart_ctx *ctx, int32_t layer, cart_r
  * request streams its whole cache).  Errors: INVALID_ARG. */
 CART_API cart_status cart_set_share_min_readers(cart_ctx *ctx, int32_t min_readers);
 
+/* How a batch with a shared part is run.  1 (default): the tensor-core kernel for the shared Cartridges and
+ * the stream kernel for the requests' own tokens are resident at the same time, each on its share of the
+ * SMs (the first is bound by latencies, the second by HBM bandwidth, which three quarters of the SMs nearly
+ * saturate); the planner chooses the division.  0: one after the other, each on all SMs.  2 .. SMs - 1:
+ * side by side with exactly this many blocks for the tensor-core kernel.  Results are the same up to fp32
+ * rounding.  Errors: INVALID_ARG. */
+CART_API cart_status cart_set_side_by_side(cart_ctx *ctx, int32_t mode);
+
 /* Planner tuning.  The stream kernel's blocks are given equal shares of tiles + tiles_per_piece * pieces,
  * a piece being the part of a (request, KV head) cache that one block handles; the constant stands
  * for what finishing a piece (combining the warps' states, writing the result) costs a block, in
  * units of the time a 64-token tile takes.  Default 3; 0 balances by tiles alone; at most 64.  The
  * results do not depend on it beyond fp32 rounding.  Errors: INVALID_ARG. */
 CART_API cart_status cart_set_piece_cost(cart_ctx *ctx, int32_t tiles_per_piece);
+
+/* Plan reuse.  The attention calls split the batch's KV tokens over the thread blocks on the host (a
+ * "plan") and upload the result.  In a decode loop (Sec. 2.3) every request grows by one token per step, so
+ * a plan is kept while the batch is the same and every request has grown by the same number of tokens, at
+ * most max_grow_tokens, since the plan was built; the kernels add that number to the last run of every
+ * request.  Default 192; 0 builds a new plan whenever a length has changed.  Results are the same up to
+ * fp32 rounding.  Errors: INVALID_ARG. */
+CART_API cart_status cart_set_plan_reuse(cart_ctx *ctx, int32_t max_grow_tokens);
+
+/* Number of plans this context has built and uploaded so far (a decode loop that keeps its plan does
+ * not advance it). */
+CART_API uint64_t cart_plan_count(const cart_ctx *ctx);
 
 /* Current suffix length of a request in a layer (host-side mirror). */
 CART_API cart_status cart_suffix_len(cart_ctx *ctx, cart_req req, int32_t layer, int32_t *out_len /*host*/);
@@ -243,7 +268,10 @@ CART_API cart_status cart_get_timing(cart_ctx *ctx, double *total_ms /*host*/, u
  * call may wait for earlier work on `stream` before it returns.  All calls share the one scratch
  * array, which keeps the previous call's contents (the call clears what it needs zeroed): calls
  * whose GPU work may overlap -- different streams, different host threads -- race and must be
- * ordered by the caller.  A device-side wait that ran out is not reported by this entry point.
+ * ordered by the caller.  The host copy of the work list is one fixed array too, so calls from different
+ * host threads must not overlap either.  A device-side wait that ran out is not reported by this entry
+ * point.  A CART_ERR_CUDA return may leave the clearing of the scratch or the copy of the work list
+ * enqueued on `stream` (harmless: the next call redoes both).
  * Errors: INVALID_ARG, SHAPE, CAPACITY, CUDA. */
 #define CART_STATIC_MAX_ROW_GROUPS 2048
 #define CART_STATIC_SCRATCH_BYTES 2228224

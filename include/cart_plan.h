@@ -32,13 +32,20 @@ typedef struct {
     uint32_t head_stride;  /* rows between consecutive KV heads (p, or the suffix capacity) */
     uint32_t layer_stride; /* rows between consecutive layers (n_kv_heads * head_stride) */
     uint32_t n_tok;        /* tokens in the segment (> 0) */
+    uint32_t flags;        /* CART_SEG_* */
 } cart_plan_seg;
+
+#define CART_SEG_SUFFIX 1u  /* the segment lies in a request's suffix buffer, which kernels write (append, extend,
+                               fused decode step); a stored Cartridge is only ever written by copies */
 
 #define CART_ITEM_BEGIN 1u  /* first item of a row-group piece in this block: load q, reset state */
 #define CART_ITEM_END 2u    /* last item of the piece: combine the warps' states and write */
 #define CART_ITEM_DIRECT 4u /* the piece is the whole row group: write out / lse, not a partial */
 #define CART_ITEM_TAIL 8u   /* the item ends with the last token of the request's cache (the token a fused
                                append + decode call writes before it attends) */
+#define CART_ITEM_SUFFIX 16u /* the item's tiles lie in suffix storage (CART_SEG_SUFFIX): a kernel earlier on the
+                               stream may have written them, so they are fetched only once those kernels are
+                               known to be complete; Cartridge tiles may be fetched ahead of that */
 
 /* A run of consecutive tiles of one segment of one row group, processed by one block. */
 typedef struct {
@@ -107,9 +114,12 @@ typedef struct {
     uint32_t n_tiles;      /* full tiles of share_tile_tokens tokens in the run (> 0) */
     uint32_t reader_begin; /* first entry of the M-tile in readers[] */
     uint32_t n_readers;    /* entries of the M-tile (1 .. 128 / group) */
-    uint32_t kv_head;
+    uint16_t kv_head;
+    uint16_t flags;        /* CART_UNIT_SUFFIX: the run lies in suffix storage (see CART_ITEM_SUFFIX) */
     uint32_t chunk;        /* ordinal of the run among the runs of its (segment, M-tile, KV head) */
 } cart_shared_unit;
+
+#define CART_UNIT_SUFFIX 1u
 
 /* Capacities (in) and results (out) of cart_plan_build_shared; all arrays are host memory. */
 typedef struct {
@@ -133,6 +143,11 @@ typedef struct {
     int64_t shared_tiles;      /* tile runs handed to the shared kernel, in share_tile_tokens tiles */
     int32_t unit_cost;         /* in: what a shared unit costs a block on top of its tiles, in tile times; the
                                   shared blocks are balanced by tiles + unit_cost * units (0: by tiles alone) */
+    int32_t side_by_side;      /* in: 0 = the shared kernel and the stream kernel each get all n_cta blocks (they run
+                                  one after the other); 1 = the n_cta blocks are divided between them so that both
+                                  are resident at once (chosen from the two parts' estimated times); > 1 = the
+                                  same with exactly this many blocks for the shared kernel (< n_cta) */
+    int32_t n_shared_ctas;     /* out: blocks set aside for the shared kernel when running side by side (else 0) */
 } cart_plan_out;
 
 /*
@@ -140,6 +155,10 @@ typedef struct {
  * tile_tokens as in cart_plan_build; group = query heads per KV head (1..8);
  * share_min_readers = 0 disables sharing (the result then equals cart_plan_build's);
  * share_tile_tokens is a multiple of tile_tokens.
+ * Side by side (out->side_by_side): the tensor-core kernel is bound by latencies and barely touches HBM,
+ * the stream kernel is bound by HBM bandwidth and loses little of it on three quarters of the SMs, so a
+ * batch with both parts finishes sooner when the two kernels share the SMs than when each has all of
+ * them in turn.  The division is chosen by minimising the larger of the two parts' estimated times.
  * If the partial slots the shared chunks need exceed slots_cap, the shared ranges are made longer
  * (fewer blocks, fewer chunks) until they fit; if they cannot fit, nothing is shared.
  * Errors: INVALID_ARG, EMPTY, CAPACITY (an output array is too small).
@@ -148,6 +167,18 @@ CART_API cart_status cart_plan_build_shared(const cart_plan_seg *segs, const int
                                             int32_t n_kv_heads, int32_t group, int32_t n_cta, int32_t tile_tokens,
                                             int32_t share_min_readers, int32_t share_tile_tokens,
                                             cart_plan_out *out);
+
+/*
+ * Plan reuse across decode steps.  A plan built for a batch whose requests had suffix lengths
+ * plan_len[i] stays usable while every request of the same batch has grown by the same number of
+ * tokens d (each fused decode step appends one token to every request, Sec. 2.3): the kernels then
+ * add d to the token count of every item marked CART_ITEM_TAIL, which only lengthens the last run of
+ * every row group.  Returns 1 and writes d to *grow when cur_len[i] - plan_len[i] == d for all i with
+ * 0 <= d <= max_grow, and, if d > 0, every plan_len[i] >= 1 (the tail item then lies in the suffix);
+ * returns 0 otherwise (re-plan).  max_grow bounds how far the blocks' shares may drift apart.
+ */
+CART_API int32_t cart_plan_reusable(const int32_t *plan_len, const int32_t *cur_len, int32_t n_reqs,
+                                    int32_t max_grow, int32_t *grow);
 
 #ifdef __cplusplus
 }

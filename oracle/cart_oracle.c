@@ -6,7 +6,7 @@
  * the benchmark's CPU-baseline leg may use it.  It shares no code with the CUDA path.
  *
  * What it computes (paper Eq. 1 evaluated at the last position i, Sec. 2.3; the Cartridge KV-cache
- * layout of Sec. 3.2; "a prefix of length p" of Sec. 3.3; composition by concatenation, Sec. 3.1
+ * layout of Sec. 3.2; served as a cached prefix of p tokens, Sec. 3.3; composition by concatenation, Sec. 3.1
  * and Sec. 5.4): for request b whose KV cache is the concatenation, in order, of its segments
  * (zero or more Cartridges followed by the request's own suffix), for query head h reading KV head
  * g = h div (Hq/Hkv):

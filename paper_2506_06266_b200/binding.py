@@ -30,6 +30,7 @@ EXPORTS = ["cart_scratch_bytes", "cart_create", "cart_destroy", "cart_register_c
            "cart_append_kv", "cart_extend_kv", "cart_decode_attention", "cart_decode_step", "cart_prefill_attention", "cart_suffix_len",
            "cart_kv_bytes", "cart_sync_status", "cart_set_timing", "cart_get_timing",
            "cart_set_share_min_readers", "cart_set_piece_cost", "cart_plan_build_shared",
+           "cart_set_plan_reuse", "cart_plan_count", "cart_plan_reusable", "cart_set_side_by_side",
            "cart_decode_attention_static", "cart_launch_count", "cart_status_string",
            "cart_last_error", "cart_plan_build"]
 
@@ -46,7 +47,7 @@ class cart_config(ctypes.Structure):
 class cart_plan_seg(ctypes.Structure):
     _fields_ = [("k_row", ctypes.c_uint32), ("v_row", ctypes.c_uint32),
                 ("head_stride", ctypes.c_uint32), ("layer_stride", ctypes.c_uint32),
-                ("n_tok", ctypes.c_uint32)]
+                ("n_tok", ctypes.c_uint32), ("flags", ctypes.c_uint32)]
 
 
 class cart_work_item(ctypes.Structure):
@@ -65,7 +66,7 @@ class cart_shared_unit(ctypes.Structure):
     _fields_ = [("k_row", ctypes.c_uint32), ("v_row", ctypes.c_uint32),
                 ("layer_stride", ctypes.c_uint32), ("n_tiles", ctypes.c_uint32),
                 ("reader_begin", ctypes.c_uint32), ("n_readers", ctypes.c_uint32),
-                ("kv_head", ctypes.c_uint32), ("chunk", ctypes.c_uint32)]
+                ("kv_head", ctypes.c_uint16), ("flags", ctypes.c_uint16), ("chunk", ctypes.c_uint32)]
 
 
 class cart_plan_out(ctypes.Structure):
@@ -82,10 +83,13 @@ class cart_plan_out(ctypes.Structure):
                 ("n_readers", ctypes.c_int32),
                 ("reader_slot", ctypes.POINTER(ctypes.c_uint32)),
                 ("reader_merge", ctypes.POINTER(ctypes.c_uint32)),
-                ("shared_tiles", ctypes.c_int64), ("unit_cost", ctypes.c_int32)]
+                ("shared_tiles", ctypes.c_int64), ("unit_cost", ctypes.c_int32),
+                ("side_by_side", ctypes.c_int32), ("n_shared_ctas", ctypes.c_int32)]
 
 
-CART_ITEM_BEGIN, CART_ITEM_END, CART_ITEM_DIRECT, CART_ITEM_TAIL = 1, 2, 4, 8
+CART_ITEM_BEGIN, CART_ITEM_END, CART_ITEM_DIRECT, CART_ITEM_TAIL, CART_ITEM_SUFFIX = 1, 2, 4, 8, 16
+CART_SEG_SUFFIX = 1
+CART_UNIT_SUFFIX = 1
 
 
 class CartError(RuntimeError):
@@ -134,6 +138,11 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.cart_decode_attention_static.argtypes = [vp, vp, i32, i32, i32, i32, ctypes.c_float, vp, vp, i32, vp]
     lib.cart_launch_count.argtypes = [vp]
     lib.cart_launch_count.restype = ctypes.c_uint64
+    lib.cart_plan_count.argtypes = [vp]
+    lib.cart_plan_count.restype = ctypes.c_uint64
+    lib.cart_set_plan_reuse.argtypes = [vp, i32]
+    lib.cart_set_side_by_side.argtypes = [vp, i32]
+    lib.cart_plan_reusable.argtypes = [i32p, i32p, i32, i32, i32p]
     lib.cart_status_string.argtypes = [ctypes.c_int]
     lib.cart_status_string.restype = ctypes.c_char_p
     lib.cart_last_error.argtypes = [vp]
@@ -146,7 +155,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
                                            ctypes.POINTER(cart_plan_out)]
     for name in EXPORTS:
         fn = getattr(lib, name)
-        if name not in ("cart_launch_count", "cart_status_string", "cart_last_error"):
+        if name not in ("cart_launch_count", "cart_plan_count", "cart_status_string", "cart_last_error"):
             fn.restype = ctypes.c_int
     if path is None:
         _lib = lib
@@ -308,6 +317,28 @@ def cart_set_piece_cost(ctx: int, tiles_per_piece: int) -> None:
     _check(load_library().cart_set_piece_cost(ctx, int(tiles_per_piece)), "cart_set_piece_cost", ctx)
 
 
+def cart_set_side_by_side(ctx: int, mode: int) -> None:
+    _check(load_library().cart_set_side_by_side(ctx, int(mode)), "cart_set_side_by_side", ctx)
+
+
+def cart_set_plan_reuse(ctx: int, max_grow_tokens: int) -> None:
+    _check(load_library().cart_set_plan_reuse(ctx, int(max_grow_tokens)), "cart_set_plan_reuse", ctx)
+
+
+def cart_plan_count(ctx: int) -> int:
+    return int(load_library().cart_plan_count(ctx))
+
+
+def cart_plan_reusable(plan_len: Sequence[int], cur_len: Sequence[int], max_grow: int) -> Optional[int]:
+    """Host-only: the common growth d if a plan built at plan_len serves cur_len, else None."""
+    n = len(plan_len)
+    a = (ctypes.c_int32 * max(n, 1))(*[int(x) for x in plan_len])
+    b = (ctypes.c_int32 * max(n, 1))(*[int(x) for x in cur_len])
+    d = ctypes.c_int32(-1)
+    ok = load_library().cart_plan_reusable(a, b, n, int(max_grow), ctypes.byref(d))
+    return int(d.value) if ok else None
+
+
 def cart_get_timing(ctx: int) -> Tuple[float, int]:
     ms, n = ctypes.c_double(0.0), ctypes.c_uint64(0)
     _check(load_library().cart_get_timing(ctx, ctypes.byref(ms), ctypes.byref(n)), "cart_get_timing", ctx)
@@ -359,7 +390,8 @@ def cart_plan_build(segs: Sequence[Sequence[Tuple[int, int, int, int, int]]], n_
 
 def cart_plan_build_shared(segs: Sequence[Sequence[Tuple[int, int, int, int, int]]], n_kv_heads: int, group: int,
                            n_cta: int, tile_tokens: int, share_min_readers: int, share_tile_tokens: int,
-                           slots_cap: int = 1 << 20, piece_cost: int = 0, unit_cost: int = 0):
+                           slots_cap: int = 1 << 20, piece_cost: int = 0, unit_cost: int = 0,
+                           side_by_side: int = 0):
     """Host-only planner with shared segments (see include/cart_plan.h).  Returns a dict with the
     stream plan (items, cta_begin, merges, ...) and the shared part (units, unit_cta_begin, readers,
     reader_slot[entry][head], reader_merge[entry][head])."""
@@ -388,6 +420,7 @@ def cart_plan_build_shared(segs: Sequence[Sequence[Tuple[int, int, int, int, int
     o.merges, o.merges_cap, o.slots_cap = merges, merges_cap, slots_cap
     o.piece_cost = piece_cost
     o.unit_cost = unit_cost
+    o.side_by_side = side_by_side
     o.units, o.units_cap, o.unit_cta_begin = units, units_cap, unit_cta_begin
     o.readers, o.readers_cap, o.reader_slot, o.reader_merge = readers, readers_cap, reader_slot, reader_merge
     st = lib.cart_plan_build_shared(seg_arr, sb, len(segs), n_kv_heads, group, n_cta, tile_tokens,
@@ -398,7 +431,7 @@ def cart_plan_build_shared(segs: Sequence[Sequence[Tuple[int, int, int, int, int
             "merges": [merges[i] for i in range(o.n_merges)], "n_cta_used": o.n_cta_used,
             "n_slots": o.n_slots, "total_tiles": o.total_tiles,
             "units": [units[i] for i in range(o.n_units)], "unit_cta_begin": list(unit_cta_begin),
-            "n_unit_cta_used": o.n_unit_cta_used, "readers": [readers[i] for i in range(nr)],
+            "n_unit_cta_used": o.n_unit_cta_used, "n_shared_ctas": o.n_shared_ctas, "readers": [readers[i] for i in range(nr)],
             "reader_slot": [[reader_slot[e * n_kv_heads + g] for g in range(n_kv_heads)] for e in range(nr)],
             "reader_merge": [[reader_merge[e * n_kv_heads + g] for g in range(n_kv_heads)] for e in range(nr)],
             "shared_tiles": o.shared_tiles}

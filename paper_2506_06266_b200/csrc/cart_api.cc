@@ -30,6 +30,9 @@ constexpr int kShareMinReaders = 4;
 constexpr int kPieceCostTiles = 3;
 // What the planner charges a shared-segment block per unit on top of its tiles, in 128-token tile times.
 constexpr int kUnitCostTiles = 4;
+// A decode plan is kept while every request of the batch has grown by the same number of tokens, up to this
+// many (the blocks' shares drift apart by one tile per 64 tokens of growth and tail item).
+constexpr int kMaxGrowTokens = 192;
 
 struct ScratchLayout {
     uint64_t status_off, tickets_off, plan_off, plan_slot_bytes, cta_begin_off, merges_off, items_off;
@@ -45,7 +48,9 @@ ScratchLayout scratch_layout(const cart_config &c)
     const int parts = c.max_parts > 0 ? c.max_parts : 8;
     const int group = c.n_q_heads / c.n_kv_heads;
     const int row_groups = c.max_requests * c.n_kv_heads;
-    s.items_cap = row_groups * (parts + 1) + kMaxCta;
+    // a row group owns at most parts + 2 segments (Cartridge parts, during prefill the shared head of the
+    // suffix, and the suffix), and every block boundary cuts one item in two
+    s.items_cap = row_groups * (parts + 2) + kMaxCta;
     // a row group with a shared part is always merged; the others only when a block boundary splits them
     s.merges_cap = row_groups + kMaxCta;
     // partial slots: stream pieces (one per row group with a shared part, two per block boundary) plus
@@ -53,7 +58,7 @@ ScratchLayout scratch_layout(const cart_config &c)
     s.slots_cap = 10 * row_groups + 2 * kMaxCta;
     s.readers_cap = c.max_requests * (parts + 1);  // + 1: the shared head of a suffix during prefill
     s.units_cap = s.readers_cap * c.n_kv_heads + kMaxCta;
-    s.status_off = 0;
+    s.status_off = 0;          // the status word; the side-by-side flag sits 128 bytes behind it
     s.tickets_off = kAlign;  // one arrival counter per merge item, zero between launches
     s.plan_off = s.tickets_off + round_up((uint64_t)s.merges_cap * 4, kAlign);
     // one plan slot: [cta_begin][merges][items] [unit_cta_begin][readers][reader_slot][reader_merge][units]
@@ -114,7 +119,10 @@ struct PlanSlot {
     bool ev_recorded = false;
     bool valid = false;
     cudaStream_t last_stream = nullptr;
-    std::vector<uint32_t> key;
+    std::vector<uint32_t> key;   // prefill plans: (request, suffix length, new tokens)
+    std::vector<int32_t> reqs;   // decode plans: the batch and its suffix lengths when the plan was built
+    std::vector<int32_t> lens;
+    bool prefill = false;
     uint64_t epoch = 0;
     int32_t n_items = 0, n_merges = 0, n_cta_used = 0, n_slots = 0;
     int32_t n_units = 0, n_unit_cta_used = 0;
@@ -130,6 +138,10 @@ struct cart_ctx {
     int n_cta = 0;
     int share_min_readers = kShareMinReaders;
     int piece_cost = kPieceCostTiles;
+    int max_grow = kMaxGrowTokens;
+    int side_by_side = 1;        // shared and stream kernel share the SMs (0: one after the other; > 1: blocks for the shared kernel)
+    uint32_t pair_seq = 0;       // counts side-by-side launches (the value the stream kernel hands to the shared kernel)
+    uint64_t plans_built = 0;
     uint64_t n_rows = 0;
     alignas(64) CUtensorMap tmap;
     alignas(64) CUtensorMap tmap_edge;
@@ -145,6 +157,7 @@ struct cart_ctx {
     std::vector<int32_t> head_tmp;
     std::vector<int32_t> seg_begin_tmp;
     std::vector<uint32_t> key_tmp;
+    std::vector<int32_t> len_tmp;
     bool timing = false;
     std::vector<cudaEvent_t> ev_pool;  // pairs: start, stop
     size_t ev_used = 0;
@@ -276,6 +289,8 @@ const char *cart_last_error(const cart_ctx *ctx) { return ctx ? ctx->err : "no c
 
 uint64_t cart_launch_count(const cart_ctx *ctx) { return ctx ? ctx->launches : 0; }
 
+uint64_t cart_plan_count(const cart_ctx *ctx) { return ctx ? ctx->plans_built : 0; }
+
 cart_status cart_scratch_bytes(const cart_config *cfg, uint64_t *out_bytes)
 {
     if (!out_bytes) return CART_ERR_INVALID_ARG;
@@ -375,6 +390,24 @@ cart_status cart_set_piece_cost(cart_ctx *ctx, int32_t tiles)
     if (tiles < 0 || tiles > 64) return fail(ctx, CART_ERR_INVALID_ARG, "piece_cost: out of range");
     ctx->piece_cost = tiles;
     ++ctx->epoch;
+    return CART_OK;
+}
+
+cart_status cart_set_side_by_side(cart_ctx *ctx, int32_t mode)
+{
+    if (!ctx) return CART_ERR_INVALID_ARG;
+    if (mode < 0 || mode >= ctx->n_cta) return fail(ctx, CART_ERR_INVALID_ARG, "side_by_side: out of range");
+    ctx->side_by_side = mode;
+    ++ctx->epoch;
+    return CART_OK;
+}
+
+cart_status cart_set_plan_reuse(cart_ctx *ctx, int32_t max_grow_tokens)
+{
+    if (!ctx) return CART_ERR_INVALID_ARG;
+    if (max_grow_tokens < 0 || max_grow_tokens > (1 << 20))
+        return fail(ctx, CART_ERR_INVALID_ARG, "plan_reuse: out of range");
+    ctx->max_grow = max_grow_tokens;
     return CART_OK;
 }
 
@@ -655,19 +688,22 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int Hkv = ctx->cfg.n_kv_heads;
 
-    // The plan depends on which requests are in the batch and on their lengths in this layer.
+    // The plan depends on which requests are in the batch and on their lengths in this layer.  A decode
+    // plan stays good while every request has grown by the same number of tokens since it was built (one
+    // per fused decode step): the kernels add that number to the tail items.
     std::vector<uint32_t> &key = ctx->key_tmp;
+    std::vector<int32_t> &cur_len = ctx->len_tmp;
     key.clear();
-    key.push_back((uint32_t)n_reqs);
+    cur_len.clear();
     if (prefill) {
         Request *r = get_req(ctx, reqs[0]);
         if (!r) return fail(ctx, CART_ERR_BAD_HANDLE, "prefill: not an open request");
         if (r->len[(size_t)layer] < n_new)
             return fail(ctx, CART_ERR_INVALID_ARG, "prefill: the suffix holds %d tokens, fewer than n_new = %d",
                         r->len[(size_t)layer], n_new);
-        key.push_back(0xFFFFFFFFu);  // no batch of requests starts like this
         key.push_back((uint32_t)reqs[0]);
         key.push_back((uint32_t)r->len[(size_t)layer]);
+        key.push_back((uint32_t)n_new);
     }
     for (int32_t i = 0; i < n_reqs && !prefill; ++i) {
         Request *r = get_req(ctx, reqs[i]);
@@ -675,12 +711,18 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
         const int32_t len = r->len[(size_t)layer];
         if (len == 0 && r->cart == CART_NONE)
             return fail(ctx, CART_ERR_EMPTY, "decode: reqs[%d] has no KV token in layer %d", i, layer);
-        key.push_back((uint32_t)reqs[i]);
-        key.push_back((uint32_t)len);
+        cur_len.push_back(len);
     }
 
     PlanSlot *sl = ctx->cur_slot >= 0 ? &ctx->slots[ctx->cur_slot] : nullptr;
-    if (!(sl && sl->valid && sl->epoch == ctx->epoch && sl->key == key)) {
+    int32_t grow = 0;
+    bool reuse = sl && sl->valid && sl->epoch == ctx->epoch && sl->prefill == prefill;
+    if (reuse && prefill) reuse = sl->key == key;
+    if (reuse && !prefill)
+        reuse = sl->reqs.size() == (size_t)n_reqs && std::memcmp(sl->reqs.data(), reqs, (size_t)n_reqs * sizeof(int32_t)) == 0 &&
+                cart_plan_reusable(sl->lens.data(), cur_len.data(), n_reqs, ctx->max_grow, &grow) != 0;
+    if (!reuse) {
+        grow = 0;
         // Build a new plan in the next ring slot.
         if (sl && sl->valid) {
             CART_CUDA(ctx, cudaEventRecord(sl->ev, sl->last_stream));
@@ -731,6 +773,7 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
                 sg.head_stride = (uint32_t)c.p;
                 sg.layer_stride = (uint32_t)((uint64_t)Hkv * c.p);
                 sg.n_tok = (uint32_t)c.p;
+                sg.flags = 0;
                 segs.push_back(sg);
             };
             if (r.cart != CART_NONE) {
@@ -752,6 +795,7 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
                     sg.head_stride = (uint32_t)r.cap;
                     sg.layer_stride = (uint32_t)((uint64_t)Hkv * r.cap);
                     sg.n_tok = (uint32_t)head;
+                    sg.flags = CART_SEG_SUFFIX;
                     segs.push_back(sg);
                     first = (uint32_t)head;
                 }
@@ -763,6 +807,7 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
                 sg.head_stride = (uint32_t)r.cap;
                 sg.layer_stride = (uint32_t)((uint64_t)Hkv * r.cap);
                 sg.n_tok = (uint32_t)len - first;
+                sg.flags = CART_SEG_SUFFIX;
                 segs.push_back(sg);
             }
             sb.push_back((int32_t)segs.size());
@@ -777,6 +822,7 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
         po.slots_cap = lay.slots_cap;
         po.piece_cost = ctx->piece_cost;
         po.unit_cost = kUnitCostTiles;
+        po.side_by_side = ctx->side_by_side;
         po.units = reinterpret_cast<cart_shared_unit *>(ns.host + lay.units_off);
         po.units_cap = lay.units_cap;
         po.unit_cta_begin = reinterpret_cast<uint32_t *>(ns.host + lay.unit_cta_begin_off);
@@ -801,8 +847,12 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
                                            cudaMemcpyHostToDevice, s));
         }
         ns.key = key;
+        ns.prefill = prefill;
+        ns.reqs.assign(reqs, reqs + (prefill ? 1 : n_reqs));
+        ns.lens = cur_len;
         ns.epoch = ctx->epoch;
         ns.valid = true;
+        ++ctx->plans_built;
         ctx->cur_slot = next;
         sl = &ns;
     }
@@ -829,6 +879,7 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
     dp.layer = layer;
     dp.group = ctx->group;
     dp.scale_log2 = ctx->scale * 1.4426950408889634f;
+    dp.grow = (uint32_t)grow;
     dp.edge_boxes = 1u;
     const bool timed = ctx->timing && ctx->ev_used + 2 <= kMaxTimedLaunches * 2;
     if (timed) {
@@ -838,6 +889,18 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
             ctx->ev_pool.push_back(e);
         }
         CART_CUDA(ctx, cudaEventRecord(ctx->ev_pool[ctx->ev_used], s));
+    }
+    // A batch with a shared part and a stream part runs the two kernels side by side: the stream kernel
+    // is launched first on its share of the SMs, the shared kernel right behind it on the rest (a dependent
+    // launch starts as soon as every block of the kernel before has started).
+    const bool pair = sl->n_units > 0 && sl->n_items > 0 && ctx->side_by_side > 0;
+    if (pair) {
+        dp.ready_flag = reinterpret_cast<uint32_t *>(arena + ctx->lay.status_off + 128);
+        dp.seq = ++ctx->pair_seq;
+    }
+    if (pair) {
+        CART_CUDA(ctx, launch_decode(ctx->tmap, ctx->tmap_edge, dp, sl->n_cta_used, s));
+        ++ctx->launches;
     }
     if (sl->n_units > 0) {
         SharedParams sp;
@@ -859,10 +922,12 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
         sp.n_kv_heads = Hkv;
         sp.n_q_heads = ctx->cfg.n_q_heads;
         sp.scale_log2 = dp.scale_log2;
+        sp.ready_flag = dp.ready_flag;
+        sp.seq = dp.seq;
         CART_CUDA(ctx, launch_shared(ctx->tmap, sp, sl->n_unit_cta_used, s));
         ++ctx->launches;
     }
-    if (sl->n_items > 0) {
+    if (sl->n_items > 0 && !pair) {
         CART_CUDA(ctx, launch_decode(ctx->tmap, ctx->tmap_edge, dp, sl->n_cta_used, s));
         ++ctx->launches;
     }

@@ -41,6 +41,14 @@ struct DecodeParams {
     int32_t layer;
     int32_t group;               // G
     float scale_log2;            // softmax scale * log2(e)
+    // Side by side with the shared-segment kernel (launched right after this one, resident at the same
+    // time): once this kernel knows that the kernels before it are complete, block 0 stores `seq` here and
+    // the shared kernel, which cannot learn it from griddepcontrol.wait without waiting for this kernel
+    // too, reads it.  Null otherwise.
+    uint32_t *ready_flag = nullptr;
+    uint32_t seq = 0;
+    uint32_t grow = 0;           // tokens every request has appended since the plan was built: added to the token
+                                 // count of every item marked CART_ITEM_TAIL
     uint32_t edge_boxes = 0;     // 1: ragged last tiles are fetched in boxes of kEdgeBoxRows rows through the second
                                  // tensor map; 0: every tile is fetched whole
 };
@@ -65,6 +73,11 @@ struct SharedParams {
     int32_t n_kv_heads;
     int32_t n_q_heads;
     float scale_log2;
+    // Side by side with the stream kernel (launched right before this one): "the kernels before the pair
+    // are complete" is read from this flag (>= seq) instead of griddepcontrol.wait, which this kernel then
+    // only executes on its way out, so that it never completes before the stream kernel.  Null: alone.
+    const uint32_t *ready_flag = nullptr;
+    uint32_t seq = 0;
 };
 
 struct MergeParams {

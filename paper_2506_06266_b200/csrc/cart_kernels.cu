@@ -86,7 +86,8 @@ __device__ __forceinline__ void process_tile(WarpState &st, const uint32_t (&qa0
 {
     const int l7 = lane & 7;
     const int lm = lane >> 3;
-    ok = mbar_wait(full_k, parity, abort_flag, status, kStatusTimeoutConsumer);
+    // (the MMA and ldmatrix instructions below are warp-wide: a wait fails for all lanes or for none)
+    ok = __all_sync(0xffffffffu, mbar_wait(full_k, parity, abort_flag, status, kStatusTimeoutConsumer));
     if (!ok) return;
 
     // ---- S = Q K^T : 16 (padded heads) x 64 tokens, fp32 ------------------------------------
@@ -143,7 +144,7 @@ __device__ __forceinline__ void process_tile(WarpState &st, const uint32_t (&qa0
     }
 
     // ---- O += P V ---------------------------------------------------------------------------------
-    ok = mbar_wait(full_v, parity, abort_flag, status, kStatusTimeoutConsumer);
+    ok = __all_sync(0xffffffffu, mbar_wait(full_v, parity, abort_flag, status, kStatusTimeoutConsumer));
     if (!ok) return;
     int ksteps = 4;
     if (valid < kTileTokens) {
@@ -234,13 +235,15 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
         bool ok = true;
         const uint64_t stream_once = l2_evict_first_policy();  // a tile is read once per launch: let it leave L2 first
         // Until the kernels before this one on the stream are known to be complete, only tiles that
-        // they cannot have written are fetched: a fused append writes a request's last token, which
-        // lies in the last tile of an item marked CART_ITEM_TAIL.  Everything else in the arena is
-        // written by copies or by kernels that complete before this one may start.
+        // none of them can have written are fetched: the tiles of stored Cartridges, which only copies
+        // write.  Suffix storage (items marked CART_ITEM_SUFFIX) is written by kernels -- the append and
+        // extend kernels, and the fused append of an earlier decode step, which may be the kernel right
+        // before this one -- so the first suffix tile is fetched only after griddepcontrol.wait.
         bool waited = false;
         uint32_t tails_seen = 0;  // tiles met so far that end with a new token
         for (uint32_t it = item_begin; it < item_end && ok; ++it) {
-            const cart_work_item w = p.items[it];
+            cart_work_item w = p.items[it];
+            if (w.flags & CART_ITEM_TAIL) w.n_tok += p.grow;  // tokens appended since the plan was built
             const uint32_t k_row = w.k_row + (uint32_t)p.layer * w.layer_stride;
             const uint32_t v_row = w.v_row + (uint32_t)p.layer * w.layer_stride;
             const uint32_t ntiles = (w.n_tok + kTileTokens - 1) / kTileTokens;
@@ -251,7 +254,7 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
                 if (lane == 0) ok0 = mbar_wait(empty(s), (round & 1u) ^ 1u, abort_flag, p.status, kStatusTimeoutProducer);
                 ok = __shfl_sync(0xffffffffu, (int)ok0, 0) != 0;
                 if (!ok) break;
-                if (!waited && (w.flags & CART_ITEM_TAIL) && j + 1 == ntiles) {
+                if (!waited && (w.flags & CART_ITEM_SUFFIX)) {
                     pdl_wait();
                     waited = true;
                 }
@@ -375,7 +378,7 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
                             const uint32_t a_v = __shfl_sync(0xffffffffu, a.v_row, src_lane);
                             const uint32_t row0 = lane < 16 ? a_k : a_v;
                             const uint32_t a_ls = __shfl_sync(0xffffffffu, a.layer_stride, src_lane);
-                            const uint32_t a_n = __shfl_sync(0xffffffffu, a.n_tok, src_lane);
+                            const uint32_t a_n = __shfl_sync(0xffffffffu, a.n_tok, src_lane) + p.grow;
                             const uint32_t a_rg = __shfl_sync(0xffffffffu, a.row_group, src_lane);
                             val[u] = __ldg(new_rows + (size_t)a_rg * 16 + c);
                             dst[u] = ((size_t)row0 + (size_t)p.layer * a_ls + (a_n - 1u)) * 16 + c;
@@ -398,6 +401,8 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
 
     // ===================== consumers ==============================================================
     pdl_wait();  // q, the partial slots and the tickets belong to the kernels before until they are done
+    if (p.ready_flag != nullptr && blockIdx.x == 0 && threadIdx.x == 0)  // tell the kernel that runs beside this one
+        asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.ready_flag), "r"(p.seq) : "memory");
     const int G = p.group;
     const int row = lane >> 2;  // query head inside the group that this thread's c0/c1 belong to
     const __nv_bfloat16 *q = reinterpret_cast<const __nv_bfloat16 *>(p.q);
@@ -412,7 +417,8 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
     uint32_t piece = 0;   // pieces this block has finished
 
     for (uint32_t it = item_begin; it < item_end; ++it) {
-        const cart_work_item w = p.items[it];
+        cart_work_item w = p.items[it];
+        if (w.flags & CART_ITEM_TAIL) w.n_tok += p.grow;
         if (w.flags & CART_ITEM_BEGIN) {
             st.m = -INFINITY;
             st.l = 0.f;

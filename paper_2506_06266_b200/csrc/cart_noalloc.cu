@@ -123,6 +123,7 @@ extern "C" cart_status cart_decode_attention_static(const void *q, const void *k
         seg[i].head_stride = (uint32_t)n_tokens;
         seg[i].layer_stride = 0;
         seg[i].n_tok = (uint32_t)n_tokens;
+        seg[i].flags = CART_SEG_SUFFIX;  // the caller's buffer: a kernel earlier on the stream may have written it
         seg_begin[i] = i;
     }
     seg_begin[n_reqs] = n_reqs;

@@ -191,10 +191,47 @@ extern "C" cart_status cart_plan_build_shared(const cart_plan_seg *segs, const i
         }
         return bal.block_has_work() ? bal.c + 1 : bal.c;
     };
+    // Side by side: how many of the n_cta blocks the shared kernel gets.  Estimated times in nanoseconds from
+    // measurements on B200: a 128-token shared tile takes a block 1.6 us and a unit 9 us on top; a 64-token
+    // stream tile takes a block at least 0.51 us (what one SM can pull) and 0.0052 us per streaming block
+    // (the SM's share of HBM bandwidth), and a row-group piece 1.5 us on top.
+    uint64_t n_cta_stream = (uint64_t)n_cta, n_cta_shared = (uint64_t)n_cta;
+    o->n_shared_ctas = 0;
+    if (W_sh > 0 && o->side_by_side > 0 && n_cta >= 2) {
+        uint64_t st_tiles = 0, st_rgs = 0;
+        for (int32_t i = 0; i < n_reqs; ++i) {
+            uint64_t t = 0;
+            for (int32_t sgi = seg_begin[i]; sgi < seg_begin[i + 1]; ++sgi) {
+                const uint64_t nt = seg_cls[(size_t)sgi] < 0 ? segs[sgi].n_tok : segs[sgi].n_tok % TS;
+                t += (nt + T - 1) / T;
+            }
+            st_tiles += t * (uint64_t)n_kv_heads;
+            if (t > 0) st_rgs += (uint64_t)n_kv_heads;
+        }
+        if (st_tiles > 0) {
+            uint64_t S = 0;
+            if (o->side_by_side > 1) {
+                S = std::min<uint64_t>((uint64_t)o->side_by_side, (uint64_t)n_cta - 1);
+            } else {
+                uint64_t best = UINT64_MAX;
+                for (uint64_t s2 = 1; s2 < (uint64_t)n_cta; ++s2) {
+                    const uint64_t c2 = (uint64_t)n_cta - s2;
+                    const uint64_t est_sh = (W_sh * 1600 + (combos.size() + s2) * 9000) / s2;
+                    const uint64_t tile_ns = std::max<uint64_t>(510, (c2 * 52) / 10);
+                    const uint64_t est_st = (st_tiles * tile_ns + (st_rgs + c2) * 1500) / c2;
+                    const uint64_t est = std::max(est_sh, est_st);
+                    if (est < best) { best = est; S = s2; }
+                }
+            }
+            n_cta_shared = S;
+            n_cta_stream = (uint64_t)n_cta - S;
+            o->n_shared_ctas = (int32_t)S;
+        }
+    }
     uint64_t C_sh = 0;
     if (W_sh > 0) {
         // a block should get at least two tiles
-        C_sh = std::min<uint64_t>((uint64_t)n_cta, std::max<uint64_t>(1, W_sh / 2));
+        C_sh = std::min<uint64_t>(n_cta_shared, std::max<uint64_t>(1, W_sh / 2));
         // every stream piece of a row group with a shared part takes a slot, and so does every split
         const int64_t stream_reserve = (int64_t)n_reqs * n_kv_heads + 2 * (int64_t)n_cta;
         for (;;) {
@@ -215,6 +252,8 @@ extern "C" cart_status cart_plan_build_shared(const cart_plan_seg *segs, const i
             std::fill(seg_cls.begin(), seg_cls.end(), -1);
             n_entries = 0;
             W_sh = 0;
+            n_cta_stream = (uint64_t)n_cta;
+            o->n_shared_ctas = 0;
         }
     }
 
@@ -239,7 +278,8 @@ extern "C" cart_status cart_plan_build_shared(const cart_plan_seg *segs, const i
                 u.n_tiles = (uint32_t)take;
                 u.reader_begin = cb.reader_begin;
                 u.n_readers = cb.n_readers;
-                u.kv_head = cb.kv_head;
+                u.kv_head = (uint16_t)cb.kv_head;
+                u.flags = (sg.flags & CART_SEG_SUFFIX) ? (uint16_t)CART_UNIT_SUFFIX : (uint16_t)0;
                 u.chunk = chunk;
             });
         if (overflow) return CART_ERR_CAPACITY;
@@ -265,7 +305,7 @@ extern "C" cart_status cart_plan_build_shared(const cart_plan_seg *segs, const i
         tiles_per_head += (nt + T - 1) / T;
     }
     const uint64_t W = tiles_per_head * (uint64_t)n_kv_heads;
-    const uint64_t C = std::min<uint64_t>((uint64_t)n_cta, W);
+    const uint64_t C = std::min<uint64_t>(n_cta_stream, W);
 
     int32_t ni = 0, nm = 0;
     uint32_t next_slot = 0;
@@ -353,6 +393,7 @@ extern "C" cart_status cart_plan_build_shared(const cart_plan_seg *segs, const i
                     it.row_group = rg;
                     it.flags = first ? CART_ITEM_BEGIN : 0u;
                     if (s == s1 - 1 && tok1 == seg_ntok) it.flags |= CART_ITEM_TAIL;
+                    if (segs[s].flags & CART_SEG_SUFFIX) it.flags |= CART_ITEM_SUFFIX;
                     it.slot = 0;
                     it.merge = 0;
                     first = false;
@@ -419,4 +460,18 @@ extern "C" cart_status cart_plan_build(const cart_plan_seg *segs, const int32_t 
     *n_slots = o.n_slots;
     *total_tiles = o.total_tiles;
     return CART_OK;
+}
+
+extern "C" int32_t cart_plan_reusable(const int32_t *plan_len, const int32_t *cur_len, int32_t n_reqs,
+                                      int32_t max_grow, int32_t *grow)
+{
+    if (!plan_len || !cur_len || !grow || n_reqs < 1 || max_grow < 0) return 0;
+    const int64_t d = (int64_t)cur_len[0] - plan_len[0];
+    if (d < 0 || d > max_grow) return 0;
+    for (int32_t i = 0; i < n_reqs; ++i) {
+        if ((int64_t)cur_len[i] - plan_len[i] != d) return 0;
+        if (d > 0 && plan_len[i] < 1) return 0;
+    }
+    *grow = (int32_t)d;
+    return 1;
 }

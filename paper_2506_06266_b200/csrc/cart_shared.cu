@@ -176,6 +176,39 @@ __device__ __forceinline__ void softmax_bar_both()  // both softmax warpgroups
     asm volatile("bar.sync 3, %0;" ::"n"(2 * kSoftmaxThreads) : "memory");
 }
 
+// "The kernels before this one on the stream are complete and their writes visible."  Alone, that is
+// griddepcontrol.wait.  Side by side with the stream kernel (launched just before, resident at the same
+// time) it is a flag that the stream kernel's block 0 sets after its own griddepcontrol.wait: waiting for
+// the stream kernel itself would put the two kernels one after the other again.  All of the stream
+// kernel's blocks are resident before this kernel is launched (a dependent launch happens once every
+// block of the kernel before has started), so the flag is on its way; the wait is bounded all the same.
+// Called by one lane per warp; the others follow through __syncwarp.
+__device__ __forceinline__ bool wait_for_prior_kernels(const SharedParams &p, volatile uint32_t *abort_flag)
+{
+    if (p.ready_flag == nullptr) {
+        pdl_wait();
+        return true;
+    }
+    uint32_t spins = 0;
+    long long t0 = 0;
+    for (;;) {
+        uint32_t v;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p.ready_flag) : "memory");
+        if ((int32_t)(v - p.seq) >= 0) return true;
+        if ((++spins & 0xFFu) == 0) {
+            if (*abort_flag) return false;
+            const long long now = clock64();
+            if (t0 == 0) {
+                t0 = now | 1;
+            } else if (now - t0 > kWaitLimitCycles) {
+                *abort_flag = 1;
+                atomicOr(p.status, kStatusTimeoutConsumer);
+                return false;
+            }
+        }
+    }
+}
+
 __global__ void __launch_bounds__(kShThreads, 1)
 cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams p)
 {
@@ -223,9 +256,12 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
-    // Shared tiles are whole tiles of stored Cartridges, which no kernel writes, and the plan is in place
-    // before any of these kernels starts; the queries, the partial slots and the tickets may still be in
-    // use by the kernels before this one: the softmax warps wait for those before they read a query.
+    // The plan is in place before any of these kernels starts.  Shared tiles of stored Cartridges are only
+    // ever written by copies and may be fetched at once; shared tiles in suffix storage (prefill: the part
+    // of the suffix that a group of rows has in common, units marked CART_UNIT_SUFFIX) may have been
+    // written by the kernel before this one, so the producers wait for the kernels before them ahead of
+    // the first such unit.  The queries, the partial slots and the tickets may still be in use by those
+    // kernels too: the softmax warps wait before they read a query.
     const uint32_t unit_begin = p.unit_cta_begin[blockIdx.x];
     const uint32_t unit_end = p.unit_cta_begin[blockIdx.x + 1];
 
@@ -243,8 +279,14 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                 asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap)) : "memory");
                 uint32_t tt = 0;
                 bool ok = true;
+                bool waited = false;
                 for (uint32_t ui = unit_begin; ui < unit_end && ok; ++ui) {
                     const cart_shared_unit u = p.units[ui];
+                    if (!waited && (u.flags & CART_UNIT_SUFFIX)) {
+                        ok = wait_for_prior_kernels(p, abort_flag);
+                        if (!ok) break;
+                        waited = true;
+                    }
                     const uint32_t row0 = (is_v ? u.v_row : u.k_row) + (uint32_t)p.layer * u.layer_stride;
                     for (uint32_t t = 0; t < u.n_tiles; ++t, ++tt) {
                         const int st = (int)(tt % nst);
@@ -380,7 +422,9 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
             // ---- this row's query into shared memory, in the swizzled K-major operand layout; each
             //      warpgroup copies one 64-dim half -------------------------------------------------
             if (!waited) {
-                pdl_wait();
+                bool ok0 = true;
+                if (lane == 0) ok0 = wait_for_prior_kernels(p, abort_flag);
+                alive = __all_sync(0xffffffffu, ok0);
                 waited = true;
             }
             {
@@ -621,6 +665,9 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
+    // Side by side: this kernel must not complete before the stream kernel does, because the kernel after
+    // this one takes this kernel's completion for that of everything before it.
+    if (p.ready_flag != nullptr && threadIdx.x == 0) pdl_wait();
 }
 
 }  // namespace

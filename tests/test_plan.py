@@ -148,3 +148,29 @@ def test_errors():
     with pytest.raises(binding.CartError) as ei:
         binding.cart_plan_build(make_segments([[1000]], 2), 2, 8, 64, items_cap=3)
     assert ei.value.status == binding.CART_ERR_CAPACITY
+
+
+def test_a_plan_is_reused_while_every_request_grows_by_the_same_amount():
+    reusable = binding.cart_plan_reusable
+    assert reusable([5, 70, 1], [5, 70, 1], 192) == 0
+    assert reusable([5, 70, 1], [6, 71, 2], 192) == 1
+    assert reusable([5, 70, 1], [135, 200, 131], 192) == 130        # two tile boundaries later
+    assert reusable([5, 70, 1], [198, 263, 194], 192) is None       # beyond the allowed drift
+    assert reusable([5, 70, 1], [6, 72, 2], 192) is None            # uneven growth
+    assert reusable([5, 70, 1], [4, 69, 0], 192) is None            # a cache never shrinks under a plan
+    assert reusable([5, 0, 1], [6, 1, 2], 192) is None              # a request had no suffix: its tail item is a Cartridge's
+    assert reusable([5, 0, 1], [5, 0, 1], 192) == 0
+    assert reusable([5, 70, 1], [6, 71, 2], 0) is None              # reuse switched off
+    assert reusable([3], [3], 0) == 0
+
+
+def test_items_in_suffix_storage_are_marked():
+    # request 0: Cartridge (not writable by kernels) + suffix; request 1: suffix only
+    segs = [[(0, 10_000, 300, 2400, 300, 0), (20_000, 30_000, 128, 1024, 70, binding.CART_SEG_SUFFIX)],
+            [(40_000, 50_000, 64, 512, 9, binding.CART_SEG_SUFFIX)]]
+    plan = binding.cart_plan_build(segs, 8, 148, 64)
+    for it in plan["items"]:
+        in_suffix = it.k_row >= 20_000
+        assert bool(it.flags & binding.CART_ITEM_SUFFIX) == in_suffix
+        if it.flags & binding.CART_ITEM_TAIL:
+            assert in_suffix

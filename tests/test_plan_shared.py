@@ -32,9 +32,16 @@ class Arena:
 
 
 def check(segs, Hkv, G, n_cta, tile=64, share_min=4, share_tile=128, slots_cap=1 << 20, piece_cost=0,
-          unit_cost=0):
+          unit_cost=0, side_by_side=0):
     plan = binding.cart_plan_build_shared(segs, Hkv, G, n_cta, tile, share_min, share_tile, slots_cap, piece_cost,
-                                          unit_cost)
+                                          unit_cost, side_by_side)
+    if plan["n_shared_ctas"]:
+        # side by side: the two kernels' blocks fit on the device together
+        assert side_by_side and plan["units"] and plan["items"]
+        assert plan["n_unit_cta_used"] <= plan["n_shared_ctas"] < n_cta
+        assert plan["n_cta_used"] <= n_cta - plan["n_shared_ctas"]
+        if side_by_side > 1:
+            assert plan["n_shared_ctas"] == min(side_by_side, n_cta - 1)
     items, cta_begin, units = plan["items"], plan["cta_begin"], plan["units"]
     R = 128 // G
 
@@ -258,6 +265,27 @@ def test_shared_blocks_balanced_by_tiles_and_units(w):
     assert len(plan["units"]) <= len(flat["units"])
 
 
+@pytest.mark.parametrize("w", [synth.config3(), synth.config4()])
+def test_side_by_side_divides_the_blocks_between_the_two_kernels(w):
+    a = Arena(w.n_kv_heads)
+    carts = [a.store(w.p) for _ in range(w.n_cartridges)]
+    suffix = w.suffix_lengths()
+    segs = [[carts[c] for c in parts] + [a.store(int(suffix[b]) + 64)] for b, parts in enumerate(w.request_parts())]
+    G = w.n_q_heads // w.n_kv_heads
+    plan = check(segs, w.n_kv_heads, G, 148, piece_cost=3, unit_cost=4, side_by_side=1)
+    S = plan["n_shared_ctas"]
+    assert 16 <= S <= 120                      # both parts are substantial on these workloads
+    assert plan["n_unit_cta_used"] >= S - 2 and plan["n_cta_used"] >= 148 - S - 2
+    forced = check(segs, w.n_kv_heads, G, 148, piece_cost=3, unit_cost=4, side_by_side=50)
+    assert forced["n_shared_ctas"] == 50
+    # a batch without a shared part, or without a stream part, keeps all blocks for the one kernel
+    alone = check([[a.store(300)] for _ in range(9)], w.n_kv_heads, G, 148, side_by_side=1)
+    assert alone["n_shared_ctas"] == 0 and alone["n_cta_used"] == 148
+    only_shared = check([[carts[0]] for _ in range(8)], w.n_kv_heads, G, 148, side_by_side=1) if w.p % 128 == 0 else None
+    if only_shared is not None:
+        assert only_shared["n_shared_ctas"] == 0 and not only_shared["items"] and only_shared["n_unit_cta_used"] >= 60
+
+
 @pytest.mark.parametrize("seed", range(40))
 def test_random_batches_keep_every_invariant(seed):
     """Random pools, compositions, suffix lengths, block counts and cost constants: coverage, slot
@@ -279,4 +307,4 @@ def test_random_batches_keep_every_invariant(seed):
         segs.append(r)
     n_cta = int(rng.choice([1, 2, 7, 37, 148]))
     check(segs, Hkv, G, n_cta, share_min=int(rng.choice([0, 2, 4])), piece_cost=int(rng.choice([0, 1, 3, 9])),
-          unit_cost=int(rng.choice([0, 2, 4])))
+          unit_cost=int(rng.choice([0, 2, 4])), side_by_side=int(rng.choice([0, 1, 1, 5, 40])))

@@ -178,3 +178,23 @@ def test_row_maxima_that_outgrow_the_reference_rescale_the_accumulator(growth):
         assert float(l1.max() - l1.min()) > 8 * 0.6931
     finally:
         sess.close()
+
+
+@pytest.mark.parametrize("mode", [0, 1, 3, 100])
+def test_side_by_side_and_one_after_the_other_agree_with_the_oracle(mode):
+    """The shared kernel and the stream kernel resident together (the planner's division, 3 and 100 blocks for
+    the shared kernel) or one after the other: the same result up to rounding, over several layers and with
+    fused decode steps in between (so that the kernels of consecutive calls follow each other closely)."""
+    w = synth.shrink(synth.config4(), n_layers=3, batch=20, pool=3, p=640, suffix_lo=1, suffix_hi=200)
+    sess, reqs = H.load_workload(w, extra_capacity=4)
+    try:
+        binding.cart_set_side_by_side(sess.ctx, mode)
+        for step in range(4):
+            kn, vn = w.appended_kv(step, "cuda:0")
+            q = w.queries(step, "cuda:0")
+            for layer in range(w.n_layers):
+                out, lse = sess.decode_step(layer, reqs, kn[layer], vn[layer], q[layer])
+                H.assert_close(out, lse, *sess.oracle_decode(layer, reqs, q[layer]),
+                               "mode %d step %d layer %d" % (mode, step, layer))
+    finally:
+        sess.close()

@@ -6,9 +6,11 @@ leftovers in the shared scratch and must not be disturbed by them.
 
 This file sorts last on purpose: a run that stops at the first failure has then already run every
 other test."""
+import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2506_06266_b200 import binding, synth
 
 import cart_harness as H
@@ -73,6 +75,23 @@ def test_static_scratch_entry_point_matches_the_context_path_twice_in_a_row():
     # and the first problem again, after the second one has overwritten the scratch
     got1b = static_path(k1, v1, q1)
     assert torch.equal(got1[0], got1b[0]) and torch.equal(got1[1], got1b[1])
+
+
+def test_static_scratch_entry_point_matches_the_cpu_oracle():
+    """Directly against the float64 oracle (not only against the context path, which runs the same kernel):
+    every request is one segment of n tokens per KV head."""
+    H.ensure_built()
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    for seed, (B, Hq, Hkv, n) in enumerate([(3, 24, 8, 1501), (7, 32, 8, 65), (2, 8, 1, 4000)]):
+        k = synth.normal_bf16((B, Hkv, n, 128), 9100 + 3 * seed, dev)
+        v = synth.normal_bf16((B, Hkv, n, 128), 9101 + 3 * seed, dev)
+        q = synth.normal_bf16((B, Hq, 128), 9102 + 3 * seed, dev)
+        kb, vb = synth.bits(k), synth.bits(v)
+        ref_o, ref_l = oracle.decode_layer(synth.bits(q), [[(kb[b], vb[b])] for b in range(B)], 128 ** -0.5)
+        for _ in range(2):                      # twice: the second call starts from the first one's leftovers
+            out, lse = static_path(k, v, q)
+            H.assert_close(out, lse, ref_o, ref_l, "static entry point, B=%d Hq=%d Hkv=%d n=%d" % (B, Hq, Hkv, n))
 
 
 def test_sizes_beyond_the_fixed_scratch_are_refused():
