@@ -8,12 +8,19 @@ before the timed region (the paper's throughput protocol pre-loads them, App. A.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl ours|reference]
 
+The headline (`value`, `roofline`, `e2e`, `cpu_baseline`) is the workload named by --workload (default: the
+Llama-3B-shaped batch of 64 private Cartridges).  With the default workload on one GPU the line also carries
+a `workloads` array: the other benchmark workloads measured one after the other in the same process with the
+paper's protocol (3 warm-up steps, then 5 timed blocks; mean and min), and the memory / throughput comparison
+of a 100 k-token in-context cache against a p = 2048 Cartridge.
+
 N > 1 is launched with torch.distributed.run: every rank runs an independent replica on its own
 GPU (the path has no exchange step), timing is the maximum over ranks.
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import subprocess
@@ -37,19 +44,47 @@ WORKLOADS = {
     "c1": synth.config1, "c2": synth.config2, "c3": synth.config3, "c4": synth.config4,
     "c5_full": synth.config5_full, "c5_cartridge": synth.config5_cartridge,
 }
+SIDE_WORKLOADS = ["c1", "c3", "c4", "c5_cartridge", "c5_full"]   # reported next to the headline workload
+TIMED_BLOCKS = 5                                                  # App. A.3: 3 warm-up runs, 5 timed runs
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the decode kernel, from the ncu capture
-# summarised under profiles/ (a smaller case of the same kernel, scaled by KV bytes); None = not captured.
-NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = {"c2": 617.90 / 608.27}   # profiles/decode_kernel_c2.md
+KERNEL_SOURCES = ["cart_kernels.cu", "cart_shared.cu", "cart_device.cuh", "cart_internal.h"]
+TRAFFIC_TABLE = os.path.join(ROOT, "profiles", "dram_traffic.txt")
 
 
-def measured_peak_gbs():
+def kernel_source_sha() -> str:
+    """Identifies the kernels' source: DRAM counters taken from another version are not reported."""
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_2506_06266_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def dram_traffic_ratio(workload: str):
+    """DRAM bytes per algorithmic byte of a workload's launch, from the table written next to the ncu
+    summaries (lines: workload, kernel, dram bytes per launch, algorithmic bytes per launch of the captured
+    case, source id).  None when the workload was not captured or the kernels have changed since."""
+    try:
+        with open(TRAFFIC_TABLE) as f:
+            for line in f:
+                parts = line.split()
+                if len(parts) >= 5 and not line.startswith("#") and parts[0] == workload:
+                    if parts[4] != kernel_source_sha():
+                        return None
+                    return float(parts[2]) / float(parts[3])
+    except OSError:
+        pass
+    return None
+
+
+def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
         with open(path) as f:
-            return float(json.load(f)["hbm_gbs"]), "measured"
+            d = json.load(f)
+        return float(d["hbm_gbs"]), float(d["bf16_tflops"]), float(d["bf16_tflops_sustained"]), "measured"
     except Exception:
-        return 6650.0, "fallback"
+        return 6650.0, 1590.0, 1400.0, "fallback"
 
 
 class ClockSampler:
@@ -129,6 +164,151 @@ def oracle_sample(w: synth.Workload, lw, layers, q_host_bits, reps_target_s: flo
             "s_per_layer": per_layer}
 
 
+def workload_config(w: synth.Workload) -> dict:
+    """What names the workload; the same keys in both arms' lines."""
+    return {"workload": w.name, "batch_per_gpu": w.batch, "layers": w.n_layers, "q_heads": w.n_q_heads,
+            "kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "cartridge_tokens": w.p,
+            "cartridges": w.cartridges, "suffix": "uniform[%d,%d]" % (w.suffix_lo, w.suffix_hi)}
+
+
+def timed_steps(lw, tensors, steps: int, blocks: int, stream, fused: bool):
+    """`steps` decode steps timed as `blocks` consecutive blocks with CUDA events on the launching stream at
+    the block boundaries.  Returns (total ms, ms per step of every block, sum over the steps of the unique
+    and of the logical bytes per layer)."""
+    q, k_new, v_new, out, lse = tensors
+    blocks = max(1, min(blocks, steps))
+    sizes = [steps // blocks + (1 if i < steps % blocks else 0) for i in range(blocks)]
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(blocks + 1)]
+    u0, l0 = lw.unique_bytes_per_layer(), lw.algorithmic_bytes_per_layer()
+    ev[0].record(stream)
+    for i, n in enumerate(sizes):
+        for _ in range(n):
+            lw.step(q, k_new, v_new, out, lse, fused=fused)
+        ev[i + 1].record(stream)
+    ev[-1].synchronize()
+    # every step appends one token per request, so the bytes per layer grow linearly over the steps: the sum
+    # over the steps (each counted with its own token already appended) follows from the two end points
+    u1, l1 = lw.unique_bytes_per_layer(), lw.algorithmic_bytes_per_layer()
+    uniq = steps * ((u0 + (u1 - u0) / steps) + u1) / 2
+    logical = steps * ((l0 + (l1 - l0) / steps) + l1) / 2
+    per_block = [ev[i].elapsed_time(ev[i + 1]) / sizes[i] for i in range(blocks)]
+    return ev[0].elapsed_time(ev[-1]), per_block, uniq, logical
+
+
+def roofline_entry(w, lw, ms, steps, uniq_sum, logical_sum, launches, workload_key, share_min=4):
+    """HBM roofline on the bytes the method must move (every stored Cartridge once, every suffix once) and,
+    where Cartridges are shared, the tensor-core side of the same launches."""
+    L = w.n_layers
+    hbm_peak, tf_burst, tf_sustained, kind = measured_peaks()
+    period_s = ms * 1e-3 / (steps * L)                  # one layer's launches, gaps included
+    uniq = uniq_sum / steps
+    logical = logical_sum / steps
+    achieved = uniq / period_s / 1e9
+    shared_flops = lw.shared_flops_per_layer(share_min)
+    kernels = ["cart_decode_kernel"]
+    if shared_flops:
+        kernels = ["cart_decode_kernel", "cart_shared_kernel"] + (["cart_merge_kernel"] if launches > 2 * steps * L else [])
+    ratio = dram_traffic_ratio(workload_key)
+    r = {"bound": "hbm", "achieved": round(achieved, 1), "peak": hbm_peak, "unit": "GB/s",
+         "frac": round(achieved / hbm_peak, 4), "peak_kind": "of " + kind,
+         "frac_of_8TBs_nominal": round(achieved / 8000.0, 4),
+         "traffic": None if ratio is None else int(ratio * uniq),
+         "kernel": "cart_decode_kernel", "kernels_per_launch_period": kernels,
+         "launches_timed": steps * L,
+         "timing": "CUDA events around the timed steps / decode calls (launch period of one layer, gaps included)",
+         "avg_kernel_us": round(period_s * 1e6, 2),
+         "algorithmic_bytes_per_launch": int(uniq),
+         "bytes": "unique: every stored Cartridge of the batch once per layer, every suffix once, q/out/lse",
+         "logical_gbs": round(logical / period_s / 1e9, 1), "logical_bytes_per_launch": int(logical)}
+    if shared_flops:
+        tf = shared_flops / period_s / 1e12
+        r["tensor"] = {"bound": "tensor", "kernel": "cart_shared_kernel", "achieved": round(tf, 1),
+                       "peak": tf_sustained, "unit": "TFLOP/s", "frac": round(tf / tf_sustained, 4),
+                       "peak_kind": "of %s (sustained bf16; burst %.0f)" % (kind, tf_burst),
+                       "flops_per_launch": int(shared_flops),
+                       "timing": "the same launch period: the tensor-core kernel runs beside the stream kernel, "
+                                 "so this is a lower bound of its own rate"}
+    return r
+
+
+def measure_side_workload(name: str, dev, stream, warmup: int, steps_per_block: int) -> dict:
+    """One of the other benchmark workloads with the paper's protocol: `warmup` steps, then 5 timed blocks."""
+    from paper_2506_06266_b200 import binding, runner
+    w = WORKLOADS[name]()
+    L, B = w.n_layers, w.batch
+    free, _ = torch.cuda.mem_get_info(dev)
+    steps = TIMED_BLOCKS * steps_per_block
+    need = runner.arena_bytes_for(w, warmup + steps + 40) + (6 << 30)
+    if free < need:
+        return {"workload": w.name, "skipped": "needs %.0f GB of device memory, %.0f GB free" % (need / 1e9, free / 1e9)}
+    lw = runner.LoadedWorkload(w, dev, extra_capacity=warmup + steps + 40, stream=stream)
+    try:
+        q = w.queries(0, dev)
+        k_new, v_new = w.appended_kv(0, dev)
+        out = torch.empty_like(q)
+        lse = torch.empty((L, B, w.n_q_heads), dtype=torch.float32, device=dev)
+        tensors = (q, k_new, v_new, out, lse)
+        for _ in range(warmup):
+            lw.step(*tensors)
+        binding.cart_sync_status(lw.ctx, stream)
+        sampler = ClockSampler(dev.index or 0)
+        sampler.start()
+        n0 = binding.cart_launch_count(lw.ctx)
+        ms, per_block, uniq, logical = timed_steps(lw, tensors, steps, TIMED_BLOCKS, stream, True)
+        launches = binding.cart_launch_count(lw.ctx) - n0
+        clocks = sampler.stop()
+        binding.cart_sync_status(lw.ctx, stream)
+        roof = roofline_entry(w, lw, ms, steps, uniq, logical, launches, name)
+        logical_b, private_b = binding.cart_kv_bytes(lw.ctx, lw.reqs[0])
+        res = {"workload": w.name, "batch": B, "layers": L, "mean_kv_tokens": round(float(lw.kv_tokens().mean()), 1),
+               "steps": steps, "warmup": warmup,
+               "tokens_per_s": round(B * steps / (ms * 1e-3), 1),
+               "tokens_per_s_best_block": round(B / (min(per_block) * 1e-3), 1),
+               "us_per_layer_mean": round(float(np.mean(per_block)) * 1e3 / L, 2),
+               "us_per_layer_min": round(min(per_block) * 1e3 / L, 2),
+               "unique_gbs": roof["achieved"], "frac_of_hbm_peak": roof["frac"], "logical_gbs": roof["logical_gbs"],
+               "kv_bytes_per_request": int(logical_b), "kv_bytes_private_per_request": int(private_b),
+               "gpu_launches": int(launches), "clocks": clocks}
+        if "tensor" in roof:
+            res["tensor_tflops"] = roof["tensor"]["achieved"]
+            res["tensor_frac"] = roof["tensor"]["frac"]
+        if L == 1:
+            res["single_call"] = single_call_latency(lw, tensors, stream, dev)
+        return res
+    finally:
+        lw.close()
+        torch.cuda.empty_cache()
+
+
+def single_call_latency(lw, tensors, stream, dev) -> dict:
+    """The single-layer workload: one decode call by itself, L2 warm and L2 cold."""
+    from paper_2506_06266_b200 import binding
+    q, _, _, out, lse = tensors
+    ca, cb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def one_call_us(flush):
+        if flush is not None:
+            flush.fill_(1)                       # 256 MB written: nothing of the KV is left in L2
+        else:
+            torch.cuda._sleep(200000)            # keeps the GPU busy while the host enqueues the call, as the
+                                                 # fill does in the cold case: the events then bracket GPU time
+        ca.record(stream)
+        binding.cart_decode_attention(lw.ctx, 0, lw.req_list, q[0], out[0], lse[0], stream)
+        cb.record(stream)
+        cb.synchronize()
+        return ca.elapsed_time(cb) * 1e3
+
+    one_call_us(None)
+    warm = [one_call_us(None) for _ in range(20)]
+    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    cold = [one_call_us(flush_buf) for _ in range(5)]
+    del flush_buf
+    binding.cart_sync_status(lw.ctx, stream)
+    return {"what": "one cart_decode_attention call, plan cached, CUDA events around the call",
+            "warm_us_mean": round(sum(warm) / len(warm), 2), "warm_us_min": round(min(warm), 2),
+            "cold_us_mean": round(sum(cold) / len(cold), 2), "cold_us_min": round(min(cold), 2)}
+
+
 def run_ours(args):
     from paper_2506_06266_b200 import binding, runner
     rank, world, local = replicas.setup()
@@ -152,88 +332,31 @@ def run_ours(args):
     k_new, v_new = w.appended_kv(0, dev)
     out = torch.empty_like(q)
     lse = torch.empty((L, B, w.n_q_heads), dtype=torch.float32, device=dev)
+    tensors = (q, k_new, v_new, out, lse)
     torch.cuda.synchronize(dev)
 
-    # ---- device-resident timing ------------------------------------------------------------
+    # ---- device-resident timing: exactly --steps steps, as five blocks ---------------------------
     for _ in range(args.warmup):
-        lw.step(q, k_new, v_new, out, lse, fused=not args.unfused)
+        lw.step(*tensors, fused=not args.unfused)
     binding.cart_sync_status(ctx, stream)
     replicas.barrier(world)
     torch.cuda.synchronize(dev)
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    binding.cart_set_timing(ctx, args.kernel_events)
     launches0 = binding.cart_launch_count(ctx)
-    bytes_before = lw.algorithmic_bytes_per_layer()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for _ in range(args.steps):
-        lw.step(q, k_new, v_new, out, lse, fused=not args.unfused)
-    e1.record(stream)
-    # every step appends one token per request, so the bytes per layer grow linearly over the steps: the sum
-    # over the steps (each counted with its own token already appended) follows from the two end points
-    bytes_after = lw.algorithmic_bytes_per_layer()
-    per_step = (bytes_after - bytes_before) / args.steps
-    bytes_layer_sum = args.steps * ((bytes_before + per_step) + bytes_after) / 2
+    plans0 = binding.cart_plan_count(ctx)
+    ms, per_block, uniq_sum, logical_sum = timed_steps(lw, tensors, args.steps, TIMED_BLOCKS, stream, not args.unfused)
     torch.cuda.synchronize(dev)
     replicas.barrier(world)
     clocks = sampler.stop() if rank == 0 else None
-    ms = e0.elapsed_time(e1)
     launches = binding.cart_launch_count(ctx) - launches0
-    kern_ms, kern_n = binding.cart_get_timing(ctx)
-    binding.cart_set_timing(ctx, False)
+    plans = binding.cart_plan_count(ctx) - plans0
     binding.cart_sync_status(ctx, stream)
     value, ms_max = replicas.whole_job_tokens_per_s(B * args.steps, ms, world, dev)
 
-    # ---- the single-layer workload: one decode call by itself, L2 warm and L2 cold ----------------
-    single_call = None
-    if L == 1 and world == 1:
-        ca, cb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-
-        def one_call_us(flush):
-            if flush is not None:
-                flush.fill_(1)                       # 256 MB written: nothing of the KV is left in L2
-            else:
-                torch.cuda._sleep(200000)            # keeps the GPU busy while the host enqueues the call, as the
-                                                     # fill does in the cold case: the events then bracket GPU time
-            ca.record(stream)
-            binding.cart_decode_attention(ctx, 0, lw.req_list, q[0], out[0], lse[0], stream)
-            cb.record(stream)
-            cb.synchronize()
-            return ca.elapsed_time(cb) * 1e3
-
-        one_call_us(None)                            # the plan for the current lengths is built here
-        warm = [one_call_us(None) for _ in range(20)]
-        flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
-        cold = [one_call_us(flush_buf) for _ in range(5)]
-        del flush_buf
-        single_call = {"what": "one cart_decode_attention call, plan cached, CUDA events around the call",
-                       "warm_us_mean": round(sum(warm) / len(warm), 2), "warm_us_min": round(min(warm), 2),
-                       "cold_us_mean": round(sum(cold) / len(cold), 2), "cold_us_min": round(min(cold), 2)}
-        binding.cart_sync_status(ctx, stream)
-
-    # ---- roofline of the dominant kernel (split-KV decode attention) -------------------------
-    peak, peak_kind = measured_peak_gbs()
-    bytes_per_launch = bytes_layer_sum / args.steps          # one launch = one layer of one step
-    timing_kind = "CUDA events around each decode call's kernels"
-    if kern_n == 0:
-        # Default: the launch period of the decode kernels = the event-timed region divided by its
-        # launches.  Consecutive layers' kernels overlap at their edges (the next one is resident and has
-        # fetched its first tiles before the last block of this one retires), so this period is what one
-        # launch costs; it includes whatever gap remains, so it cannot flatter the kernel.
-        kern_ms, kern_n = ms, args.steps * L
-        timing_kind = "timed region / decode calls (launch period, gaps included)"
-    avg_kernel_s = kern_ms * 1e-3 / max(kern_n, 1)
-    achieved = bytes_per_launch / avg_kernel_s / 1e9
-    ratio = NCU_TRAFFIC_PER_ALGORITHMIC_BYTE.get(args.workload)
-    roofline = {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
-                "frac": round(achieved / peak, 4), "peak_kind": "of " + peak_kind,
-                "frac_of_8TBs_nominal": round(achieved / 8000.0, 4),
-                "traffic": None if ratio is None else int(ratio * bytes_per_launch),
-                "kernel": "cart_decode_kernel", "launches_timed": kern_n, "timing": timing_kind,
-                "avg_kernel_us": round(avg_kernel_s * 1e6, 2),
-                "algorithmic_bytes_per_launch": int(bytes_per_launch)}
+    single_call = single_call_latency(lw, tensors, stream, dev) if (L == 1 and world == 1) else None
+    roofline = roofline_entry(w, lw, ms, args.steps, uniq_sum, logical_sum, launches, args.workload)
 
     # ---- end to end through the C ABI from pinned host buffers -------------------------------
     e2e = None
@@ -314,28 +437,53 @@ def run_ours(args):
     logical, private = binding.cart_kv_bytes(ctx, lw.reqs[0])
     kv_tokens = lw.kv_tokens()
     lw.close()
+    del tensors, q, k_new, v_new, out, lse
+    torch.cuda.empty_cache()
+
+    # ---- the other workloads and the in-context-cache comparison (default run on one GPU only) --------
+    side, comparison = None, None
+    if world == 1 and not args.no_side and args.workload == "c2" and not args.layers:
+        side = []
+        for name in SIDE_WORKLOADS:
+            n = {"c1": 40, "c3": 4, "c4": 4, "c5_cartridge": 2, "c5_full": 2}[name]
+            side.append(measure_side_workload(name, dev, stream, 3, n))
+        by = {s["workload"]: s for s in side}
+        full, cart = by.get(synth.config5_full().name), by.get(synth.config5_cartridge().name)
+        if full and cart and "skipped" not in full and "skipped" not in cart:
+            comparison = {"what": "in-context KV cache of 100 000 tokens at batch 8 against a Cartridge of p = 2048 at "
+                                  "batch 256, Llama-8B attention shapes, same GPU",
+                          "kv_bytes_per_request_ratio": round(full["kv_bytes_per_request"] / cart["kv_bytes_per_request"], 2),
+                          "tokens_per_s_ratio": round(cart["tokens_per_s"] / full["tokens_per_s"], 2),
+                          "paper_context": "38.6x less memory, 26.4x more tokens/s on 1xH100 with a serving stack "
+                                           "(whole model, not attention alone)"}
     if world > 1:
         replicas.barrier(world)
         replicas.shutdown()
     if rank != 0:
         return
+    cfg = workload_config(w)
+    cfg.update({"mean_kv_tokens": round(float(kv_tokens.mean()), 1),
+                "step": ("per layer: cart_append_kv, then cart_decode_attention" if args.unfused else
+                         "per layer: cart_decode_step (append 1 KV token per request and attend, one call)"),
+                "l2": "inputs larger than L2 (%.0f MB of KV per layer, %.1f GB per step)"
+                      % (roofline["algorithmic_bytes_per_launch"] / 1e6, roofline["algorithmic_bytes_per_launch"] * L / 1e9),
+                "parallelism": "replicas only" if world > 1 else "single GPU",
+                "attention_us_per_layer": round(ms_max * 1e3 / args.steps / L, 2),
+                "kv_bytes_per_request": int(logical), "kv_bytes_private_per_request": int(private)})
     line = {
         "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": round(ms_max / args.steps, 4), "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": w.name, "batch_per_gpu": B, "layers": L, "q_heads": w.n_q_heads,
-                   "kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "cartridge_tokens": w.p,
-                   "cartridges": w.cartridges, "suffix": "uniform[%d,%d]" % (w.suffix_lo, w.suffix_hi),
-                   "mean_kv_tokens": round(float(kv_tokens.mean()), 1),
-                   "step": ("per layer: cart_append_kv, then cart_decode_attention" if args.unfused else
-                            "per layer: cart_decode_step (append 1 KV token per request and attend, one call)"),
-                   "l2": "inputs larger than L2 (%.0f MB of KV per layer, %.1f GB per step)"
-                         % (bytes_per_launch / 1e6, bytes_per_launch * L / 1e9),
-                   "parallelism": "replicas only" if world > 1 else "single GPU",
-                   "attention_us_per_layer": round(ms_max * 1e3 / args.steps / L, 2),
-                   "kv_bytes_per_request": int(logical), "kv_bytes_private_per_request": int(private)},
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": cfg,
+        "repeats": {"blocks": len(per_block), "protocol": "warm-up steps, then the timed steps as consecutive blocks "
+                                                          "(App. A.3: 3 warm-up and 5 timed runs)",
+                    "ms_per_step_mean": round(float(np.mean(per_block)), 4),
+                    "ms_per_step_min": round(min(per_block), 4),
+                    "tokens_per_s_best_block": round(B * world / (min(per_block) * 1e-3), 1)},
         "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
-        "clocks": clocks, **({"single_call": single_call} if single_call else {}),
+        "plans_built_in_timed_region": int(plans), "clocks": clocks,
+        **({"single_call": single_call} if single_call else {}),
+        **({"workloads": side} if side is not None else {}),
+        **({"comparison_100k_context_vs_cartridge": comparison} if comparison else {}),
     }
     print(json.dumps(line))
 
@@ -393,6 +541,8 @@ def run_prefill(args):
     mean_ctx = w.p + s_old + (args.warmup + (args.steps - 1) / 2.0) * T + (T + 1) / 2.0
     flops = 4.0 * w.n_q_heads * 128 * mean_ctx * T                    # per layer
     us_layer = ms * 1e3 / args.steps / L
+    _, tf_burst, tf_sustained, kind = measured_peaks()
+    tflops = flops / (us_layer * 1e-6) / 1e12
     binding.cart_destroy(ctx)
     print(json.dumps({"metric": "prefill_attention_tokens_per_s", "value": round(T * args.steps / (ms * 1e-3), 1),
                       "unit": "tokens/s", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
@@ -401,7 +551,10 @@ def run_prefill(args):
                       "config": {"workload": "prefill of %d tokens over %s shapes" % (T, w0.name), "layers": L,
                                  "cartridge_tokens": w.p, "suffix_before": s_old, "mean_context": round(mean_ctx, 1),
                                  "attention_us_per_layer": round(us_layer, 2),
-                                 "tflops": round(flops / (us_layer * 1e-6) / 1e12, 2)},
+                                 "tflops": round(tflops, 2)},
+                      "roofline": {"bound": "tensor", "achieved": round(tflops, 1), "peak": tf_sustained,
+                                   "unit": "TFLOP/s", "frac": round(tflops / tf_sustained, 4),
+                                   "peak_kind": "of %s (sustained bf16)" % kind, "traffic": None},
                       "gpu_launches": int(launches)}))
 
 
@@ -445,14 +598,19 @@ def run_reference(args):
     for _ in range(args.steps):
         step()
     el = time.perf_counter() - t0
+    sample_ms = el / args.steps * 1e3                      # what one timed step (the sampled layers) took
     per_step_full = el / args.steps * (L / n_layers)
     value = B / per_step_full
-    sample = ("each step = layers 0..%d of %d, all %d requests (inputs of the GPU arm's recipe, "
-              "generated per sampled layer); extrapolated to %d layers" % (n_layers - 1, L, B, L))
+    sample = ("each timed step = layers 0..%d of %d, all %d requests (inputs of the GPU arm's recipe, generated per "
+              "sampled layer); ms_per_step is that sample's time, value is extrapolated to %d layers "
+              "(%.1f ms per whole step)" % (n_layers - 1, L, B, L, per_step_full * 1e3))
+    cfg = workload_config(w)
+    cfg["sampled_layers_per_step"] = n_layers
     line = {"impl": "reference", "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(per_step_full * 1e3, 3),
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(sample_ms, 3),
+            "ms_per_whole_step_extrapolated": round(per_step_full * 1e3, 3),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-            "data": "synthetic", "config": {"workload": w.name, "batch_per_gpu": B, "layers": L},
+            "data": "synthetic", "config": cfg,
             "cpu_baseline": {"value": round(value, 3), "unit": UNIT, "cores": oracle.num_threads(),
                              "kind": "oracle", "sample": sample},
             "e2e": {"value": round(value, 3), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -471,6 +629,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=50)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-side", action="store_true",
+                    help="skip the other workloads that the default run reports next to the headline")
     ap.add_argument("--prefill", type=int, default=0,
                     help="side measurement: prefill attention of a message of this many tokens over one Cartridge "
                          "of the workload's shape (prints its own JSON line)")
@@ -482,13 +642,14 @@ def main():
                     help="planner tuning (cart_set_side_by_side): 0 = shared and stream kernel one after the other, "
                          "1 = side by side with the planner's division, N > 1 = N blocks for the shared kernel; "
                          "-1 keeps the library's default")
-    ap.add_argument("--kernel-events", action="store_true",
-                    help="bracket every decode call's kernels with a pair of CUDA events and report their mean "
-                         "duration; the events sit between the kernels, so a kernel can then no longer start "
-                         "under the tail of the one before (programmatic dependent launch) and the step slows down")
     ap.add_argument("--cpu-layers", type=int, default=4, help="layers the CPU oracle sample covers")
     ap.add_argument("--ref-layers", type=int, default=2, help="layers per step of the reference arm")
+    ap.add_argument("--kernel-sha", action="store_true",
+                    help="print the id of the kernels' source that profiles/dram_traffic.txt records, and exit")
     args = ap.parse_args()
+    if args.kernel_sha:
+        print(kernel_source_sha())
+        return
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     if args.prefill > 0:

@@ -10,10 +10,10 @@
 // consumer multiplies the group's G query heads (padded to the 16 rows of an m16n8k16 bf16 MMA, so
 // a K/V tile is read once per group) with the tile, keeps an fp32 online softmax (running max, sum,
 // rescaled output) in registers, and multiplies the probabilities with V.  At the end of a row-group
-// piece every warp deposits its state in shared memory and moves on; the warp that deposits last
-// combines the six states and writes either the final bf16 output + lse (piece = whole row group) or
-// an fp32 partial; the block that delivers the last partial of a split row group merges them (an
-// arrival ticket per split row group, no waiting), unless a merge kernel follows.
+// piece every warp deposits its state in shared memory and moves on; a warp of its own combines the
+// six states and writes either the final bf16 output + lse (piece = whole row group) or an fp32
+// partial; the block that delivers the last partial of a split row group merges them (an arrival
+// ticket per split row group, no waiting), unless a merge kernel follows.
 // Arithmetic follows Eq. 1 of the paper evaluated at the last position; the split and the merge use
 // that a softmax over a union of token sets is the lse-weighted mix of the softmaxes over the sets.
 #include <cuda_bf16.h>
@@ -31,7 +31,7 @@ constexpr int kStages = 6;
 // current phase from the one before.)
 constexpr int kConsumerWarps = kStages;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
-constexpr int kThreads = kConsumerThreads + 64;      // + the producer warp + the append warp
+constexpr int kThreads = kConsumerThreads + 96;      // + the producer warp + the append warp + the combine warp
 constexpr uint32_t kHalfBytes = kTileTokens * 128;    // 64 tokens x 64 dims of bf16
 constexpr uint32_t kTileBytes = 2 * kHalfBytes;       // K or V tile: 64 tokens x 128 dims
 constexpr uint32_t kStageBytes = 2 * kTileBytes;      // K tile then V tile
@@ -42,7 +42,7 @@ static_assert(kEdgeRows % 16 == 0 && kTileTokens % kEdgeRows == 0,
 constexpr int kScratchStride = 132;                   // floats per scratch row (128 + pad)
 constexpr uint32_t kScratchOBytes = kConsumerWarps * kMaxGroup * kScratchStride * 4;
 constexpr uint32_t kScratchMLBytes = 2 * kConsumerWarps * kMaxGroup * 2 * 4;  // two buffers
-constexpr uint32_t kBarrierBytes = (3 * kStages + 2) * 8;
+constexpr uint32_t kBarrierBytes = (3 * kStages + 4) * 8;
 constexpr uint32_t kSmemUsed = kStages * kStageBytes + kScratchOBytes + kScratchMLBytes + kBarrierBytes + 16;  // + flags
 constexpr uint32_t kSmemBytes = kSmemUsed + 1024;     // slack to align the stages to 1024 bytes
 static_assert(kSmemBytes <= 232448, "shared memory budget of one sm_100 block exceeded");
@@ -194,11 +194,12 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
     const uint32_t bars = base + kStages * kStageBytes + kScratchOBytes + kScratchMLBytes;
     volatile uint32_t *abort_flag =
         reinterpret_cast<volatile uint32_t *>(smem + kStages * kStageBytes + kScratchOBytes + kScratchMLBytes + kBarrierBytes);
-    volatile uint32_t *arrivals = abort_flag + 1;   // [0], [1]: warps that have deposited their state of a piece; [2]: see append_count
+    volatile uint32_t *arrivals = abort_flag + 1;   // [2]: see append_count ([0], [1] unused)
     auto full_k = [&](int s) { return bars + (uint32_t)s * 8u; };
     auto full_v = [&](int s) { return bars + (uint32_t)(kStages + s) * 8u; };
     auto empty = [&](int s) { return bars + (uint32_t)(2 * kStages + s) * 8u; };
     auto scratch_free = [&](uint32_t b) { return bars + (uint32_t)(3 * kStages) * 8u + b * 8u; };
+    auto deposited = [&](uint32_t b) { return bars + (uint32_t)(3 * kStages + 2) * 8u + b * 8u; };
     // [1] how many of the block's new tokens (in work-list order) are in the arena: append warp -> producer
     const uint32_t append_count = smem_u32(const_cast<uint32_t *>(arrivals + 2));
 
@@ -214,6 +215,8 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
         }
         mbar_init(scratch_free(0), 1);
         mbar_init(scratch_free(1), 1);
+        mbar_init(deposited(0), kConsumerWarps);
+        mbar_init(deposited(1), kConsumerWarps);
         *abort_flag = 0;
         arrivals[0] = 0;
         arrivals[1] = 0;
@@ -283,46 +286,33 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
                                 }
                             }
                         }
-                        asm volatile("fence.proxy.async;" ::: "memory");  // those generic-proxy stores before this TMA read
                     }
                     ok = __shfl_sync(0xffffffffu, (int)ok1, 0) != 0;
                     if (!ok) break;
+                    // those generic-proxy stores before the TMA reads below (every issuing lane fences for itself)
+                    asm volatile("fence.proxy.async;" ::: "memory");
                 }
-                if (lane == 0) {
+                {
+                    // The tile's four boxes (K and V, each as two 64-dim halves) are requested by four lanes in
+                    // one instruction: a copy instruction costs the issuing thread about a hundred cycles,
+                    // and one thread issuing all of them one after the other is what limits the tile rate of
+                    // a block when the batch is made of many short runs.
                     const uint32_t kdst = stages + (uint32_t)s * kStageBytes;
-                    const uint32_t vdst = kdst + kTileBytes;
-                    const int32_t yk = (int32_t)(k_row + j * kTileTokens);
-                    const int32_t yv = (int32_t)(v_row + j * kTileTokens);
+                    const uint32_t is_v = ((uint32_t)lane >> 1) & 1u, hi = (uint32_t)lane & 1u;
+                    const uint32_t dst = kdst + is_v * kTileBytes + hi * kHalfBytes;
+                    const int32_t y = (int32_t)((is_v ? v_row : k_row) + j * kTileTokens);
+                    const uint32_t bar = is_v ? full_v(s) : full_k(s);
                     const uint32_t valid = min((uint32_t)kTileTokens, w.n_tok - j * kTileTokens);
-                    if (p.edge_boxes != 0u && valid + kEdgeRows <= (uint32_t)kTileTokens) {
-                        // Ragged last tile of a segment that leaves at least one small box empty: only the boxes
-                        // that hold tokens are fetched (the consumers read no row past the 16-row step that
-                        // holds the last token), not the rows that follow the segment in memory.  A small box
-                        // is a whole number of 8-row swizzle groups, so the tile's layout is unchanged.  (Boxes
-                        // of 16 rows save more bytes but cost up to three times the copy instructions, which
-                        // made batches of many short segments slower.)
-                        const uint32_t nb = (valid + kEdgeRows - 1u) / kEdgeRows;
-                        mbar_expect_tx(full_k(s), nb * 2u * kEdgeBoxBytes);
-                        for (uint32_t b = 0; b < nb; ++b) {
-                            tma_load_2d_hint(kdst + b * kEdgeBoxBytes, &tmap_edge, 0, yk + (int32_t)(b * kEdgeRows),
-                                             full_k(s), stream_once);
-                            tma_load_2d_hint(kdst + kHalfBytes + b * kEdgeBoxBytes, &tmap_edge, 64,
-                                             yk + (int32_t)(b * kEdgeRows), full_k(s), stream_once);
-                        }
-                        mbar_expect_tx(full_v(s), nb * 2u * kEdgeBoxBytes);
-                        for (uint32_t b = 0; b < nb; ++b) {
-                            tma_load_2d_hint(vdst + b * kEdgeBoxBytes, &tmap_edge, 0, yv + (int32_t)(b * kEdgeRows),
-                                             full_v(s), stream_once);
-                            tma_load_2d_hint(vdst + kHalfBytes + b * kEdgeBoxBytes, &tmap_edge, 64,
-                                             yv + (int32_t)(b * kEdgeRows), full_v(s), stream_once);
-                        }
-                    } else {
-                        mbar_expect_tx(full_k(s), kTileBytes);
-                        tma_load_2d_hint(kdst, &tmap, 0, yk, full_k(s), stream_once);
-                        tma_load_2d_hint(kdst + kHalfBytes, &tmap, 64, yk, full_k(s), stream_once);
-                        mbar_expect_tx(full_v(s), kTileBytes);
-                        tma_load_2d_hint(vdst, &tmap, 0, yv, full_v(s), stream_once);
-                        tma_load_2d_hint(vdst + kHalfBytes, &tmap, 64, yv, full_v(s), stream_once);
+                    // Ragged last tile of a segment with at most kEdgeRows tokens: only one small box per half
+                    // is fetched (the consumers read no row past the 16-row step that holds the last token),
+                    // not the rows that follow the segment in memory.  A small box is a whole number of 8-row
+                    // swizzle groups, so the tile's layout is unchanged.  (Boxes of 16 rows save more bytes
+                    // but cost up to three times the copy instructions.)
+                    const bool edge = p.edge_boxes != 0u && valid <= kEdgeRows;
+                    static_assert(2 * kEdgeRows == kTileTokens, "a ragged tile is fetched as one small box or whole");
+                    if (lane < 4) {
+                        if (hi == 0u) mbar_expect_tx(bar, edge ? 2u * kEdgeBoxBytes : kTileBytes);
+                        tma_load_2d_hint(dst, edge ? &tmap_edge : &tmap, (int32_t)(hi * 64u), y, bar, stream_once);
                     }
                 }
             }
@@ -399,6 +389,93 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
         return;
     }
 
+    if (warp == kConsumerWarps + 2) {
+        // ================= combine warp ================================================================
+        // At the end of a row-group piece every consumer warp deposits its online-softmax state in shared
+        // memory and goes straight on to its tiles of the next piece; this warp combines the six states
+        // and writes the piece -- the final bf16 output and lse when the piece is the whole row group,
+        // else a normalised fp32 partial followed by the arrival ticket and, if it was the last one, the
+        // merge.  On a consumer warp the combine (about a microsecond of dependent shared-memory reads)
+        // held up that warp's ring stage, and the producer, which refills the stages in order, with it.
+        pdl_wait();  // out, the partial slots and the tickets belong to the kernels before until they are done
+        const int G = p.group;
+        const uint32_t nbuf = G <= kMaxGroup / 2 ? 2u : 1u;
+        const int rows_buf = G <= kMaxGroup / 2 ? kMaxGroup / 2 : kMaxGroup;
+        uint32_t piece = 0;
+        cart_work_item w_next{};
+        if (item_begin < item_end) w_next = p.items[item_begin];
+        for (uint32_t it = item_begin; it < item_end; ++it) {
+            const cart_work_item w = w_next;
+            if (it + 1 < item_end) w_next = p.items[it + 1];
+            if (!(w.flags & CART_ITEM_END)) continue;
+            const uint32_t b = piece % nbuf, use = piece / nbuf;
+            ++piece;
+            if (!__all_sync(0xffffffffu, mbar_wait(deposited(b), use & 1u, abort_flag, p.status, kStatusTimeoutConsumer)))
+                return;
+            const float *buf_o = scratch_o + (size_t)b * kConsumerWarps * rows_buf * kScratchStride;
+            const float *buf_ml = scratch_ml + (size_t)b * kConsumerWarps * kMaxGroup * 2;
+            const int quad = lane;  // four output dims per lane
+#pragma unroll 2
+            for (int r = 0; r < G; ++r) {
+                float mw[kConsumerWarps], lw[kConsumerWarps];
+                float4 v[kConsumerWarps];
+                float M = -INFINITY;
+#pragma unroll
+                for (int wv = 0; wv < kConsumerWarps; ++wv) {  // all loads of the row in flight together
+                    mw[wv] = buf_ml[(wv * kMaxGroup + r) * 2];
+                    lw[wv] = buf_ml[(wv * kMaxGroup + r) * 2 + 1];
+                    v[wv] = *reinterpret_cast<const float4 *>(buf_o + ((size_t)wv * rows_buf + r) * kScratchStride + 4 * quad);
+                }
+#pragma unroll
+                for (int wv = 0; wv < kConsumerWarps; ++wv) M = fmaxf(M, mw[wv]);
+                float L = 0.f;
+                float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int wv = 0; wv < kConsumerWarps; ++wv) {
+                    if (mw[wv] == -INFINITY) continue;  // that warp had no tile of the piece (its slot holds old data)
+                    const float wgt = fast_exp2(mw[wv] - M);
+                    L += wgt * lw[wv];
+                    a.x += wgt * v[wv].x;
+                    a.y += wgt * v[wv].y;
+                    a.z += wgt * v[wv].z;
+                    a.w += wgt * v[wv].w;
+                }
+                const float inv = 1.f / L;
+                const float lse2 = M + log2f(L);
+                if (w.flags & CART_ITEM_DIRECT) {
+                    const size_t orow = (size_t)w.row_group * G + r;
+                    uint2 packed;
+                    packed.x = pack_bf16(a.x * inv, a.y * inv);
+                    packed.y = pack_bf16(a.z * inv, a.w * inv);
+                    *reinterpret_cast<uint2 *>(reinterpret_cast<__nv_bfloat16 *>(p.out) + orow * kHeadDim + 4 * quad) = packed;
+                    if (quad == 0 && p.lse) p.lse[orow] = lse2 * 0.6931471805599453f;
+                } else {
+                    float4 *pp = reinterpret_cast<float4 *>(p.part_o + ((size_t)w.slot * G + r) * kHeadDim) + quad;
+                    *pp = make_float4(a.x * inv, a.y * inv, a.z * inv, a.w * inv);
+                    if (quad == 0) p.part_lse2[(size_t)w.slot * kMaxGroup + r] = lse2;
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(scratch_free(b));  // the buffer may be refilled from here on
+            if (!(w.flags & CART_ITEM_DIRECT) && p.tickets != nullptr) {
+                // Split row group: the block whose piece arrives last merges all pieces.  Nobody waits.
+                __threadfence();  // publish the partial before the ticket
+                __syncwarp();
+                const cart_merge_item mi = p.merges[w.merge];
+                uint32_t mine = 0;
+                if (lane == 0) mine = (atomicAdd(&p.tickets[w.merge], 1u) + 1u == mi.slot_end - mi.slot_begin) ? 1u : 0u;
+                mine = __shfl_sync(0xffffffffu, mine, 0);
+                if (mine) {
+                    __threadfence();
+                    merge_row_group<4, 2>(mi, G, p.part_o, p.part_lse2, p.out, p.lse, lane, 32);
+                    __syncwarp();
+                    if (lane == 0) p.tickets[w.merge] = 0;  // ready for the next launch
+                }
+            }
+        }
+        return;
+    }
+
     // ===================== consumers ==============================================================
     pdl_wait();  // q, the partial slots and the tickets belong to the kernels before until they are done
     if (p.ready_flag != nullptr && blockIdx.x == 0 && threadIdx.x == 0)  // tell the kernel that runs beside this one
@@ -457,7 +534,7 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
         t += ntiles;
 
         if (w.flags & CART_ITEM_END) {
-            // ---- hand this warp's state of the piece to whichever warp arrives last ----------------
+            // ---- hand this warp's state of the piece to the combine warp ------------------------------
             // No block-wide barrier: a warp that has deposited goes straight on to its tiles of the next
             // piece.  Pieces alternate between the scratch buffers; a buffer is free again once the
             // combine of the piece that used it before is done.
@@ -483,75 +560,7 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
                 }
             }
             __syncwarp();
-            uint32_t last = 0;
-            if (lane == 0) {
-                __threadfence_block();
-                last = (atomicAdd(const_cast<uint32_t *>(&arrivals[b]), 1u) == (uint32_t)kConsumerWarps - 1u) ? 1u : 0u;
-                __threadfence_block();
-            }
-            last = __shfl_sync(0xffffffffu, last, 0);
-            __syncwarp();
-            if (!last) continue;
-
-            // ---- this warp arrived last: combine the six states and write the piece -------------------
-            for (int idx = lane; idx < G * 32; idx += 32) {  // one query row, four output dims
-                const int r = idx >> 5, quad = idx & 31;
-                float mw[kConsumerWarps];
-                float M = -INFINITY;
-#pragma unroll
-                for (int wv = 0; wv < kConsumerWarps; ++wv) {
-                    mw[wv] = buf_ml[(wv * kMaxGroup + r) * 2];
-                    M = fmaxf(M, mw[wv]);
-                }
-                float L = 0.f;
-                float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-                for (int wv = 0; wv < kConsumerWarps; ++wv) {
-                    if (mw[wv] == -INFINITY) continue;  // that warp had no tile of the piece
-                    const float wgt = fast_exp2(mw[wv] - M);
-                    L += wgt * buf_ml[(wv * kMaxGroup + r) * 2 + 1];
-                    const float4 v = *reinterpret_cast<const float4 *>(
-                        buf_o + ((size_t)wv * rows_buf + r) * kScratchStride + 4 * quad);
-                    a.x += wgt * v.x;
-                    a.y += wgt * v.y;
-                    a.z += wgt * v.z;
-                    a.w += wgt * v.w;
-                }
-                const float inv = 1.f / L;
-                const float lse2 = M + log2f(L);
-                if (w.flags & CART_ITEM_DIRECT) {
-                    const size_t orow = (size_t)w.row_group * G + r;
-                    uint2 packed;
-                    packed.x = pack_bf16(a.x * inv, a.y * inv);
-                    packed.y = pack_bf16(a.z * inv, a.w * inv);
-                    *reinterpret_cast<uint2 *>(reinterpret_cast<__nv_bfloat16 *>(p.out) + orow * kHeadDim + 4 * quad) = packed;
-                    if (quad == 0 && p.lse) p.lse[orow] = lse2 * 0.6931471805599453f;
-                } else {
-                    float4 *pp = reinterpret_cast<float4 *>(p.part_o + ((size_t)w.slot * G + r) * kHeadDim) + quad;
-                    *pp = make_float4(a.x * inv, a.y * inv, a.z * inv, a.w * inv);
-                    if (quad == 0) p.part_lse2[(size_t)w.slot * kMaxGroup + r] = lse2;
-                }
-            }
-            __syncwarp();
-            if (lane == 0) {
-                arrivals[b] = 0;
-                mbar_arrive(scratch_free(b));  // the buffer may be refilled from here on
-            }
-            if (!(w.flags & CART_ITEM_DIRECT) && p.tickets != nullptr) {
-                // Split row group: the block whose piece arrives last merges all pieces.  Nobody waits.
-                __threadfence();  // publish the partial before the ticket
-                __syncwarp();
-                const cart_merge_item mi = p.merges[w.merge];
-                uint32_t mine = 0;
-                if (lane == 0) mine = (atomicAdd(&p.tickets[w.merge], 1u) + 1u == mi.slot_end - mi.slot_begin) ? 1u : 0u;
-                mine = __shfl_sync(0xffffffffu, mine, 0);
-                if (mine) {
-                    __threadfence();
-                    merge_row_group<4, 2>(mi, G, p.part_o, p.part_lse2, p.out, p.lse, lane, 32);
-                    __syncwarp();
-                    if (lane == 0) p.tickets[w.merge] = 0;  // ready for the next launch
-                }
-            }
+            if (lane == 0) mbar_arrive(deposited(b));  // (release) the combine warp takes it from here
         }
     }
 }

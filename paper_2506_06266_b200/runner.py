@@ -106,6 +106,27 @@ class LoadedWorkload:
         io = w.batch * w.n_q_heads * (w.head_dim * 2 * 2 + 4)
         return kv + io
 
+    def unique_bytes_per_layer(self) -> int:
+        """What the method itself has to read per layer: every stored Cartridge the batch attends to once,
+        however many requests share it, every request's own suffix, plus q, out and lse traffic."""
+        w = self.w
+        carts = {c for parts in self.parts for c in parts}
+        suffix_tokens = int(self.suffix.sum()) + self.appended * w.batch
+        kv = (len(carts) * w.p + suffix_tokens) * w.kv_bytes_per_token_layer()
+        io = w.batch * w.n_q_heads * (w.head_dim * 2 * 2 + 4)
+        return kv + io
+
+    def shared_flops_per_layer(self, min_readers: int = 4, tile: int = 128) -> int:
+        """Floating-point operations of the two dense products (q K^T and P V) over the full tiles of the
+        Cartridges that at least `min_readers` requests of the batch share: the tensor-core kernel's work."""
+        w = self.w
+        readers: Dict[int, int] = {}
+        for parts in self.parts:
+            for c in parts:
+                readers[c] = readers.get(c, 0) + 1
+        full = w.p // tile * tile
+        return sum(4 * r * w.n_q_heads * w.head_dim * full for r in readers.values() if r >= min_readers and full)
+
     def step(self, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor, out: torch.Tensor,
              lse: Optional[torch.Tensor], layers: Optional[Iterable[int]] = None, fused: bool = True) -> None:
         """One decode step: per layer, append every request's new token, then attend -- in one call
