@@ -191,10 +191,13 @@ extern "C" cart_status cart_plan_build_shared(const cart_plan_seg *segs, const i
         }
         return bal.block_has_work() ? bal.c + 1 : bal.c;
     };
-    // Side by side: how many of the n_cta blocks the shared kernel gets.  Estimated times in nanoseconds from
-    // measurements on B200: a 128-token shared tile takes a block 1.6 us and a unit 9 us on top; a 64-token
-    // stream tile takes a block at least 0.51 us (what one SM can pull) and 0.0052 us per streaming block
-    // (the SM's share of HBM bandwidth), and a row-group piece 1.5 us on top.
+    // Side by side: how many of the n_cta blocks the shared kernel gets.  Estimated times in nanoseconds,
+    // fitted to measurements on B200 (launch lists of the two kernels at several divisions of the SMs):
+    //   shared kernel on s blocks   3000 + (1340 per 128-token tile + 6500 per unit) / s
+    //   stream kernel on c blocks   3000 + max((510 per 64-token tile + 1500 per row-group piece) / c,
+    //                                          5.1 per tile)      -- the second term is the HBM bound
+    // One after the other costs the sum of the two on all blocks less 6000 (the second kernel starts under the
+    // first one's tail); side by side the larger of the two on their shares.  The division with the smallest estimate is taken if it beats one-after-the-other by 5 %.
     uint64_t n_cta_stream = (uint64_t)n_cta, n_cta_shared = (uint64_t)n_cta;
     o->n_shared_ctas = 0;
     if (W_sh > 0 && o->side_by_side > 0 && n_cta >= 2) {
@@ -209,23 +212,35 @@ extern "C" cart_status cart_plan_build_shared(const cart_plan_seg *segs, const i
             if (t > 0) st_rgs += (uint64_t)n_kv_heads;
         }
         if (st_tiles > 0) {
+            auto est_shared = [&](uint64_t blocks) {
+                // runs of equal length that divide evenly over the blocks are not cut; otherwise every block
+                // boundary but the last cuts one
+                const uint64_t cuts = combos.size() % blocks == 0 ? 0 : blocks - 1;
+                return 3000 + (W_sh * 1340 + (combos.size() + cuts) * 6500) / blocks;
+            };
+            auto est_stream = [&](uint64_t blocks) {
+                return 3000 + std::max<uint64_t>((st_tiles * 510 + (st_rgs + blocks) * 1500) / blocks, (st_tiles * 51) / 10);
+            };
             uint64_t S = 0;
             if (o->side_by_side > 1) {
                 S = std::min<uint64_t>((uint64_t)o->side_by_side, (uint64_t)n_cta - 1);
             } else {
                 uint64_t best = UINT64_MAX;
                 for (uint64_t s2 = 1; s2 < (uint64_t)n_cta; ++s2) {
-                    const uint64_t c2 = (uint64_t)n_cta - s2;
-                    const uint64_t est_sh = (W_sh * 1600 + (combos.size() + s2) * 9000) / s2;
-                    const uint64_t tile_ns = std::max<uint64_t>(510, (c2 * 52) / 10);
-                    const uint64_t est_st = (st_tiles * tile_ns + (st_rgs + c2) * 1500) / c2;
-                    const uint64_t est = std::max(est_sh, est_st);
+                    // (a division that leaves the runs whole is preferred to one that is a hair faster on paper)
+                    const uint64_t est = std::max(est_shared(s2), est_stream((uint64_t)n_cta - s2)) +
+                                         (combos.size() % s2 == 0 ? 0 : 1500);
                     if (est < best) { best = est; S = s2; }
                 }
+                // one after the other, the second kernel's start-up and first tiles hide under the first one's tail
+                const uint64_t serial = est_shared((uint64_t)n_cta) + est_stream((uint64_t)n_cta) - 6000;
+                if (best * 100 >= serial * 95) S = 0;  // not worth it: each kernel gets all blocks in turn
             }
-            n_cta_shared = S;
-            n_cta_stream = (uint64_t)n_cta - S;
-            o->n_shared_ctas = (int32_t)S;
+            if (S > 0) {
+                n_cta_shared = S;
+                n_cta_stream = (uint64_t)n_cta - S;
+                o->n_shared_ctas = (int32_t)S;
+            }
         }
     }
     uint64_t C_sh = 0;

@@ -274,8 +274,14 @@ def test_side_by_side_divides_the_blocks_between_the_two_kernels(w):
     G = w.n_q_heads // w.n_kv_heads
     plan = check(segs, w.n_kv_heads, G, 148, piece_cost=3, unit_cost=4, side_by_side=1)
     S = plan["n_shared_ctas"]
-    assert 16 <= S <= 120                      # both parts are substantial on these workloads
-    assert plan["n_unit_cta_used"] >= S - 2 and plan["n_cta_used"] >= 148 - S - 2
+    if w.cartridges == "shared":
+        # one long Cartridge and long suffixes: a quarter of the blocks or so for the tensor-core kernel, and a
+        # division that leaves the 32 (M-tile, KV head) runs whole
+        assert 16 <= S <= 64 and len(plan["units"]) == 32
+        assert plan["n_unit_cta_used"] >= S - 2 and plan["n_cta_used"] >= 148 - S - 2
+    else:
+        # many short runs: the estimate does not favour either order by the required margin
+        assert S == 0 or plan["n_unit_cta_used"] >= S - 2
     forced = check(segs, w.n_kv_heads, G, 148, piece_cost=3, unit_cost=4, side_by_side=50)
     assert forced["n_shared_ctas"] == 50
     # a batch without a shared part, or without a stream part, keeps all blocks for the one kernel
