@@ -193,11 +193,10 @@ extern "C" cart_status cart_plan_build_shared(const cart_plan_seg *segs, const i
     };
     // Side by side: how many of the n_cta blocks the shared kernel gets.  Estimated times in nanoseconds,
     // fitted to measurements on B200 (launch lists of the two kernels at several divisions of the SMs):
-    //   shared kernel on s blocks   3000 + (1340 per 128-token tile + 6500 per unit) / s
+    //   shared kernel on s blocks   3000 + (1200 per 128-token tile + 4000 per unit) / s
     //   stream kernel on c blocks   3000 + max((510 per 64-token tile + 1500 per row-group piece) / c,
     //                                          5.1 per tile)      -- the second term is the HBM bound
-    // One after the other costs the sum of the two on all blocks less 6000 (the second kernel starts under the
-    // first one's tail); side by side the larger of the two on their shares.  The division with the smallest estimate is taken if it beats one-after-the-other by 5 %.
+    // One after the other costs the sum of the two on all blocks; side by side the larger of the two on their shares.  The division with the smallest estimate is taken if it beats one-after-the-other by 5 %.
     uint64_t n_cta_stream = (uint64_t)n_cta, n_cta_shared = (uint64_t)n_cta;
     o->n_shared_ctas = 0;
     if (W_sh > 0 && o->side_by_side > 0 && n_cta >= 2) {
@@ -216,7 +215,7 @@ extern "C" cart_status cart_plan_build_shared(const cart_plan_seg *segs, const i
                 // runs of equal length that divide evenly over the blocks are not cut; otherwise every block
                 // boundary but the last cuts one
                 const uint64_t cuts = combos.size() % blocks == 0 ? 0 : blocks - 1;
-                return 3000 + (W_sh * 1340 + (combos.size() + cuts) * 6500) / blocks;
+                return 3000 + (W_sh * 1200 + (combos.size() + cuts) * 4000) / blocks;
             };
             auto est_stream = [&](uint64_t blocks) {
                 return 3000 + std::max<uint64_t>((st_tiles * 510 + (st_rgs + blocks) * 1500) / blocks, (st_tiles * 51) / 10);
@@ -227,13 +226,13 @@ extern "C" cart_status cart_plan_build_shared(const cart_plan_seg *segs, const i
             } else {
                 uint64_t best = UINT64_MAX;
                 for (uint64_t s2 = 1; s2 < (uint64_t)n_cta; ++s2) {
-                    // (a division that leaves the runs whole is preferred to one that is a hair faster on paper)
+                    // (a division that leaves the runs whole is preferred: measured on one shared Cartridge of 32 runs, 28 blocks
+                    //  for the tensor-core kernel took 8 us longer per layer than 32)
                     const uint64_t est = std::max(est_shared(s2), est_stream((uint64_t)n_cta - s2)) +
-                                         (combos.size() % s2 == 0 ? 0 : 1500);
+                                         (combos.size() % s2 == 0 ? 0 : 6000);
                     if (est < best) { best = est; S = s2; }
                 }
-                // one after the other, the second kernel's start-up and first tiles hide under the first one's tail
-                const uint64_t serial = est_shared((uint64_t)n_cta) + est_stream((uint64_t)n_cta) - 6000;
+                const uint64_t serial = est_shared((uint64_t)n_cta) + est_stream((uint64_t)n_cta);
                 if (best * 100 >= serial * 95) S = 0;  // not worth it: each kernel gets all blocks in turn
             }
             if (S > 0) {

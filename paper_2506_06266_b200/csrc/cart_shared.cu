@@ -10,25 +10,26 @@
 //   producer warps  TMA loads of K tiles (warp 0, three stages) and V tiles (warp 2, two stages), 128 tokens
 //                   x 128 dims, 128-byte swizzle, completion on mbarriers
 //   MMA warp        one thread issues  S = Q K^T  (128 x 128 x 128, both operands from shared memory,
-//                   accumulator in tensor memory) and  O += P V  (A operand P from tensor memory, V from
-//                   shared memory, accumulating in tensor memory over the warpgroup's tiles of the unit);
+//                   accumulator in tensor memory) two tiles ahead of the softmax, and  O += P V  (A operand
+//                   P from tensor memory, V from shared memory, one accumulator for the whole unit);
 //                   tcgen05.commit signals mbarriers
-//   2 x 4 softmax  two warpgroups take alternate tiles (warpgroup w owns S buffer w and accumulator w).
-//   warps           Thread r of a warpgroup owns query row r: reads S from tensor memory (two loads in
-//                   flight), keeps a reference maximum and the sum of an online softmax over its
-//                   warpgroup's tiles in fp32, and writes P = 2^(s - m) as bf16 pairs back over the first
-//                   half of the S buffer (tcgen05.st).  The reference maximum only moves when a row's
-//                   maximum has grown by more than 2^8 (then the warp rescales its lanes of the accumulator
-//                   in tensor memory); sum and accumulator always refer to the same reference, so the
-//                   result is exact.  At the end of a unit the warpgroups read their accumulators and
-//                   combine their states through shared memory.
+//   2 x 4 softmax   both warpgroups work on every tile: thread (w, r) owns query row r (tensor-memory
+//   warps           lane r) and the 64 score columns of half w.  It reads its 64 scores once, the two
+//                   owners of a row exchange their maxima through shared memory, and each writes
+//                   P = 2^(s - m) as bf16 pairs over its own half of the score buffer (tcgen05.st).  The
+//                   reference m of a row only moves when the row's maximum has outgrown it by more
+//                   than 2^8 (then the two owners rescale their halves of the accumulator in tensor
+//                   memory); sums and accumulator always refer to the same reference, so the result is
+//                   exact.  At the end of a unit each thread reads its 64 columns of the accumulator,
+//                   the two owners add their sums, and the row leaves as a normalised fp32 partial.
 //
-// S (with P in it) is double-buffered in tensor memory and each warpgroup has its own accumulator
-// (4 x 128 columns), so the products of tile t+1 run while the softmax of tile t does.  At the end of a
-// unit every row is written as a
-// normalised fp32 partial (o, lse); the partials of a (request, KV head) row group are merged by
-// log-sum-exp either by the block that delivers the last one -- this kernel's or the stream kernel's --
-// or, when the batch has more split row groups than blocks, by a merge kernel that runs afterwards.
+// Tensor memory: three score buffers (S0 S1 S2, with P inside) and one accumulator, 128 fp32 columns
+// each.  With three buffers the score products of tiles t+1 and t+2 are complete or in flight while the
+// softmax of tile t runs, so neither side waits for the other's latency: the tile rate is set by the
+// tensor pipe (16 instructions per tile) or by the exponentials (128 x 128 per tile), whichever is slower.
+// The partials of a (request, KV head) row group are merged by log-sum-exp either by the block that
+// delivers the last one -- this kernel's or the stream kernel's -- or, when the batch has more split row
+// groups than blocks, by a merge kernel that runs afterwards.
 //
 // Every wait is bounded; on expiry the block raises a flag in the device status word, stops issuing
 // work, waits (bounded) for what is in flight, frees its tensor memory and returns.
@@ -45,43 +46,48 @@ constexpr uint32_t kShBlock = 128u * 128u;            // 128 rows x 128 bytes: o
 constexpr uint32_t kShTileBytes = 2u * kShBlock;      // 128 x 128 bf16
 constexpr int kKStages = 3;                           // K tiles in flight (each ring has its own producer warp)
 constexpr int kVStages = 2;
+constexpr int kSBufs = 3;                             // score buffers in tensor memory
 constexpr int kShThreads = 384;                       // utility warpgroup (K producer, MMA, V producer, 1 idle) + 2 softmax warpgroups
 // Registers per thread after the warpgroups have re-divided the block's allocation (384 x 168): the
-// utility warps need few, the softmax threads hold a 128-float accumulator at the end of a unit.  4 x 32 x 40 + 8 x 32 x 232
+// utility warps need few, a softmax thread holds 64 scores and 32 packed probabilities.  4 x 32 x 40 + 8 x 32 x 232
 // = 64512 registers, and per SM sub-partition 1 utility + 2 softmax warps = 16128 of its 16384.
 constexpr int kRegsUtility = 40;
 constexpr int kRegsSoftmax = 232;
 constexpr int kSoftmaxThreads = 128;                  // one softmax warpgroup
-constexpr uint32_t kTmemCols = 512;                   // S0 S1 (scores, then P), O0 O1 (accumulators): 128 fp32 columns each
+constexpr uint32_t kTmemCols = 512;                   // S0 S1 S2 (scores, then P), O (accumulator): 128 fp32 columns each
+constexpr uint32_t kTmemO = 3u * 128u;                // first column of the accumulator
 constexpr float kRescaleStep = 8.f;                   // how far a row's maximum may outgrow its reference (base-2 units)
 
 // shared-memory layout (offsets from a 1024-byte aligned base)
-constexpr uint32_t kOffQ = 0;
-constexpr uint32_t kOffX = kOffQ + kShTileBytes;       // with Q: the 64 KB scratch of a unit's end
-constexpr uint32_t kOffK = kOffX + kShTileBytes;
+constexpr uint32_t kOffQ = 0;                          // two query buffers
+constexpr uint32_t kOffK = kOffQ + 2u * kShTileBytes;
 constexpr uint32_t kOffV = kOffK + kKStages * kShTileBytes;
 constexpr uint32_t kOffBar = kOffV + kVStages * kShTileBytes;
-constexpr uint32_t kOffMisc = kOffBar + 32 * 8;        // room for 32 barriers (22 used); then: tmem address, abort flag, unit flag
+constexpr uint32_t kOffMisc = kOffBar + 32 * 8;        // room for 32 barriers; then: tmem address, abort flag, unit flag
 constexpr uint32_t kOffFlags = kOffMisc + 16;          // one word per reader: "merge this row group"
-constexpr uint32_t kOffComb = kOffFlags + 128 * 4;     // running maximum and sum of the second warpgroup's rows
-constexpr uint32_t kShSmemUsed = kOffComb + 2 * 128 * 4;
+// what the two owners of a row tell each other: per tile their maxima (bf16 bits, [tile parity][half][row]);
+// at a unit's end their sums (fp32 [half][row], over the same bytes, behind a barrier)
+constexpr uint32_t kOffXchg = kOffFlags + 128 * 4;
+constexpr uint32_t kShSmemUsed = kOffXchg + 2 * 128 * 4;
 constexpr uint32_t kShSmemBytes = kShSmemUsed + 1024;  // slack to align the base
 static_assert(kShSmemBytes <= 232448, "shared memory budget of one sm_100 block exceeded");
 
 enum Bar : int {
     kBarKFull = 0,   // [kKStages] TMA -> MMA
-    kBarKEmpty = 3,  // [kKStages] MMA (commit) -> TMA
+    kBarKEmpty = 3,  // (unused: the K producer listens on kBarSFull)
     kBarVFull = 6,   // [kVStages]
     kBarVEmpty = 8,  // [kVStages]
-    kBarSFull = 10,  // [2] MMA (commit) -> softmax
-    kBarSFree = 12,  // [2] MMA (commit of P V: the probabilities live in the S buffer) -> MMA
-    kBarPReady = 14, // [2] softmax -> MMA          (4 arrivals: one per warp of the warpgroup)
-    kBarOFull = 16,  // [2] MMA (commit of P V) -> softmax: the accumulator holds the product
-    kBarQReady = 20, // softmax -> MMA              (8 arrivals: every softmax warp)
-    kBarDrain = 21,  // MMA (commit) -> MMA, on the way out
+    kBarSFull = 10,  // [kSBufs] MMA (commit) -> softmax
+    kBarSFree = 13,  // [kSBufs] MMA (commit of P V) -> softmax: the accumulator holds the products up to this tile
+    kBarPReady = 16, // [kSBufs] softmax -> MMA         (8 arrivals: one per softmax warp)
+    kBarQReady = 20, // [2] softmax -> MMA: a unit's query rows are in their buffer  (8 arrivals: one per softmax warp)
+    kBarDrain = 24,  // MMA (commit) -> MMA, on the way out
 };
+static_assert(kKStages == kSBufs, "the K ring's stages are released through the score buffers' barriers");
 static_assert(kBarKEmpty - kBarKFull >= kKStages && kBarVFull - kBarKEmpty >= kKStages &&
-              kBarVEmpty - kBarVFull >= kVStages && kBarSFull - kBarVEmpty >= kVStages, "barrier indices overlap");
+              kBarVEmpty - kBarVFull >= kVStages && kBarSFull - kBarVEmpty >= kVStages &&
+              kBarSFree - kBarSFull >= kSBufs && kBarPReady - kBarSFree >= kSBufs && kBarQReady - kBarPReady >= kSBufs,
+              "barrier indices overlap");
 
 // ---- tcgen05 wrappers ---------------------------------------------------------------------------
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -103,32 +109,42 @@ constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) <<
 constexpr uint32_t kIdescS = kIdesc;                  // A (Q) and B (K tile) both K-major
 constexpr uint32_t kIdescPV = kIdesc | (1u << 16);    // B (V tile) is MN-major: dims contiguous
 
+// The issuing warp runs its loop with all lanes (uniform control flow, so that addresses and descriptors
+// can live in uniform registers); `issue` is non-zero in the one lane that executes the instruction.
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                          uint32_t accumulate)
+                                          uint32_t accumulate, uint32_t issue)
 {
     asm volatile(
         "{\n"
-        ".reg .pred p;\n"
+        ".reg .pred p, q;\n"
         "setp.ne.b32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
-        "}\n" ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        "setp.ne.b32 q, %5, 0;\n"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+        "}\n" ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(issue)
         : "memory");
 }
 // The same with the A operand in tensor memory (lane = row, 8 columns of bf16 pairs per 16-wide step).
 __device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
-                                             uint32_t accumulate)
+                                             uint32_t accumulate, uint32_t issue)
 {
     asm volatile(
         "{\n"
-        ".reg .pred p;\n"
+        ".reg .pred p, q;\n"
         "setp.ne.b32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n"
-        "}\n" ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        "setp.ne.b32 q, %5, 0;\n"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n"
+        "}\n" ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(issue)
         : "memory");
 }
-__device__ __forceinline__ void umma_commit(uint32_t bar)
+__device__ __forceinline__ void umma_commit(uint32_t bar, uint32_t issue)
 {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    asm volatile(
+        "{\n"
+        ".reg .pred q;\n"
+        "setp.ne.b32 q, %1, 0;\n"
+        "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n"
+        "}\n" ::"r"(bar), "r"(issue)
+        : "memory");
 }
 // Writes 16 consecutive 32-bit columns of this thread's tensor-memory lane.
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&w)[16])
@@ -174,6 +190,13 @@ __device__ __forceinline__ void softmax_bar()  // the first softmax warpgroup
 __device__ __forceinline__ void softmax_bar_both()  // both softmax warpgroups
 {
     asm volatile("bar.sync 3, %0;" ::"n"(2 * kSoftmaxThreads) : "memory");
+}
+// A float rounded up to the next bf16 (upper 16 bits), for finite inputs: the exchanged row maxima only
+// have to be the same number for both owners of a row and not below the true maximum.
+__device__ __forceinline__ uint32_t bf16_ceil_bits(float x)
+{
+    const uint32_t b = __float_as_uint(x);
+    return ((b & 0x80000000u) ? b : b + 0xFFFFu) >> 16;  // negative: truncation already rounds up
 }
 
 // "The kernels before this one on the stream are complete and their writes visible."  Alone, that is
@@ -225,21 +248,36 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     pdl_launch_dependents();
+    // The plan is in place before any of these kernels starts: read it at once.
+    const uint32_t unit_begin = p.unit_cta_begin[blockIdx.x];
+    const uint32_t unit_end = p.unit_cta_begin[blockIdx.x + 1];
+    // ... as far as the first unit and, for the softmax threads, the batch index of the row's reader: these
+    // dependent loads run under the set-up below (and, in a sequence of dependent launches, under the tail
+    // of the kernel before)
+    cart_shared_unit u_first{};
+    uint32_t first_batch = 0;
+    if (unit_begin < unit_end) {
+        u_first = p.units[unit_begin];
+        const uint32_t r0 = (threadIdx.x & 127u) / (uint32_t)p.group;
+        if (threadIdx.x >= 128u && r0 < u_first.n_readers) first_batch = p.readers[u_first.reader_begin + r0];
+    }
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < kKStages; ++i) {
             mbar_init(bar(kBarKFull + i), 1);
-            mbar_init(bar(kBarKEmpty + i), 1);
         }
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < kVStages; ++i) {
             mbar_init(bar(kBarVFull + i), 1);
             mbar_init(bar(kBarVEmpty + i), 1);
+        }
+        for (int i = 0; i < kSBufs; ++i) {
             mbar_init(bar(kBarSFull + i), 1);
             mbar_init(bar(kBarSFree + i), 1);
-            mbar_init(bar(kBarOFull + i), 1);
-            mbar_init(bar(kBarPReady + i), 4);
+            mbar_init(bar(kBarPReady + i), 8);
         }
-        mbar_init(bar(kBarQReady), 8);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bar(kBarQReady + i), 8);
+        }
         mbar_init(bar(kBarDrain), 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -256,14 +294,12 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
-    // The plan is in place before any of these kernels starts.  Shared tiles of stored Cartridges are only
-    // ever written by copies and may be fetched at once; shared tiles in suffix storage (prefill: the part
-    // of the suffix that a group of rows has in common, units marked CART_UNIT_SUFFIX) may have been
-    // written by the kernel before this one, so the producers wait for the kernels before them ahead of
-    // the first such unit.  The queries, the partial slots and the tickets may still be in use by those
-    // kernels too: the softmax warps wait before they read a query.
-    const uint32_t unit_begin = p.unit_cta_begin[blockIdx.x];
-    const uint32_t unit_end = p.unit_cta_begin[blockIdx.x + 1];
+    // Shared tiles of stored Cartridges are only ever written by copies and may be fetched at once; shared
+    // tiles in suffix storage (prefill: the part of the suffix that a group of rows has in common, units
+    // marked CART_UNIT_SUFFIX) may have been written by the kernel before this one, so the producers wait
+    // for the kernels before them ahead of the first such unit.  The queries, the partial slots and the
+    // tickets may still be in use by those kernels too: the softmax warps wait before they read a query, and
+    // nothing is written before the first scores exist.
 
     if (warp < 4) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsUtility));
@@ -273,7 +309,8 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
             //  V ring is waiting for)
             if (lane == 0) {
                 const bool is_v = warp == 2;
-                const int full0 = is_v ? kBarVFull : kBarKFull, empty0 = is_v ? kBarVEmpty : kBarKEmpty;
+                // (a K stage is free once the score product that read it is complete: the barrier of score buffer tt % 3)
+                const int full0 = is_v ? kBarVFull : kBarKFull, empty0 = is_v ? kBarVEmpty : kBarSFull;
                 const uint32_t ring = base + (is_v ? kOffV : kOffK);
                 const uint32_t nst = is_v ? (uint32_t)kVStages : (uint32_t)kKStages;
                 asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap)) : "memory");
@@ -316,178 +353,235 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
             __syncwarp();
         } else if (warp == 1) {
             // ================= MMA issuer ===================================================================
-            if (lane == 0) {
-                const uint32_t q_lo = base + kOffQ;
-                uint32_t tt0 = 0;   // tiles of earlier units
-                uint32_t nunit = 0;
-                bool ok = true;
-                // S(tt) = Q K^T into S buffer tt & 1
-                auto issue_s = [&](uint32_t tt) -> bool {
-                    const int st = (int)(tt & 1u);
-                    const uint32_t par = (tt >> 1) & 1u;
-                    const uint32_t kst = tt % (uint32_t)kKStages, kpar = (tt / (uint32_t)kKStages) & 1u;
-                    if (!mbar_wait(bar(kBarKFull + (int)kst), kpar, abort_flag, p.status, kStatusTimeoutMma)) return false;
-                    if (!mbar_wait(bar(kBarSFree + st), par ^ 1u, abort_flag, p.status, kStatusTimeoutMma)) return false;
-                    tc_fence_after();
-                    const uint32_t k_lo = base + kOffK + kst * kShTileBytes;
-                    // the operands' descriptors differ from step to step only in the start address field
-                    // (units of 16 bytes): the next 16 dims are 32 bytes on, the second 64-dim block kShBlock on
-                    const uint64_t a0 = umma_desc(q_lo, 16, 1024), b0 = umma_desc(k_lo, 16, 1024);
-                    const uint32_t d_s = tmem + (uint32_t)st * 128u;
-    #pragma unroll
-                    for (uint32_t k = 0; k < 8; ++k) {  // 16 dims per instruction
-                        const uint64_t off16 = (uint64_t)(((k >> 2) * kShBlock + (k & 3u) * 32u) >> 4);
-                        umma_bf16(d_s, a0 + off16, b0 + off16, kIdescS, k);
-                    }
-                    umma_commit(bar(kBarSFull + st));
-                    umma_commit(bar(kBarKEmpty + (int)kst));
-                    return true;
-                };
-                // O += P V into the accumulator of warpgroup tt & 1; `first`: the warpgroup's first tile of the unit
-                auto issue_pv = [&](uint32_t tt, bool first) -> bool {
-                    const int st = (int)(tt & 1u);
-                    const uint32_t par = (tt >> 1) & 1u;
-                    if (!mbar_wait(bar(kBarVFull + st), par, abort_flag, p.status, kStatusTimeoutMma)) return false;
-                    if (!mbar_wait(bar(kBarPReady + st), par, abort_flag, p.status, kStatusTimeoutMma)) return false;
-                    tc_fence_after();
-                    const uint32_t v_lo = base + kOffV + (uint32_t)st * kShTileBytes;
-                    // P: the A operand comes from tensor memory, where the softmax warps left it in the first
-                    // 64 columns of the S buffer (two bf16 per column, 16 tokens = 8 columns per step).
-                    // V: tokens are rows of 128 bytes (8-token groups 1024 bytes apart, 16 tokens = 2048 bytes
-                    // per step); the two 64-dim blocks of the tile are kShBlock bytes apart.
-                    const uint64_t b0 = umma_desc(v_lo, kShBlock, 1024);
-                    const uint32_t p_tm = tmem + (uint32_t)st * 128u;
-                    const uint32_t d_o = tmem + 256u + (uint32_t)st * 128u;
-    #pragma unroll
-                    for (uint32_t k = 0; k < 8; ++k)  // 16 tokens per instruction
-                        umma_bf16_ts(d_o, p_tm + 8u * k, b0 + (uint64_t)(k * 128u), kIdescPV, (first && k == 0u) ? 0u : 1u);
-                    umma_commit(bar(kBarOFull + st));
-                    umma_commit(bar(kBarVEmpty + st));
-                    umma_commit(bar(kBarSFree + st));  // the S buffer (and the P in it) may be overwritten
-                    return true;
-                };
-                for (uint32_t ui = unit_begin; ui < unit_end && ok; ++ui, ++nunit) {
-                    const uint32_t n = p.units[ui].n_tiles;
-                    ok = mbar_wait(bar(kBarQReady), nunit & 1u, abort_flag, p.status, kStatusTimeoutMma);
-                    if (!ok) break;
-                    tc_fence_after();
-                    ok = issue_s(tt0);
-                    for (uint32_t t = 0; t < n && ok; ++t) {
-                        if (t + 1 < n) ok = issue_s(tt0 + t + 1);
-                        if (ok) ok = issue_pv(tt0 + t, t < 2u);
-                    }
-                    tt0 += n;
+            // All lanes walk the loop and wait together; lane 0 issues.
+            const uint32_t issue = lane == 0 ? 1u : 0u;
+            bool ok = true;
+            auto wait_all = [&](int b, uint32_t parity) -> bool {
+                return __all_sync(0xffffffffu, mbar_wait(bar(b), parity, abort_flag, p.status, kStatusTimeoutMma));
+            };
+            // Two cursors walk the block's tiles in order: `qk` names the next score product to issue (it
+            // runs two tiles ahead), `pv` the next P V product.  tt = tile index counted over the block.
+            struct Cursor { uint32_t ui, t, n, unit_no; };
+            auto tiles_of = [&](uint32_t ui) { return ui < unit_end ? p.units[ui].n_tiles : 0u; };
+            Cursor qk{unit_begin, 0u, tiles_of(unit_begin), 0u}, pv = qk;
+            auto advance = [&](Cursor &c) {
+                if (++c.t == c.n) {
+                    ++c.ui;
+                    ++c.unit_no;
+                    c.t = 0;
+                    c.n = tiles_of(c.ui);
                 }
-                // products still in flight must finish before the tensor memory is given back
-                umma_commit(bar(kBarDrain));
-                const uint64_t t0 = global_timer_ns();
-                while (!mbar_try_wait(bar(kBarDrain), 0) && global_timer_ns() - t0 < kWaitLimitNs) {}
+            };
+            uint32_t total = 0;
+            for (uint32_t ui = unit_begin; ui < unit_end; ++ui) total += p.units[ui].n_tiles;
+            // S(tt) = Q K^T into score buffer tt % 3.  The buffer last held the probabilities of tile tt - 3,
+            // read by that tile's P V product, which this thread issued earlier: the tensor pipe executes one
+            // thread's products in the order of issue, so no completion has to be waited for here.
+            auto issue_s = [&](uint32_t tt) -> bool {
+                const uint32_t sb = tt % (uint32_t)kSBufs;
+                const uint32_t kst = tt % (uint32_t)kKStages, kpar = (tt / (uint32_t)kKStages) & 1u;
+                const uint32_t qb = qk.unit_no & 1u;
+                if (qk.t == 0u && !wait_all(kBarQReady + (int)qb, (qk.unit_no >> 1) & 1u)) return false;
+                if (!wait_all(kBarKFull + (int)kst, kpar)) return false;
+                tc_fence_after();
+                const uint32_t q_lo = base + kOffQ + qb * kShTileBytes;
+                const uint32_t k_lo = base + kOffK + kst * kShTileBytes;
+                // the operands' descriptors differ from step to step only in the start address field
+                // (units of 16 bytes): the next 16 dims are 32 bytes on, the second 64-dim block kShBlock on
+                const uint64_t a0 = umma_desc(q_lo, 16, 1024), b0 = umma_desc(k_lo, 16, 1024);
+                const uint32_t d_s = tmem + sb * 128u;
+#pragma unroll
+                for (uint32_t k = 0; k < 8; ++k) {  // 16 dims per instruction
+                    const uint64_t off16 = (uint64_t)(((k >> 2) * kShBlock + (k & 3u) * 32u) >> 4);
+                    umma_bf16(d_s, a0 + off16, b0 + off16, kIdescS, k, issue);
+                }
+                // one commit tells the softmax warps that the scores are there and the K producer that its
+                // stage is free (the K ring and the score buffers are both indexed by tt % 3)
+                umma_commit(bar(kBarSFull + (int)sb), issue);
+                advance(qk);
+                return true;
+            };
+            // O += P V (O = P V for a unit's first tile)
+            auto issue_pv = [&](uint32_t tt) -> bool {
+                const uint32_t sb = tt % (uint32_t)kSBufs, spar = (tt / (uint32_t)kSBufs) & 1u;
+                const uint32_t vst = tt % (uint32_t)kVStages, vpar = (tt / (uint32_t)kVStages) & 1u;
+                if (!wait_all(kBarVFull + (int)vst, vpar)) return false;
+                if (!wait_all(kBarPReady + (int)sb, spar)) return false;
+                tc_fence_after();
+                const uint32_t v_lo = base + kOffV + vst * kShTileBytes;
+                // P: the A operand comes from tensor memory, where the softmax warps left it inside the
+                // score buffer: two bf16 per column, 16 tokens = 8 columns per step; tokens 0-63 in columns
+                // 0-31 (written by the first warpgroup over its own scores), tokens 64-127 in columns 64-95.
+                // V: tokens are rows of 128 bytes (8-token groups 1024 bytes apart, 16 tokens = 2048 bytes
+                // per step); the two 64-dim blocks of the tile are kShBlock bytes apart.
+                const uint64_t b0 = umma_desc(v_lo, kShBlock, 1024);
+                const uint32_t p_tm = tmem + sb * 128u;
+                const uint32_t d_o = tmem + kTmemO;
+                const bool first = pv.t == 0u;
+#pragma unroll
+                for (uint32_t k = 0; k < 8; ++k)  // 16 tokens per instruction
+                    umma_bf16_ts(d_o, p_tm + (k < 4u ? 8u * k : 64u + 8u * (k - 4u)), b0 + (uint64_t)(k * 128u), kIdescPV,
+                                 (first && k == 0u) ? 0u : 1u, issue);
+                umma_commit(bar(kBarVEmpty + (int)vst), issue);
+                umma_commit(bar(kBarSFree + (int)sb), issue);  // the accumulator holds the products up to this tile
+                advance(pv);
+                return true;
+            };
+            if (total > 0u) ok = issue_s(0u);
+            if (ok && total > 1u) ok = issue_s(1u);
+            for (uint32_t tt = 0; tt < total && ok; ++tt) {
+                // The score product two tiles on goes first, so that it is queued on the tensor pipe while the
+                // softmax of tile tt still runs -- unless it opens a unit whose query rows are not there yet:
+                // the softmax warps store them while they work on the unit before, which (for units of one
+                // tile) may need this tile's P V product first.
+                bool s_issued = tt + 2u >= total;
+                if (!s_issued) {
+                    const bool q_there = qk.t != 0u || __all_sync(0xffffffffu, mbar_try_wait(bar(kBarQReady + (int)(qk.unit_no & 1u)),
+                                                                                         (qk.unit_no >> 1) & 1u));
+                    if (q_there) {
+                        ok = issue_s(tt + 2u);
+                        s_issued = true;
+                    }
+                }
+                if (ok) ok = issue_pv(tt);
+                if (ok && !s_issued) ok = issue_s(tt + 2u);
             }
+            // products still in flight must finish before the tensor memory is given back
+            umma_commit(bar(kBarDrain), issue);
+            const uint64_t t0 = global_timer_ns();
+            while (!mbar_try_wait(bar(kBarDrain), 0) && global_timer_ns() - t0 < kWaitLimitNs) {}
             __syncwarp();
         }
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
         // ================= softmax / epilogue warps ====================================================
         const int G = p.group;
-        const int wg = (warp - 4) >> 2;       // softmax warpgroup 0 or 1: owns the tiles with (index & 1) == wg
+        const int wg = (warp - 4) >> 2;       // which 64 score columns (tokens) of every tile this thread owns
         const int sw = warp & 3;              // the tensor-memory lanes this warp may read: 32 sw .. 32 sw + 31
         const int row = 32 * sw + lane;       // query row of the M-tile = tensor-memory lane
         const int tid = row;                  // index among the 128 threads of the warpgroup
         const uint32_t lane_addr = tmem + ((uint32_t)(32 * sw) << 16);
-        const __nv_bfloat16 *q = reinterpret_cast<const __nv_bfloat16 *>(p.q);
-        const uint32_t swz = (uint32_t)(row & 7);
-        float *comb_ml = reinterpret_cast<float *>(smem + kOffComb); // [2][128 rows]
-        uint32_t tt0 = 0;
-        bool alive = true;
-        bool waited = false;  // for the kernels before this one on the stream
-        float o_acc[128];
+        const uint32_t col0 = 64u * (uint32_t)wg;
+        uint16_t *xchg_mx = reinterpret_cast<uint16_t *>(smem + kOffXchg);  // [tile parity][half][row]
+        float *xchg_l = reinterpret_cast<float *>(smem + kOffXchg);         // [half][row]
+        uint32_t tt = 0;      // tiles of the block so far
+        bool alive = true;    // false once the block has given up: work is skipped, barriers are still met
         // the warp's lanes must stay together (the tensor-memory loads are warp-wide): a wait fails for
         // all of them or for none
         auto warp_wait = [&](uint32_t b, uint32_t parity) -> bool {
             return __all_sync(0xffffffffu, mbar_wait(b, parity, abort_flag, p.status, kStatusTimeoutConsumer));
         };
-        const uint32_t s_addr = lane_addr + (uint32_t)wg * 128u;
-        const uint32_t o_addr = lane_addr + 256u + (uint32_t)wg * 128u;
+        const uint32_t o_addr = lane_addr + kTmemO + col0;
 
-        for (uint32_t ui = unit_begin; ui < unit_end && alive; ++ui) {
-            const cart_shared_unit u = p.units[ui];
-            const int i_reader = row / G, h = row - i_reader * G;
+        // Query rows.  Thread (w, r) copies the 64-dim half w of row r (head r % G of the M-tile's reader r / G)
+        // into the unit's query buffer, in the swizzled K-major operand layout: block w, row r, 16-byte chunk c
+        // at position c ^ (r % 8).  Rows past the unit's readers are zeros.  Unit number n of the block uses
+        // buffer n & 1.  The first unit's rows are fetched at once; the rows of unit n + 1 are requested after
+        // the first tile of unit n and stored a tile later, when the loads have landed (all products of unit
+        // n - 1, the buffer's last readers, were complete before the first scores of unit n arrived).
+        const int i_reader = row / G, h = row - i_reader * G;
+        const __nv_bfloat16 *q = reinterpret_cast<const __nv_bfloat16 *>(p.q);
+        uint4 qv[8];
+        auto load_q = [&](const cart_shared_unit &uu, uint32_t batch, bool on) {
+            const uint4 *src = reinterpret_cast<const uint4 *>(
+                q + ((size_t)batch * p.n_q_heads + (size_t)uu.kv_head * G + h) * kHeadDim) + 8 * wg;
+#pragma unroll
+            for (uint32_t c = 0; c < 8; ++c) qv[c] = on ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);  // all in flight
+        };
+        auto store_q = [&](uint32_t buf) {
+            const uint32_t qrow = base + kOffQ + buf * kShTileBytes + (uint32_t)wg * kShBlock + (uint32_t)row * 128u;
+            const uint32_t swz = (uint32_t)(row & 7);
+#pragma unroll
+            for (uint32_t c = 0; c < 8; ++c)
+                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(qrow + ((c ^ swz) << 4)), "r"(qv[c].x),
+                             "r"(qv[c].y), "r"(qv[c].z), "r"(qv[c].w)
+                             : "memory");
+            fence_async_smem();   // these writes before the tensor core's reads of the operand
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kBarQReady + (int)buf));
+        };
+        cart_shared_unit u{}, u_next{};
+        u = u_first;
+        if (unit_begin + 1u < unit_end) u_next = p.units[unit_begin + 1u];
+        {
+            // the first unit's queries: everything up to the rows themselves is part of the plan
+            const bool on = unit_begin < unit_end && (uint32_t)i_reader < u.n_readers;
+            const uint32_t batch = first_batch;
+            bool ok0 = true;
+            if (lane == 0) ok0 = wait_for_prior_kernels(p, abort_flag);
+            alive = __all_sync(0xffffffffu, ok0);  // (from here on the partial slots and the tickets are this kernel's too)
+            if (unit_begin < unit_end) {
+                load_q(u, batch, on && alive);
+                store_q(0u);
+            }
+        }
+
+        uint32_t unit_no = 0;
+        for (uint32_t ui = unit_begin; ui < unit_end; ++ui, ++unit_no) {
+            if (ui != unit_begin) {
+                u = u_next;
+                u_next = cart_shared_unit{};
+                if (ui + 1u < unit_end) u_next = p.units[ui + 1u];
+            }
+            const bool has_next = ui + 1u < unit_end;
             const bool valid = (uint32_t)i_reader < u.n_readers;
-            uint32_t entry = 0, batch = 0, slot = 0;
-            if (valid) {
-                entry = u.reader_begin + (uint32_t)i_reader;
-                batch = p.readers[entry];
-                slot = p.reader_slot[(size_t)entry * p.n_kv_heads + u.kv_head] + u.chunk;  // where this row's partial goes
-            }
-            // ---- this row's query into shared memory, in the swizzled K-major operand layout; each
-            //      warpgroup copies one 64-dim half -------------------------------------------------
-            if (!waited) {
-                bool ok0 = true;
-                if (lane == 0) ok0 = wait_for_prior_kernels(p, abort_flag);
-                alive = __all_sync(0xffffffffu, ok0);
-                waited = true;
-            }
-            {
-                const uint4 *src = reinterpret_cast<const uint4 *>(
-                    q + ((size_t)batch * p.n_q_heads + (size_t)u.kv_head * G + h) * kHeadDim) + 8 * wg;
-                const uint32_t qrow = base + kOffQ + (uint32_t)wg * kShBlock + (uint32_t)row * 128u;
-                uint4 v[8];
-#pragma unroll
-                for (uint32_t c = 0; c < 8; ++c) v[c] = valid ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);  // all in flight
-#pragma unroll
-                for (uint32_t c = 0; c < 8; ++c) {
-                    const uint32_t a = qrow + ((c ^ swz) << 4);
-                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(v[c].x), "r"(v[c].y), "r"(v[c].z),
-                                 "r"(v[c].w)
-                                 : "memory");
-                }
-                fence_async_smem();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(kBarQReady));
-            }
-            // m_run: the reference maximum that l_run and the warpgroup's accumulator in tensor memory refer to.
-            // It only moves when a row's maximum has outgrown it by more than kRescaleStep (base 2); until then
-            // probabilities may exceed 1 (by at most that factor), which bf16 and the fp32 sums hold easily.
+            const bool valid_next = has_next && (uint32_t)i_reader < u_next.n_readers;
+            uint32_t batch_next = 0;
+            if (valid_next) batch_next = p.readers[u_next.reader_begin + (uint32_t)i_reader];
+            const uint32_t t_store = u.n_tiles > 1u ? 1u : 0u;  // the tile after which the next unit's rows are stored
+            uint32_t slot = 0;
+            if (valid)  // where this row's partial goes (needed at the unit's end: the load has the tiles' time)
+                slot = p.reader_slot[(size_t)(u.reader_begin + (uint32_t)i_reader) * p.n_kv_heads + u.kv_head] + u.chunk;
+            // m_run: the reference that l_run and the accumulator in tensor memory refer to, the same for both
+            // owners of the row.  It only moves when the row's maximum has outgrown it by more than
+            // kRescaleStep (base 2); until then probabilities may exceed 1 (by at most that factor), which
+            // bf16 and the fp32 sums hold easily.  l_run: the sum over this thread's columns.
             float m_run = -INFINITY, l_run = 0.f;
 
-            // this warpgroup's tiles of the unit: those whose block-wide index is congruent to wg mod 2
-            bool have_prev = false;
-            uint32_t prev_tt = 0;
-            for (uint32_t t = ((uint32_t)wg ^ tt0) & 1u; t < u.n_tiles; t += 2) {
-                const uint32_t tt = tt0 + t;
-                const uint32_t par = (tt >> 1) & 1u;
-                alive = warp_wait(bar(kBarSFull + wg), par);
-                if (!alive) break;
-                tc_fence_after();
-                // pass 1: the row's maximum over the tile
+            for (uint32_t t = 0; t < u.n_tiles; ++t, ++tt) {
+                const uint32_t sb = tt % (uint32_t)kSBufs, spar = (tt / (uint32_t)kSBufs) & 1u;
+                const uint32_t s_addr = lane_addr + sb * 128u + col0;
+                uint32_t s[64];
                 float mx = -INFINITY;
+                if (alive) alive = warp_wait(bar(kBarSFull + (int)sb), spar);
+                if (alive) {
+                    tc_fence_after();
+                    tmem_ld32_issue(s_addr, reinterpret_cast<uint32_t(&)[32]>(s[0]));
+                    tmem_ld32_issue(s_addr + 32u, reinterpret_cast<uint32_t(&)[32]>(s[32]));
+                    tmem_ld_wait(reinterpret_cast<uint32_t(&)[32]>(s[0]));
+                    tmem_ld_wait(reinterpret_cast<uint32_t(&)[32]>(s[32]));
 #pragma unroll
-                for (int c2 = 0; c2 < 2; ++c2) {  // two loads of 32 columns in flight
-                    uint32_t a[32], b[32];
-                    tmem_ld32_issue(s_addr + (uint32_t)c2 * 64u, a);
-                    tmem_ld32_issue(s_addr + (uint32_t)c2 * 64u + 32u, b);
-                    tmem_ld_wait(a);
-                    tmem_ld_wait(b);
-#pragma unroll
-                    for (int k = 0; k < 32; ++k) mx = fmaxf(mx, fmaxf(__uint_as_float(a[k]), __uint_as_float(b[k])));
+                    for (int k = 0; k < 64; k += 2) mx = fmaxf(mx, fmaxf(__uint_as_float(s[k]), __uint_as_float(s[k + 1])));
+                    mx *= p.scale_log2;
                 }
-                mx *= p.scale_log2;
-                if (!have_prev) {
-                    m_run = mx;
-                } else if (__any_sync(0xffffffffu, mx > m_run + kRescaleStep)) {
-                    // a row of this warp has outgrown its reference: every row moves up to its maximum and the
-                    // warp rescales its lanes of the accumulator (tensor-memory accesses are warp-wide, so the
-                    // warp decides together; the other rows' factors are 1 or close to it)
-                    const float m_new = fmaxf(m_run, mx);
+                // the row's maximum over the whole tile: the two owners trade their halves' maxima (rounded up to
+                // bf16, the same numbers on both sides, so both keep the same reference)
+                const uint32_t mine = bf16_ceil_bits(mx);
+                xchg_mx[((tt & 1u) * 2u + (uint32_t)wg) * 128u + (uint32_t)row] = (uint16_t)mine;
+                softmax_bar_both();
+                const uint32_t theirs = xchg_mx[((tt & 1u) * 2u + (uint32_t)(wg ^ 1)) * 128u + (uint32_t)row];
+                if (!alive) continue;
+                const float m_tile = fmaxf(__uint_as_float(mine << 16), __uint_as_float(theirs << 16));
+                if (t == 0) {
+                    m_run = m_tile;
+                } else if (__any_sync(0xffffffffu, m_tile > m_run + kRescaleStep)) {
+                    // a row of this warp has outgrown its reference: every row of the warp moves up to its
+                    // maximum and the two owners rescale their halves of the accumulator's lanes (tensor-memory
+                    // accesses are warp-wide, so the warp decides together, and its twin in the other warpgroup
+                    // sees the same numbers and decides the same; the other rows' factors are 1 or close to it)
+                    const float m_new = fmaxf(m_run, m_tile);
                     const float f = fast_exp2(m_run - m_new);
                     m_run = m_new;
                     l_run *= f;
-                    // the product of this warpgroup's previous tile must have landed first
-                    alive = warp_wait(bar(kBarOFull + wg), (prev_tt >> 1) & 1u);
-                    if (!alive) break;
+                    // The product of the tile before must have landed first.  Its completion is read from the
+                    // barrier of the score buffer it used: a barrier that completes once per tile could be two
+                    // phases behind this warp (the tensor pipe also holds score products queued ahead), which a
+                    // parity cannot tell from none; a score buffer's barrier is at most one behind.
+                    alive = warp_wait(bar(kBarSFree + (int)((tt - 1u) % (uint32_t)kSBufs)), ((tt - 1u) / (uint32_t)kSBufs) & 1u);
+                    if (!alive) continue;
                     tc_fence_after();
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
+                    for (int c = 0; c < 2; ++c) {
                         uint32_t o[32];
                         tmem_ld32_issue(o_addr + (uint32_t)c * 32u, o);
                         tmem_ld_wait(o);
@@ -498,142 +592,72 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                     }
                     // (these stores are waited for with those of P below, before the MMA warp hears of the tile)
                 }
-                const float m_new = m_run;
-                // pass 2: probabilities, as bf16 pairs, back into tensor memory over the first half of the
-                // scores they came from (32 scores are read, then 16 columns behind the read position are
-                // written): the A operand of the second product
-                float psum = 0.f;
-                {
-                    uint32_t buf[2][32];  // the load of the next 32 scores runs under the arithmetic on these
-                    tmem_ld32_issue(s_addr, buf[0]);
-                    tmem_ld_wait(buf[0]);
+                // probabilities of this thread's 64 tokens, as bf16 pairs (the even token in the low half), written
+                // over the first 32 columns of the scores they came from: the A operand of the second product
+                float psum0 = 0.f, psum1 = 0.f;
 #pragma unroll
-                    for (int c4 = 0; c4 < 4; ++c4) {
-                        uint32_t(&v)[32] = buf[c4 & 1];
-                        if (c4 < 3) tmem_ld32_issue(s_addr + (uint32_t)(c4 + 1) * 32u, buf[(c4 + 1) & 1]);
-                        uint32_t w[16];
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t w[16];
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            const float p0 = fast_exp2(fmaf(__uint_as_float(v[2 * j]), p.scale_log2, -m_new));
-                            const float p1 = fast_exp2(fmaf(__uint_as_float(v[2 * j + 1]), p.scale_log2, -m_new));
-                            psum += p0 + p1;
-                            w[j] = pack_bf16(p0, p1);  // the even token in the low half
-                        }
-                        tmem_st16(s_addr + (uint32_t)c4 * 16u, w);
-                        if (c4 < 3) tmem_ld_wait(buf[(c4 + 1) & 1]);
+                    for (int j = 0; j < 16; ++j) {
+                        const float p0 = fast_exp2(fmaf(__uint_as_float(s[32 * c + 2 * j]), p.scale_log2, -m_run));
+                        const float p1 = fast_exp2(fmaf(__uint_as_float(s[32 * c + 2 * j + 1]), p.scale_log2, -m_run));
+                        psum0 += p0;
+                        psum1 += p1;
+                        w[j] = pack_bf16(p0, p1);
                     }
+                    tmem_st16(s_addr + (uint32_t)c * 16u, w);
                 }
-                l_run += psum;
+                l_run += psum0 + psum1;
                 tmem_st_wait();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(kBarPReady + wg));
-                prev_tt = tt;
-                have_prev = true;
-            }
-            // the warpgroup's share of the unit's output, out of tensor memory
-            if (alive && have_prev) {
-                alive = warp_wait(bar(kBarOFull + wg), (prev_tt >> 1) & 1u);
-                if (alive) {
-                    tc_fence_after();
-#pragma unroll
-                    for (int c2 = 0; c2 < 2; ++c2) {  // two loads of 32 columns in flight
-                        uint32_t a[32], b[32];
-                        tmem_ld32_issue(o_addr + (uint32_t)c2 * 64u, a);
-                        tmem_ld32_issue(o_addr + (uint32_t)c2 * 64u + 32u, b);
-                        tmem_ld_wait(a);
-                        tmem_ld_wait(b);
-#pragma unroll
-                        for (int k = 0; k < 32; ++k) {
-                            o_acc[c2 * 64 + k] = __uint_as_float(a[k]);
-                            o_acc[c2 * 64 + 32 + k] = __uint_as_float(b[k]);
-                        }
-                    }
-                    tc_fence_before();
+                if (lane == 0) mbar_arrive(bar(kBarPReady + (int)sb));
+                if (has_next) {
+                    if (t == 0u) load_q(u_next, batch_next, valid_next);
+                    if (t == t_store) store_q((unit_no + 1u) & 1u);
                 }
-            } else {
-#pragma unroll
-                for (int d = 0; d < 128; ++d) o_acc[d] = 0.f;
             }
-            tt0 += u.n_tiles;
 
-            // ---- combine the two warpgroups' states of each row and write the partials ------------------
-            // All products of the unit are complete once both warpgroups have taken their last O, so the P
-            // buffers can serve as scratch: row r lives at r * 512 bytes, its 16-byte quad q at position
-            // q ^ (r & 31), which keeps both the row-per-lane and the quad-per-lane accesses free of bank
-            // conflicts.
-            softmax_bar_both();
-            uint8_t *comb = smem + kOffQ;   // the query buffer and the block behind it: 64 KB
-            const uint32_t rsw = (uint32_t)(row & 31);
-            if (wg == 1) {
-#pragma unroll
-                for (uint32_t q4 = 0; q4 < 32; ++q4)
-                    *reinterpret_cast<float4 *>(comb + (size_t)row * 512 + ((q4 ^ rsw) << 4)) =
-                        make_float4(o_acc[4 * q4], o_acc[4 * q4 + 1], o_acc[4 * q4 + 2], o_acc[4 * q4 + 3]);
-                comb_ml[row] = m_run;
-                comb_ml[128 + row] = l_run;
+            // ---- the unit's rows leave as normalised partials -------------------------------------------
+            // Each thread reads its 64 columns of the accumulator once the last product has landed; the two
+            // owners of a row add their sums (in a fixed order, so the result does not depend on timing).
+            uint32_t o[64];
+            if (alive) alive = warp_wait(bar(kBarSFree + (int)((tt - 1u) % (uint32_t)kSBufs)), ((tt - 1u) / (uint32_t)kSBufs) & 1u);
+            if (alive) {
+                tc_fence_after();
+                tmem_ld32_issue(o_addr, reinterpret_cast<uint32_t(&)[32]>(o[0]));
+                tmem_ld32_issue(o_addr + 32u, reinterpret_cast<uint32_t(&)[32]>(o[32]));
+                tmem_ld_wait(reinterpret_cast<uint32_t(&)[32]>(o[0]));
+                tmem_ld_wait(reinterpret_cast<uint32_t(&)[32]>(o[32]));
+                tc_fence_before();
             }
+            softmax_bar_both();  // nobody reads the maxima of the last tile any more: the sums go over them
+            xchg_l[wg * 128 + row] = l_run;
             softmax_bar_both();
-            if (wg == 0) {
-                const float m1 = comb_ml[row], l1 = comb_ml[128 + row];
-                const float M = fmaxf(m_run, m1);   // finite: the unit has at least one tile
-                const float w0 = fast_exp2(m_run - M), w1 = fast_exp2(m1 - M);
-                const float l = l_run * w0 + l1 * w1;
+            if (alive && valid) {
+                const float l = xchg_l[row] + xchg_l[128 + row];
                 const float inv = 1.f / l;
-                const float c0 = w0 * inv, c1 = w1 * inv;
+                float4 *dst = reinterpret_cast<float4 *>(p.part_o + ((size_t)slot * G + h) * kHeadDim + col0);
 #pragma unroll
-                for (uint32_t q0 = 0; q0 < 32; q0 += 8) {  // eight loads in flight, then eight stores
-                    float4 v[8];
-#pragma unroll
-                    for (uint32_t j = 0; j < 8; ++j)
-                        v[j] = *reinterpret_cast<const float4 *>(comb + (size_t)row * 512 + (((q0 + j) ^ rsw) << 4));
-#pragma unroll
-                    for (uint32_t j = 0; j < 8; ++j) {
-                        const uint32_t q4 = q0 + j;
-                        *reinterpret_cast<float4 *>(comb + (size_t)row * 512 + ((q4 ^ rsw) << 4)) =
-                            make_float4(o_acc[4 * q4] * c0 + v[j].x * c1, o_acc[4 * q4 + 1] * c0 + v[j].y * c1,
-                                        o_acc[4 * q4 + 2] * c0 + v[j].z * c1, o_acc[4 * q4 + 3] * c0 + v[j].w * c1);
-                    }
-                }
-                uint32_t dst_row = 0xFFFFFFFFu;  // row of part_o ([slot][G] flattened) this query row goes to
-                if (alive && valid) {
-                    dst_row = slot * (uint32_t)G + (uint32_t)h;
-                    p.part_lse2[(size_t)slot * kMaxGroup + h] = M + log2f(l);
-                }
-                flags[row] = dst_row;
+                for (int q4 = 0; q4 < 16; ++q4)
+                    dst[q4] = make_float4(__uint_as_float(o[4 * q4]) * inv, __uint_as_float(o[4 * q4 + 1]) * inv,
+                                          __uint_as_float(o[4 * q4 + 2]) * inv, __uint_as_float(o[4 * q4 + 3]) * inv);
+                if (wg == 0) p.part_lse2[(size_t)slot * kMaxGroup + h] = m_run + log2f(l);
             }
-            softmax_bar_both();
-            // both warpgroups copy the normalised rows out, a warp writing one 512-byte row per instruction
-            {
-                const uint32_t *dst_rows = reinterpret_cast<const uint32_t *>(smem + kOffFlags);
-                const uint32_t q4 = (uint32_t)lane;                       // a warp = one row per pass
-                const uint32_t r0 = (uint32_t)(wg * 4 + (warp & 3));      // 8 softmax warps, 16 rows each
-#pragma unroll
-                for (uint32_t rb = 0; rb < 16; rb += 8) {  // eight rows' loads in flight, then their stores
-                    uint32_t dst[8];
-                    float4 v[8];
-#pragma unroll
-                    for (uint32_t j = 0; j < 8; ++j) {
-                        const uint32_t r = r0 + 8u * (rb + j);
-                        dst[j] = dst_rows[r];
-                        v[j] = *reinterpret_cast<const float4 *>(comb + (size_t)r * 512 + ((q4 ^ (r & 31u)) << 4));
-                    }
-#pragma unroll
-                    for (uint32_t j = 0; j < 8; ++j)
-                        if (dst[j] != 0xFFFFFFFFu)
-                            reinterpret_cast<float4 *>(p.part_o + (size_t)dst[j] * kHeadDim)[q4] = v[j];
-                }
+            if (p.tickets == nullptr) {
+                softmax_bar_both();  // the sums have been read: the next unit's maxima may be written
+                continue;
             }
-            if (p.tickets) __threadfence();  // publish the partials before the tickets
-            softmax_bar_both();
 
             // ---- arrival tickets (when no merge kernel follows) -------------------------------------------
+            __threadfence();  // publish the partials before the tickets
+            softmax_bar_both();
             if (wg == 0) {
-                // one thread decides for all whether the block is still in business, so that all softmax
-                // threads leave the unit loop together
+                // one thread decides for all whether the block is still in business
                 if (tid == 0) *unit_ok = (*abort_flag == 0u) ? 1u : 0u;
-                if (p.tickets && tid < 128 / G) {
-                    uint32_t mine = 0;
+                if (tid < 128 / G) {
+                    uint32_t won = 0;
                     if (*abort_flag == 0u && (uint32_t)tid < u.n_readers) {
                         // thread tid speaks for reader tid (rows tid * G .. tid * G + G - 1): the block that
                         // delivers the last partial of the reader's row group merges it
@@ -641,12 +665,12 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                         const uint32_t mg = p.reader_merge[(size_t)e2 * p.n_kv_heads + u.kv_head];
                         const cart_merge_item mi = p.merges[mg];
                         const uint32_t seen = atomicAdd(&p.tickets[mg], 1u);
-                        if (seen + 1u == mi.slot_end - mi.slot_begin) mine = mg + 1u;
+                        if (seen + 1u == mi.slot_end - mi.slot_begin) won = mg + 1u;
                     }
-                    flags[tid] = mine;
+                    flags[tid] = won;
                 }
                 softmax_bar();
-                for (uint32_t r = 0; p.tickets && *unit_ok != 0u && r < u.n_readers; ++r) {
+                for (uint32_t r = 0; *unit_ok != 0u && r < u.n_readers; ++r) {
                     const uint32_t f = flags[r];
                     if (f == 0) continue;
                     __threadfence();
@@ -654,8 +678,7 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                     if (tid == 0) p.tickets[f - 1u] = 0;  // ready for the next launch
                 }
             }
-            softmax_bar_both();  // scratch, flags and unit_ok may be rewritten by the next unit from here on
-            alive = *unit_ok != 0u;
+            softmax_bar_both();  // flags, unit_ok and the exchange area may be rewritten by the next unit from here on
         }
     }
 
