@@ -321,7 +321,8 @@ def run_ours(args):
     total_steps = args.warmup + args.steps + (0 if args.no_e2e else args.warmup + args.e2e_steps) + 2
     sample_layers = list(range(min(args.cpu_layers, L))) if (rank == 0 and world == 1 and not args.no_cpu) else []
     stream = torch.cuda.current_stream(dev)
-    lw = runner.LoadedWorkload(w, dev, extra_capacity=total_steps, keep_layers=sample_layers, stream=stream)
+    lw = runner.LoadedWorkload(w, dev, extra_capacity=total_steps, keep_layers=sample_layers, stream=stream,
+                               paged=args.paged)
     ctx = lw.ctx
     if args.piece_cost >= 0:
         binding.cart_set_piece_cost(ctx, args.piece_cost)
@@ -462,6 +463,8 @@ def run_ours(args):
     if rank != 0:
         return
     cfg = workload_config(w)
+    if args.paged:
+        cfg["suffix_storage"] = "pages of 64 tokens, taken as the suffixes grow"
     cfg.update({"mean_kv_tokens": round(float(kv_tokens.mean()), 1),
                 "step": ("per layer: cart_append_kv, then cart_decode_attention" if args.unfused else
                          "per layer: cart_decode_step (append 1 KV token per request and attend, one call)"),
@@ -634,6 +637,8 @@ def main():
     ap.add_argument("--prefill", type=int, default=0,
                     help="side measurement: prefill attention of a message of this many tokens over one Cartridge "
                          "of the workload's shape (prints its own JSON line)")
+    ap.add_argument("--paged", action="store_true",
+                    help="the requests' suffixes are stored in pages of 64 tokens (cart_request_open_paged)")
     ap.add_argument("--unfused", action="store_true",
                     help="append and attend with two calls per layer instead of cart_decode_step")
     ap.add_argument("--piece-cost", type=int, default=-1,

@@ -62,7 +62,8 @@ typedef enum {
     CART_ERR_EMPTY = 6,       /* a request has no KV token at all in the layer asked for */
     CART_ERR_IN_USE = 7,      /* releasing a Cartridge that an open request or composition uses */
     CART_ERR_CUDA = 8,        /* a CUDA runtime / driver call failed (see cart_last_error) */
-    CART_ERR_TIMEOUT = 9      /* a bounded device-side wait ran out (reported by cart_sync_status) */
+    CART_ERR_TIMEOUT = 9,     /* a bounded device-side wait ran out (reported by cart_sync_status) */
+    CART_ERR_EVICTED = 10     /* the request, or a Cartridge it attends to, is swapped out of the arena */
 } cart_status;
 
 typedef struct {
@@ -97,6 +98,9 @@ CART_API cart_status cart_destroy(cart_ctx *ctx);
  * memory makes the copy asynchronous); they are copied into the arena on `stream` (the caller may free
  * or reuse them once the stream has passed this point).  p >= 1, the same in every layer.  A Cartridge
  * is stored once however many requests open on it; cart_release_cartridge gives its space back.
+ * The Cartridge is always copied: every tile of the arena is fetched through one tensor map, and a block left in
+ * the caller's memory would need a map of its own in every kernel, so borrowing a caller's buffer is not offered (a
+ * cache too large to hold twice is registered from host memory, or in parts that are then composed).
  * Errors: INVALID_ARG, CAPACITY (table full), OOM, CUDA. */
 CART_API cart_status cart_register_cartridge(cart_ctx *ctx, const void *k /*device or host*/, const void *v /*device or host*/,
                                     int32_t p, void *stream /*cudaStream_t*/, cart_id *out /*host*/);
@@ -121,6 +125,20 @@ CART_API cart_status cart_release_cartridge(cart_ctx *ctx, cart_id id);
 CART_API cart_status cart_request_open(cart_ctx *ctx, cart_id cartridge, int32_t suffix_capacity,
                               cart_req *out /*host*/);
 
+/* The same with the suffix stored in pages (Sec. 3.3: a Cartridge is served by the mechanisms that handle cached
+ * prefixes and per-user KV caches; paging is how such caches grow without being moved).  A page holds CART_PAGE_TOKENS
+ * tokens of the request for every layer and KV head -- per (layer, KV head) the K rows, then the V rows -- and may lie
+ * anywhere in the arena; the attention kernels find a tile through the request's page list.  initial_capacity tokens
+ * (rounded up to whole pages, may be 0) are reserved now; cart_append_kv, cart_extend_kv and cart_decode_step take
+ * further pages from the arena as the suffix grows (CART_ERR_OOM when none is left; nothing is appended then), and
+ * cart_request_reserve takes pages instead of copying.  Pages return to the arena with cart_request_close or
+ * cart_evict_request.  Everything else is as for cart_request_open; results are bitwise those of a request with a
+ * contiguous suffix.  One attention call may name at most 256 * max_requests + 8192 pages over its whole batch
+ * (CART_ERR_CAPACITY beyond).  Errors: BAD_HANDLE, CAPACITY (table full), OOM. */
+#define CART_PAGE_TOKENS 64
+CART_API cart_status cart_request_open_paged(cart_ctx *ctx, cart_id cartridge, int32_t initial_capacity,
+                                             cart_req *out /*host*/);
+
 /* Grows the suffix buffer of an open request to at least suffix_capacity tokens per layer (rounded up
  * to a multiple of 64), for conversations that outlive the capacity they were opened with (Sec. 3.3:
  * per-user KV caches of any length next to the shared prefix).  A new buffer is taken from the arena,
@@ -130,6 +148,33 @@ CART_API cart_status cart_request_open(cart_ctx *ctx, cart_id cartridge, int32_t
  * changes nothing.  The arena must have room for the new buffer while the old one is still held.
  * Errors: BAD_HANDLE, INVALID_ARG, OOM (nothing has changed), CUDA. */
 CART_API cart_status cart_request_reserve(cart_ctx *ctx, cart_req req, int32_t suffix_capacity, void *stream);
+
+/* Eviction (Sec. 3.3: many users' caches share one GPU; a scheduler keeps the active ones resident).
+ *
+ * cart_evict_request swaps a paused request's suffix out: the tokens stored so far are copied on `stream` to k_out /
+ * v_out (host memory -- page-locked makes the copy asynchronous -- or device memory outside the arena), each laid out
+ * bf16 [n_layers][n_kv_heads][n][128] with n = *n_tokens_out = the longest layer's length, and the request's pages or
+ * buffer return to the arena at once (later calls on the same stream may reuse them; the caller orders other
+ * streams).  The handle stays open and keeps its lengths; until it is restored, every call that would read or write
+ * its suffix returns CART_ERR_EVICTED.  With n = 0 nothing is copied and k_out / v_out may be NULL.
+ * cart_restore_request takes storage for n tokens again (pages for a paged request, else a buffer of the old
+ * capacity) and copies k_in / v_in back (same layout and n as evict returned).
+ * Errors: BAD_HANDLE, INVALID_ARG, EVICTED (evict: already out; restore: not out), OOM (restore; nothing changed), CUDA. */
+CART_API cart_status cart_evict_request(cart_ctx *ctx, cart_req req, void *k_out /*host or device*/,
+                                        void *v_out /*host or device*/, int32_t *n_tokens_out /*host*/, void *stream);
+CART_API cart_status cart_restore_request(cart_ctx *ctx, cart_req req, const void *k_in /*host or device*/,
+                                          const void *v_in /*host or device*/, void *stream);
+
+/* cart_evict_cartridge returns a registered Cartridge's arena space while its handle, the compositions that contain
+ * it and the requests opened on it stay valid.  A Cartridge is never written after registration, so nothing is copied
+ * out: the caller restores it from wherever it keeps trained Cartridges.  Refused with CART_ERR_IN_USE while a request
+ * that is not itself evicted attends to it (directly or through a composition): evict those requests first.  While
+ * it is out, decode and prefill calls on requests that attend to it return CART_ERR_EVICTED.
+ * cart_restore_cartridge takes space again and copies k / v in (as cart_register_cartridge; same p).
+ * Errors: BAD_HANDLE (also: a composition), IN_USE, EVICTED (as above), OOM, INVALID_ARG, CUDA. */
+CART_API cart_status cart_evict_cartridge(cart_ctx *ctx, cart_id id);
+CART_API cart_status cart_restore_cartridge(cart_ctx *ctx, cart_id id, const void *k /*device or host*/,
+                                            const void *v /*device or host*/, void *stream);
 
 /* Closes a request and returns its suffix buffer to the arena.  Errors: BAD_HANDLE. */
 CART_API cart_status cart_request_close(cart_ctx *ctx, cart_req req);

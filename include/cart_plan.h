@@ -37,6 +37,11 @@ typedef struct {
 
 #define CART_SEG_SUFFIX 1u  /* the segment lies in a request's suffix buffer, which kernels write (append, extend,
                                fused decode step); a stored Cartridge is only ever written by copies */
+#define CART_SEG_PAGED 2u   /* the segment is stored in pages of tile_tokens tokens (a paged suffix): k_row is the index
+                               of the page that holds the segment's first token in the batch's page list (a device
+                               array of page base rows), v_row is unused, head_stride = rows between consecutive KV
+                               heads inside a page (2 * tile_tokens: the head's K rows, then its V rows), layer_stride =
+                               rows between consecutive layers inside a page.  The segment starts on a page boundary. */
 
 #define CART_ITEM_BEGIN 1u  /* first item of a row-group piece in this block: load q, reset state */
 #define CART_ITEM_END 2u    /* last item of the piece: combine the warps' states and write */
@@ -46,6 +51,9 @@ typedef struct {
 #define CART_ITEM_SUFFIX 16u /* the item's tiles lie in suffix storage (CART_SEG_SUFFIX): a kernel earlier on the
                                stream may have written them, so they are fetched only once those kernels are
                                known to be complete; Cartridge tiles may be fetched ahead of that */
+#define CART_ITEM_PAGED 32u  /* the item's tiles are pages (CART_SEG_PAGED): k_row is the index of the first tile's
+                               entry in the page list, v_row the row of the KV head's K block inside a page (its V
+                               block follows tile_tokens rows later); tile j of the item lies in page k_row + j */
 
 /* A run of consecutive tiles of one segment of one row group, processed by one block. */
 typedef struct {
@@ -120,6 +128,10 @@ typedef struct {
 } cart_shared_unit;
 
 #define CART_UNIT_SUFFIX 1u
+#define CART_UNIT_PAGED 2u    /* the run lies in pages: k_row = index of its first page in the page list (a shared
+                                 tile of share_tile_tokens tokens spans share_tile_tokens / tile_tokens consecutive
+                                 entries), v_row = row of the KV head's K block inside a page, layer_stride as in
+                                 CART_SEG_PAGED */
 
 /* Capacities (in) and results (out) of cart_plan_build_shared; all arrays are host memory. */
 typedef struct {

@@ -20,9 +20,10 @@ CART_NONE = -1
 CART_OK = 0
 STATUS_NAMES = ["CART_OK", "CART_ERR_INVALID_ARG", "CART_ERR_SHAPE", "CART_ERR_BAD_HANDLE",
                 "CART_ERR_CAPACITY", "CART_ERR_OOM", "CART_ERR_EMPTY", "CART_ERR_IN_USE",
-                "CART_ERR_CUDA", "CART_ERR_TIMEOUT"]
+                "CART_ERR_CUDA", "CART_ERR_TIMEOUT", "CART_ERR_EVICTED"]
 (CART_ERR_INVALID_ARG, CART_ERR_SHAPE, CART_ERR_BAD_HANDLE, CART_ERR_CAPACITY, CART_ERR_OOM,
- CART_ERR_EMPTY, CART_ERR_IN_USE, CART_ERR_CUDA, CART_ERR_TIMEOUT) = range(1, 10)
+ CART_ERR_EMPTY, CART_ERR_IN_USE, CART_ERR_CUDA, CART_ERR_TIMEOUT, CART_ERR_EVICTED) = range(1, 11)
+CART_PAGE_TOKENS = 64
 
 # every symbol include/cart.h and include/cart_plan.h declare
 EXPORTS = ["cart_scratch_bytes", "cart_create", "cart_destroy", "cart_register_cartridge",
@@ -31,6 +32,8 @@ EXPORTS = ["cart_scratch_bytes", "cart_create", "cart_destroy", "cart_register_c
            "cart_kv_bytes", "cart_sync_status", "cart_set_timing", "cart_get_timing",
            "cart_set_share_min_readers", "cart_set_piece_cost", "cart_plan_build_shared",
            "cart_set_plan_reuse", "cart_plan_count", "cart_plan_reusable", "cart_set_side_by_side",
+           "cart_request_open_paged", "cart_evict_request", "cart_restore_request", "cart_evict_cartridge",
+           "cart_restore_cartridge",
            "cart_decode_attention_static", "cart_launch_count", "cart_status_string",
            "cart_last_error", "cart_plan_build"]
 
@@ -87,8 +90,9 @@ class cart_plan_out(ctypes.Structure):
                 ("side_by_side", ctypes.c_int32), ("n_shared_ctas", ctypes.c_int32)]
 
 
-CART_ITEM_BEGIN, CART_ITEM_END, CART_ITEM_DIRECT, CART_ITEM_TAIL, CART_ITEM_SUFFIX = 1, 2, 4, 8, 16
-CART_SEG_SUFFIX = 1
+CART_ITEM_BEGIN, CART_ITEM_END, CART_ITEM_DIRECT, CART_ITEM_TAIL, CART_ITEM_SUFFIX, CART_ITEM_PAGED = 1, 2, 4, 8, 16, 32
+CART_SEG_SUFFIX, CART_SEG_PAGED = 1, 2
+CART_UNIT_SUFFIX, CART_UNIT_PAGED = 1, 2
 CART_UNIT_SUFFIX = 1
 
 
@@ -122,6 +126,11 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.cart_release_cartridge.argtypes = [vp, i32]
     lib.cart_request_open.argtypes = [vp, i32, i32, i32p]
     lib.cart_request_close.argtypes = [vp, i32]
+    lib.cart_request_open_paged.argtypes = [vp, i32, i32, i32p]
+    lib.cart_evict_request.argtypes = [vp, i32, vp, vp, i32p, vp]
+    lib.cart_restore_request.argtypes = [vp, i32, vp, vp, vp]
+    lib.cart_evict_cartridge.argtypes = [vp, i32]
+    lib.cart_restore_cartridge.argtypes = [vp, i32, vp, vp, vp]
     lib.cart_request_reserve.argtypes = [vp, i32, i32, vp]
     lib.cart_append_kv.argtypes = [vp, i32, i32p, i32, vp, vp, vp]
     lib.cart_extend_kv.argtypes = [vp, i32, i32, vp, vp, i32, vp]
@@ -237,6 +246,35 @@ def cart_request_open(ctx: int, cartridge: int, suffix_capacity: int) -> int:
     _check(load_library().cart_request_open(ctx, int(cartridge), int(suffix_capacity), ctypes.byref(out)),
            "cart_request_open", ctx)
     return int(out.value)
+
+
+def cart_request_open_paged(ctx: int, cartridge: int, initial_capacity: int = 0) -> int:
+    out = ctypes.c_int32(-1)
+    _check(load_library().cart_request_open_paged(ctx, int(cartridge), int(initial_capacity), ctypes.byref(out)),
+           "cart_request_open_paged", ctx)
+    return int(out.value)
+
+
+def cart_evict_request(ctx: int, req: int, k_out, v_out, stream=None) -> int:
+    """Returns n, the number of tokens per (layer, KV head) written to k_out / v_out."""
+    n = ctypes.c_int32(0)
+    _check(load_library().cart_evict_request(ctx, int(req), _ptr(k_out), _ptr(v_out), ctypes.byref(n), _stream(stream)),
+           "cart_evict_request", ctx)
+    return int(n.value)
+
+
+def cart_restore_request(ctx: int, req: int, k_in, v_in, stream=None) -> None:
+    _check(load_library().cart_restore_request(ctx, int(req), _ptr(k_in), _ptr(v_in), _stream(stream)),
+           "cart_restore_request", ctx)
+
+
+def cart_evict_cartridge(ctx: int, cid: int) -> None:
+    _check(load_library().cart_evict_cartridge(ctx, int(cid)), "cart_evict_cartridge", ctx)
+
+
+def cart_restore_cartridge(ctx: int, cid: int, k, v, stream=None) -> None:
+    _check(load_library().cart_restore_cartridge(ctx, int(cid), _ptr(k), _ptr(v), _stream(stream)),
+           "cart_restore_cartridge", ctx)
 
 
 def cart_request_reserve(ctx: int, req: int, suffix_capacity: int, stream=None) -> None:

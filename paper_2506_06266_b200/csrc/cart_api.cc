@@ -38,8 +38,9 @@ struct ScratchLayout {
     uint64_t status_off, tickets_off, plan_off, plan_slot_bytes, cta_begin_off, merges_off, items_off;
     // shared-segment part of a plan slot
     uint64_t shared_off, unit_cta_begin_off, readers_off, reader_slot_off, reader_merge_off, units_off;
+    uint64_t pages_off;  // page list of the batch's paged suffixes (base row per page)
     uint64_t part_o_off, part_lse_off, total;
-    int items_cap, slots_cap, merges_cap, units_cap, readers_cap;
+    int items_cap, slots_cap, merges_cap, units_cap, readers_cap, pages_cap;
 };
 
 ScratchLayout scratch_layout(const cart_config &c)
@@ -71,7 +72,11 @@ ScratchLayout scratch_layout(const cart_config &c)
     s.reader_slot_off = s.readers_off + round_up((uint64_t)s.readers_cap * 4, kAlign);
     s.reader_merge_off = s.reader_slot_off + round_up((uint64_t)s.readers_cap * c.n_kv_heads * 4, kAlign);
     s.units_off = s.reader_merge_off + round_up((uint64_t)s.readers_cap * c.n_kv_heads * 4, kAlign);
-    s.plan_slot_bytes = s.units_off + round_up((uint64_t)s.units_cap * sizeof(cart_shared_unit), kAlign);
+    s.pages_off = s.units_off + round_up((uint64_t)s.units_cap * sizeof(cart_shared_unit), kAlign);
+    // (a function of the table sizes alone, like the rest of the layout: 16 k tokens of paged suffix per request
+    //  on average, and room for a few very long ones)
+    s.pages_cap = 256 * c.max_requests + 8192;
+    s.plan_slot_bytes = s.pages_off + round_up((uint64_t)s.pages_cap * 4, kAlign);
     s.part_o_off = s.plan_off + (uint64_t)kPlanSlots * s.plan_slot_bytes;
     s.part_lse_off = s.part_o_off + round_up((uint64_t)s.slots_cap * group * kHeadDim * 4, kAlign);
     s.total = s.part_lse_off + round_up((uint64_t)s.slots_cap * kMaxGroup * 4, kAlign);
@@ -100,6 +105,7 @@ struct Cartridge {
     uint64_t alloc_start = 0, alloc_rows = 0;
     std::vector<int32_t> parts;    // composed: registered ids, flattened, in order
     int32_t refs = 0;              // open requests + compositions that hold it
+    bool evicted = false;          // registered only: the arena space has been given back
 };
 
 struct Request {
@@ -110,6 +116,11 @@ struct Request {
     uint64_t alloc_start = 0, alloc_rows = 0;
     std::vector<int32_t> len;  // per layer
     uint64_t stamp = 0;
+    bool paged = false;            // the suffix lives in pages (base rows in `pages`); k_row / v_row / alloc_* unused
+    std::vector<uint32_t> pages;
+    bool evicted = false;          // the suffix is swapped out: no storage, lengths kept
+    uint64_t list_stamp = 0;       // plan building: the request's pages are in the page list at list_base
+    uint32_t list_base = 0;
 };
 
 struct PlanSlot {
@@ -152,6 +163,7 @@ struct cart_ctx {
     int cur_slot = -1;
     uint64_t epoch = 1;
     uint64_t stamp = 0;
+    uint64_t list_stamp = 0;
     uint64_t launches = 0;
     std::vector<cart_plan_seg> seg_tmp;
     std::vector<int32_t> head_tmp;
@@ -232,6 +244,62 @@ Request *get_req(cart_ctx *ctx, cart_req r)
 
 uint8_t *arena_ptr(cart_ctx *ctx, uint64_t row) { return static_cast<uint8_t *>(ctx->cfg.arena) + row * kRowBytes; }
 
+// A page holds kTileTokens tokens of a request for every layer and KV head: [layer][KV head][K rows, V rows].
+uint64_t page_rows(const cart_ctx *ctx) { return (uint64_t)ctx->cfg.n_layers * ctx->cfg.n_kv_heads * 2 * kTileTokens; }
+// Row of token `pos` of (layer, KV head 0) in a paged suffix: K rows; the V rows are kTileTokens further on, the
+// next KV head 2 * kTileTokens.
+uint64_t paged_row(const cart_ctx *ctx, const Request &r, int32_t layer, int32_t pos)
+{
+    return (uint64_t)r.pages[(size_t)(pos / kTileTokens)] + (uint64_t)layer * ctx->cfg.n_kv_heads * 2 * kTileTokens +
+           (uint64_t)(pos % kTileTokens);
+}
+// Takes pages until the paged request holds at least `tokens` tokens.  False: the arena is full (pages taken so
+// far are kept).  A new page changes the page list, so cached plans are dropped.
+bool grow_pages(cart_ctx *ctx, Request &r, int64_t tokens)
+{
+    while ((int64_t)r.cap < tokens) {
+        uint64_t start = 0;
+        if (!arena_alloc(ctx, page_rows(ctx), &start)) return false;
+        r.pages.push_back((uint32_t)start);
+        r.cap += kTileTokens;
+        ++ctx->epoch;
+    }
+    return true;
+}
+void drop_storage(cart_ctx *ctx, Request &r)
+{
+    if (r.paged) {
+        for (uint32_t pg : r.pages) arena_free(ctx, pg, page_rows(ctx));
+        r.pages.clear();
+    } else if (r.alloc_rows > 0) {
+        arena_free(ctx, r.alloc_start, r.alloc_rows);
+    }
+    r.alloc_rows = 0;
+}
+// Does a request that is resident attend to registered Cartridge `id`?
+bool cartridge_has_active_reader(const cart_ctx *ctx, int32_t id)
+{
+    for (const Request &r : ctx->reqs) {
+        if (!r.live || r.evicted || r.cart == CART_NONE) continue;
+        const Cartridge &c = ctx->carts[(size_t)r.cart];
+        if (r.cart == id) return true;
+        if (c.composed)
+            for (int32_t b : c.parts)
+                if (b == id) return true;
+    }
+    return false;
+}
+// The first evicted registered Cartridge a request attends to, or -1.
+int32_t evicted_part(const cart_ctx *ctx, const Request &r)
+{
+    if (r.cart == CART_NONE) return -1;
+    const Cartridge &c = ctx->carts[(size_t)r.cart];
+    if (!c.composed) return c.evicted ? r.cart : -1;
+    for (int32_t b : c.parts)
+        if (ctx->carts[(size_t)b].evicted) return b;
+    return -1;
+}
+
 cart_status encode_tensor_map(cart_ctx *ctx)
 {
     typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
@@ -281,6 +349,7 @@ const char *cart_status_string(cart_status s)
     case CART_ERR_IN_USE: return "CART_ERR_IN_USE";
     case CART_ERR_CUDA: return "CART_ERR_CUDA";
     case CART_ERR_TIMEOUT: return "CART_ERR_TIMEOUT";
+    case CART_ERR_EVICTED: return "CART_ERR_EVICTED";
     }
     return "CART_ERR_UNKNOWN";
 }
@@ -504,7 +573,7 @@ cart_status cart_release_cartridge(cart_ctx *ctx, cart_id id)
     if (c->refs > 0) return fail(ctx, CART_ERR_IN_USE, "release: %d users still hold the Cartridge", c->refs);
     if (c->composed) {
         for (int32_t b : c->parts) --ctx->carts[(size_t)b].refs;
-    } else {
+    } else if (!c->evicted) {
         arena_free(ctx, c->alloc_start, c->alloc_rows);
     }
     *c = Cartridge();
@@ -512,7 +581,10 @@ cart_status cart_release_cartridge(cart_ctx *ctx, cart_id id)
     return CART_OK;
 }
 
-cart_status cart_request_open(cart_ctx *ctx, cart_id cartridge, int32_t suffix_capacity, cart_req *out)
+}  // extern "C"
+
+namespace {
+cart_status open_impl(cart_ctx *ctx, cart_id cartridge, int32_t suffix_capacity, bool paged, cart_req *out)
 {
     if (!ctx) return CART_ERR_INVALID_ARG;
     if (!out || suffix_capacity < 0) return fail(ctx, CART_ERR_INVALID_ARG, "open: bad argument");
@@ -523,24 +595,47 @@ cart_status cart_request_open(cart_ctx *ctx, cart_id cartridge, int32_t suffix_c
         if (!ctx->reqs[i].live) { id = (int32_t)i; break; }
     if (id < 0) return fail(ctx, CART_ERR_CAPACITY, "open: request table full (%d)", ctx->cfg.max_requests);
     const int64_t cap = ((int64_t)suffix_capacity + kTileTokens - 1) / kTileTokens * kTileTokens;
-    const uint64_t rows_one = (uint64_t)ctx->cfg.n_layers * ctx->cfg.n_kv_heads * (uint64_t)cap;
-    uint64_t start = 0;
-    if (rows_one > 0 && !arena_alloc(ctx, 2 * rows_one, &start))
-        return fail(ctx, CART_ERR_OOM, "open: arena has no room for a suffix of %lld tokens", (long long)cap);
     Request &r = ctx->reqs[(size_t)id];
-    r = Request();
+    if (paged) {
+        r = Request();
+        r.paged = true;
+        if (!grow_pages(ctx, r, cap)) {
+            drop_storage(ctx, r);
+            r = Request();
+            return fail(ctx, CART_ERR_OOM, "open: arena has no room for %lld tokens of pages", (long long)cap);
+        }
+    } else {
+        const uint64_t rows_one = (uint64_t)ctx->cfg.n_layers * ctx->cfg.n_kv_heads * (uint64_t)cap;
+        uint64_t start = 0;
+        if (rows_one > 0 && !arena_alloc(ctx, 2 * rows_one, &start))
+            return fail(ctx, CART_ERR_OOM, "open: arena has no room for a suffix of %lld tokens", (long long)cap);
+        r = Request();
+        r.cap = (int32_t)cap;
+        r.k_row = start;
+        r.v_row = start + rows_one;
+        r.alloc_start = start;
+        r.alloc_rows = 2 * rows_one;
+    }
     r.live = true;
     r.cart = cartridge;
-    r.cap = (int32_t)cap;
-    r.k_row = start;
-    r.v_row = start + rows_one;
-    r.alloc_start = start;
-    r.alloc_rows = 2 * rows_one;
     r.len.assign((size_t)ctx->cfg.n_layers, 0);
     if (cartridge != CART_NONE) ++ctx->carts[(size_t)cartridge].refs;
     ++ctx->epoch;
     *out = id;
     return CART_OK;
+}
+}  // namespace
+
+extern "C" {
+
+cart_status cart_request_open(cart_ctx *ctx, cart_id cartridge, int32_t suffix_capacity, cart_req *out)
+{
+    return open_impl(ctx, cartridge, suffix_capacity, false, out);
+}
+
+cart_status cart_request_open_paged(cart_ctx *ctx, cart_id cartridge, int32_t initial_capacity, cart_req *out)
+{
+    return open_impl(ctx, cartridge, initial_capacity, true, out);
 }
 
 cart_status cart_request_reserve(cart_ctx *ctx, cart_req req, int32_t suffix_capacity, void *stream)
@@ -549,8 +644,22 @@ cart_status cart_request_reserve(cart_ctx *ctx, cart_req req, int32_t suffix_cap
     Request *r = get_req(ctx, req);
     if (!r) return fail(ctx, CART_ERR_BAD_HANDLE, "reserve: not an open request");
     if (suffix_capacity < 0) return fail(ctx, CART_ERR_INVALID_ARG, "reserve: negative capacity");
+    if (r->evicted) return fail(ctx, CART_ERR_EVICTED, "reserve: the request is swapped out");
     const int64_t cap = ((int64_t)suffix_capacity + kTileTokens - 1) / kTileTokens * kTileTokens;
     if (cap <= r->cap) return CART_OK;  // a buffer never shrinks
+    if (r->paged) {
+        // pages instead of a copy; on failure the pages taken by this call go back
+        const size_t had = r->pages.size();
+        if (!grow_pages(ctx, *r, cap)) {
+            while (r->pages.size() > had) {
+                arena_free(ctx, r->pages.back(), page_rows(ctx));
+                r->pages.pop_back();
+                r->cap -= kTileTokens;
+            }
+            return fail(ctx, CART_ERR_OOM, "reserve: arena has no room for %lld tokens of pages", (long long)cap);
+        }
+        return CART_OK;
+    }
     const uint64_t heads = (uint64_t)ctx->cfg.n_layers * ctx->cfg.n_kv_heads;
     const uint64_t rows_one = heads * (uint64_t)cap;
     uint64_t start = 0;
@@ -589,8 +698,143 @@ cart_status cart_request_close(cart_ctx *ctx, cart_req req)
     Request *r = get_req(ctx, req);
     if (!r) return fail(ctx, CART_ERR_BAD_HANDLE, "close: not an open request");
     if (r->cart != CART_NONE) --ctx->carts[(size_t)r->cart].refs;
-    arena_free(ctx, r->alloc_start, r->alloc_rows);
+    drop_storage(ctx, *r);
     *r = Request();
+    ++ctx->epoch;
+    return CART_OK;
+}
+
+}  // extern "C"
+
+namespace {
+// Copies the first n tokens of every (layer, KV head) run of a request's suffix to (out = true) or from a dense
+// [L][Hkv][n][128] pair of buffers.  A paged suffix moves page by page: inside a page the (layer, KV head) blocks of
+// K (and of V) are 2 * kTileTokens rows apart.
+cart_status swap_copy(cart_ctx *ctx, const Request &r, void *k_buf, void *v_buf, int32_t n, bool out, cudaStream_t s)
+{
+    const uint64_t heads = (uint64_t)ctx->cfg.n_layers * ctx->cfg.n_kv_heads;
+    const size_t dense_pitch = (size_t)n * kRowBytes;
+    auto copy2d = [&](void *dense, size_t dense_off, uint64_t arena_row, size_t arena_pitch, size_t width) -> cudaError_t {
+        uint8_t *d = static_cast<uint8_t *>(dense) + dense_off;
+        uint8_t *a = arena_ptr(ctx, arena_row);
+        return out ? cudaMemcpy2DAsync(d, dense_pitch, a, arena_pitch, width, heads, cudaMemcpyDefault, s)
+                   : cudaMemcpy2DAsync(a, arena_pitch, d, dense_pitch, width, heads, cudaMemcpyDefault, s);
+    };
+    if (r.paged) {
+        for (int32_t t0 = 0; t0 < n; t0 += kTileTokens) {
+            const size_t width = (size_t)std::min(kTileTokens, n - t0) * kRowBytes;
+            const uint64_t pg = r.pages[(size_t)(t0 / kTileTokens)];
+            CART_CUDA(ctx, copy2d(k_buf, (size_t)t0 * kRowBytes, pg, 2 * kTileTokens * kRowBytes, width));
+            CART_CUDA(ctx, copy2d(v_buf, (size_t)t0 * kRowBytes, pg + kTileTokens, 2 * kTileTokens * kRowBytes, width));
+        }
+    } else {
+        CART_CUDA(ctx, copy2d(k_buf, 0, r.k_row, (size_t)r.cap * kRowBytes, dense_pitch));
+        CART_CUDA(ctx, copy2d(v_buf, 0, r.v_row, (size_t)r.cap * kRowBytes, dense_pitch));
+    }
+    return CART_OK;
+}
+}  // namespace
+
+extern "C" {
+
+cart_status cart_evict_request(cart_ctx *ctx, cart_req req, void *k_out, void *v_out, int32_t *n_tokens_out, void *stream)
+{
+    if (!ctx) return CART_ERR_INVALID_ARG;
+    Request *r = get_req(ctx, req);
+    if (!r) return fail(ctx, CART_ERR_BAD_HANDLE, "evict: not an open request");
+    if (!n_tokens_out) return fail(ctx, CART_ERR_INVALID_ARG, "evict: null n_tokens_out");
+    if (r->evicted) return fail(ctx, CART_ERR_EVICTED, "evict: the request is already swapped out");
+    int32_t n = 0;
+    for (int32_t l : r->len) n = std::max(n, l);
+    if (n > 0 && (!k_out || !v_out)) return fail(ctx, CART_ERR_INVALID_ARG, "evict: null buffer for %d tokens", n);
+    if (n > 0) {
+        const cart_status st = swap_copy(ctx, *r, k_out, v_out, n, true, static_cast<cudaStream_t>(stream));
+        if (st != CART_OK) return st;
+    }
+    drop_storage(ctx, *r);
+    r->evicted = true;
+    ++ctx->epoch;
+    *n_tokens_out = n;
+    return CART_OK;
+}
+
+cart_status cart_restore_request(cart_ctx *ctx, cart_req req, const void *k_in, const void *v_in, void *stream)
+{
+    if (!ctx) return CART_ERR_INVALID_ARG;
+    Request *r = get_req(ctx, req);
+    if (!r) return fail(ctx, CART_ERR_BAD_HANDLE, "restore: not an open request");
+    if (!r->evicted) return fail(ctx, CART_ERR_EVICTED, "restore: the request is not swapped out");
+    int32_t n = 0;
+    for (int32_t l : r->len) n = std::max(n, l);
+    if (n > 0 && (!k_in || !v_in)) return fail(ctx, CART_ERR_INVALID_ARG, "restore: null buffer for %d tokens", n);
+    if (r->paged) {
+        r->cap = 0;
+        if (!grow_pages(ctx, *r, n)) {
+            drop_storage(ctx, *r);
+            return fail(ctx, CART_ERR_OOM, "restore: arena has no room for %d tokens of pages", n);
+        }
+    } else {
+        const uint64_t rows_one = (uint64_t)ctx->cfg.n_layers * ctx->cfg.n_kv_heads * (uint64_t)r->cap;
+        uint64_t start = 0;
+        if (rows_one > 0 && !arena_alloc(ctx, 2 * rows_one, &start))
+            return fail(ctx, CART_ERR_OOM, "restore: arena has no room for a suffix of %d tokens", r->cap);
+        r->k_row = start;
+        r->v_row = start + rows_one;
+        r->alloc_start = start;
+        r->alloc_rows = 2 * rows_one;
+    }
+    if (n > 0) {
+        const cart_status st = swap_copy(ctx, *r, const_cast<void *>(k_in), const_cast<void *>(v_in), n, false,
+                                         static_cast<cudaStream_t>(stream));
+        if (st != CART_OK) {
+            drop_storage(ctx, *r);
+            return st;
+        }
+    }
+    r->evicted = false;
+    ++ctx->epoch;
+    return CART_OK;
+}
+
+cart_status cart_evict_cartridge(cart_ctx *ctx, cart_id id)
+{
+    if (!ctx) return CART_ERR_INVALID_ARG;
+    Cartridge *c = get_cart(ctx, id);
+    if (!c || c->composed) return fail(ctx, CART_ERR_BAD_HANDLE, "evict: not a registered Cartridge");
+    if (c->evicted) return fail(ctx, CART_ERR_EVICTED, "evict: the Cartridge is already swapped out");
+    if (cartridge_has_active_reader(ctx, id))
+        return fail(ctx, CART_ERR_IN_USE, "evict: a resident request attends to the Cartridge");
+    arena_free(ctx, c->alloc_start, c->alloc_rows);
+    c->alloc_rows = 0;
+    c->evicted = true;
+    ++ctx->epoch;
+    return CART_OK;
+}
+
+cart_status cart_restore_cartridge(cart_ctx *ctx, cart_id id, const void *k, const void *v, void *stream)
+{
+    if (!ctx) return CART_ERR_INVALID_ARG;
+    Cartridge *c = get_cart(ctx, id);
+    if (!c || c->composed) return fail(ctx, CART_ERR_BAD_HANDLE, "restore: not a registered Cartridge");
+    if (!c->evicted) return fail(ctx, CART_ERR_EVICTED, "restore: the Cartridge is not swapped out");
+    if (!aligned16(k) || !aligned16(v)) return fail(ctx, CART_ERR_INVALID_ARG, "restore: null/misaligned pointer");
+    const uint64_t rows_one = (uint64_t)ctx->cfg.n_layers * ctx->cfg.n_kv_heads * (uint64_t)c->p;
+    uint64_t start = 0;
+    if (!arena_alloc(ctx, 2 * rows_one, &start))
+        return fail(ctx, CART_ERR_OOM, "restore: arena has no room for %llu bytes", (unsigned long long)(2 * rows_one * kRowBytes));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(arena_ptr(ctx, start), k, rows_one * kRowBytes, cudaMemcpyDefault, s);
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(arena_ptr(ctx, start + rows_one), v, rows_one * kRowBytes, cudaMemcpyDefault, s);
+    if (e != cudaSuccess) {
+        arena_free(ctx, start, 2 * rows_one);
+        return fail(ctx, CART_ERR_CUDA, "restore: copy failed: %s", cudaGetErrorString(e));
+    }
+    c->k_row = start;
+    c->v_row = start + rows_one;
+    c->alloc_start = start;
+    c->alloc_rows = 2 * rows_one;
+    c->evicted = false;
     ++ctx->epoch;
     return CART_OK;
 }
@@ -608,8 +852,14 @@ cart_status cart_append_kv(cart_ctx *ctx, int32_t layer, const cart_req *reqs, i
         if (!r) return fail(ctx, CART_ERR_BAD_HANDLE, "append: reqs[%d] is not an open request", i);
         if (r->stamp == stamp) return fail(ctx, CART_ERR_INVALID_ARG, "append: reqs[%d] appears twice", i);
         r->stamp = stamp;
-        if (r->len[(size_t)layer] >= r->cap)
+        if (r->evicted) return fail(ctx, CART_ERR_EVICTED, "append: reqs[%d] is swapped out", i);
+        if (!r->paged && r->len[(size_t)layer] >= r->cap)
             return fail(ctx, CART_ERR_CAPACITY, "append: suffix of reqs[%d] is full (%d tokens)", i, r->cap);
+    }
+    for (int32_t i = 0; i < n_reqs; ++i) {  // paged suffixes take a page when the token opens one
+        Request &r = ctx->reqs[(size_t)reqs[i]];
+        if (r.paged && !grow_pages(ctx, r, (int64_t)r.len[(size_t)layer] + 1))
+            return fail(ctx, CART_ERR_OOM, "append: arena has no page left for reqs[%d]", i);
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int Hkv = ctx->cfg.n_kv_heads;
@@ -619,6 +869,13 @@ cart_status cart_append_kv(cart_ctx *ctx, int32_t layer, const cart_req *reqs, i
         const int32_t n = std::min(kAppendBatch, n_reqs - b0);
         for (int32_t i = 0; i < n; ++i) {
             const Request &r = ctx->reqs[(size_t)reqs[b0 + i]];
+            if (r.paged) {
+                const uint64_t row = paged_row(ctx, r, layer, r.len[(size_t)layer]);
+                ap.e[i].k_row = (uint32_t)row;
+                ap.e[i].v_row = (uint32_t)(row + kTileTokens);
+                ap.e[i].head_stride = 2u * kTileTokens;
+                continue;
+            }
             const uint64_t off = (uint64_t)layer * Hkv * (uint64_t)r.cap + (uint64_t)r.len[(size_t)layer];
             ap.e[i].k_row = (uint32_t)(r.k_row + off);
             ap.e[i].v_row = (uint32_t)(r.v_row + off);
@@ -645,6 +902,33 @@ cart_status cart_extend_kv(cart_ctx *ctx, int32_t layer, cart_req req, const voi
     if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, CART_ERR_BAD_HANDLE, "extend: layer out of range");
     Request *r = get_req(ctx, req);
     if (!r) return fail(ctx, CART_ERR_BAD_HANDLE, "extend: not an open request");
+    if (r->evicted) return fail(ctx, CART_ERR_EVICTED, "extend: the request is swapped out");
+    if (r->paged) {
+        if (!grow_pages(ctx, *r, (int64_t)r->len[(size_t)layer] + n_tokens))
+            return fail(ctx, CART_ERR_OOM, "extend: arena has no pages left for %d more tokens", n_tokens);
+        // one scatter per page touched
+        const int Hkv = ctx->cfg.n_kv_heads;
+        int32_t done = 0;
+        while (done < n_tokens) {
+            const int32_t pos = r->len[(size_t)layer] + done;
+            const int32_t n = std::min(n_tokens - done, kTileTokens - pos % kTileTokens);
+            ExtendParams ep;
+            const uint64_t row = paged_row(ctx, *r, layer, pos);
+            ep.arena = ctx->cfg.arena;
+            ep.k = static_cast<const uint8_t *>(k) + (uint64_t)done * Hkv * kRowBytes;
+            ep.v = static_cast<const uint8_t *>(v) + (uint64_t)done * Hkv * kRowBytes;
+            ep.k_row = (uint32_t)row;
+            ep.v_row = (uint32_t)(row + kTileTokens);
+            ep.head_stride = 2u * kTileTokens;
+            ep.n_tokens = n;
+            ep.n_kv_heads = Hkv;
+            CART_CUDA(ctx, launch_extend(ep, static_cast<cudaStream_t>(stream)));
+            ++ctx->launches;
+            done += n;
+        }
+        r->len[(size_t)layer] += n_tokens;
+        return CART_OK;
+    }
     if ((int64_t)r->len[(size_t)layer] + n_tokens > r->cap)
         return fail(ctx, CART_ERR_CAPACITY, "extend: %d + %d tokens exceed the capacity %d", r->len[(size_t)layer],
                     n_tokens, r->cap);
@@ -698,6 +982,9 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
     if (prefill) {
         Request *r = get_req(ctx, reqs[0]);
         if (!r) return fail(ctx, CART_ERR_BAD_HANDLE, "prefill: not an open request");
+        if (r->evicted) return fail(ctx, CART_ERR_EVICTED, "prefill: the request is swapped out");
+        if (evicted_part(ctx, *r) >= 0)
+            return fail(ctx, CART_ERR_EVICTED, "prefill: Cartridge %d is swapped out", evicted_part(ctx, *r));
         if (r->len[(size_t)layer] < n_new)
             return fail(ctx, CART_ERR_INVALID_ARG, "prefill: the suffix holds %d tokens, fewer than n_new = %d",
                         r->len[(size_t)layer], n_new);
@@ -708,6 +995,10 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
     for (int32_t i = 0; i < n_reqs && !prefill; ++i) {
         Request *r = get_req(ctx, reqs[i]);
         if (!r) return fail(ctx, CART_ERR_BAD_HANDLE, "decode: reqs[%d] is not an open request", i);
+        if (r->evicted) return fail(ctx, CART_ERR_EVICTED, "decode: reqs[%d] is swapped out", i);
+        if (evicted_part(ctx, *r) >= 0)
+            return fail(ctx, CART_ERR_EVICTED, "decode: reqs[%d] attends to Cartridge %d, which is swapped out", i,
+                        evicted_part(ctx, *r));
         const int32_t len = r->len[(size_t)layer];
         if (len == 0 && r->cart == CART_NONE)
             return fail(ctx, CART_ERR_EMPTY, "decode: reqs[%d] has no KV token in layer %d", i, layer);
@@ -735,6 +1026,18 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
             ns.ev_recorded = false;
         }
         ns.valid = false;
+        // Paged suffixes.  In a fused decode loop every request takes a new page once per 64 steps, each at a step
+        // of its own, and a new page means a new plan; so when a plan is built anyway, requests with less than a
+        // page of room are given their next page now (if the arena has one), and the plan lasts 64 steps or more.
+        if (k_new != nullptr)
+            for (int32_t i = 0; i < n_reqs; ++i) {
+                Request &r = ctx->reqs[(size_t)reqs[i]];
+                if (r.paged) (void)grow_pages(ctx, r, (int64_t)r.len[(size_t)layer] + kTileTokens);
+            }
+        // the batch's page list: every page of every paged request, request by request
+        uint32_t *page_list = reinterpret_cast<uint32_t *>(ns.host + ctx->lay.pages_off);
+        uint32_t n_listed = 0;
+        const uint64_t list_stamp = ++ctx->list_stamp;
         auto &segs = ctx->seg_tmp;
         auto &sb = ctx->seg_begin_tmp;
         segs.clear();
@@ -764,8 +1067,23 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
                 head_of_group.push_back(cur);
             }
         }
+        bool list_full = false;
+        // describes the part of a paged suffix that starts at token `first` (a multiple of the page size)
+        auto paged_seg = [&](Request &r, uint32_t first, cart_plan_seg *sg) {
+            if (r.list_stamp != list_stamp) {
+                if (n_listed + r.pages.size() > (size_t)ctx->lay.pages_cap) { list_full = true; return; }
+                r.list_stamp = list_stamp;
+                r.list_base = n_listed;
+                for (uint32_t pg : r.pages) page_list[n_listed++] = pg;
+            }
+            sg->k_row = r.list_base + first / (uint32_t)kTileTokens;
+            sg->v_row = 0;
+            sg->head_stride = 2u * kTileTokens;
+            sg->layer_stride = (uint32_t)Hkv * 2u * kTileTokens;
+            sg->flags |= CART_SEG_PAGED;
+        };
         for (int32_t i = 0; i < n_reqs; ++i) {
-            const Request &r = ctx->reqs[(size_t)reqs[prefill ? 0 : i]];
+            Request &r = ctx->reqs[(size_t)reqs[prefill ? 0 : i]];
             auto push_cart = [&](const Cartridge &c) {
                 cart_plan_seg sg;
                 sg.k_row = (uint32_t)c.k_row;
@@ -796,6 +1114,7 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
                     sg.layer_stride = (uint32_t)((uint64_t)Hkv * r.cap);
                     sg.n_tok = (uint32_t)head;
                     sg.flags = CART_SEG_SUFFIX;
+                    if (r.paged) paged_seg(r, 0u, &sg);
                     segs.push_back(sg);
                     first = (uint32_t)head;
                 }
@@ -808,10 +1127,12 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
                 sg.layer_stride = (uint32_t)((uint64_t)Hkv * r.cap);
                 sg.n_tok = (uint32_t)len - first;
                 sg.flags = CART_SEG_SUFFIX;
+                if (r.paged) paged_seg(r, first, &sg);
                 segs.push_back(sg);
             }
             sb.push_back((int32_t)segs.size());
         }
+        if (list_full) return fail(ctx, CART_ERR_CAPACITY, "decode: the batch names more than %d pages", ctx->lay.pages_cap);
         const ScratchLayout &lay = ctx->lay;
         cart_plan_out po{};
         po.items = reinterpret_cast<cart_work_item *>(ns.host + lay.items_off);
@@ -846,6 +1167,9 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
             CART_CUDA(ctx, cudaMemcpyAsync(ns.dev + lay.shared_off, ns.host + lay.shared_off, sh_bytes,
                                            cudaMemcpyHostToDevice, s));
         }
+        if (n_listed > 0)
+            CART_CUDA(ctx, cudaMemcpyAsync(ns.dev + lay.pages_off, ns.host + lay.pages_off, (uint64_t)n_listed * 4,
+                                           cudaMemcpyHostToDevice, s));
         ns.key = key;
         ns.prefill = prefill;
         ns.reqs.assign(reqs, reqs + (prefill ? 1 : n_reqs));
@@ -881,6 +1205,7 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
     dp.scale_log2 = ctx->scale * 1.4426950408889634f;
     dp.grow = (uint32_t)grow;
     dp.edge_boxes = 1u;
+    dp.pages = reinterpret_cast<const uint32_t *>(sl->dev + ctx->lay.pages_off);
     const bool timed = ctx->timing && ctx->ev_used + 2 <= kMaxTimedLaunches * 2;
     if (timed) {
         while (ctx->ev_pool.size() < ctx->ev_used + 2) {
@@ -924,6 +1249,7 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
         sp.scale_log2 = dp.scale_log2;
         sp.ready_flag = dp.ready_flag;
         sp.seq = dp.seq;
+        sp.pages = dp.pages;
         CART_CUDA(ctx, launch_shared(ctx->tmap, sp, sl->n_unit_cta_used, s));
         ++ctx->launches;
     }
@@ -981,8 +1307,14 @@ cart_status cart_decode_step(cart_ctx *ctx, int32_t layer, const cart_req *reqs,
         if (!r) return fail(ctx, CART_ERR_BAD_HANDLE, "decode_step: reqs[%d] is not an open request", i);
         if (r->stamp == stamp) return fail(ctx, CART_ERR_INVALID_ARG, "decode_step: reqs[%d] appears twice", i);
         r->stamp = stamp;
-        if (r->len[(size_t)layer] >= r->cap)
+        if (r->evicted) return fail(ctx, CART_ERR_EVICTED, "decode_step: reqs[%d] is swapped out", i);
+        if (!r->paged && r->len[(size_t)layer] >= r->cap)
             return fail(ctx, CART_ERR_CAPACITY, "decode_step: suffix of reqs[%d] is full (%d tokens)", i, r->cap);
+    }
+    for (int32_t i = 0; i < n_reqs; ++i) {  // paged suffixes take a page when the new token opens one
+        Request &r = ctx->reqs[(size_t)reqs[i]];
+        if (r.paged && !grow_pages(ctx, r, (int64_t)r.len[(size_t)layer] + 1))
+            return fail(ctx, CART_ERR_OOM, "decode_step: arena has no page left for reqs[%d]", i);
     }
     // The plan must see the new token: count it first, take it back if nothing was launched.
     for (int32_t i = 0; i < n_reqs; ++i) ++ctx->reqs[(size_t)reqs[i]].len[(size_t)layer];

@@ -51,6 +51,8 @@ struct DecodeParams {
                                  // count of every item marked CART_ITEM_TAIL
     uint32_t edge_boxes = 0;     // 1: ragged last tiles are fetched in boxes of kEdgeBoxRows rows through the second
                                  // tensor map; 0: every tile is fetched whole
+    const uint32_t *pages = nullptr;  // page list of the batch (base row of every page of every paged suffix), read by
+                                      // items marked CART_ITEM_PAGED
 };
 
 // Parameters of the shared-segment kernel (units and reader tables as the planner lays them out).
@@ -78,6 +80,7 @@ struct SharedParams {
     // only executes on its way out, so that it never completes before the stream kernel.  Null: alone.
     const uint32_t *ready_flag = nullptr;
     uint32_t seq = 0;
+    const uint32_t *pages = nullptr;  // page list (units marked CART_UNIT_PAGED)
 };
 
 struct MergeParams {

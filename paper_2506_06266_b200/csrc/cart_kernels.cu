@@ -250,7 +250,14 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
             const uint32_t k_row = w.k_row + (uint32_t)p.layer * w.layer_stride;
             const uint32_t v_row = w.v_row + (uint32_t)p.layer * w.layer_stride;
             const uint32_t ntiles = (w.n_tok + kTileTokens - 1) / kTileTokens;
+            // Paged suffix (Sec. 3.3: per-user KV caches of any length): tile j of the item is page w.k_row + j of the
+            // batch's page list.  Lane l holds the base row of the page of tile 32 c + l, fetched 32 tiles at a time.
+            const bool paged = (w.flags & CART_ITEM_PAGED) != 0u;
+            const uint32_t in_page = (uint32_t)p.layer * w.layer_stride + w.v_row;  // the head's K block inside a page
+            uint32_t page_row = 0;
             for (uint32_t j = 0; j < ntiles; ++j, ++t) {
+                if (paged && (j & 31u) == 0u) page_row = j + (uint32_t)lane < ntiles ? __ldg(p.pages + w.k_row + j + (uint32_t)lane) : 0u;
+                const uint32_t page_base = __shfl_sync(0xffffffffu, page_row, (int)(j & 31u)) + in_page;
                 const int s = (int)(t % kStages);
                 const uint32_t round = t / kStages;
                 bool ok0 = true;
@@ -300,7 +307,8 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
                     const uint32_t kdst = stages + (uint32_t)s * kStageBytes;
                     const uint32_t is_v = ((uint32_t)lane >> 1) & 1u, hi = (uint32_t)lane & 1u;
                     const uint32_t dst = kdst + is_v * kTileBytes + hi * kHalfBytes;
-                    const int32_t y = (int32_t)((is_v ? v_row : k_row) + j * kTileTokens);
+                    const int32_t y = paged ? (int32_t)(page_base + is_v * (uint32_t)kTileTokens)
+                                            : (int32_t)((is_v ? v_row : k_row) + j * kTileTokens);
                     const uint32_t bar = is_v ? full_v(s) : full_k(s);
                     const uint32_t valid = min((uint32_t)kTileTokens, w.n_tok - j * kTileTokens);
                     // Ragged last tile of a segment with at most kEdgeRows tokens: only one small box per half
@@ -370,8 +378,16 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
                             const uint32_t a_ls = __shfl_sync(0xffffffffu, a.layer_stride, src_lane);
                             const uint32_t a_n = __shfl_sync(0xffffffffu, a.n_tok, src_lane) + p.grow;
                             const uint32_t a_rg = __shfl_sync(0xffffffffu, a.row_group, src_lane);
+                            const uint32_t a_fl = __shfl_sync(0xffffffffu, a.flags, src_lane);
                             val[u] = __ldg(new_rows + (size_t)a_rg * 16 + c);
-                            dst[u] = ((size_t)row0 + (size_t)p.layer * a_ls + (a_n - 1u)) * 16 + c;
+                            if (a_fl & CART_ITEM_PAGED) {
+                                // the page that holds the item's last token, then the head's K or V block in it
+                                const uint32_t page = __ldg(p.pages + a_k + ((a_n - 1u) / (uint32_t)kTileTokens));
+                                dst[u] = ((size_t)page + (size_t)p.layer * a_ls + a_v + (lane < 16 ? 0u : (uint32_t)kTileTokens) +
+                                          ((a_n - 1u) % (uint32_t)kTileTokens)) * 16 + c;
+                            } else {
+                                dst[u] = ((size_t)row0 + (size_t)p.layer * a_ls + (a_n - 1u)) * 16 + c;
+                            }
                             n = u + 1;
                         }
                     }

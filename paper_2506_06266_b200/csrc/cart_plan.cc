@@ -76,7 +76,7 @@ struct Balancer {
 bool same_storage(const cart_plan_seg &a, const cart_plan_seg &b)
 {
     return a.k_row == b.k_row && a.v_row == b.v_row && a.n_tok == b.n_tok && a.head_stride == b.head_stride &&
-           a.layer_stride == b.layer_stride;
+           a.layer_stride == b.layer_stride && (a.flags & CART_SEG_PAGED) == (b.flags & CART_SEG_PAGED);
 }
 
 }  // namespace
@@ -286,14 +286,20 @@ extern "C" cart_status cart_plan_build_shared(const cart_plan_seg *segs, const i
                 const cart_plan_seg &sg = classes[(size_t)cb.cls].seg;
                 cart_shared_unit &u = o->units[nu++];
                 const uint32_t tok0 = (uint32_t)(done * TS);
-                u.k_row = sg.k_row + cb.kv_head * sg.head_stride + tok0;
-                u.v_row = sg.v_row + cb.kv_head * sg.head_stride + tok0;
+                u.flags = (sg.flags & CART_SEG_SUFFIX) ? (uint16_t)CART_UNIT_SUFFIX : (uint16_t)0;
+                if (sg.flags & CART_SEG_PAGED) {
+                    u.k_row = sg.k_row + (uint32_t)(tok0 / T);
+                    u.v_row = cb.kv_head * sg.head_stride;
+                    u.flags |= (uint16_t)CART_UNIT_PAGED;
+                } else {
+                    u.k_row = sg.k_row + cb.kv_head * sg.head_stride + tok0;
+                    u.v_row = sg.v_row + cb.kv_head * sg.head_stride + tok0;
+                }
                 u.layer_stride = sg.layer_stride;
                 u.n_tiles = (uint32_t)take;
                 u.reader_begin = cb.reader_begin;
                 u.n_readers = cb.n_readers;
                 u.kv_head = (uint16_t)cb.kv_head;
-                u.flags = (sg.flags & CART_SEG_SUFFIX) ? (uint16_t)CART_UNIT_SUFFIX : (uint16_t)0;
                 u.chunk = chunk;
             });
         if (overflow) return CART_ERR_CAPACITY;
@@ -400,12 +406,19 @@ extern "C" cart_status cart_plan_build_shared(const cart_plan_seg *segs, const i
                     cart_work_item &it = o->items[ni++];
                     const uint64_t tok0 = seg_tile * T;
                     const uint64_t tok1 = std::min<uint64_t>(seg_ntok, (seg_tile + take) * T);
-                    it.k_row = segs[s].k_row + (uint32_t)g * segs[s].head_stride + seg_tok0 + (uint32_t)tok0;
-                    it.v_row = segs[s].v_row + (uint32_t)g * segs[s].head_stride + seg_tok0 + (uint32_t)tok0;
+                    it.flags = first ? CART_ITEM_BEGIN : 0u;
+                    if (segs[s].flags & CART_SEG_PAGED) {
+                        // a page holds one tile: the run starts (seg_tok0 + tok0) / T pages into the segment
+                        it.k_row = segs[s].k_row + (uint32_t)((seg_tok0 + tok0) / T);
+                        it.v_row = (uint32_t)g * segs[s].head_stride;
+                        it.flags |= CART_ITEM_PAGED;
+                    } else {
+                        it.k_row = segs[s].k_row + (uint32_t)g * segs[s].head_stride + seg_tok0 + (uint32_t)tok0;
+                        it.v_row = segs[s].v_row + (uint32_t)g * segs[s].head_stride + seg_tok0 + (uint32_t)tok0;
+                    }
                     it.layer_stride = segs[s].layer_stride;
                     it.n_tok = (uint32_t)(tok1 - tok0);
                     it.row_group = rg;
-                    it.flags = first ? CART_ITEM_BEGIN : 0u;
                     if (s == s1 - 1 && tok1 == seg_ntok) it.flags |= CART_ITEM_TAIL;
                     if (segs[s].flags & CART_SEG_SUFFIX) it.flags |= CART_ITEM_SUFFIX;
                     it.slot = 0;

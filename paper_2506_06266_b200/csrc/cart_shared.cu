@@ -325,19 +325,34 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                         waited = true;
                     }
                     const uint32_t row0 = (is_v ? u.v_row : u.k_row) + (uint32_t)p.layer * u.layer_stride;
+                    // Paged suffix storage: a 128-token tile is two pages of 64 tokens, entries u.k_row + 2 t and
+                    // + 2 t + 1 of the page list; inside a page the head's K block is at u.v_row, its V block 64
+                    // rows later.  The entries of the next tile are read while this tile's stage is waited for.
+                    const bool paged = (u.flags & CART_UNIT_PAGED) != 0u;
+                    const uint32_t in_page = (uint32_t)p.layer * u.layer_stride + u.v_row + (is_v ? 64u : 0u);
+                    uint32_t pg0 = 0, pg1 = 0;
+                    if (paged) {
+                        pg0 = __ldg(p.pages + u.k_row);
+                        pg1 = __ldg(p.pages + u.k_row + 1u);
+                    }
                     for (uint32_t t = 0; t < u.n_tiles; ++t, ++tt) {
                         const int st = (int)(tt % nst);
                         const uint32_t par = (tt / nst) & 1u;
-                        const int32_t y = (int32_t)(row0 + t * kShTile);
+                        const int32_t y = paged ? (int32_t)(pg0 + in_page) : (int32_t)(row0 + t * kShTile);
+                        const int32_t y2 = paged ? (int32_t)(pg1 + in_page) : y + 64;
+                        if (paged && t + 1u < u.n_tiles) {
+                            pg0 = __ldg(p.pages + u.k_row + 2u * (t + 1u));
+                            pg1 = __ldg(p.pages + u.k_row + 2u * (t + 1u) + 1u);
+                        }
                         ok = mbar_wait(bar(empty0 + st), par ^ 1u, abort_flag, p.status, kStatusTimeoutProducer);
                         if (!ok) break;
                         const uint32_t dst = ring + (uint32_t)st * kShTileBytes;
                         mbar_expect_tx(bar(full0 + st), kShTileBytes);
                         // a block of the tile = 128 rows x 64 dims = two boxes of 64 rows
                         tma_load_2d(dst, &tmap, 0, y, bar(full0 + st));
-                        tma_load_2d(dst + kShBlock / 2, &tmap, 0, y + 64, bar(full0 + st));
+                        tma_load_2d(dst + kShBlock / 2, &tmap, 0, y2, bar(full0 + st));
                         tma_load_2d(dst + kShBlock, &tmap, 64, y, bar(full0 + st));
-                        tma_load_2d(dst + kShBlock + kShBlock / 2, &tmap, 64, y + 64, bar(full0 + st));
+                        tma_load_2d(dst + kShBlock + kShBlock / 2, &tmap, 64, y2, bar(full0 + st));
                     }
                 }
                 if (!ok) {

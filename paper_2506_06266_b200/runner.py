@@ -14,9 +14,10 @@ import torch
 from . import binding, buildlib, synth
 
 
-def arena_bytes_for(w: synth.Workload, extra_capacity: int) -> int:
+def arena_bytes_for(w: synth.Workload, extra_capacity: int, paged: bool = False) -> int:
     per_tok = w.n_layers * w.kv_bytes_per_token_layer()
-    caps = [-(-(int(s) + extra_capacity) // 64) * 64 for s in w.suffix_lengths()]
+    # (a paged request may hold one page of room more than it needs: pages are taken a plan's lifetime ahead)
+    caps = [-(-(int(s) + extra_capacity) // 64) * 64 + (128 if paged else 0) for s in w.suffix_lengths()]
     return (w.n_cartridges * w.p + sum(caps)) * per_tok
 
 
@@ -25,11 +26,12 @@ class LoadedWorkload:
 
     keep_layers / keep_requests: layers and batch indices whose KV bits are also copied to the host
     while loading (``host_segments``), in cache order [Cartridge part(s)..., suffix].
+    paged: the requests' suffixes live in pages of 64 tokens taken as they grow, not in one buffer each.
     """
 
     def __init__(self, w: synth.Workload, device: torch.device, extra_capacity: int = 0,
                  keep_layers: Sequence[int] = (), keep_requests: Optional[Sequence[int]] = None,
-                 stream: Optional[torch.cuda.Stream] = None):
+                 stream: Optional[torch.cuda.Stream] = None, paged: bool = False):
         buildlib.build()
         binding.load_library()
         self.w = w
@@ -41,7 +43,7 @@ class LoadedWorkload:
                                   w.n_cartridges + w.batch + 1, device=self.dev.index or 0,
                                   softmax_scale=w.scale)
         scratch = binding.cart_scratch_bytes(cfg)
-        total = scratch + arena_bytes_for(w, extra_capacity) + 4096
+        total = scratch + arena_bytes_for(w, extra_capacity, paged) + 4096
         self.arena = torch.empty(total, dtype=torch.uint8, device=self.dev)
         cfg.arena, cfg.arena_bytes = self.arena.data_ptr(), total
         self.cfg = cfg
@@ -71,7 +73,10 @@ class LoadedWorkload:
             else:
                 cart = binding.cart_compose(self.ctx, [self.cart_ids[p] for p in parts])
                 self.composed.append(cart)
-            r = binding.cart_request_open(self.ctx, cart, int(self.suffix[b]) + extra_capacity)
+            if paged:
+                r = binding.cart_request_open_paged(self.ctx, cart, 0)
+            else:
+                r = binding.cart_request_open(self.ctx, cart, int(self.suffix[b]) + extra_capacity)
             n = int(self.suffix[b])
             if n > 0:
                 k, v = w.suffix_kv(b, n, self.dev)      # [L][T][Hkv][D]

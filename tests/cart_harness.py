@@ -84,8 +84,8 @@ class Session:
             self.cart_map[cid] = self.oc.compose([self.cart_map[p] for p in parts])
         return cid
 
-    def open(self, cart: int, capacity: int) -> int:
-        rid = binding.cart_request_open(self.ctx, cart, capacity)
+    def open(self, cart: int, capacity: int, paged: bool = False) -> int:
+        rid = (binding.cart_request_open_paged if paged else binding.cart_request_open)(self.ctx, cart, capacity)
         if self.oc is not None:
             self.req_map[rid] = self.oc.open(None if cart == binding.CART_NONE else self.cart_map[cart])
         return rid
@@ -155,7 +155,7 @@ def workload_arena_bytes(w: synth.Workload, extra_capacity: int = 0) -> int:
 
 def load_workload(w: synth.Workload, extra_capacity: int = 0, with_oracle: bool = True,
                   gen_device: str = "cuda:0", extra_bytes: int = 0, extra_requests: int = 0,
-                  extra_cartridges: int = 0, **kw) -> tuple:
+                  extra_cartridges: int = 0, paged: bool = False, **kw) -> tuple:
     """Creates a Session for ``w``: registers its Cartridges, opens one request per batch entry
     (composing pool members where the workload says so) and fills the suffixes.  Returns
     (session, request handles)."""
@@ -177,7 +177,7 @@ def load_workload(w: synth.Workload, extra_capacity: int = 0, with_oracle: bool 
             cart = cids[parts[0]]
         else:
             cart = sess.compose([cids[p] for p in parts])
-        r = sess.open(cart, int(suffix[b]) + extra_capacity)
+        r = sess.open(cart, int(suffix[b]) + extra_capacity, paged=paged)
         k, v = w.suffix_kv(b, int(suffix[b]), gen_device)
         sess.extend(r, k, v)
         reqs.append(r)

@@ -174,3 +174,43 @@ def test_items_in_suffix_storage_are_marked():
         assert bool(it.flags & binding.CART_ITEM_SUFFIX) == in_suffix
         if it.flags & binding.CART_ITEM_TAIL:
             assert in_suffix
+
+
+def test_paged_segments_become_runs_of_page_list_entries():
+    """A paged suffix is named by the index of its first page in the batch's page list; the items that cover it
+    carry the index of their first tile's page, the row of the KV head's block inside a page and the paged flag,
+    and cover every page exactly once per KV head.  A shared paged segment (the common head of a prefill's rows)
+    becomes units of two pages per 128-token tile."""
+    Hkv, T = 2, 64
+    SUF, PAGED = binding.CART_SEG_SUFFIX, binding.CART_SEG_PAGED
+    cart = (5000, 9000, 300, Hkv * 300, 300)
+    # request 0: Cartridge + paged suffix of 200 tokens whose pages start at list entry 7; request 1: paged, entry 20
+    segs = [[cart, (7, 0, 2 * T, Hkv * 2 * T, 200, SUF | PAGED)], [(20, 0, 2 * T, Hkv * 2 * T, 65, SUF | PAGED)]]
+    plan = binding.cart_plan_build_shared(segs, Hkv, 4, 5, T, 0, 2 * T)
+    seen = {}
+    for it in plan["items"]:
+        if not it.flags & binding.CART_ITEM_PAGED:
+            assert it.k_row >= 5000
+            continue
+        assert it.flags & binding.CART_ITEM_SUFFIX and it.layer_stride == Hkv * 2 * T
+        head = it.row_group % Hkv
+        assert it.v_row == head * 2 * T
+        for j in range(-(-it.n_tok // T)):
+            key = (it.row_group, it.k_row + j)
+            assert key not in seen
+            seen[key] = min(T, it.n_tok - j * T)
+    expect = {}
+    for rg_req, first, n in [(0, 7, 200), (1, 20, 65)]:
+        for g in range(Hkv):
+            for j in range(-(-n // T)):
+                expect[(rg_req * Hkv + g, first + j)] = min(T, n - j * T)
+    assert seen == expect
+    # five rows of a prefill that share 256 tokens of paged suffix (entries 3..6) and own a ragged rest
+    rows = [[(3, 0, 2 * T, Hkv * 2 * T, 256, SUF | PAGED), (7, 0, 2 * T, Hkv * 2 * T, 10 + i, SUF | PAGED)] for i in range(5)]
+    plan = binding.cart_plan_build_shared(rows, Hkv, 4, 3, T, 4, 2 * T)
+    units = plan["units"]
+    assert units and all(u.flags & binding.CART_UNIT_PAGED and u.flags & binding.CART_UNIT_SUFFIX for u in units)
+    pages = sorted((u.kv_head, u.k_row + 2 * t) for u in units for t in range(u.n_tiles))
+    assert pages == [(g, 3 + 2 * t) for g in range(Hkv) for t in range(2)]
+    assert all(u.v_row == u.kv_head * 2 * T for u in units)
+    assert all(it.flags & binding.CART_ITEM_PAGED and it.k_row == 7 for it in plan["items"])
