@@ -233,6 +233,40 @@ CART_API cart_status cart_prefill_attention(cart_ctx *ctx, int32_t layer, cart_r
                                    int32_t n_new, void *out /*device*/, float *lse /*device or NULL*/,
                                    void *stream);
 
+/* Training-time attention over a shared trainable Cartridge.  Self-Study (Sec. 4.2) trains the key and value vectors
+ * of a Cartridge (Sec. 3.2: Z holds p trainable key and value vectors per layer and KV head) by back-propagating
+ * through attention of many short conversations that all attend to Z; Sec. 6 names shared-prefix attention kernels as
+ * the way to make that cheaper.  These two calls are that attention layer, forward and backward.
+ *
+ * convs: n_convs open requests, all on the same registered Cartridge Z (or all on CART_NONE), with contiguous (not
+ * paged) suffix storage; request c's suffix in `layer` holds conversation c's keys and values (cart_extend_kv).  The
+ * conversations are packed back to back on one token axis: conversation c owns tokens cu[c] .. cu[c+1] - 1 with cu the
+ * running sum of the suffix lengths, T = cu[n_convs] <= max_requests.  Token i of a conversation attends, per Eq. 1
+ * (Sec. 2.3) with its causal sum over j <= i, to all of Z and to the conversation's tokens 0 .. i.
+ *
+ * cart_train_attention_fwd: q device bf16 [T][n_q_heads][128] -> out device bf16 [T][n_q_heads][128] and lse device
+ * fp32 [T][n_q_heads] (natural log; required, the backward reads it).  Z is read once per 128 query rows by the
+ * tensor-core kernel, whichever conversations the rows belong to.
+ *
+ * cart_train_attention_bwd: given q, out, lse of the forward and dout (device bf16 [T][n_q_heads][128], the gradient
+ * of the loss with respect to out), writes the gradients with respect to q (dq, device fp32 [T][n_q_heads][128]), to
+ * the conversations' keys and values (dk, dv, device fp32 [T][n_kv_heads][128], token-major like the tensors
+ * cart_extend_kv took) and to the Cartridge (dzk, dzv, device fp32 [n_kv_heads][p][128], summed over all
+ * conversations; may be NULL without a Cartridge).  delta is device scratch, fp32 [T][n_q_heads].  All outputs are
+ * overwritten.  Products run on the tensor cores in bf16 with fp32 accumulation; sums over blocks use fp32 atomic
+ * adds, so the last bits depend on the order of arrival.
+ * Errors: INVALID_ARG (also: requests on different Cartridges, a composition, a paged request), BAD_HANDLE, EVICTED,
+ * EMPTY (a conversation without tokens), CAPACITY (T > max_requests, or more work items than the scratch holds), CUDA. */
+CART_API cart_status cart_train_attention_fwd(cart_ctx *ctx, int32_t layer, const cart_req *convs /*host*/, int32_t n_convs,
+                                              const void *q /*device*/, void *out /*device*/, float *lse /*device*/,
+                                              void *stream);
+CART_API cart_status cart_train_attention_bwd(cart_ctx *ctx, int32_t layer, const cart_req *convs /*host*/, int32_t n_convs,
+                                              const void *q /*device*/, const void *out /*device*/,
+                                              const float *lse /*device*/, const void *dout /*device*/,
+                                              float *delta /*device scratch*/, float *dq /*device*/, float *dk /*device*/,
+                                              float *dv /*device*/, float *dzk /*device or NULL*/,
+                                              float *dzv /*device or NULL*/, void *stream);
+
 /* Sharing policy.  When at least min_readers requests of a decode batch attend to the same stored
  * Cartridge (one Cartridge serving many users, Sec. 1 and Sec. 3.3; pool members composed by many
  * requests, Sec. 5.4), cart_decode_attention reads each of its K/V tiles once for up to 128 query

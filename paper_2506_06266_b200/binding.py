@@ -33,7 +33,7 @@ EXPORTS = ["cart_scratch_bytes", "cart_create", "cart_destroy", "cart_register_c
            "cart_set_share_min_readers", "cart_set_piece_cost", "cart_plan_build_shared",
            "cart_set_plan_reuse", "cart_plan_count", "cart_plan_reusable", "cart_set_side_by_side",
            "cart_request_open_paged", "cart_evict_request", "cart_restore_request", "cart_evict_cartridge",
-           "cart_restore_cartridge",
+           "cart_restore_cartridge", "cart_train_attention_fwd", "cart_train_attention_bwd",
            "cart_decode_attention_static", "cart_launch_count", "cart_status_string",
            "cart_last_error", "cart_plan_build"]
 
@@ -130,6 +130,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.cart_evict_request.argtypes = [vp, i32, vp, vp, i32p, vp]
     lib.cart_restore_request.argtypes = [vp, i32, vp, vp, vp]
     lib.cart_evict_cartridge.argtypes = [vp, i32]
+    lib.cart_train_attention_fwd.argtypes = [vp, i32, i32p, i32, vp, vp, vp, vp]
+    lib.cart_train_attention_bwd.argtypes = [vp, i32, i32p, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.cart_restore_cartridge.argtypes = [vp, i32, vp, vp, vp]
     lib.cart_request_reserve.argtypes = [vp, i32, i32, vp]
     lib.cart_append_kv.argtypes = [vp, i32, i32p, i32, vp, vp, vp]
@@ -275,6 +277,20 @@ def cart_evict_cartridge(ctx: int, cid: int) -> None:
 def cart_restore_cartridge(ctx: int, cid: int, k, v, stream=None) -> None:
     _check(load_library().cart_restore_cartridge(ctx, int(cid), _ptr(k), _ptr(v), _stream(stream)),
            "cart_restore_cartridge", ctx)
+
+
+def cart_train_attention_fwd(ctx: int, layer: int, convs, q, out, lse, stream=None) -> None:
+    arr, n = _reqs(convs)
+    _check(load_library().cart_train_attention_fwd(ctx, int(layer), arr, n, _ptr(q), _ptr(out), _ptr(lse), _stream(stream)),
+           "cart_train_attention_fwd", ctx)
+
+
+def cart_train_attention_bwd(ctx: int, layer: int, convs, q, out, lse, dout, delta, dq, dk, dv, dzk=None, dzv=None,
+                             stream=None) -> None:
+    arr, n = _reqs(convs)
+    _check(load_library().cart_train_attention_bwd(ctx, int(layer), arr, n, _ptr(q), _ptr(out), _ptr(lse), _ptr(dout),
+                                                   _ptr(delta), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dzk), _ptr(dzv),
+                                                   _stream(stream)), "cart_train_attention_bwd", ctx)
 
 
 def cart_request_reserve(ctx: int, req: int, suffix_capacity: int, stream=None) -> None:

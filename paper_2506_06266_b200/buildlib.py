@@ -10,7 +10,7 @@ _ROOT = os.path.dirname(_PKG)
 CSRC = os.path.join(_PKG, "csrc")
 INCLUDE = os.path.join(_ROOT, "include")
 LIB = os.path.join(_PKG, "libcart.so")
-SOURCES = ["cart_kernels.cu", "cart_shared.cu", "cart_noalloc.cu", "cart_api.cc", "cart_plan.cc"]
+SOURCES = ["cart_kernels.cu", "cart_shared.cu", "cart_train.cu", "cart_noalloc.cu", "cart_api.cc", "cart_plan.cc"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "-cudart", "static"]
 

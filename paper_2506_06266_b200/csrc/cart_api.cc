@@ -156,6 +156,7 @@ struct cart_ctx {
     uint64_t n_rows = 0;
     alignas(64) CUtensorMap tmap;
     alignas(64) CUtensorMap tmap_edge;
+    void *encode_fn = nullptr;  // cuTensorMapEncodeTiled
     std::vector<FreeBlock> free_list;
     std::vector<Cartridge> carts;
     std::vector<Request> reqs;
@@ -300,17 +301,18 @@ int32_t evicted_part(const cart_ctx *ctx, const Request &r)
     return -1;
 }
 
+typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                             const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                             CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
 cart_status encode_tensor_map(cart_ctx *ctx)
 {
-    typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                 const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
-                                 CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
-                                 CUtensorMapFloatOOBfill);
     void *fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
     CART_CUDA(ctx, cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
     if (!fn || qres != cudaDriverEntryPointSuccess)
         return fail(ctx, CART_ERR_CUDA, "the driver does not provide cuTensorMapEncodeTiled");
+    ctx->encode_fn = fn;
     // The whole arena as a matrix of rows of 128 bf16; a KV tile is 64 consecutive rows, fetched as
     // two boxes of 64 rows x 64 elements (128 bytes, the widest row a 128-byte swizzle allows).
     const cuuint64_t gdim[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)ctx->n_rows};
@@ -403,7 +405,9 @@ cart_status cart_create(const cart_config *cfg, cart_ctx **out)
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, cfg->device);
     if (e != cudaSuccess || sms < 1) return bail(CART_ERR_CUDA);
     ctx->n_cta = std::min(sms, kMaxCta);
-    if (prepare_kernels() != cudaSuccess || prepare_shared_kernel() != cudaSuccess) return bail(CART_ERR_CUDA);
+    if (prepare_kernels() != cudaSuccess || prepare_shared_kernel() != cudaSuccess ||
+        prepare_train_kernels() != cudaSuccess)
+        return bail(CART_ERR_CUDA);
     if (encode_tensor_map(ctx) != CART_OK) return bail(CART_ERR_CUDA);
     for (int i = 0; i < kPlanSlots; ++i) {
         PlanSlot &sl = ctx->slots[i];
@@ -954,16 +958,28 @@ namespace {
 
 // Decode attention for a batch; with k_new / v_new non-null the stream kernel first writes each
 // request's new token at position len - 1 of its suffix (the host lengths already count it).
-// Prefill mode (n_new > 0): reqs[0] is one request, and the batch is its last n_new suffix tokens as
-// n_new query rows; row i attends over the Cartridge(s) and the suffix up to and including its own
-// token (Eq. 1 for the rows of the new block).  The rows are planned like n_new requests that share the
-// Cartridge(s) and, group by group, the part of the suffix before the group's first token, so those go
-// through the shared-segment kernel.
+// Prefill mode (n_pre > 0): reqs[0 .. n_pre) are requests, and the batch is, request after request, the last
+// n_new_list[c] suffix tokens of request c as query rows; a row attends over the Cartridge(s) and the suffix up
+// to and including its own token (Eq. 1 for the rows of the new block).  The rows are planned like requests
+// that share the Cartridge(s) and, group by group, the part of the suffix before the group's first token, so
+// those go through the shared-segment kernel.  (One request: prefill of a user's message.  Many requests
+// that are whole conversations over one Cartridge: the forward of training-time attention.)
 cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int32_t n_reqs, const void *q,
-                        void *out, float *lse, const void *k_new, const void *v_new, void *stream, int32_t n_new = 0)
+                        void *out, float *lse, const void *k_new, const void *v_new, void *stream,
+                        const int32_t *n_new_list = nullptr, int32_t n_pre = 0)
 {
-    const bool prefill = n_new > 0;
-    if (prefill) n_reqs = n_new;
+    const bool prefill = n_pre > 0;
+    if (prefill) {
+        int64_t rows = 0;
+        for (int32_t c = 0; c < n_pre; ++c) {
+            if (n_new_list[c] < 1) return fail(ctx, CART_ERR_INVALID_ARG, "prefill: n_new < 1");
+            rows += n_new_list[c];
+        }
+        if (rows > ctx->cfg.max_requests)
+            return fail(ctx, CART_ERR_CAPACITY, "prefill: %lld rows exceed max_requests %d", (long long)rows,
+                        ctx->cfg.max_requests);
+        n_reqs = (int32_t)rows;
+    }
     if (!reqs || n_reqs < 1 || !aligned16(q) || !aligned16(out) || (lse && (reinterpret_cast<uintptr_t>(lse) & 3u)))
         return fail(ctx, CART_ERR_INVALID_ARG, "decode: null/misaligned pointer or empty batch");
     if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, CART_ERR_BAD_HANDLE, "decode: layer out of range");
@@ -979,18 +995,18 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
     std::vector<int32_t> &cur_len = ctx->len_tmp;
     key.clear();
     cur_len.clear();
-    if (prefill) {
-        Request *r = get_req(ctx, reqs[0]);
+    for (int32_t c = 0; c < n_pre; ++c) {
+        Request *r = get_req(ctx, reqs[c]);
         if (!r) return fail(ctx, CART_ERR_BAD_HANDLE, "prefill: not an open request");
         if (r->evicted) return fail(ctx, CART_ERR_EVICTED, "prefill: the request is swapped out");
         if (evicted_part(ctx, *r) >= 0)
             return fail(ctx, CART_ERR_EVICTED, "prefill: Cartridge %d is swapped out", evicted_part(ctx, *r));
-        if (r->len[(size_t)layer] < n_new)
+        if (r->len[(size_t)layer] < n_new_list[c])
             return fail(ctx, CART_ERR_INVALID_ARG, "prefill: the suffix holds %d tokens, fewer than n_new = %d",
-                        r->len[(size_t)layer], n_new);
-        key.push_back((uint32_t)reqs[0]);
+                        r->len[(size_t)layer], n_new_list[c]);
+        key.push_back((uint32_t)reqs[c]);
         key.push_back((uint32_t)r->len[(size_t)layer]);
-        key.push_back((uint32_t)n_new);
+        key.push_back((uint32_t)n_new_list[c]);
     }
     for (int32_t i = 0; i < n_reqs && !prefill; ++i) {
         Request *r = get_req(ctx, reqs[i]);
@@ -1048,24 +1064,32 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
         // tiles, is visible to all of its rows: that is the group's shared head of the suffix, a
         // staircase that follows the causal diagonal, so a row streams fewer than 128 + 128 / G tokens
         // by itself.  A step is only taken if enough rows stand on it to be shared.
-        std::vector<int32_t> &head_of_group = ctx->head_tmp;
-        head_of_group.clear();
+        // row_of[i] = (request of row i, its index among the request's new tokens, its group's shared head)
+        struct RowOf { int32_t c, i, head; };
+        std::vector<RowOf> row_of;
         const int32_t rows_per_tile = 128 / ctx->group;
-        if (prefill && ctx->share_min_readers > 0 && n_new >= ctx->share_min_readers) {
-            const int32_t s_old = ctx->reqs[(size_t)reqs[0]].len[(size_t)layer] - n_new;
-            const int32_t n_groups = (n_new + rows_per_tile - 1) / rows_per_tile;
-            auto natural = [&](int32_t g) { return (s_old + g * rows_per_tile) / kShareTileTokens * kShareTileTokens; };
-            int32_t cur = natural(0);
-            for (int32_t g = 0; g < n_groups; ++g) {
-                const int32_t nat = natural(g);
-                if (nat != cur) {
-                    int32_t g2 = g;
-                    while (g2 < n_groups && natural(g2) == nat) ++g2;
-                    const int32_t rows = std::min(n_new, g2 * rows_per_tile) - g * rows_per_tile;
-                    if (rows >= ctx->share_min_readers) cur = nat;
+        for (int32_t c = 0; c < n_pre; ++c) {
+            const int32_t n_new = n_new_list[c];
+            std::vector<int32_t> &head_of_group = ctx->head_tmp;
+            head_of_group.clear();
+            if (ctx->share_min_readers > 0 && n_new >= ctx->share_min_readers) {
+                const int32_t s_old = ctx->reqs[(size_t)reqs[c]].len[(size_t)layer] - n_new;
+                const int32_t n_groups = (n_new + rows_per_tile - 1) / rows_per_tile;
+                auto natural = [&](int32_t g) { return (s_old + g * rows_per_tile) / kShareTileTokens * kShareTileTokens; };
+                int32_t cur = natural(0);
+                for (int32_t g = 0; g < n_groups; ++g) {
+                    const int32_t nat = natural(g);
+                    if (nat != cur) {
+                        int32_t g2 = g;
+                        while (g2 < n_groups && natural(g2) == nat) ++g2;
+                        const int32_t rows = std::min(n_new, g2 * rows_per_tile) - g * rows_per_tile;
+                        if (rows >= ctx->share_min_readers) cur = nat;
+                    }
+                    head_of_group.push_back(cur);
                 }
-                head_of_group.push_back(cur);
             }
+            for (int32_t i = 0; i < n_new; ++i)
+                row_of.push_back(RowOf{c, i, head_of_group.empty() ? 0 : head_of_group[(size_t)(i / rows_per_tile)]});
         }
         bool list_full = false;
         // describes the part of a paged suffix that starts at token `first` (a multiple of the page size)
@@ -1083,7 +1107,7 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
             sg->flags |= CART_SEG_PAGED;
         };
         for (int32_t i = 0; i < n_reqs; ++i) {
-            Request &r = ctx->reqs[(size_t)reqs[prefill ? 0 : i]];
+            Request &r = ctx->reqs[(size_t)reqs[prefill ? row_of[(size_t)i].c : i]];
             auto push_cart = [&](const Cartridge &c) {
                 cart_plan_seg sg;
                 sg.k_row = (uint32_t)c.k_row;
@@ -1103,9 +1127,9 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
             uint32_t first = 0;  // first suffix token of the segment
             if (prefill) {
                 // row i sees the suffix up to its own token; its group's shared head is a segment of its own
-                const int32_t s_old = len - n_new;
-                len = s_old + i + 1;
-                const int32_t head = head_of_group.empty() ? 0 : head_of_group[(size_t)(i / rows_per_tile)];
+                const int32_t s_old = len - n_new_list[row_of[(size_t)i].c];
+                len = s_old + row_of[(size_t)i].i + 1;
+                const int32_t head = row_of[(size_t)i].head;
                 if (head > 0) {
                     cart_plan_seg sg;
                     sg.k_row = (uint32_t)r.k_row;
@@ -1172,7 +1196,7 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
                                            cudaMemcpyHostToDevice, s));
         ns.key = key;
         ns.prefill = prefill;
-        ns.reqs.assign(reqs, reqs + (prefill ? 1 : n_reqs));
+        ns.reqs.assign(reqs, reqs + (prefill ? n_pre : n_reqs));
         ns.lens = cur_len;
         ns.epoch = ctx->epoch;
         ns.valid = true;
@@ -1291,7 +1315,7 @@ cart_status cart_prefill_attention(cart_ctx *ctx, int32_t layer, cart_req req, c
 {
     if (!ctx) return CART_ERR_INVALID_ARG;
     if (n_new < 1) return fail(ctx, CART_ERR_INVALID_ARG, "prefill: n_new < 1");
-    return decode_impl(ctx, layer, &req, 1, q, out, lse, nullptr, nullptr, stream, n_new);
+    return decode_impl(ctx, layer, &req, 1, q, out, lse, nullptr, nullptr, stream, &n_new, 1);
 }
 
 cart_status cart_decode_step(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int32_t n_reqs, const void *k_new,
@@ -1323,6 +1347,219 @@ cart_status cart_decode_step(cart_ctx *ctx, int32_t layer, const cart_req *reqs,
     if (st != CART_OK && ctx->launches == launches_before)
         for (int32_t i = 0; i < n_reqs; ++i) --ctx->reqs[(size_t)reqs[i]].len[(size_t)layer];
     return st;
+}
+
+}  // extern "C"
+
+namespace {
+
+// What the two training calls share: the conversations' lengths in `layer`, their common Cartridge (or none).
+struct TrainBatch {
+    std::vector<int32_t> len;   // tokens per conversation
+    std::vector<int32_t> cu;    // running sum, n_convs + 1 entries
+    int32_t T = 0;
+    const Cartridge *z = nullptr;
+};
+
+cart_status train_batch(cart_ctx *ctx, int32_t layer, const cart_req *convs, int32_t n_convs, TrainBatch *tb)
+{
+    if (!convs || n_convs < 1) return fail(ctx, CART_ERR_INVALID_ARG, "train: no conversations");
+    if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, CART_ERR_BAD_HANDLE, "train: layer out of range");
+    tb->cu.assign(1, 0);
+    int32_t cart = CART_NONE;
+    const uint64_t stamp = ++ctx->stamp;
+    for (int32_t c = 0; c < n_convs; ++c) {
+        Request *r = get_req(ctx, convs[c]);
+        if (!r) return fail(ctx, CART_ERR_BAD_HANDLE, "train: convs[%d] is not an open request", c);
+        if (r->stamp == stamp) return fail(ctx, CART_ERR_INVALID_ARG, "train: convs[%d] appears twice", c);
+        r->stamp = stamp;
+        if (r->evicted) return fail(ctx, CART_ERR_EVICTED, "train: convs[%d] is swapped out", c);
+        if (r->paged) return fail(ctx, CART_ERR_INVALID_ARG, "train: convs[%d] has a paged suffix", c);
+        if (c == 0) cart = r->cart;
+        if (r->cart != cart) return fail(ctx, CART_ERR_INVALID_ARG, "train: the conversations attend to different Cartridges");
+        const int32_t n = r->len[(size_t)layer];
+        if (n < 1) return fail(ctx, CART_ERR_EMPTY, "train: convs[%d] has no token in layer %d", c, layer);
+        tb->len.push_back(n);
+        tb->cu.push_back(tb->cu.back() + n);
+    }
+    tb->T = tb->cu.back();
+    if (tb->T > ctx->cfg.max_requests)
+        return fail(ctx, CART_ERR_CAPACITY, "train: %d tokens exceed max_requests %d", tb->T, ctx->cfg.max_requests);
+    if (cart != CART_NONE) {
+        const Cartridge &z = ctx->carts[(size_t)cart];
+        if (z.composed) return fail(ctx, CART_ERR_INVALID_ARG, "train: the Cartridge is a composition");
+        if (z.evicted) return fail(ctx, CART_ERR_EVICTED, "train: the Cartridge is swapped out");
+        tb->z = &z;
+    }
+    return CART_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+cart_status cart_train_attention_fwd(cart_ctx *ctx, int32_t layer, const cart_req *convs, int32_t n_convs, const void *q,
+                                     void *out, float *lse, void *stream)
+{
+    if (!ctx) return CART_ERR_INVALID_ARG;
+    if (!lse) return fail(ctx, CART_ERR_INVALID_ARG, "train: the forward must write lse");
+    TrainBatch tb;
+    const cart_status st = train_batch(ctx, layer, convs, n_convs, &tb);
+    if (st != CART_OK) return st;
+    // every conversation is a block of new tokens over an empty suffix: the rows of all conversations share Z
+    return decode_impl(ctx, layer, convs, n_convs, q, out, lse, nullptr, nullptr, stream, tb.len.data(), n_convs);
+}
+
+cart_status cart_train_attention_bwd(cart_ctx *ctx, int32_t layer, const cart_req *convs, int32_t n_convs, const void *q,
+                                     const void *out, const float *lse, const void *dout, float *delta, float *dq, float *dk,
+                                     float *dv, float *dzk, float *dzv, void *stream)
+{
+    if (!ctx) return CART_ERR_INVALID_ARG;
+    TrainBatch tb;
+    cart_status st = train_batch(ctx, layer, convs, n_convs, &tb);
+    if (st != CART_OK) return st;
+    if (!aligned16(q) || !aligned16(out) || !aligned16(dout) || !aligned16(dq) || !aligned16(dk) || !aligned16(dv) || !lse ||
+        !delta || (tb.z && (!aligned16(dzk) || !aligned16(dzv))))
+        return fail(ctx, CART_ERR_INVALID_ARG, "train: null/misaligned pointer");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int Hkv = ctx->cfg.n_kv_heads, Hq = ctx->cfg.n_q_heads, G = ctx->group;
+    const uint32_t tpt = 128u / (uint32_t)G;
+    const uint32_t T = (uint32_t)tb.T;
+    const uint32_t n_rt = (T + tpt - 1) / tpt;
+    const uint32_t p = tb.z ? (uint32_t)tb.z->p : 0u;
+
+    // ---- work items: Cartridge tiles first (long), then the conversations' own key tiles ------------
+    // They go through the next buffer of the plan ring (a decode plan kept there is dropped).
+    PlanSlot *cur = ctx->cur_slot >= 0 ? &ctx->slots[ctx->cur_slot] : nullptr;
+    if (cur && cur->valid) {
+        CART_CUDA(ctx, cudaEventRecord(cur->ev, cur->last_stream));
+        cur->ev_recorded = true;
+    }
+    const int next = (ctx->cur_slot + 1) % kPlanSlots;
+    PlanSlot &ns = ctx->slots[next];
+    if (ns.ev_recorded) {
+        CART_CUDA(ctx, cudaEventSynchronize(ns.ev));
+        ns.ev_recorded = false;
+    }
+    ns.valid = false;
+    TrainItem *items = reinterpret_cast<TrainItem *>(ns.host + ctx->lay.items_off);
+    const size_t items_cap = (size_t)ctx->lay.items_cap * sizeof(cart_work_item) / sizeof(TrainItem);
+    size_t n_items = 0;
+    const uint32_t z_tiles = (p + 127u) / 128u;
+    // a Cartridge tile's rows are divided among several blocks when there are fewer tiles than SMs
+    uint32_t nsplit = 1;
+    if (z_tiles > 0) nsplit = std::max<uint32_t>(1u, std::min<uint32_t>(n_rt, (uint32_t)ctx->n_cta / (z_tiles * (uint32_t)Hkv)));
+    bool full = false;
+    auto push = [&](const TrainItem &ti) {
+        if (n_items >= items_cap) { full = true; return; }
+        items[n_items++] = ti;
+    };
+    for (uint32_t zt = 0; zt < z_tiles; ++zt)
+        for (int g = 0; g < Hkv; ++g)
+            for (uint32_t sp = 0; sp < nsplit; ++sp) {
+                TrainItem ti{};
+                ti.k_row = (uint32_t)(tb.z->k_row + (uint64_t)g * p + zt * 128u);
+                ti.v_row = (uint32_t)(tb.z->v_row + (uint64_t)g * p + zt * 128u);
+                ti.layer_stride = (uint32_t)Hkv * p;
+                ti.n_keys = std::min(128u, p - zt * 128u);
+                ti.kv_head = (uint32_t)g;
+                ti.rt_begin = (uint32_t)((uint64_t)n_rt * sp / nsplit);
+                ti.rt_end = (uint32_t)((uint64_t)n_rt * (sp + 1) / nsplit);
+                if (ti.rt_end == ti.rt_begin) continue;
+                // blocks that add into the same rows of dq (the tiles of one KV head) start at different row tiles
+                ti.rt_first = ti.rt_begin + (zt * 5u) % (ti.rt_end - ti.rt_begin);
+                ti.key_tok0 = 0;
+                ti.tok_end = T;
+                ti.causal = 0;
+                ti.dst_row = (uint32_t)g * p + zt * 128u;
+                ti.dst_stride = 1;
+                ti.is_z = 1;
+                push(ti);
+            }
+    for (int32_t c = 0; c < n_convs; ++c) {
+        const Request &r = ctx->reqs[(size_t)convs[c]];
+        const uint32_t n = (uint32_t)tb.len[(size_t)c], t0 = (uint32_t)tb.cu[(size_t)c], t1 = (uint32_t)tb.cu[(size_t)c + 1];
+        for (uint32_t kc = 0; kc * 128u < n; ++kc)
+            for (int g = 0; g < Hkv; ++g) {
+                TrainItem ti{};
+                ti.k_row = (uint32_t)(r.k_row + (uint64_t)g * r.cap + kc * 128u);
+                ti.v_row = (uint32_t)(r.v_row + (uint64_t)g * r.cap + kc * 128u);
+                ti.layer_stride = (uint32_t)((uint64_t)Hkv * r.cap);
+                ti.n_keys = std::min(128u, n - kc * 128u);
+                ti.kv_head = (uint32_t)g;
+                ti.key_tok0 = t0 + kc * 128u;
+                ti.tok_end = t1;
+                ti.rt_begin = ti.key_tok0 / tpt;
+                ti.rt_end = (t1 + tpt - 1) / tpt;
+                ti.rt_first = ti.rt_begin;
+                ti.causal = 1;
+                ti.dst_row = ti.key_tok0 * (uint32_t)Hkv + (uint32_t)g;
+                ti.dst_stride = (uint32_t)Hkv;
+                ti.is_z = 0;
+                push(ti);
+            }
+    }
+    if (full) return fail(ctx, CART_ERR_CAPACITY, "train: more than %zu work items", items_cap);
+    uint8_t *dev_items = ns.dev + ctx->lay.items_off;
+    CART_CUDA(ctx, cudaMemcpyAsync(dev_items, items, n_items * sizeof(TrainItem), cudaMemcpyHostToDevice, s));
+    ns.last_stream = s;
+    ns.epoch = 0;
+    ctx->cur_slot = next;
+    CART_CUDA(ctx, cudaEventRecord(ns.ev, s));  // (recorded again below, after the kernels)
+    ns.ev_recorded = true;
+
+    // ---- q and dout as [T][Hq][128], fetched in boxes of 128 / G tokens x G heads x 64 dims -----------
+    alignas(64) CUtensorMap tmap_q, tmap_do;
+    {
+        const cuuint64_t gdim[3] = {(cuuint64_t)kHeadDim, (cuuint64_t)Hq, (cuuint64_t)T};
+        const cuuint64_t gstride[2] = {(cuuint64_t)kRowBytes, (cuuint64_t)Hq * kRowBytes};
+        const cuuint32_t box[3] = {64u, (cuuint32_t)G, (cuuint32_t)tpt};
+        const cuuint32_t estride[3] = {1u, 1u, 1u};
+        EncodeFn enc = reinterpret_cast<EncodeFn>(ctx->encode_fn);
+        CUresult r1 = enc(&tmap_q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(q), gdim, gstride, box, estride,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        CUresult r2 = enc(&tmap_do, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(dout), gdim, gstride, box, estride,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r1 != CUDA_SUCCESS || r2 != CUDA_SUCCESS)
+            return fail(ctx, CART_ERR_CUDA, "train: cuTensorMapEncodeTiled failed with code %d", (int)(r1 != CUDA_SUCCESS ? r1 : r2));
+    }
+    // ---- zero the outputs (they are accumulated into), D, then the kernel ----------------------------
+    CART_CUDA(ctx, cudaMemsetAsync(dq, 0, (size_t)T * Hq * kHeadDim * 4, s));
+    CART_CUDA(ctx, cudaMemsetAsync(dk, 0, (size_t)T * Hkv * kHeadDim * 4, s));
+    CART_CUDA(ctx, cudaMemsetAsync(dv, 0, (size_t)T * Hkv * kHeadDim * 4, s));
+    if (tb.z) {
+        CART_CUDA(ctx, cudaMemsetAsync(dzk, 0, (size_t)Hkv * p * kHeadDim * 4, s));
+        CART_CUDA(ctx, cudaMemsetAsync(dzv, 0, (size_t)Hkv * p * kHeadDim * 4, s));
+    }
+    TrainDeltaParams dpm;
+    dpm.out = out;
+    dpm.dout = dout;
+    dpm.delta = delta;
+    dpm.n_rows = (int32_t)(T * (uint32_t)Hq);
+    CART_CUDA(ctx, launch_train_delta(dpm, s));
+    ++ctx->launches;
+    TrainBwdParams bp;
+    bp.items = reinterpret_cast<const TrainItem *>(dev_items);
+    bp.lse = lse;
+    bp.delta = delta;
+    bp.dq = dq;
+    bp.dk = dk;
+    bp.dv = dv;
+    bp.dzk = dzk;
+    bp.dzv = dzv;
+    bp.status = reinterpret_cast<uint32_t *>(static_cast<uint8_t *>(ctx->cfg.arena) + ctx->lay.status_off);
+    bp.layer = layer;
+    bp.group = G;
+    bp.n_q_heads = Hq;
+    bp.n_tokens = (int32_t)T;
+    bp.scale = ctx->scale;
+    CART_CUDA(ctx, launch_train_bwd(ctx->tmap, tmap_q, tmap_do, bp, (int)n_items, s));
+    ++ctx->launches;
+    CART_CUDA(ctx, cudaEventRecord(ns.ev, s));
+    ns.ev_recorded = true;
+    return CART_OK;
 }
 
 cart_status cart_suffix_len(cart_ctx *ctx, cart_req req, int32_t layer, int32_t *out_len)

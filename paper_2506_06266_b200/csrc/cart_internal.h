@@ -118,6 +118,51 @@ struct ExtendParams {
     int32_t n_kv_heads;
 };
 
+// ---- training-time attention (backward) ---------------------------------------------------------
+// One unit of the backward kernel's work: a tile of up to 128 keys of one KV head -- of the shared Cartridge
+// or of a conversation -- against a range of row tiles.  Rows are (token, head of the group) pairs in
+// token-major order; a row tile holds the 128 / G tokens [rt * tpt, (rt + 1) * tpt) of the packed batch.
+struct TrainItem {
+    uint32_t k_row;       // arena row of the tile's first key in layer 0 (KV head applied); values at v_row
+    uint32_t v_row;
+    uint32_t layer_stride;
+    uint32_t n_keys;      // valid keys in the tile (1 .. 128)
+    uint32_t kv_head;
+    uint32_t rt_begin;    // row tiles [rt_begin, rt_end)
+    uint32_t rt_end;
+    uint32_t rt_first;    // the tile the loop starts with (it wraps around): items that share rows start apart
+    uint32_t key_tok0;    // conversation tile: packed token index of key 0; Cartridge tile: 0
+    uint32_t tok_end;     // conversation tile: one past the conversation's last token; Cartridge tile: T
+    uint32_t causal;      // 1: key j is seen by rows of tokens >= key_tok0 + j only (conversation tile)
+    uint32_t dst_row;     // row of key 0 in the gradient tensors: Cartridge [Hkv][p] -> kv_head * p + key;
+                          // conversation [T][Hkv] -> token * Hkv + kv_head (dst_stride = Hkv rows between keys)
+    uint32_t dst_stride;
+    uint32_t is_z;        // 1: gradients go to dzk / dzv, else to dk / dv
+    uint32_t pad[2];
+};
+
+struct TrainBwdParams {
+    const TrainItem *items;
+    const float *lse;     // fp32 [T][Hq], natural log (forward)
+    const float *delta;   // fp32 [T][Hq]: <dout, out> per row
+    float *dq;            // fp32 [T][Hq][128]
+    float *dk, *dv;       // fp32 [T][Hkv][128]
+    float *dzk, *dzv;     // fp32 [Hkv][p][128]
+    uint32_t *status;
+    int32_t layer;
+    int32_t group;        // G
+    int32_t n_q_heads;
+    int32_t n_tokens;     // T
+    float scale;          // softmax scale
+};
+
+struct TrainDeltaParams {
+    const void *out;      // bf16 [T][Hq][128]
+    const void *dout;     // bf16 [T][Hq][128]
+    float *delta;         // fp32 [T][Hq]
+    int32_t n_rows;       // T * Hq
+};
+
 // Launch configuration shared by the decode kernels: the kernel may start (become resident, run its
 // prologue) before the kernel before it on the stream has finished; it orders itself with
 // griddepcontrol.wait.
@@ -148,6 +193,12 @@ cudaError_t launch_shared(const CUtensorMap &tmap, const SharedParams &p, int gr
 cudaError_t launch_merge(const MergeParams &p, int n_merges, cudaStream_t s);
 cudaError_t launch_append(const AppendParams &p, cudaStream_t s);
 cudaError_t launch_extend(const ExtendParams &p, cudaStream_t s);
+cudaError_t prepare_train_kernels();
+cudaError_t launch_train_delta(const TrainDeltaParams &p, cudaStream_t s);
+// tmap: the arena (boxes of 64 rows x 64 elements); tmap_q / tmap_do: q and dout as [T][Hq][128] in boxes of
+// 128 / G tokens x G heads x 64 elements
+cudaError_t launch_train_bwd(const CUtensorMap &tmap, const CUtensorMap &tmap_q, const CUtensorMap &tmap_do,
+                             const TrainBwdParams &p, int n_items, cudaStream_t s);
 
 }  // namespace cart
 #endif
