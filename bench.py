@@ -47,7 +47,7 @@ WORKLOADS = {
 SIDE_WORKLOADS = ["c1", "c3", "c4", "c5_cartridge", "c5_full"]   # reported next to the headline workload
 TIMED_BLOCKS = 5                                                  # App. A.3: 3 warm-up runs, 5 timed runs
 
-KERNEL_SOURCES = ["cart_kernels.cu", "cart_shared.cu", "cart_device.cuh", "cart_internal.h"]
+KERNEL_SOURCES = ["cart_kernels.cu", "cart_shared.cu", "cart_train.cu", "cart_tc.cuh", "cart_device.cuh", "cart_internal.h"]
 TRAFFIC_TABLE = os.path.join(ROOT, "profiles", "dram_traffic.txt")
 
 
@@ -561,6 +561,90 @@ def run_prefill(args):
                       "gpu_launches": int(launches)}))
 
 
+def run_train(args):
+    """Side measurement (its own JSON line, not the headline): one layer of training-time attention over a shared
+    trainable Cartridge -- args.train conversations of 64 .. 512 tokens (seeded) over a Cartridge of the chosen
+    workload's shape, cart_train_attention_fwd and cart_train_attention_bwd timed separately."""
+    from paper_2506_06266_b200 import binding
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    w0 = WORKLOADS[args.workload]()
+    Hq, Hkv, p = w0.n_q_heads, w0.n_kv_heads, w0.p
+    lens = [int(x) for x in np.random.default_rng(w0.seed + 5).integers(64, 513, size=args.train)]
+    T = int(sum(lens))
+    cu = np.concatenate([[0], np.cumsum(lens)])
+    stream = torch.cuda.current_stream(dev)
+    cfg = binding.make_config(1, Hq, Hkv, T, 4, device=0, softmax_scale=w0.scale)
+    per_tok = 2 * Hkv * 256
+    arena_bytes = binding.cart_scratch_bytes(cfg) + (p + sum(-(-n // 64) * 64 for n in lens) + 128) * per_tok + 4096
+    arena = torch.empty(arena_bytes, dtype=torch.uint8, device=dev)
+    cfg.arena, cfg.arena_bytes = arena.data_ptr(), arena_bytes
+    ctx = binding.cart_create(cfg)
+    zk = synth.normal_bf16((1, Hkv, p, 128), w0.seed + 71, dev)
+    zv = synth.normal_bf16((1, Hkv, p, 128), w0.seed + 72, dev)
+    cart = binding.cart_register_cartridge(ctx, zk, zv, p, stream)
+    k = synth.normal_bf16((T, Hkv, 128), w0.seed + 73, dev)
+    v = synth.normal_bf16((T, Hkv, 128), w0.seed + 74, dev)
+    q = synth.normal_bf16((T, Hq, 128), w0.seed + 75, dev)
+    dout = synth.normal_bf16((T, Hq, 128), w0.seed + 76, dev)
+    convs = []
+    for c, n in enumerate(lens):
+        r = binding.cart_request_open(ctx, cart, n)
+        binding.cart_extend_kv(ctx, 0, r, k[cu[c]:cu[c + 1]], v[cu[c]:cu[c + 1]], n, stream)
+        convs.append(r)
+    convs = binding.ReqList(convs)
+    out = torch.empty_like(q)
+    lse = torch.empty((T, Hq), dtype=torch.float32, device=dev)
+    delta = torch.empty_like(lse)
+    dq = torch.empty((T, Hq, 128), dtype=torch.float32, device=dev)
+    dk = torch.empty((T, Hkv, 128), dtype=torch.float32, device=dev)
+    dv = torch.empty_like(dk)
+    dzk = torch.empty((Hkv, p, 128), dtype=torch.float32, device=dev)
+    dzv = torch.empty_like(dzk)
+
+    def fwd():
+        binding.cart_train_attention_fwd(ctx, 0, convs, q, out, lse, stream)
+
+    def bwd():
+        binding.cart_train_attention_bwd(ctx, 0, convs, q, out, lse, dout, delta, dq, dk, dv, dzk, dzv, stream)
+
+    times = {}
+    n0 = binding.cart_launch_count(ctx)
+    for name, fn in (("fwd", fwd), ("bwd", bwd)):
+        for _ in range(args.warmup):
+            fn()
+        binding.cart_sync_status(ctx, stream)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(args.steps):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize(dev)
+        binding.cart_sync_status(ctx, stream)
+        times[name] = e0.elapsed_time(e1) / args.steps
+    launches = binding.cart_launch_count(ctx) - n0
+    binding.cart_destroy(ctx)
+    # a token of a conversation sees the Cartridge and its own conversation up to itself: 2 products forward, 5 backward
+    pairs = float(T) * p + sum(n * (n + 1) / 2.0 for n in lens)
+    flops_fwd = 4.0 * Hq * 128 * pairs
+    flops_bwd = 10.0 * Hq * 128 * pairs
+    _, tf_burst, tf_sustained, kind = measured_peaks()
+    tf = {"fwd": flops_fwd / (times["fwd"] * 1e-3) / 1e12, "bwd": flops_bwd / (times["bwd"] * 1e-3) / 1e12}
+    total_ms = times["fwd"] + times["bwd"]
+    print(json.dumps({"metric": "train_attention_tokens_per_s", "value": round(T / (total_ms * 1e-3), 1),
+                      "unit": "tokens/s", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
+                      "ms_per_step": round(total_ms, 4), "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
+                      "config": {"workload": "one layer of training attention, %d conversations of 64..512 tokens over a "
+                                             "Cartridge of %s shape" % (args.train, w0.name),
+                                 "tokens": T, "cartridge_tokens": p, "q_heads": Hq, "kv_heads": Hkv,
+                                 "fwd_ms": round(times["fwd"], 4), "bwd_ms": round(times["bwd"], 4),
+                                 "fwd_tflops": round(tf["fwd"], 1), "bwd_tflops": round(tf["bwd"], 1)},
+                      "roofline": {"bound": "tensor", "kernel": "cart_train_bwd_kernel", "achieved": round(tf["bwd"], 1),
+                                   "peak": tf_sustained, "unit": "TFLOP/s", "frac": round(tf["bwd"] / tf_sustained, 4),
+                                   "peak_kind": "of %s (sustained bf16)" % kind, "traffic": None},
+                      "gpu_launches": int(launches)}))
+
+
 def run_reference(args):
     """The reference arm is the CPU oracle, as it stands, timed on the host cores."""
     rank = int(os.environ.get("RANK", "0"))
@@ -637,6 +721,9 @@ def main():
     ap.add_argument("--prefill", type=int, default=0,
                     help="side measurement: prefill attention of a message of this many tokens over one Cartridge "
                          "of the workload's shape (prints its own JSON line)")
+    ap.add_argument("--train", type=int, default=0,
+                    help="side measurement: training-time attention (forward and backward) of this many conversations "
+                         "over one Cartridge of the workload's shape, one layer")
     ap.add_argument("--paged", action="store_true",
                     help="the requests' suffixes are stored in pages of 64 tokens (cart_request_open_paged)")
     ap.add_argument("--unfused", action="store_true",
@@ -659,6 +746,8 @@ def main():
         args.warmup = 3
     if args.prefill > 0:
         run_prefill(args)
+    elif args.train > 0:
+        run_train(args)
     elif args.impl == "reference":
         run_reference(args)
     else:

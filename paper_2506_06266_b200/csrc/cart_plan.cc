@@ -38,6 +38,7 @@ struct Balancer {
     uint64_t c = 0;        // block being filled
     uint64_t acc = 0;      // weight block c holds
     uint64_t budget = 0;
+    bool whole = false;    // every block takes exactly one whole group (small batches: see the stream part)
 
     Balancer(uint64_t blocks, uint64_t unit_cost, uint64_t tiles, uint64_t groups)
         : C(blocks), A(unit_cost), tiles_left(tiles), groups_left(groups) { open(false); }
@@ -53,6 +54,10 @@ struct Balancer {
     // first if the current one cannot pay for another unit.  `fresh`: nothing of the group was taken yet.
     uint64_t take(uint64_t rem, bool fresh)
     {
+        if (whole) {
+            if (acc > 0 && c + 1 < C) { ++c; open(false); }
+            return rem;
+        }
         for (;;) {
             const uint64_t paid = acc + A;
             uint64_t room = budget > paid ? budget - paid : 0;
@@ -68,6 +73,7 @@ struct Balancer {
         acc += A + t;
         tiles_left -= t;
         if (fresh) --groups_left;
+        if (whole) return;
         if (acc >= budget && c + 1 < C) { ++c; open(more); }
     }
     bool block_has_work() const { return acc > 0; }
@@ -344,7 +350,24 @@ extern "C" cart_status cart_plan_build_shared(const cart_plan_seg *segs, const i
         }
         if (any) rgs_with_tiles += (uint64_t)n_kv_heads;
     }
-    Balancer bal(C ? C : 1, A, W, rgs_with_tiles);
+    // Small batches are bound by latencies, not by bandwidth: when every row group can have a block of its own and
+    // an even split would leave a block only a few tiles, a row group is not cut at all -- a block streams it whole
+    // and writes the result itself (or one partial, if part of the cache is shared), which saves the partials,
+    // the arrival tickets and the merge, a chain of dependent memory round trips longer than the tiles it spares.
+    uint64_t longest_rg = 0;
+    for (int32_t i = 0; i < n_reqs; ++i) {
+        uint64_t t = 0;
+        for (int32_t sgi = seg_begin[i]; sgi < seg_begin[i + 1]; ++sgi) {
+            uint32_t t0, nt;
+            stream_part(sgi, &t0, &nt);
+            t += (nt + T - 1) / T;
+        }
+        longest_rg = std::max(longest_rg, t);
+    }
+    const bool whole = A > 0 && rgs_with_tiles > 0 && rgs_with_tiles <= n_cta_stream && W <= 4 * n_cta_stream &&
+                       longest_rg <= 24;
+    Balancer bal(whole ? rgs_with_tiles : (C ? C : 1), A, W, rgs_with_tiles);
+    bal.whole = whole;
     o->cta_begin[0] = 0;
 
     for (int32_t i = 0; i < n_reqs; ++i) {

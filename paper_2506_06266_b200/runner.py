@@ -138,13 +138,20 @@ class LoadedWorkload:
         (cart_decode_step) or, with fused=False, as cart_append_kv followed by cart_decode_attention.
         q, out: [L][B][Hq][D]; k_new, v_new: [L][B][Hkv][D]; lse: [L][B][Hq] or None."""
         ctx, rl, s = self.ctx, self.req_list, self.stream
+        # (addresses instead of per-layer tensor views: slicing five tensors costs more host time than a small
+        #  batch's kernel takes)
+        qp, op, kp, vp = q.data_ptr(), out.data_ptr(), k_new.data_ptr(), v_new.data_ptr()
+        qs, ks = q.stride(0) * q.element_size(), k_new.stride(0) * k_new.element_size()
+        lp = 0 if lse is None else lse.data_ptr()
+        lstride = 0 if lse is None else lse.stride(0) * lse.element_size()
         for layer in (range(self.w.n_layers) if layers is None else layers):
-            ls = None if lse is None else lse[layer]
+            ls = None if lse is None else lp + layer * lstride
             if fused:
-                binding.cart_decode_step(ctx, layer, rl, k_new[layer], v_new[layer], q[layer], out[layer], ls, s)
+                binding.cart_decode_step(ctx, layer, rl, kp + layer * ks, vp + layer * ks, qp + layer * qs,
+                                         op + layer * qs, ls, s)
             else:
-                binding.cart_append_kv(ctx, layer, rl, k_new[layer], v_new[layer], s)
-                binding.cart_decode_attention(ctx, layer, rl, q[layer], out[layer], ls, s)
+                binding.cart_append_kv(ctx, layer, rl, kp + layer * ks, vp + layer * ks, s)
+                binding.cart_decode_attention(ctx, layer, rl, qp + layer * qs, op + layer * qs, ls, s)
         self.appended += 1
 
     def close(self) -> None:

@@ -75,6 +75,11 @@ def check(segs, Hkv, G, n_cta, tile=64, share_min=4, share_tile=128, slots_cap=1
     assert sum(per_cta) == plan["total_tiles"] and all(t == 0 for t in per_cta[used:])
     if used and piece_cost == 0:
         assert max(per_cta[:used]) - min(per_cta[:used]) <= 1 and min(per_cta[:used]) >= 1
+    elif used and used == len(pieces) and all(len(v) == 1 for v in pieces.values()) and \
+            all(n == 1 for n in per_cta_pieces[:used]):
+        # a small batch: every row group has a block of its own and is streamed whole (no cut, no stream-side merge),
+        # which the planner only does when the blocks stay short
+        assert max(per_cta[:used]) <= 24 and sum(per_cta) <= 4 * n_cta and min(per_cta[:used]) >= 1
     elif used:
         # balanced by weight = tiles + piece_cost * pieces: no block is more than one piece and one tile
         # above the even share (the last block takes what is left and may be lighter)
