@@ -1509,7 +1509,7 @@ cart_status cart_train_attention_bwd(cart_ctx *ctx, int32_t layer, const cart_re
     ns.ev_recorded = true;
 
     // ---- q and dout as [T][Hq][128], fetched in boxes of 128 / G tokens x G heads x 64 dims -----------
-    alignas(64) CUtensorMap tmap_q, tmap_do;
+    alignas(64) CUtensorMap tmap_q, tmap_do, tmap_dq;
     {
         const cuuint64_t gdim[3] = {(cuuint64_t)kHeadDim, (cuuint64_t)Hq, (cuuint64_t)T};
         const cuuint64_t gstride[2] = {(cuuint64_t)kRowBytes, (cuuint64_t)Hq * kRowBytes};
@@ -1522,8 +1522,15 @@ cart_status cart_train_attention_bwd(cart_ctx *ctx, int32_t layer, const cart_re
         CUresult r2 = enc(&tmap_do, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(dout), gdim, gstride, box, estride,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-        if (r1 != CUDA_SUCCESS || r2 != CUDA_SUCCESS)
-            return fail(ctx, CART_ERR_CUDA, "train: cuTensorMapEncodeTiled failed with code %d", (int)(r1 != CUDA_SUCCESS ? r1 : r2));
+        // dq as fp32 [T][Hq][128]: boxes of 128 / G tokens x G heads x 32 dims (128 bytes, the swizzle's span)
+        const cuuint64_t dstride[2] = {(cuuint64_t)kHeadDim * 4, (cuuint64_t)Hq * kHeadDim * 4};
+        const cuuint32_t dbox[3] = {32u, (cuuint32_t)G, (cuuint32_t)tpt};
+        CUresult r3 = enc(&tmap_dq, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, dq, gdim, dstride, dbox, estride,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r1 != CUDA_SUCCESS || r2 != CUDA_SUCCESS || r3 != CUDA_SUCCESS)
+            return fail(ctx, CART_ERR_CUDA, "train: cuTensorMapEncodeTiled failed with code %d",
+                        (int)(r1 != CUDA_SUCCESS ? r1 : r2 != CUDA_SUCCESS ? r2 : r3));
     }
     // ---- zero the outputs (they are accumulated into), D, then the kernel ----------------------------
     CART_CUDA(ctx, cudaMemsetAsync(dq, 0, (size_t)T * Hq * kHeadDim * 4, s));
@@ -1555,7 +1562,7 @@ cart_status cart_train_attention_bwd(cart_ctx *ctx, int32_t layer, const cart_re
     bp.n_q_heads = Hq;
     bp.n_tokens = (int32_t)T;
     bp.scale = ctx->scale;
-    CART_CUDA(ctx, launch_train_bwd(ctx->tmap, tmap_q, tmap_do, bp, (int)n_items, s));
+    CART_CUDA(ctx, launch_train_bwd(ctx->tmap, tmap_q, tmap_do, tmap_dq, bp, (int)n_items, s));
     ++ctx->launches;
     CART_CUDA(ctx, cudaEventRecord(ns.ev, s));
     ns.ev_recorded = true;

@@ -197,8 +197,9 @@ cudaError_t prepare_train_kernels();
 cudaError_t launch_train_delta(const TrainDeltaParams &p, cudaStream_t s);
 // tmap: the arena (boxes of 64 rows x 64 elements); tmap_q / tmap_do: q and dout as [T][Hq][128] in boxes of
 // 128 / G tokens x G heads x 64 elements
+// tmap_dq: dq as fp32 [T][Hq][128] in boxes of 128 / G tokens x G heads x 32 elements (written by bulk reductions)
 cudaError_t launch_train_bwd(const CUtensorMap &tmap, const CUtensorMap &tmap_q, const CUtensorMap &tmap_do,
-                             const TrainBwdParams &p, int n_items, cudaStream_t s);
+                             const CUtensorMap &tmap_dq, const TrainBwdParams &p, int n_items, cudaStream_t s);
 
 }  // namespace cart
 #endif

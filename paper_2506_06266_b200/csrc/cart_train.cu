@@ -26,13 +26,14 @@
 //     dV  += P^T dO       (A operand from tensor memory, dO tile as the MN-major B operand)
 //     dK  += dS^T Q
 //     dQ_part = dS K      (dS from shared memory as an MN-major A operand, into the columns S^T held)
-//     the same threads, now as row owners, add dQ_part to dq with vector atomics.
+//     the same threads, now as row owners, put dQ_part into shared memory (the row tile's Q and dO stage, spent by
+//     then) and a bulk tensor reduction adds it into dq.
 //
 // Tensor memory: S^T / P^T / dQ_part, dP^T / dS^T, the dV accumulator, the dK accumulator: 4 x 128 columns.
 // The tensor pipe executes one thread's instructions in the order of issue, which orders dV += P^T dO before the
-// product that overwrites P^T.  All gradients are accumulated into zero-initialised fp32 tensors with atomic adds
-// (several blocks share a Cartridge tile when its rows are split, every key tile adds into dq), so the last bits
-// depend on the order of arrival.  Every wait is bounded, as in the other kernels.
+// product that overwrites P^T.  All gradients are accumulated into zero-initialised fp32 tensors by additions in the
+// memory system (every key tile adds into dq; several blocks share a Cartridge tile when its rows are split), so the
+// last bits depend on the order of arrival.  Every wait is bounded, as in the other kernels.
 #include <cuda_bf16.h>
 
 #include "cart_device.cuh"
@@ -45,8 +46,8 @@ namespace {
 constexpr uint32_t kTBlock = 128u * 128u;         // 128 rows x 128 bytes: one swizzled block (64 bf16 wide)
 constexpr uint32_t kTTile = 2u * kTBlock;         // 128 x 128 bf16
 constexpr int kTrThreads = 384;                   // utility warpgroup (producer, MMA, 2 idle) + 2 compute warpgroups
-constexpr int kTrRegsUtility = 40;
-constexpr int kTrRegsCompute = 232;
+constexpr int kTrRegsUtility = 96;
+constexpr int kTrRegsCompute = 176;
 constexpr uint32_t kTrTmemCols = 512;
 constexpr uint32_t kTmS = 0, kTmDP = 128, kTmDV = 256, kTmDK = 384;
 
@@ -59,14 +60,16 @@ constexpr uint32_t kTrOffLD = kTrOffDS + kTTile;        // [stage][128] (lse * l
 constexpr uint32_t kTrOffTok = kTrOffLD + 2u * 128u * 8u;  // [128] token offset of row i inside its row tile (i / G)
 constexpr uint32_t kTrOffBar = kTrOffTok + 128u;
 constexpr uint32_t kTrOffMisc = kTrOffBar + 16u * 8u;   // tensor-memory address, abort flag
-constexpr uint32_t kTrSmemUsed = kTrOffMisc + 16u;
+constexpr uint32_t kTrOffItem = kTrOffMisc + 16u;       // the block's work item (read by every warp, all through the loop)
+constexpr uint32_t kTrSmemUsed = kTrOffItem + 64u;
+static_assert(sizeof(TrainItem) == 64, "the work item's copy in shared memory is 64 bytes");
 constexpr uint32_t kTrSmemBytes = 232448u;              // all of it: what is left over is the room to align the base
 static_assert(kTrSmemUsed <= kTrSmemBytes, "shared memory budget of one sm_100 block exceeded");
 
 enum TrBar : int {
     kTbKV = 0,       // TMA -> all: the key tile's K and V are in shared memory
     kTbQFull = 1,    // [2] TMA + producer warp (2 arrivals) -> MMA, compute: a row tile's Q, dO, lse and D
-    kTbQEmpty = 3,   // [2] MMA (commit) -> producer
+    kTbQEmpty = 3,   // [2] compute (2 arrivals: one per warpgroup, once its dq reduction has left the stage) -> producer
     kTbSFull = 5,    // MMA (commit) -> compute: S^T and dP^T
     kTbPReady = 6,   // compute (8 arrivals) -> MMA: P^T, dS^T in tensor memory, dS in shared memory
     kTbDQFull = 7,   // MMA (commit) -> compute: dQ_part (and the accumulators up to this row tile)
@@ -85,6 +88,15 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tma
         "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(z), "r"(bar)
         : "memory");
+}
+
+// Adds a box of fp32 from shared memory into global memory (dq as [T][Hq][128], boxes of 128 / G tokens x G heads x
+// 32 dims): the additions happen in the memory system, one instruction per box instead of one atomic per 16 bytes.
+__device__ __forceinline__ void tma_reduce_add_3d(const CUtensorMap *tmap, uint32_t src, int32_t x, int32_t y, int32_t z)
+{
+    asm volatile("cp.reduce.async.bulk.tensor.3d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2, %3}], [%4];"
+                 ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(z), "r"(src)
+                 : "memory");
 }
 
 // D_i = <dout_i, out_i> per query row: one warp per row of 128 bf16 pairs.
@@ -107,7 +119,8 @@ __global__ void __launch_bounds__(256) cart_train_delta_kernel(const TrainDeltaP
 
 __global__ void __launch_bounds__(kTrThreads, 1)
 cart_train_bwd_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ CUtensorMap tmap_q,
-                      const __grid_constant__ CUtensorMap tmap_do, const TrainBwdParams p)
+                      const __grid_constant__ CUtensorMap tmap_do, const __grid_constant__ CUtensorMap tmap_dq,
+                      const TrainBwdParams p)
 {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -123,7 +136,13 @@ cart_train_bwd_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_con
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
 
-    const TrainItem it = p.items[blockIdx.x];
+    // The item lives in shared memory: the warps with few registers would otherwise keep its fields in local memory
+    // and wait for them, row tile after row tile.
+    if (threadIdx.x < 16)
+        reinterpret_cast<uint32_t *>(smem + kTrOffItem)[threadIdx.x] =
+            reinterpret_cast<const uint32_t *>(p.items + blockIdx.x)[threadIdx.x];
+    __syncthreads();
+    const TrainItem &it = *reinterpret_cast<const TrainItem *>(smem + kTrOffItem);
     const int G = p.group;
     const uint32_t tpt = 128u / (uint32_t)G;          // tokens per row tile
     const uint32_t rows_valid = tpt * (uint32_t)G;    // rows of a row tile that exist (128 unless G does not divide it)
@@ -133,7 +152,7 @@ cart_train_bwd_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_con
         mbar_init(bar(kTbKV), 1);
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar(kTbQFull + i), 2);
-            mbar_init(bar(kTbQEmpty + i), 1);
+            mbar_init(bar(kTbQEmpty + i), 2);
         }
         mbar_init(bar(kTbSFull), 1);
         mbar_init(bar(kTbPReady), 8);
@@ -178,6 +197,7 @@ cart_train_bwd_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_con
                 asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap)) : "memory");
                 asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap_q)) : "memory");
                 asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap_do)) : "memory");
+                asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap_dq)) : "memory");
                 // the key tile: 128 keys x 128 dims of K and of V, each as four boxes of 64 rows x 64 dims
                 mbar_expect_tx(bar(kTbKV), 2u * kTTile);
                 const int32_t ky = (int32_t)(it.k_row + (uint32_t)p.layer * it.layer_stride);
@@ -275,8 +295,7 @@ cart_train_bwd_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_con
 #pragma unroll
                     for (uint32_t k = 0; k < 8; ++k)
                         umma_bf16(tmem + kTmS, ads + (uint64_t)(k * 128u), bk + (uint64_t)(k * 128u), kIdMnMn, k, issue);
-                    umma_commit(bar(kTbDQFull), issue);
-                    umma_commit(bar(kTbQEmpty + (int)st), issue);
+                    umma_commit(bar(kTbDQFull), issue);  // (the stage's Q and dO tiles have been consumed with it)
                 }
             }
             umma_commit(bar(kTbDrain), issue);
@@ -294,20 +313,22 @@ cart_train_bwd_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_con
         const uint32_t lane_addr = tmem + ((uint32_t)(32 * sw) << 16);
         const uint8_t *tokoff = reinterpret_cast<const uint8_t *>(smem + kTrOffTok);
         const float sl2 = p.scale * 1.4426950408889634f;
-        const bool key_valid = j < it.n_keys;
+        const uint32_t n_keys = it.n_keys, rt_begin = it.rt_begin, rt_first = it.rt_first, kv_head = it.kv_head;
+        const uint32_t causal = it.causal, key_tok0 = it.key_tok0;
+        const bool key_valid = j < n_keys;
         // key j is seen by the rows of tokens lo .. hi - 1
-        const uint32_t lo = it.causal ? it.key_tok0 + j : 0u, hi = it.tok_end;
+        const uint32_t lo = causal ? key_tok0 + j : 0u, hi = it.tok_end;
         bool alive = true;
         auto warp_wait = [&](int b, uint32_t parity) -> bool {
             return __all_sync(0xffffffffu, mbar_wait(bar(b), parity, abort_flag, p.status, kStatusTimeoutConsumer));
         };
         alive = warp_wait(kTbKV, 0u);
-        if (alive && it.n_keys < 128u) {
+        if (alive && n_keys < 128u) {
             // keys past the tile's end hold whatever follows in the arena; dS is zero there, but 0 * NaN would poison
             // dQ_part = dS K, so those rows of K are cleared (dS K reads them as the B operand)
-            const uint32_t n_bad = 128u - it.n_keys;
+            const uint32_t n_bad = 128u - n_keys;
             for (uint32_t x = threadIdx.x - 128u; x < n_bad * 16u; x += 256u) {
-                const uint32_t r = it.n_keys + x / 16u, c = x % 16u;
+                const uint32_t r = n_keys + x / 16u, c = x % 16u;
                 const uint32_t a = base + kTrOffK + (c >> 3) * kTBlock + r * 128u + ((c & 7u) << 4);
                 asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0u) : "memory");
             }
@@ -315,9 +336,11 @@ cart_train_bwd_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_con
         }
         for (uint32_t i = 0; i < n_it; ++i) {
             const uint32_t st = i & 1u;
-            const uint32_t rt = it.rt_begin + (it.rt_first - it.rt_begin + i) % n_it;
+            const uint32_t rt = rt_begin + (rt_first - rt_begin + i) % n_it;
             const uint32_t tok0 = rt * tpt;
             const float2 *ld = reinterpret_cast<const float2 *>(smem + kTrOffLD) + st * 128u;
+            // a Cartridge tile whose keys all exist against a row tile whose rows all exist needs no mask
+            const bool full = !causal && n_keys == 128u && rows_valid == 128u && tok0 + tpt <= hi;
             if (alive) alive = warp_wait(kTbQFull + (int)st, (i >> 1) & 1u);   // the row tile's lse and D are in shared memory
             if (alive) alive = warp_wait(kTbSFull, i & 1u);
             if (alive) {
@@ -337,8 +360,11 @@ cart_train_bwd_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_con
                         for (uint32_t e = 0; e < 2; ++e) {
                             const uint32_t r = c_base + c + e;            // row of the row tile
                             const float2 l = ld[r];
-                            const uint32_t tk = tok0 + tokoff[r];
-                            const bool on = key_valid && r < rows_valid && tk >= lo && tk < hi;
+                            bool on = true;
+                            if (!full) {
+                                const uint32_t tk = tok0 + tokoff[r];
+                                on = key_valid && r < rows_valid && tk >= lo && tk < hi;
+                            }
                             const float pr = on ? fast_exp2(fmaf(__uint_as_float(s[c + e]), sl2, -l.x)) : 0.f;
                             pv[e] = pr;
                             // (what the key does not see may hold anything, NaN included: it is left out, not weighted by 0)
@@ -369,27 +395,41 @@ cart_train_bwd_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_con
             if (alive) alive = warp_wait(kTbDQFull, i & 1u);
             if (alive) {
                 tc_fence_after();
-                // dQ_part: this thread now owns ROW j of the row tile (tensor-memory lane j), dims col0 .. col0 + 63
-                const uint32_t tk = tok0 + tokoff[j];
-                // (a conversation tile only reaches rows of its own conversation at or after its first key)
-                const bool row_on = j < rows_valid && tk < hi && tk >= (it.causal ? it.key_tok0 : 0u);
+                // dQ_part: this thread now owns ROW j of the row tile (tensor-memory lane j), dims col0 .. col0 + 63.  The
+                // row goes to shared memory -- the stage's Q tile (first warpgroup) or dO tile (second), which the
+                // products no longer need -- as two blocks of 128 rows x 32 dims with the 128-byte swizzle, and one
+                // thread per warpgroup has the memory system add the blocks into dq: rows of tokens past the end of
+                // the batch are clipped by the tensor map, rows the key tile does not reach hold zeros.
+                const uint32_t stage_lo = base + (wg == 0 ? kTrOffQ : kTrOffDO) + st * kTTile;
 #pragma unroll
                 for (uint32_t half = 0; half < 2; ++half) {
                     uint32_t v[32];
                     tmem_ld32_issue(lane_addr + kTmS + col0 + 32u * half, v);
                     tmem_ld_wait(v);
-                    if (row_on) {
-                        float4 *dst = reinterpret_cast<float4 *>(
-                            p.dq + ((size_t)tk * p.n_q_heads + it.kv_head * (uint32_t)G + (j % (uint32_t)G)) * kHeadDim + col0 + 32u * half);
+                    const uint32_t row_addr = stage_lo + half * kTBlock + j * 128u;
 #pragma unroll
-                        for (uint32_t q4 = 0; q4 < 8; ++q4)
-                            atomicAdd(dst + q4, make_float4(__uint_as_float(v[4 * q4]), __uint_as_float(v[4 * q4 + 1]),
-                                                            __uint_as_float(v[4 * q4 + 2]), __uint_as_float(v[4 * q4 + 3])));
-                    }
+                    for (uint32_t c8 = 0; c8 < 8; ++c8)
+                        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(row_addr + ((c8 ^ (j & 7u)) << 4)),
+                                     "r"(v[4 * c8]), "r"(v[4 * c8 + 1]), "r"(v[4 * c8 + 2]), "r"(v[4 * c8 + 3])
+                                     : "memory");
                 }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(kTbTmFree));
+            }
+            // the warpgroup's rows are all in shared memory: one thread sends them off and, once they have been read,
+            // gives the stage back to the producer (the barrier is met by every warp, also by one that has given up)
+            if (wg == 0) asm volatile("bar.sync 5, 128;" ::: "memory");
+            else asm volatile("bar.sync 6, 128;" ::: "memory");
+            if (alive && sw == 0 && lane == 0) {
+                const uint32_t stage_lo = base + (wg == 0 ? kTrOffQ : kTrOffDO) + st * kTTile;
+                const int32_t y = (int32_t)(kv_head * (uint32_t)G), z = (int32_t)tok0;
+                tma_reduce_add_3d(&tmap_dq, stage_lo, (int32_t)col0, y, z);
+                tma_reduce_add_3d(&tmap_dq, stage_lo + kTBlock, (int32_t)col0 + 32, y, z);
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                mbar_arrive(bar(kTbQEmpty + (int)st));
             }
         }
         // the key tile's gradients: lane j = key j, dims col0 .. col0 + 63 of dV and dK (complete with the last dQ_part)
@@ -442,9 +482,9 @@ cudaError_t launch_train_delta(const TrainDeltaParams &p, cudaStream_t s)
 }
 
 cudaError_t launch_train_bwd(const CUtensorMap &tmap, const CUtensorMap &tmap_q, const CUtensorMap &tmap_do,
-                             const TrainBwdParams &p, int n_items, cudaStream_t s)
+                             const CUtensorMap &tmap_dq, const TrainBwdParams &p, int n_items, cudaStream_t s)
 {
-    cart_train_bwd_kernel<<<n_items, kTrThreads, kTrSmemBytes, s>>>(tmap, tmap_q, tmap_do, p);
+    cart_train_bwd_kernel<<<n_items, kTrThreads, kTrSmemBytes, s>>>(tmap, tmap_q, tmap_do, tmap_dq, p);
     return cudaGetLastError();
 }
 
