@@ -123,11 +123,27 @@ typedef struct {
     uint32_t reader_begin; /* first entry of the M-tile in readers[] */
     uint32_t n_readers;    /* entries of the M-tile (1 .. 128 / group) */
     uint16_t kv_head;
-    uint16_t flags;        /* CART_UNIT_SUFFIX: the run lies in suffix storage (see CART_ITEM_SUFFIX) */
+    uint16_t flags;        /* CART_UNIT_*: CART_UNIT_SUFFIX = the run lies in suffix storage (see CART_ITEM_SUFFIX) */
     uint32_t chunk;        /* ordinal of the run among the runs of its (segment, M-tile, KV head) */
+    /* Masked runs (CART_UNIT_MASKED; the planner does not emit them, the training forward builds them): row r of the
+     * M-tile (token offset tr = r / group) sees the run's keys 0 .. limit with
+     *     limit = tr < tr_hi ? min(lim_base + tr, lim_cap) : -1        (negative: the row sees nothing of the run)
+     * so a causal run has lim_base = first row's token - run's first token, and a run every row sees whole but that
+     * ends inside a tile has lim_base = lim_cap = its last key.  n_tiles then counts the ragged last tile too. */
+    int32_t lim_base;
+    int32_t lim_cap;
+    uint32_t tr_hi;
+    uint32_t reserved;
 } cart_shared_unit;
 
 #define CART_UNIT_SUFFIX 1u
+#define CART_UNIT_MASKED 4u   /* see lim_base */
+#define CART_UNIT_CONT 8u     /* the unit continues the M-tile of the unit before it in the same block: the softmax state
+                                 and the accumulator carry over (same readers, same KV head) */
+#define CART_UNIT_HOLD 16u    /* nothing is written at the unit's end: the next unit (CART_UNIT_CONT) goes on */
+#define CART_UNIT_DIRECT 32u  /* the unit's end writes the rows' final bf16 output and lse (row i of reader j goes to
+                                 query row readers[reader_begin + j]), not a partial: the chain covers the rows' whole
+                                 caches */
 #define CART_UNIT_PAGED 2u    /* the run lies in pages: k_row = index of its first page in the page list (a shared
                                  tile of share_tile_tokens tokens spans share_tile_tokens / tile_tokens consecutive
                                  entries), v_row = row of the KV head's K block inside a page, layer_stride as in

@@ -69,7 +69,9 @@ class cart_shared_unit(ctypes.Structure):
     _fields_ = [("k_row", ctypes.c_uint32), ("v_row", ctypes.c_uint32),
                 ("layer_stride", ctypes.c_uint32), ("n_tiles", ctypes.c_uint32),
                 ("reader_begin", ctypes.c_uint32), ("n_readers", ctypes.c_uint32),
-                ("kv_head", ctypes.c_uint16), ("flags", ctypes.c_uint16), ("chunk", ctypes.c_uint32)]
+                ("kv_head", ctypes.c_uint16), ("flags", ctypes.c_uint16), ("chunk", ctypes.c_uint32),
+                ("lim_base", ctypes.c_int32), ("lim_cap", ctypes.c_int32), ("tr_hi", ctypes.c_uint32),
+                ("reserved", ctypes.c_uint32)]
 
 
 class cart_plan_out(ctypes.Structure):

@@ -1406,8 +1406,145 @@ cart_status cart_train_attention_fwd(cart_ctx *ctx, int32_t layer, const cart_re
     TrainBatch tb;
     const cart_status st = train_batch(ctx, layer, convs, n_convs, &tb);
     if (st != CART_OK) return st;
-    // every conversation is a block of new tokens over an empty suffix: the rows of all conversations share Z
-    return decode_impl(ctx, layer, convs, n_convs, q, out, lse, nullptr, nullptr, stream, tb.len.data(), n_convs);
+    if (!aligned16(q) || !aligned16(out)) return fail(ctx, CART_ERR_INVALID_ARG, "train: null/misaligned pointer");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int Hkv = ctx->cfg.n_kv_heads, G = ctx->group;
+    const uint32_t tpt = 128u / (uint32_t)G;   // tokens (readers) per M-tile
+    const uint32_t T = (uint32_t)tb.T, n_rt = (T + tpt - 1) / tpt;
+    const uint32_t p = tb.z ? (uint32_t)tb.z->p : 0u;
+
+    // One chain of units per (M-tile of 128 / G consecutive tokens, KV head), all on the tensor-core kernel: the
+    // Cartridge's tiles (every row sees all of them), then, conversation by conversation, the tiles of the
+    // conversations the M-tile's tokens belong to, masked causally; the chain's last unit writes out and lse
+    // directly -- no partials, no merge, and no row streams its diagonal by itself.
+    PlanSlot *cur = ctx->cur_slot >= 0 ? &ctx->slots[ctx->cur_slot] : nullptr;
+    if (cur && cur->valid) {
+        CART_CUDA(ctx, cudaEventRecord(cur->ev, cur->last_stream));
+        cur->ev_recorded = true;
+    }
+    const int next = (ctx->cur_slot + 1) % kPlanSlots;
+    PlanSlot &ns = ctx->slots[next];
+    if (ns.ev_recorded) {
+        CART_CUDA(ctx, cudaEventSynchronize(ns.ev));
+        ns.ev_recorded = false;
+    }
+    ns.valid = false;
+    const ScratchLayout &lay = ctx->lay;
+    cart_shared_unit *units = reinterpret_cast<cart_shared_unit *>(ns.host + lay.units_off);
+    uint32_t *unit_cta_begin = reinterpret_cast<uint32_t *>(ns.host + lay.unit_cta_begin_off);
+    uint32_t *readers = reinterpret_cast<uint32_t *>(ns.host + lay.readers_off);
+    if ((int64_t)T > lay.readers_cap) return fail(ctx, CART_ERR_CAPACITY, "train: %u tokens exceed the reader table", T);
+    for (uint32_t t = 0; t < T; ++t) readers[t] = t;   // reader entry t = token t = query row t
+    // tiles of every chain, to balance the blocks
+    std::vector<uint32_t> chain_tiles(n_rt, 0);
+    std::vector<int32_t> first_conv(n_rt, 0);
+    {
+        int32_t c = 0;
+        for (uint32_t rt = 0; rt < n_rt; ++rt) {
+            const uint32_t a = rt * tpt, b = std::min(T, a + tpt);
+            while ((uint32_t)tb.cu[(size_t)c + 1] <= a) ++c;
+            first_conv[rt] = c;
+            uint32_t tiles = (p + 127u) / 128u;
+            for (int32_t cc = c; cc < n_convs && (uint32_t)tb.cu[(size_t)cc] < b; ++cc) {
+                const uint32_t last = std::min<uint32_t>(b, (uint32_t)tb.cu[(size_t)cc + 1]) - 1u;   // last token of cc in the tile
+                tiles += (last - (uint32_t)tb.cu[(size_t)cc] + 1u + 127u) / 128u;
+            }
+            chain_tiles[rt] = tiles;
+        }
+    }
+    uint64_t total_tiles = 0;
+    for (uint32_t rt = 0; rt < n_rt; ++rt) total_tiles += (uint64_t)chain_tiles[rt] * (uint64_t)Hkv;
+    const uint32_t n_blocks = (uint32_t)std::min<uint64_t>((uint64_t)ctx->n_cta, (uint64_t)n_rt * Hkv);
+    size_t nu = 0;
+    uint32_t blk = 0;
+    uint64_t given = 0;
+    bool full = false;
+    unit_cta_begin[0] = 0;
+    for (int g = 0; g < Hkv && !full; ++g)
+        for (uint32_t rt = 0; rt < n_rt && !full; ++rt) {
+            // a chain goes to the block whose share of the tiles it starts in
+            while (blk + 1 < n_blocks && given * n_blocks >= (uint64_t)(blk + 1) * total_tiles) unit_cta_begin[++blk] = (uint32_t)nu;
+            given += chain_tiles[rt];
+            const uint32_t a = rt * tpt, b = std::min(T, a + tpt);
+            bool first = true;
+            auto emit = [&](cart_shared_unit u, bool last) {
+                if (nu >= (size_t)lay.units_cap) { full = true; return; }
+                u.reader_begin = a;
+                u.n_readers = b - a;
+                u.kv_head = (uint16_t)g;
+                u.chunk = 0;
+                u.reserved = 0;
+                if (!first) u.flags |= CART_UNIT_CONT;
+                u.flags |= last ? CART_UNIT_DIRECT : CART_UNIT_HOLD;
+                first = false;
+                units[nu++] = u;
+            };
+            int32_t c_last = first_conv[rt];
+            while (c_last + 1 < n_convs && (uint32_t)tb.cu[(size_t)c_last + 1] < b) ++c_last;
+            if (p > 0) {
+                cart_shared_unit u{};
+                u.k_row = (uint32_t)(tb.z->k_row + (uint64_t)g * p);
+                u.v_row = (uint32_t)(tb.z->v_row + (uint64_t)g * p);
+                u.layer_stride = (uint32_t)Hkv * p;
+                u.n_tiles = (p + 127u) / 128u;
+                u.flags = (p % 128u) ? CART_UNIT_MASKED : 0;
+                u.lim_base = (int32_t)p - 1;
+                u.lim_cap = (int32_t)p - 1;
+                u.tr_hi = tpt;
+                emit(u, false);
+            }
+            for (int32_t c = first_conv[rt]; c <= c_last; ++c) {
+                const Request &r = ctx->reqs[(size_t)convs[c]];
+                const uint32_t c0 = (uint32_t)tb.cu[(size_t)c], c1 = (uint32_t)tb.cu[(size_t)c + 1];
+                const uint32_t last = std::min(b, c1) - 1u;   // last token of the conversation in the M-tile
+                cart_shared_unit u{};
+                u.k_row = (uint32_t)(r.k_row + (uint64_t)g * r.cap);
+                u.v_row = (uint32_t)(r.v_row + (uint64_t)g * r.cap);
+                u.layer_stride = (uint32_t)((uint64_t)Hkv * r.cap);
+                u.n_tiles = (last - c0 + 1u + 127u) / 128u;
+                u.flags = CART_UNIT_MASKED | CART_UNIT_SUFFIX;
+                u.lim_base = (int32_t)a - (int32_t)c0;      // token offset 0 of the M-tile sees keys 0 .. a - c0
+                u.lim_cap = (int32_t)(c1 - c0) - 1;         // the conversation's last stored key
+                u.tr_hi = c1 - a;                           // tokens from here on belong to later conversations
+                emit(u, c == c_last);
+            }
+        }
+    if (full) return fail(ctx, CART_ERR_CAPACITY, "train: more than %d units", lay.units_cap);
+    while (blk + 1 <= n_blocks) unit_cta_begin[++blk] = (uint32_t)nu;
+    for (uint32_t b2 = blk; b2 < (uint32_t)kMaxCta; ++b2) unit_cta_begin[b2 + 1] = (uint32_t)nu;
+    const uint64_t sh_bytes = lay.units_off + (uint64_t)nu * sizeof(cart_shared_unit) - lay.shared_off;
+    CART_CUDA(ctx, cudaMemcpyAsync(ns.dev + lay.shared_off, ns.host + lay.shared_off, sh_bytes, cudaMemcpyHostToDevice, s));
+    ns.last_stream = s;
+    ns.epoch = 0;
+    ctx->cur_slot = next;
+    CART_CUDA(ctx, cudaEventRecord(ns.ev, s));
+    ns.ev_recorded = true;
+
+    uint8_t *arena = static_cast<uint8_t *>(ctx->cfg.arena);
+    SharedParams sp;
+    sp.unit_cta_begin = reinterpret_cast<const uint32_t *>(ns.dev + lay.unit_cta_begin_off);
+    sp.units = reinterpret_cast<const cart_shared_unit *>(ns.dev + lay.units_off);
+    sp.readers = reinterpret_cast<const uint32_t *>(ns.dev + lay.readers_off);
+    sp.reader_slot = reinterpret_cast<const uint32_t *>(ns.dev + lay.reader_slot_off);
+    sp.reader_merge = reinterpret_cast<const uint32_t *>(ns.dev + lay.reader_merge_off);
+    sp.merges = reinterpret_cast<const cart_merge_item *>(ns.dev + lay.merges_off);
+    sp.q = q;
+    sp.out = out;
+    sp.lse = lse;
+    sp.part_o = reinterpret_cast<float *>(arena + lay.part_o_off);
+    sp.part_lse2 = reinterpret_cast<float *>(arena + lay.part_lse_off);
+    sp.tickets = nullptr;
+    sp.status = reinterpret_cast<uint32_t *>(arena + lay.status_off);
+    sp.layer = layer;
+    sp.group = G;
+    sp.n_kv_heads = Hkv;
+    sp.n_q_heads = ctx->cfg.n_q_heads;
+    sp.scale_log2 = ctx->scale * 1.4426950408889634f;
+    sp.pages = nullptr;
+    CART_CUDA(ctx, launch_shared(ctx->tmap, sp, (int)n_blocks, s, true));
+    ++ctx->launches;
+    CART_CUDA(ctx, cudaEventRecord(ns.ev, s));
+    return CART_OK;
 }
 
 cart_status cart_train_attention_bwd(cart_ctx *ctx, int32_t layer, const cart_req *convs, int32_t n_convs, const void *q,

@@ -189,7 +189,8 @@ cudaError_t prepare_kernels();  // sets the dynamic shared-memory attribute; cal
 cudaError_t launch_decode(const CUtensorMap &tmap, const CUtensorMap &tmap_edge, const DecodeParams &p, int grid,
                           cudaStream_t s);
 cudaError_t prepare_shared_kernel();
-cudaError_t launch_shared(const CUtensorMap &tmap, const SharedParams &p, int grid, cudaStream_t s);
+// chains: the plan holds chained / masked / directly written units (see CART_UNIT_CONT in cart_plan.h)
+cudaError_t launch_shared(const CUtensorMap &tmap, const SharedParams &p, int grid, cudaStream_t s, bool chains = false);
 cudaError_t launch_merge(const MergeParams &p, int n_merges, cudaStream_t s);
 cudaError_t launch_append(const AppendParams &p, cudaStream_t s);
 cudaError_t launch_extend(const ExtendParams &p, cudaStream_t s);

@@ -307,6 +307,10 @@ extern "C" cart_status cart_plan_build_shared(const cart_plan_seg *segs, const i
                 u.n_readers = cb.n_readers;
                 u.kv_head = (uint16_t)cb.kv_head;
                 u.chunk = chunk;
+                u.lim_base = 0;
+                u.lim_cap = 0;
+                u.tr_hi = 0;
+                u.reserved = 0;
             });
         if (overflow) return CART_ERR_CAPACITY;
         for (uint64_t b = cur; b < (uint64_t)n_cta; ++b) o->unit_cta_begin[b + 1] = (uint32_t)nu;

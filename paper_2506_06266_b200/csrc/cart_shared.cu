@@ -144,6 +144,10 @@ __device__ __forceinline__ bool wait_for_prior_kernels(const SharedParams &p, vo
     }
 }
 
+// kChains: the kernel also understands chained, masked and directly written units (CART_UNIT_CONT / _HOLD / _MASKED /
+// _DIRECT: the forward of training attention).  The decode and prefill plans never contain them, and their
+// instantiation carries none of that code in its tile loop.
+template <bool kChains>
 __global__ void __launch_bounds__(kShThreads, 1)
 cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams p)
 {
@@ -288,15 +292,19 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
             };
             // Two cursors walk the block's tiles in order: `qk` names the next score product to issue (it
             // runs two tiles ahead), `pv` the next P V product.  tt = tile index counted over the block.
-            struct Cursor { uint32_t ui, t, n, unit_no; };
+            struct Cursor { uint32_t ui, t, n, unit_no, cont; };
             auto tiles_of = [&](uint32_t ui) { return ui < unit_end ? p.units[ui].n_tiles : 0u; };
-            Cursor qk{unit_begin, 0u, tiles_of(unit_begin), 0u}, pv = qk;
+            auto cont_of = [&](uint32_t ui) {
+                return kChains && ui < unit_end ? (uint32_t)(p.units[ui].flags & CART_UNIT_CONT) : 0u;
+            };
+            Cursor qk{unit_begin, 0u, tiles_of(unit_begin), 0u, cont_of(unit_begin)}, pv = qk;
             auto advance = [&](Cursor &c) {
                 if (++c.t == c.n) {
                     ++c.ui;
                     ++c.unit_no;
                     c.t = 0;
                     c.n = tiles_of(c.ui);
+                    c.cont = cont_of(c.ui);
                 }
             };
             uint32_t total = 0;
@@ -344,7 +352,7 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                 const uint64_t b0 = umma_desc(v_lo, kShBlock, 1024);
                 const uint32_t p_tm = tmem + sb * 128u;
                 const uint32_t d_o = tmem + kTmemO;
-                const bool first = pv.t == 0u;
+                const bool first = pv.t == 0u && pv.cont == 0u;  // (a unit that continues a chain adds to its accumulator)
 #pragma unroll
                 for (uint32_t k = 0; k < 8; ++k)  // 16 tokens per instruction
                     umma_bf16_ts(d_o, p_tm + (k < 4u ? 8u * k : 64u + 8u * (k - 4u)), b0 + (uint64_t)(k * 128u), kIdescPV,
@@ -443,6 +451,8 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
             }
         }
 
+        float m_run = -INFINITY, l_run = 0.f;
+        bool fresh = true;   // no tile of the chain has been seen yet
         uint32_t unit_no = 0;
         for (uint32_t ui = unit_begin; ui < unit_end; ++ui, ++unit_no) {
             if (ui != unit_begin) {
@@ -456,20 +466,35 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
             uint32_t batch_next = 0;
             if (valid_next) batch_next = p.readers[u_next.reader_begin + (uint32_t)i_reader];
             const uint32_t t_store = u.n_tiles > 1u ? 1u : 0u;  // the tile after which the next unit's rows are stored
-            uint32_t slot = 0;
-            if (valid)  // where this row's partial goes (needed at the unit's end: the load has the tiles' time)
-                slot = p.reader_slot[(size_t)(u.reader_begin + (uint32_t)i_reader) * p.n_kv_heads + u.kv_head] + u.chunk;
+            const bool direct = kChains && (u.flags & CART_UNIT_DIRECT) != 0u, hold = kChains && (u.flags & CART_UNIT_HOLD) != 0u;
+            const bool masked = kChains && (u.flags & CART_UNIT_MASKED) != 0u;
+            uint32_t slot = 0;   // where this row's partial goes, or (direct) its query row: needed at the unit's end
+            if (valid && !hold)
+                slot = direct ? p.readers[u.reader_begin + (uint32_t)i_reader]
+                              : p.reader_slot[(size_t)(u.reader_begin + (uint32_t)i_reader) * p.n_kv_heads + u.kv_head] + u.chunk;
             // m_run: the reference that l_run and the accumulator in tensor memory refer to, the same for both
             // owners of the row.  It only moves when the row's maximum has outgrown it by more than
             // kRescaleStep (base 2); until then probabilities may exceed 1 (by at most that factor), which
-            // bf16 and the fp32 sums hold easily.  l_run: the sum over this thread's columns.
-            float m_run = -INFINITY, l_run = 0.f;
+            // bf16 and the fp32 sums hold easily.  l_run: the sum over this thread's columns.  A unit that
+            // continues the one before it (a chain over the same rows) inherits all three.
+            if (!kChains || !(u.flags & CART_UNIT_CONT)) {
+                m_run = -INFINITY;
+                l_run = 0.f;
+                fresh = true;
+            }
+            // masked run: the last key of the run this row sees (-1: none)
+            int32_t limit = 0x7FFFFFFF;
+            if (masked) {
+                const int32_t lb = u.lim_base + i_reader;
+                limit = (uint32_t)i_reader < u.tr_hi ? (lb < u.lim_cap ? lb : u.lim_cap) : -1;
+            }
 
             for (uint32_t t = 0; t < u.n_tiles; ++t, ++tt) {
                 const uint32_t sb = tt % (uint32_t)kSBufs, spar = (tt / (uint32_t)kSBufs) & 1u;
                 const uint32_t s_addr = lane_addr + sb * 128u + col0;
                 uint32_t s[64];
                 float mx = -INFINITY;
+                bool all_on = true;
                 if (alive) alive = warp_wait(bar(kBarSFull + (int)sb), spar);
                 if (alive) {
                     tc_fence_after();
@@ -477,8 +502,18 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                     tmem_ld32_issue(s_addr + 32u, reinterpret_cast<uint32_t(&)[32]>(s[32]));
                     tmem_ld_wait(reinterpret_cast<uint32_t(&)[32]>(s[0]));
                     tmem_ld_wait(reinterpret_cast<uint32_t(&)[32]>(s[32]));
+                    // keys of this thread's columns: kidx0 .. kidx0 + 63 of the run; all of them seen unless masked
+                    const int32_t kidx0 = (int32_t)(t * (uint32_t)kShTile + col0);
+                    all_on = !masked || kidx0 + 63 <= limit;
+                    if (all_on) {
 #pragma unroll
-                    for (int k = 0; k < 64; k += 2) mx = fmaxf(mx, fmaxf(__uint_as_float(s[k]), __uint_as_float(s[k + 1])));
+                        for (int k = 0; k < 64; k += 2) mx = fmaxf(mx, fmaxf(__uint_as_float(s[k]), __uint_as_float(s[k + 1])));
+                    } else {
+                        // (what lies past a row's limit may be anything, NaN included: it is left out, not compared)
+#pragma unroll
+                        for (int k = 0; k < 64; ++k)
+                            if (kidx0 + k <= limit) mx = fmaxf(mx, __uint_as_float(s[k]));
+                    }
                     mx *= p.scale_log2;
                 }
                 // the row's maximum over the whole tile: the two owners trade their halves' maxima (rounded up to
@@ -489,15 +524,17 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                 const uint32_t theirs = xchg_mx[((tt & 1u) * 2u + (uint32_t)(wg ^ 1)) * 128u + (uint32_t)row];
                 if (!alive) continue;
                 const float m_tile = fmaxf(__uint_as_float(mine << 16), __uint_as_float(theirs << 16));
-                if (t == 0) {
+                if (fresh) {
                     m_run = m_tile;
+                    fresh = false;
                 } else if (__any_sync(0xffffffffu, m_tile > m_run + kRescaleStep)) {
                     // a row of this warp has outgrown its reference: every row of the warp moves up to its
                     // maximum and the two owners rescale their halves of the accumulator's lanes (tensor-memory
                     // accesses are warp-wide, so the warp decides together, and its twin in the other warpgroup
                     // sees the same numbers and decides the same; the other rows' factors are 1 or close to it)
                     const float m_new = fmaxf(m_run, m_tile);
-                    const float f = fast_exp2(m_run - m_new);
+                    // (a row of a masked run may not have seen a key yet: its reference stays at -inf, factor 1)
+                    const float f = m_new == -INFINITY ? 1.f : fast_exp2(m_run - m_new);
                     m_run = m_new;
                     l_run *= f;
                     // The product of the tile before must have landed first.  Its completion is read from the
@@ -527,8 +564,13 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                     uint32_t w[16];
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
-                        const float p0 = fast_exp2(fmaf(__uint_as_float(s[32 * c + 2 * j]), p.scale_log2, -m_run));
-                        const float p1 = fast_exp2(fmaf(__uint_as_float(s[32 * c + 2 * j + 1]), p.scale_log2, -m_run));
+                        float p0 = fast_exp2(fmaf(__uint_as_float(s[32 * c + 2 * j]), p.scale_log2, -m_run));
+                        float p1 = fast_exp2(fmaf(__uint_as_float(s[32 * c + 2 * j + 1]), p.scale_log2, -m_run));
+                        if (!all_on) {
+                            const int32_t kidx = (int32_t)(t * (uint32_t)kShTile + col0) + 32 * c + 2 * j;
+                            if (kidx > limit) p0 = 0.f;
+                            if (kidx + 1 > limit) p1 = 0.f;
+                        }
                         psum0 += p0;
                         psum1 += p1;
                         w[j] = pack_bf16(p0, p1);
@@ -536,6 +578,23 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                     tmem_st16(s_addr + (uint32_t)c * 16u, w);
                 }
                 l_run += psum0 + psum1;
+                if (masked && t + 1u == u.n_tiles && (uint32_t)(u.lim_cap + 1) < u.n_tiles * (uint32_t)kShTile) {
+                    // The run ends inside this tile.  The rows behind its last key hold whatever follows in memory;
+                    // their probabilities are zero, but 0 * NaN would poison the product, so those rows of the V tile
+                    // are cleared (both softmax warpgroups share the work) before the MMA warp hears of the tile.
+                    const uint32_t vst = tt % (uint32_t)kVStages, vpar = (tt / (uint32_t)kVStages) & 1u;
+                    alive = warp_wait(bar(kBarVFull + (int)vst), vpar);
+                    if (!alive) continue;
+                    const uint32_t first_bad = (uint32_t)(u.lim_cap + 1) - t * (uint32_t)kShTile;   // 1 .. 127
+                    const uint32_t v_lo = base + kOffV + vst * kShTileBytes;
+                    for (uint32_t x = (uint32_t)(wg * kSoftmaxThreads + tid); x < (128u - first_bad) * 16u; x += 2u * kSoftmaxThreads) {
+                        const uint32_t r = first_bad + x / 16u, c = x % 16u;
+                        asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(v_lo + (c >> 3) * kShBlock + r * 128u + ((c & 7u) << 4)),
+                                     "r"(0u)
+                                     : "memory");
+                    }
+                    fence_async_smem();
+                }
                 tmem_st_wait();
                 tc_fence_before();
                 __syncwarp();
@@ -547,6 +606,8 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
             }
 
             // ---- the unit's rows leave as normalised partials -------------------------------------------
+            // (unless the next unit continues the same rows: then the state simply stays)
+            if (hold) continue;
             // Each thread reads its 64 columns of the accumulator once the last product has landed; the two
             // owners of a row add their sums (in a fixed order, so the result does not depend on timing).
             uint32_t o[64];
@@ -562,7 +623,23 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
             softmax_bar_both();  // nobody reads the maxima of the last tile any more: the sums go over them
             xchg_l[wg * 128 + row] = l_run;
             softmax_bar_both();
-            if (alive && valid) {
+            if (alive && valid && direct) {
+                // the chain covered the row's whole cache: the final output, rounded to bf16, and the lse
+                const float l = xchg_l[row] + xchg_l[128 + row];
+                const float inv = 1.f / l;
+                const size_t orow = (size_t)slot * p.n_q_heads + (size_t)u.kv_head * G + h;
+                uint4 *dst = reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(p.out) + orow * kHeadDim + col0);
+#pragma unroll
+                for (int c8 = 0; c8 < 8; ++c8) {
+                    uint4 w;
+                    w.x = pack_bf16(__uint_as_float(o[8 * c8]) * inv, __uint_as_float(o[8 * c8 + 1]) * inv);
+                    w.y = pack_bf16(__uint_as_float(o[8 * c8 + 2]) * inv, __uint_as_float(o[8 * c8 + 3]) * inv);
+                    w.z = pack_bf16(__uint_as_float(o[8 * c8 + 4]) * inv, __uint_as_float(o[8 * c8 + 5]) * inv);
+                    w.w = pack_bf16(__uint_as_float(o[8 * c8 + 6]) * inv, __uint_as_float(o[8 * c8 + 7]) * inv);
+                    dst[c8] = w;
+                }
+                if (wg == 0 && p.lse) p.lse[orow] = (m_run + log2f(l)) * 0.6931471805599453f;
+            } else if (alive && valid) {
                 const float l = xchg_l[row] + xchg_l[128 + row];
                 const float inv = 1.f / l;
                 float4 *dst = reinterpret_cast<float4 *>(p.part_o + ((size_t)slot * G + h) * kHeadDim + col0);
@@ -572,7 +649,7 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                                           __uint_as_float(o[4 * q4 + 2]) * inv, __uint_as_float(o[4 * q4 + 3]) * inv);
                 if (wg == 0) p.part_lse2[(size_t)slot * kMaxGroup + h] = m_run + log2f(l);
             }
-            if (p.tickets == nullptr) {
+            if (p.tickets == nullptr || direct) {
                 softmax_bar_both();  // the sums have been read: the next unit's maxima may be written
                 continue;
             }
@@ -624,14 +701,17 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
 
 cudaError_t prepare_shared_kernel()
 {
-    return cudaFuncSetAttribute(cart_shared_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kShSmemBytes);
+    cudaError_t e = cudaFuncSetAttribute(cart_shared_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kShSmemBytes);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(cart_shared_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kShSmemBytes);
 }
 
-cudaError_t launch_shared(const CUtensorMap &tmap, const SharedParams &p, int grid, cudaStream_t s)
+cudaError_t launch_shared(const CUtensorMap &tmap, const SharedParams &p, int grid, cudaStream_t s, bool chains)
 {
     cudaLaunchAttribute attr;
     const cudaLaunchConfig_t cfg = pdl_config(grid, kShThreads, kShSmemBytes, s, &attr);
-    return cudaLaunchKernelEx(&cfg, cart_shared_kernel, tmap, p);
+    return chains ? cudaLaunchKernelEx(&cfg, cart_shared_kernel<true>, tmap, p)
+                  : cudaLaunchKernelEx(&cfg, cart_shared_kernel<false>, tmap, p);
 }
 
 }  // namespace cart
