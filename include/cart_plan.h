@@ -133,7 +133,8 @@ typedef struct {
     int32_t lim_base;
     int32_t lim_cap;
     uint32_t tr_hi;
-    uint32_t reserved;
+    uint32_t reserved;     /* plans with chains: on a chain's first unit, how many units on the next chain begins (0: none follows
+                              in the block); else 0 */
 } cart_shared_unit;
 
 #define CART_UNIT_SUFFIX 1u

@@ -179,6 +179,11 @@ struct cart_ctx {
 
 namespace {
 
+struct ChainPart { uint64_t k_row, v_row; uint32_t p; };
+struct ChainStrand { uint64_t k_row, v_row; uint32_t cap, len, row_begin, n_rows, key_first; };
+cart_status launch_chains(cart_ctx *ctx, int32_t layer, const std::vector<ChainPart> &parts, const std::vector<ChainStrand> &strands,
+                          uint32_t T, const void *q, void *out, float *lse, cudaStream_t s);
+
 cart_status fail(cart_ctx *ctx, cart_status st, const char *fmt, ...)
 {
     if (ctx) {
@@ -1315,6 +1320,26 @@ cart_status cart_prefill_attention(cart_ctx *ctx, int32_t layer, cart_req req, c
 {
     if (!ctx) return CART_ERR_INVALID_ARG;
     if (n_new < 1) return fail(ctx, CART_ERR_INVALID_ARG, "prefill: n_new < 1");
+    // A message long enough to give every SM a chain (an M-tile of 128 / G tokens times a KV head) goes through
+    // chains of masked tiles: one kernel, the diagonal on the tensor cores too (1024 tokens over a 2048-token
+    // Cartridge: 218 us per layer against 256).  Shorter messages have too few chains to fill the device (256
+    // tokens: 110 us against 90) and go, like paged suffixes, through the decode kernels, which split the keys.
+    Request *r = get_req(ctx, req);
+    const int32_t tpt = 128 / ctx->group;
+    if (r && !r->paged && !r->evicted && ctx->share_min_readers > 0 && n_new <= ctx->cfg.max_requests &&
+        (int64_t)((n_new + tpt - 1) / tpt) * ctx->cfg.n_kv_heads >= ctx->n_cta &&
+        layer >= 0 && layer < ctx->cfg.n_layers && r->len[(size_t)layer] >= n_new && evicted_part(ctx, *r) < 0 && aligned16(q) &&
+        aligned16(out)) {
+        std::vector<ChainPart> parts;
+        if (r->cart != CART_NONE) {
+            const Cartridge &c = ctx->carts[(size_t)r->cart];
+            if (c.composed) for (int32_t b : c.parts) parts.push_back(ChainPart{ctx->carts[(size_t)b].k_row, ctx->carts[(size_t)b].v_row, (uint32_t)ctx->carts[(size_t)b].p});
+            else parts.push_back(ChainPart{c.k_row, c.v_row, (uint32_t)c.p});
+        }
+        const uint32_t len = (uint32_t)r->len[(size_t)layer];
+        std::vector<ChainStrand> strands{ChainStrand{r->k_row, r->v_row, (uint32_t)r->cap, len, 0u, (uint32_t)n_new, len - (uint32_t)n_new}};
+        return launch_chains(ctx, layer, parts, strands, (uint32_t)n_new, q, out, lse, static_cast<cudaStream_t>(stream));
+    }
     return decode_impl(ctx, layer, &req, 1, q, out, lse, nullptr, nullptr, stream, &n_new, 1);
 }
 
@@ -1398,25 +1423,25 @@ cart_status train_batch(cart_ctx *ctx, int32_t layer, const cart_req *convs, int
 
 extern "C" {
 
-cart_status cart_train_attention_fwd(cart_ctx *ctx, int32_t layer, const cart_req *convs, int32_t n_convs, const void *q,
-                                     void *out, float *lse, void *stream)
+}  // extern "C"
+
+namespace {
+
+// Rows that attend causally, as chains of units on the tensor-core kernel (prefill of a long message; the forward
+// of training attention).  The rows are numbered 0 .. T - 1 (row t = query row t of q / out / lse); every row sees
+// all of `parts` (Cartridge blocks, in order) and then its own "strand": strand c owns the rows row_begin ..
+// row_begin + n_rows - 1, its keys are the first key_first + i + 1 tokens of a contiguous suffix buffer for its row i.
+
+// One chain of units per (M-tile of 128 / G consecutive rows' tokens, KV head): the parts' tiles (every row sees all
+// of them), then, strand by strand, the tiles of the strands the M-tile's rows belong to, masked causally; the
+// chain's last unit writes out and lse directly -- no partials, no merge, and no row streams its diagonal by itself.
+cart_status launch_chains(cart_ctx *ctx, int32_t layer, const std::vector<ChainPart> &parts, const std::vector<ChainStrand> &strands,
+                          uint32_t T, const void *q, void *out, float *lse, cudaStream_t s)
 {
-    if (!ctx) return CART_ERR_INVALID_ARG;
-    if (!lse) return fail(ctx, CART_ERR_INVALID_ARG, "train: the forward must write lse");
-    TrainBatch tb;
-    const cart_status st = train_batch(ctx, layer, convs, n_convs, &tb);
-    if (st != CART_OK) return st;
-    if (!aligned16(q) || !aligned16(out)) return fail(ctx, CART_ERR_INVALID_ARG, "train: null/misaligned pointer");
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int Hkv = ctx->cfg.n_kv_heads, G = ctx->group;
     const uint32_t tpt = 128u / (uint32_t)G;   // tokens (readers) per M-tile
-    const uint32_t T = (uint32_t)tb.T, n_rt = (T + tpt - 1) / tpt;
-    const uint32_t p = tb.z ? (uint32_t)tb.z->p : 0u;
-
-    // One chain of units per (M-tile of 128 / G consecutive tokens, KV head), all on the tensor-core kernel: the
-    // Cartridge's tiles (every row sees all of them), then, conversation by conversation, the tiles of the
-    // conversations the M-tile's tokens belong to, masked causally; the chain's last unit writes out and lse
-    // directly -- no partials, no merge, and no row streams its diagonal by itself.
+    const uint32_t n_rt = (T + tpt - 1) / tpt;
+    const int32_t n_strands = (int32_t)strands.size();
     PlanSlot *cur = ctx->cur_slot >= 0 ? &ctx->slots[ctx->cur_slot] : nullptr;
     if (cur && cur->valid) {
         CART_CUDA(ctx, cudaEventRecord(cur->ev, cur->last_stream));
@@ -1433,22 +1458,26 @@ cart_status cart_train_attention_fwd(cart_ctx *ctx, int32_t layer, const cart_re
     cart_shared_unit *units = reinterpret_cast<cart_shared_unit *>(ns.host + lay.units_off);
     uint32_t *unit_cta_begin = reinterpret_cast<uint32_t *>(ns.host + lay.unit_cta_begin_off);
     uint32_t *readers = reinterpret_cast<uint32_t *>(ns.host + lay.readers_off);
-    if ((int64_t)T > lay.readers_cap) return fail(ctx, CART_ERR_CAPACITY, "train: %u tokens exceed the reader table", T);
-    for (uint32_t t = 0; t < T; ++t) readers[t] = t;   // reader entry t = token t = query row t
-    // tiles of every chain, to balance the blocks
+    if ((int64_t)T > lay.readers_cap) return fail(ctx, CART_ERR_CAPACITY, "%u rows exceed the reader table", T);
+    for (uint32_t t = 0; t < T; ++t) readers[t] = t;   // reader entry t = query row t
+    uint32_t part_tiles = 0;
+    for (const ChainPart &pt : parts) part_tiles += (pt.p + 127u) / 128u;
+    // keys of strand c that the rows of [a, b) need: up to the last of its rows in the tile
+    auto needed = [&](const ChainStrand &st, uint32_t b) {
+        const uint32_t last_row = std::min(b, st.row_begin + st.n_rows) - 1u;
+        return st.key_first + (last_row - st.row_begin) + 1u;
+    };
     std::vector<uint32_t> chain_tiles(n_rt, 0);
-    std::vector<int32_t> first_conv(n_rt, 0);
+    std::vector<int32_t> first_strand(n_rt, 0);
     {
         int32_t c = 0;
         for (uint32_t rt = 0; rt < n_rt; ++rt) {
             const uint32_t a = rt * tpt, b = std::min(T, a + tpt);
-            while ((uint32_t)tb.cu[(size_t)c + 1] <= a) ++c;
-            first_conv[rt] = c;
-            uint32_t tiles = (p + 127u) / 128u;
-            for (int32_t cc = c; cc < n_convs && (uint32_t)tb.cu[(size_t)cc] < b; ++cc) {
-                const uint32_t last = std::min<uint32_t>(b, (uint32_t)tb.cu[(size_t)cc + 1]) - 1u;   // last token of cc in the tile
-                tiles += (last - (uint32_t)tb.cu[(size_t)cc] + 1u + 127u) / 128u;
-            }
+            while (strands[(size_t)c].row_begin + strands[(size_t)c].n_rows <= a) ++c;
+            first_strand[rt] = c;
+            uint32_t tiles = part_tiles;
+            for (int32_t cc = c; cc < n_strands && strands[(size_t)cc].row_begin < b; ++cc)
+                tiles += (needed(strands[(size_t)cc], b) + 127u) / 128u;
             chain_tiles[rt] = tiles;
         }
     }
@@ -1479,37 +1508,45 @@ cart_status cart_train_attention_fwd(cart_ctx *ctx, int32_t layer, const cart_re
                 first = false;
                 units[nu++] = u;
             };
-            int32_t c_last = first_conv[rt];
-            while (c_last + 1 < n_convs && (uint32_t)tb.cu[(size_t)c_last + 1] < b) ++c_last;
-            if (p > 0) {
+            int32_t c_last = first_strand[rt];
+            while (c_last + 1 < n_strands && strands[(size_t)c_last + 1].row_begin < b) ++c_last;
+            for (const ChainPart &pt : parts) {
                 cart_shared_unit u{};
-                u.k_row = (uint32_t)(tb.z->k_row + (uint64_t)g * p);
-                u.v_row = (uint32_t)(tb.z->v_row + (uint64_t)g * p);
-                u.layer_stride = (uint32_t)Hkv * p;
-                u.n_tiles = (p + 127u) / 128u;
-                u.flags = (p % 128u) ? CART_UNIT_MASKED : 0;
-                u.lim_base = (int32_t)p - 1;
-                u.lim_cap = (int32_t)p - 1;
+                u.k_row = (uint32_t)(pt.k_row + (uint64_t)g * pt.p);
+                u.v_row = (uint32_t)(pt.v_row + (uint64_t)g * pt.p);
+                u.layer_stride = (uint32_t)Hkv * pt.p;
+                u.n_tiles = (pt.p + 127u) / 128u;
+                u.flags = (pt.p % 128u) ? CART_UNIT_MASKED : 0;
+                u.lim_base = (int32_t)pt.p - 1;
+                u.lim_cap = (int32_t)pt.p - 1;
                 u.tr_hi = tpt;
                 emit(u, false);
             }
-            for (int32_t c = first_conv[rt]; c <= c_last; ++c) {
-                const Request &r = ctx->reqs[(size_t)convs[c]];
-                const uint32_t c0 = (uint32_t)tb.cu[(size_t)c], c1 = (uint32_t)tb.cu[(size_t)c + 1];
-                const uint32_t last = std::min(b, c1) - 1u;   // last token of the conversation in the M-tile
+            for (int32_t c = first_strand[rt]; c <= c_last; ++c) {
+                const ChainStrand &st = strands[(size_t)c];
                 cart_shared_unit u{};
-                u.k_row = (uint32_t)(r.k_row + (uint64_t)g * r.cap);
-                u.v_row = (uint32_t)(r.v_row + (uint64_t)g * r.cap);
-                u.layer_stride = (uint32_t)((uint64_t)Hkv * r.cap);
-                u.n_tiles = (last - c0 + 1u + 127u) / 128u;
+                u.k_row = (uint32_t)(st.k_row + (uint64_t)g * st.cap);
+                u.v_row = (uint32_t)(st.v_row + (uint64_t)g * st.cap);
+                u.layer_stride = (uint32_t)((uint64_t)Hkv * st.cap);
+                u.n_tiles = (needed(st, b) + 127u) / 128u;
                 u.flags = CART_UNIT_MASKED | CART_UNIT_SUFFIX;
-                u.lim_base = (int32_t)a - (int32_t)c0;      // token offset 0 of the M-tile sees keys 0 .. a - c0
-                u.lim_cap = (int32_t)(c1 - c0) - 1;         // the conversation's last stored key
-                u.tr_hi = c1 - a;                           // tokens from here on belong to later conversations
+                // token offset 0 of the M-tile is the strand's row a - row_begin (negative: the strand starts inside the tile)
+                u.lim_base = (int32_t)st.key_first + ((int32_t)a - (int32_t)st.row_begin);
+                u.lim_cap = (int32_t)st.len - 1;                   // the strand's last stored key
+                u.tr_hi = st.row_begin + st.n_rows - a;            // tokens from here on belong to later strands
                 emit(u, c == c_last);
             }
         }
-    if (full) return fail(ctx, CART_ERR_CAPACITY, "train: more than %d units", lay.units_cap);
+    if (full) return fail(ctx, CART_ERR_CAPACITY, "more than %d units", lay.units_cap);
+    // a chain's first unit names the distance to the next chain (the kernel fetches that chain's query rows ahead)
+    {
+        size_t next_start = nu;
+        for (size_t i = nu; i-- > 0;) {
+            if (units[i].flags & CART_UNIT_CONT) continue;
+            units[i].reserved = next_start < nu ? (uint32_t)(next_start - i) : 0u;
+            next_start = i;
+        }
+    }
     while (blk + 1 <= n_blocks) unit_cta_begin[++blk] = (uint32_t)nu;
     for (uint32_t b2 = blk; b2 < (uint32_t)kMaxCta; ++b2) unit_cta_begin[b2 + 1] = (uint32_t)nu;
     const uint64_t sh_bytes = lay.units_off + (uint64_t)nu * sizeof(cart_shared_unit) - lay.shared_off;
@@ -1545,6 +1582,30 @@ cart_status cart_train_attention_fwd(cart_ctx *ctx, int32_t layer, const cart_re
     ++ctx->launches;
     CART_CUDA(ctx, cudaEventRecord(ns.ev, s));
     return CART_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+cart_status cart_train_attention_fwd(cart_ctx *ctx, int32_t layer, const cart_req *convs, int32_t n_convs, const void *q,
+                                     void *out, float *lse, void *stream)
+{
+    if (!ctx) return CART_ERR_INVALID_ARG;
+    if (!lse) return fail(ctx, CART_ERR_INVALID_ARG, "train: the forward must write lse");
+    TrainBatch tb;
+    const cart_status st = train_batch(ctx, layer, convs, n_convs, &tb);
+    if (st != CART_OK) return st;
+    if (!aligned16(q) || !aligned16(out)) return fail(ctx, CART_ERR_INVALID_ARG, "train: null/misaligned pointer");
+    std::vector<ChainPart> parts;
+    if (tb.z) parts.push_back(ChainPart{tb.z->k_row, tb.z->v_row, (uint32_t)tb.z->p});
+    std::vector<ChainStrand> strands;
+    for (int32_t c = 0; c < n_convs; ++c) {
+        const Request &r = ctx->reqs[(size_t)convs[c]];
+        strands.push_back(ChainStrand{r.k_row, r.v_row, (uint32_t)r.cap, (uint32_t)tb.len[(size_t)c],
+                                      (uint32_t)tb.cu[(size_t)c], (uint32_t)tb.len[(size_t)c], 0u});
+    }
+    return launch_chains(ctx, layer, parts, strands, (uint32_t)tb.T, q, out, lse, static_cast<cudaStream_t>(stream));
 }
 
 cart_status cart_train_attention_bwd(cart_ctx *ctx, int32_t layer, const cart_req *convs, int32_t n_convs, const void *q,

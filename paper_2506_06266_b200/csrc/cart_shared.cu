@@ -292,7 +292,7 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
             };
             // Two cursors walk the block's tiles in order: `qk` names the next score product to issue (it
             // runs two tiles ahead), `pv` the next P V product.  tt = tile index counted over the block.
-            struct Cursor { uint32_t ui, t, n, unit_no, cont; };
+            struct Cursor { uint32_t ui, t, n, unit_no, cont; };  // unit_no counts the units that bring their own query rows
             auto tiles_of = [&](uint32_t ui) { return ui < unit_end ? p.units[ui].n_tiles : 0u; };
             auto cont_of = [&](uint32_t ui) {
                 return kChains && ui < unit_end ? (uint32_t)(p.units[ui].flags & CART_UNIT_CONT) : 0u;
@@ -301,10 +301,10 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
             auto advance = [&](Cursor &c) {
                 if (++c.t == c.n) {
                     ++c.ui;
-                    ++c.unit_no;
                     c.t = 0;
                     c.n = tiles_of(c.ui);
                     c.cont = cont_of(c.ui);
+                    if (c.cont == 0u) ++c.unit_no;   // (a unit that continues a chain keeps its rows and their query buffer)
                 }
             };
             uint32_t total = 0;
@@ -316,7 +316,7 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                 const uint32_t sb = tt % (uint32_t)kSBufs;
                 const uint32_t kst = tt % (uint32_t)kKStages, kpar = (tt / (uint32_t)kKStages) & 1u;
                 const uint32_t qb = qk.unit_no & 1u;
-                if (qk.t == 0u && !wait_all(kBarQReady + (int)qb, (qk.unit_no >> 1) & 1u)) return false;
+                if (qk.t == 0u && qk.cont == 0u && !wait_all(kBarQReady + (int)qb, (qk.unit_no >> 1) & 1u)) return false;
                 if (!wait_all(kBarKFull + (int)kst, kpar)) return false;
                 tc_fence_after();
                 const uint32_t q_lo = base + kOffQ + qb * kShTileBytes;
@@ -371,7 +371,7 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                 // tile) may need this tile's P V product first.
                 bool s_issued = tt + 2u >= total;
                 if (!s_issued) {
-                    const bool q_there = qk.t != 0u || __all_sync(0xffffffffu, mbar_try_wait(bar(kBarQReady + (int)(qk.unit_no & 1u)),
+                    const bool q_there = qk.t != 0u || qk.cont != 0u || __all_sync(0xffffffffu, mbar_try_wait(bar(kBarQReady + (int)(qk.unit_no & 1u)),
                                                                                          (qk.unit_no >> 1) & 1u));
                     if (q_there) {
                         ok = issue_s(tt + 2u);
@@ -416,21 +416,23 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
         // n - 1, the buffer's last readers, were complete before the first scores of unit n arrived).
         const int i_reader = row / G, h = row - i_reader * G;
         const __nv_bfloat16 *q = reinterpret_cast<const __nv_bfloat16 *>(p.q);
-        uint4 qv[8];
-        auto load_q = [&](const cart_shared_unit &uu, uint32_t batch, bool on) {
-            const uint4 *src = reinterpret_cast<const uint4 *>(
-                q + ((size_t)batch * p.n_q_heads + (size_t)uu.kv_head * G + h) * kHeadDim) + 8 * wg;
-#pragma unroll
-            for (uint32_t c = 0; c < 8; ++c) qv[c] = on ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);  // all in flight
+        // The copies are cp.async (global to shared memory without passing through registers: 32 registers held over a
+        // tile's arithmetic were what made this loop spill); load_q requests a unit's rows into buffer `buf`, store_q
+        // waits for them and tells the MMA warp.
+        auto q_src = [&](uint32_t kv_head, uint32_t batch) {   // this thread's 128 bytes of a unit's query rows
+            return reinterpret_cast<const uint8_t *>(q + ((size_t)batch * p.n_q_heads + (size_t)kv_head * G + h) * kHeadDim) + 128 * wg;
         };
-        auto store_q = [&](uint32_t buf) {
+        auto load_q = [&](const uint8_t *src, bool on, uint32_t buf) {
             const uint32_t qrow = base + kOffQ + buf * kShTileBytes + (uint32_t)wg * kShBlock + (uint32_t)row * 128u;
             const uint32_t swz = (uint32_t)(row & 7);
 #pragma unroll
-            for (uint32_t c = 0; c < 8; ++c)
-                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(qrow + ((c ^ swz) << 4)), "r"(qv[c].x),
-                             "r"(qv[c].y), "r"(qv[c].z), "r"(qv[c].w)
+            for (uint32_t c = 0; c < 8; ++c)   // (size 0: zeros are written instead)
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(qrow + ((c ^ swz) << 4)),
+                             "l"(on ? src + 16u * c : reinterpret_cast<const uint8_t *>(q)), "r"(on ? 16u : 0u)
                              : "memory");
+        };
+        auto store_q = [&](uint32_t buf) {
+            asm volatile("cp.async.wait_all;" ::: "memory");
             fence_async_smem();   // these writes before the tensor core's reads of the operand
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(kBarQReady + (int)buf));
@@ -446,26 +448,39 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
             if (lane == 0) ok0 = wait_for_prior_kernels(p, abort_flag);
             alive = __all_sync(0xffffffffu, ok0);  // (from here on the partial slots and the tickets are this kernel's too)
             if (unit_begin < unit_end) {
-                load_q(u, batch, on && alive);
+                load_q(q_src(u.kv_head, batch), on && alive, 0u);
                 store_q(0u);
             }
         }
 
         float m_run = -INFINITY, l_run = 0.f;
         bool fresh = true;   // no tile of the chain has been seen yet
-        uint32_t unit_no = 0;
-        for (uint32_t ui = unit_begin; ui < unit_end; ++ui, ++unit_no) {
+        uint32_t unit_no = 0;   // counts the units that bring their own query rows (not those that continue a chain)
+        for (uint32_t ui = unit_begin; ui < unit_end; ++ui) {
             if (ui != unit_begin) {
                 u = u_next;
                 u_next = cart_shared_unit{};
                 if (ui + 1u < unit_end) u_next = p.units[ui + 1u];
             }
-            const bool has_next = ui + 1u < unit_end;
+            const bool brings_rows = !kChains || !(u.flags & CART_UNIT_CONT);
+            if (brings_rows && ui != unit_begin) ++unit_no;
+            // the next unit with rows of its own (the units of a chain in between reuse this one's)
+            bool has_next = false;
+            cart_shared_unit uq{};
+            if (brings_rows) {
+                // (in a plan with chains the unit says how many units on the next chain begins)
+                const uint32_t uj = kChains ? ui + (u.reserved ? u.reserved : (unit_end - ui)) : ui + 1u;
+                has_next = uj < unit_end;
+                if (has_next) uq = uj == ui + 1u ? u_next : p.units[uj];
+            }
             const bool valid = (uint32_t)i_reader < u.n_readers;
-            const bool valid_next = has_next && (uint32_t)i_reader < u_next.n_readers;
-            uint32_t batch_next = 0;
-            if (valid_next) batch_next = p.readers[u_next.reader_begin + (uint32_t)i_reader];
-            const uint32_t t_store = u.n_tiles > 1u ? 1u : 0u;  // the tile after which the next unit's rows are stored
+            const bool valid_next = has_next && (uint32_t)i_reader < uq.n_readers;
+            const uint8_t *src_next = reinterpret_cast<const uint8_t *>(q);
+            if (valid_next) src_next = q_src(uq.kv_head, p.readers[uq.reader_begin + (uint32_t)i_reader]);
+            // the tiles after which the next unit's rows are requested and stored: in a plan with chains the request
+            // hangs on two dependent reads issued above, which get two tiles' time
+            const uint32_t t_load = kChains ? (u.n_tiles > 2u ? 2u : u.n_tiles - 1u) : 0u;
+            const uint32_t t_store = kChains ? (u.n_tiles > 4u ? 4u : u.n_tiles - 1u) : (u.n_tiles > 1u ? 1u : 0u);
             const bool direct = kChains && (u.flags & CART_UNIT_DIRECT) != 0u, hold = kChains && (u.flags & CART_UNIT_HOLD) != 0u;
             const bool masked = kChains && (u.flags & CART_UNIT_MASKED) != 0u;
             uint32_t slot = 0;   // where this row's partial goes, or (direct) its query row: needed at the unit's end
@@ -509,10 +524,13 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
 #pragma unroll
                         for (int k = 0; k < 64; k += 2) mx = fmaxf(mx, fmaxf(__uint_as_float(s[k]), __uint_as_float(s[k + 1])));
                     } else {
-                        // (what lies past a row's limit may be anything, NaN included: it is left out, not compared)
+                        // (what lies past a row's limit may be anything, NaN included: it is left out of the maximum
+                        //  and replaced by -inf, which the exponential below turns into a probability of zero)
 #pragma unroll
-                        for (int k = 0; k < 64; ++k)
+                        for (int k = 0; k < 64; ++k) {
                             if (kidx0 + k <= limit) mx = fmaxf(mx, __uint_as_float(s[k]));
+                            else s[k] = 0xFF800000u;
+                        }
                     }
                     mx *= p.scale_log2;
                 }
@@ -559,18 +577,15 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                 // probabilities of this thread's 64 tokens, as bf16 pairs (the even token in the low half), written
                 // over the first 32 columns of the scores they came from: the A operand of the second product
                 float psum0 = 0.f, psum1 = 0.f;
+                // (a row of a masked run that has not seen a key yet has no reference: all its scores are -inf here)
+                const float m_use = kChains && m_run == -INFINITY ? 0.f : m_run;
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
                     uint32_t w[16];
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
-                        float p0 = fast_exp2(fmaf(__uint_as_float(s[32 * c + 2 * j]), p.scale_log2, -m_run));
-                        float p1 = fast_exp2(fmaf(__uint_as_float(s[32 * c + 2 * j + 1]), p.scale_log2, -m_run));
-                        if (!all_on) {
-                            const int32_t kidx = (int32_t)(t * (uint32_t)kShTile + col0) + 32 * c + 2 * j;
-                            if (kidx > limit) p0 = 0.f;
-                            if (kidx + 1 > limit) p1 = 0.f;
-                        }
+                        const float p0 = fast_exp2(fmaf(__uint_as_float(s[32 * c + 2 * j]), p.scale_log2, -m_use));
+                        const float p1 = fast_exp2(fmaf(__uint_as_float(s[32 * c + 2 * j + 1]), p.scale_log2, -m_use));
                         psum0 += p0;
                         psum1 += p1;
                         w[j] = pack_bf16(p0, p1);
@@ -600,7 +615,7 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(kBarPReady + (int)sb));
                 if (has_next) {
-                    if (t == 0u) load_q(u_next, batch_next, valid_next);
+                    if (t == t_load) load_q(src_next, valid_next, (unit_no + 1u) & 1u);
                     if (t == t_store) store_q((unit_no + 1u) & 1u);
                 }
             }

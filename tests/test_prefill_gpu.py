@@ -91,6 +91,15 @@ def test_prefill_of_a_long_message_shares_the_suffix_in_causal_steps(Hq, Hkv, s_
     run(Hq, Hkv, 200, s_old, n_new, layers=1, seed=6)
 
 
+@pytest.mark.parametrize("Hq,Hkv,p,parts,s_old,n_new", [(32, 8, 300, 1, 100, 640), (24, 8, 128, 2, 0, 820),
+                                                        (8, 8, 0, 1, 77, 2500)])
+def test_prefill_of_a_message_that_fills_the_device_runs_as_chains_of_masked_tiles(Hq, Hkv, p, parts, s_old, n_new):
+    # 128 / G new tokens x a KV head make one chain on the tensor-core kernel: the Cartridge part(s), then the suffix up
+    # to each row's own token under a causal mask (Cartridge and suffix ends inside tiles, a group of three heads whose
+    # row tiles hold two rows no token owns, no Cartridge at all); with at least one chain per SM the call takes this path
+    run(Hq, Hkv, p, s_old, n_new, parts=parts, layers=1, seed=8)
+
+
 def test_prefill_errors():
     sess = H.Session(1, 32, 8, 8 << 20, max_requests=8)
     try:
