@@ -1323,11 +1323,13 @@ cart_status cart_prefill_attention(cart_ctx *ctx, int32_t layer, cart_req req, c
     // A message long enough to give every SM a chain (an M-tile of 128 / G tokens times a KV head) goes through
     // chains of masked tiles: one kernel, the diagonal on the tensor cores too (1024 tokens over a 2048-token
     // Cartridge: 218 us per layer against 256).  Shorter messages have too few chains to fill the device (256
-    // tokens: 110 us against 90) and go, like paged suffixes, through the decode kernels, which split the keys.
+    // tokens: 110 us against 90) and go, like paged suffixes, through the decode kernels, which split the keys; so
+    // do suffixes beyond 16 k tokens, where every chain re-reads the whole suffix and the decode kernels' shared
+    // steps read it once per group of steps (1024 tokens behind 30 k: 775 us against 680).
     Request *r = get_req(ctx, req);
     const int32_t tpt = 128 / ctx->group;
     if (r && !r->paged && !r->evicted && ctx->share_min_readers > 0 && n_new <= ctx->cfg.max_requests &&
-        (int64_t)((n_new + tpt - 1) / tpt) * ctx->cfg.n_kv_heads >= ctx->n_cta &&
+        (int64_t)((n_new + tpt - 1) / tpt) * ctx->cfg.n_kv_heads >= ctx->n_cta && r->len[(size_t)std::max(0, std::min(layer, ctx->cfg.n_layers - 1))] <= 16384 &&
         layer >= 0 && layer < ctx->cfg.n_layers && r->len[(size_t)layer] >= n_new && evicted_part(ctx, *r) < 0 && aligned16(q) &&
         aligned16(out)) {
         std::vector<ChainPart> parts;
