@@ -474,9 +474,14 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                 if (has_next) uq = uj == ui + 1u ? u_next : p.units[uj];
             }
             const bool valid = (uint32_t)i_reader < u.n_readers;
-            const bool valid_next = has_next && (uint32_t)i_reader < uq.n_readers;
-            const uint8_t *src_next = reinterpret_cast<const uint8_t *>(q);
-            if (valid_next) src_next = q_src(uq.kv_head, p.readers[uq.reader_begin + (uint32_t)i_reader]);
+            // (in a plan with chains uq is a load in flight here, and the reader's batch index one more: they are looked
+            //  at a tile later, so that nothing waits for them at the start of a chain)
+            bool valid_next = false;
+            uint32_t batch_next = 0;
+            if (!kChains && has_next) {
+                valid_next = (uint32_t)i_reader < uq.n_readers;
+                if (valid_next) batch_next = p.readers[uq.reader_begin + (uint32_t)i_reader];
+            }
             // the tiles after which the next unit's rows are requested and stored: in a plan with chains the request
             // hangs on two dependent reads issued above, which get two tiles' time
             const uint32_t t_load = kChains ? (u.n_tiles > 2u ? 2u : u.n_tiles - 1u) : 0u;
@@ -615,7 +620,11 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(kBarPReady + (int)sb));
                 if (has_next) {
-                    if (t == t_load) load_q(src_next, valid_next, (unit_no + 1u) & 1u);
+                    if (kChains && t == 0u) {
+                        valid_next = (uint32_t)i_reader < uq.n_readers;
+                        if (valid_next) batch_next = p.readers[uq.reader_begin + (uint32_t)i_reader];
+                    }
+                    if (t == t_load) load_q(q_src(uq.kv_head, batch_next), valid_next, (unit_no + 1u) & 1u);
                     if (t == t_store) store_q((unit_no + 1u) & 1u);
                 }
             }
