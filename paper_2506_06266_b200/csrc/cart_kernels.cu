@@ -244,8 +244,13 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
         // before this one -- so the first suffix tile is fetched only after griddepcontrol.wait.
         bool waited = false;
         uint32_t tails_seen = 0;  // tiles met so far that end with a new token
+        // The next work item is requested while the copies of this one are issued: read at the item's start, it
+        // held the ring back by a memory round trip per item, which short row groups cannot spare.
+        cart_work_item w_next{};
+        if (item_begin < item_end) w_next = p.items[item_begin];
         for (uint32_t it = item_begin; it < item_end && ok; ++it) {
-            cart_work_item w = p.items[it];
+            cart_work_item w = w_next;
+            if (it + 1 < item_end) w_next = p.items[it + 1];
             if (w.flags & CART_ITEM_TAIL) w.n_tok += p.grow;  // tokens appended since the plan was built
             const uint32_t k_row = w.k_row + (uint32_t)p.layer * w.layer_stride;
             const uint32_t v_row = w.v_row + (uint32_t)p.layer * w.layer_stride;
@@ -296,8 +301,8 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
                     }
                     ok = __shfl_sync(0xffffffffu, (int)ok1, 0) != 0;
                     if (!ok) break;
-                    // those generic-proxy stores before the TMA reads below (every issuing lane fences for itself)
-                    asm volatile("fence.proxy.async;" ::: "memory");
+                    // (the append warp has ordered its generic-proxy stores before the TMA reads that follow its
+                    // release: the proxy fence is on the writer's side, off the path of the copies)
                 }
                 {
                     // The tile's four boxes (K and V, each as two 64-dim halves) are requested by four lanes in
@@ -395,6 +400,7 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
                     for (int u = 0; u < 4; ++u)
                         if (u < n) reinterpret_cast<uint4 *>(p.arena)[dst[u]] = val[u];
                     __threadfence();  // the rows are in memory before the producer hears of them
+                    asm volatile("fence.proxy.async;" ::: "memory");  // ... and before the TMA reads it then issues
                     __syncwarp();
                     n_done += (uint32_t)n;
                     if (lane == 0)
