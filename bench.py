@@ -514,6 +514,8 @@ def run_prefill(args):
     ctx = binding.cart_create(cfg)
     k, v = w.cartridge_kv(0, dev)
     cart = binding.cart_register_cartridge(ctx, k, v, w.p, stream)
+    if args.prefill_split >= 0:
+        binding.cart_set_prefill_split(ctx, args.prefill_split)
     req = binding.cart_request_open(ctx, cart, s_old + reps * T)
     ks, vs = w.suffix_kv(0, s_old, dev)
     for layer in range(L):
@@ -728,6 +730,8 @@ def main():
                     help="the requests' suffixes are stored in pages of 64 tokens (cart_request_open_paged)")
     ap.add_argument("--unfused", action="store_true",
                     help="append and attend with two calls per layer instead of cart_decode_step")
+    ap.add_argument("--prefill-split", type=int, default=-1,
+                    help="pieces a short message's chains are cut into (cart_set_prefill_split); -1 keeps the library's choice")
     ap.add_argument("--piece-cost", type=int, default=-1,
                     help="planner tuning (cart_set_piece_cost); -1 keeps the library's default")
     ap.add_argument("--side-by-side", type=int, default=-1,

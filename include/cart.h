@@ -224,10 +224,12 @@ CART_API cart_status cart_decode_step(cart_ctx *ctx, int32_t layer, const cart_r
  * [n_new][n_q_heads][128], token-major as the projection produces it) is the query of the i-th new
  * token and attends, per Eq. 1 with its causal sum over j <= i, to the request's Cartridge(s), the
  * suffix tokens before the new ones and the new tokens 0 .. i.  out, lse as in cart_decode_attention,
- * with n_new rows.  When n_new reaches the sharing threshold, the Cartridge(s) are read once for all
- * rows and the suffix before each group of 128 / (n_q_heads / n_kv_heads) consecutive new tokens once
- * for that group (tensor-core kernel); a row reads by itself only the fewer than 128 + 128 / G tokens
- * around the causal diagonal.  n_new <= max_requests.
+ * with n_new rows.  A message of 4 tokens or more behind a contiguous suffix of at most 16 k tokens runs on the
+ * tensor cores throughout: per group of 128 / (n_q_heads / n_kv_heads) consecutive new tokens and KV head, the
+ * Cartridge(s) and the suffix up to the group's last token are read once, the tiles on the causal diagonal masked
+ * per row (see cart_set_prefill_split for short messages).  Otherwise, when n_new reaches the sharing threshold,
+ * the Cartridge(s) are read once for all rows and the suffix before each group once for that group, and a row
+ * reads by itself only the fewer than 128 + 128 / G tokens around the causal diagonal.  n_new <= max_requests.
  * Errors: INVALID_ARG (also: the suffix holds fewer than n_new tokens), BAD_HANDLE, CAPACITY, CUDA. */
 CART_API cart_status cart_prefill_attention(cart_ctx *ctx, int32_t layer, cart_req req, const void *q /*device*/,
                                    int32_t n_new, void *out /*device*/, float *lse /*device or NULL*/,
@@ -289,6 +291,16 @@ CART_API cart_status cart_set_side_by_side(cart_ctx *ctx, int32_t mode);
  * units of the time a 64-token tile takes.  Default 3; 0 balances by tiles alone; at most 64.  The
  * results do not depend on it beyond fp32 rounding.  Errors: INVALID_ARG. */
 CART_API cart_status cart_set_piece_cost(cart_ctx *ctx, int32_t tiles_per_piece);
+
+/* How cart_prefill_attention runs a message that is too short to give every SM a chain of tensor-core tiles (a
+ * chain: 128 / G consecutive new tokens times a KV head, over the Cartridge(s) and the suffix up to the causal
+ * diagonal).  -1 (default): with fewer chains than half the SMs, every chain is cut along its keys into as many
+ * pieces of two tiles or more as give every SM one, and a merge kernel combines the pieces' partial results;
+ * messages of fewer than 4 tokens go through the decode kernels.  0: short messages go through the decode kernels
+ * (the shared tiles on the tensor cores, each row's stretch of the causal diagonal streamed by itself).  1 .. 64:
+ * cut into this many pieces (1: whole chains, however few).  Results are the same up to fp32 rounding.
+ * Errors: INVALID_ARG. */
+CART_API cart_status cart_set_prefill_split(cart_ctx *ctx, int32_t pieces);
 
 /* Plan reuse.  The attention calls split the batch's KV tokens over the thread blocks on the host (a
  * "plan") and upload the result.  In a decode loop (Sec. 2.3) every request grows by one token per step, so

@@ -31,7 +31,7 @@ EXPORTS = ["cart_scratch_bytes", "cart_create", "cart_destroy", "cart_register_c
            "cart_append_kv", "cart_extend_kv", "cart_decode_attention", "cart_decode_step", "cart_prefill_attention", "cart_suffix_len",
            "cart_kv_bytes", "cart_sync_status", "cart_set_timing", "cart_get_timing",
            "cart_set_share_min_readers", "cart_set_piece_cost", "cart_plan_build_shared",
-           "cart_set_plan_reuse", "cart_plan_count", "cart_plan_reusable", "cart_set_side_by_side",
+           "cart_set_plan_reuse", "cart_set_prefill_split", "cart_plan_count", "cart_plan_reusable", "cart_set_side_by_side",
            "cart_request_open_paged", "cart_evict_request", "cart_restore_request", "cart_evict_cartridge",
            "cart_restore_cartridge", "cart_train_attention_fwd", "cart_train_attention_bwd",
            "cart_decode_attention_static", "cart_launch_count", "cart_status_string",
@@ -154,6 +154,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.cart_plan_count.argtypes = [vp]
     lib.cart_plan_count.restype = ctypes.c_uint64
     lib.cart_set_plan_reuse.argtypes = [vp, i32]
+    lib.cart_set_prefill_split.argtypes = [vp, i32]
     lib.cart_set_side_by_side.argtypes = [vp, i32]
     lib.cart_plan_reusable.argtypes = [i32p, i32p, i32, i32, i32p]
     lib.cart_status_string.argtypes = [ctypes.c_int]
@@ -375,6 +376,10 @@ def cart_set_piece_cost(ctx: int, tiles_per_piece: int) -> None:
 
 def cart_set_side_by_side(ctx: int, mode: int) -> None:
     _check(load_library().cart_set_side_by_side(ctx, int(mode)), "cart_set_side_by_side", ctx)
+
+
+def cart_set_prefill_split(ctx: int, pieces: int) -> None:
+    _check(load_library().cart_set_prefill_split(ctx, int(pieces)), "cart_set_prefill_split", ctx)
 
 
 def cart_set_plan_reuse(ctx: int, max_grow_tokens: int) -> None:

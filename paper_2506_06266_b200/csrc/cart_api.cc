@@ -137,6 +137,11 @@ struct PlanSlot {
     uint64_t epoch = 0;
     int32_t n_items = 0, n_merges = 0, n_cta_used = 0, n_slots = 0;
     int32_t n_units = 0, n_unit_cta_used = 0;
+    // a plan of chains (prefill of a message, training forward): what it was built from and where its tables are
+    bool chain = false;
+    std::vector<uint64_t> chain_key;
+    uint32_t chain_blocks = 0, chain_merges = 0;
+    uint64_t chain_off[6] = {0, 0, 0, 0, 0, 0};
 };
 
 }  // namespace
@@ -151,6 +156,7 @@ struct cart_ctx {
     int piece_cost = kPieceCostTiles;
     int max_grow = kMaxGrowTokens;
     int side_by_side = 1;        // shared and stream kernel share the SMs (0: one after the other; > 1: blocks for the shared kernel)
+    int prefill_split = -1;      // pieces a short message's chains are cut into along the keys (-1: chosen per call; 0: never)
     uint32_t pair_seq = 0;       // counts side-by-side launches (the value the stream kernel hands to the shared kernel)
     uint64_t plans_built = 0;
     uint64_t n_rows = 0;
@@ -171,6 +177,9 @@ struct cart_ctx {
     std::vector<int32_t> seg_begin_tmp;
     std::vector<uint32_t> key_tmp;
     std::vector<int32_t> len_tmp;
+    std::vector<uint64_t> chain_key_tmp;
+    std::vector<cart_shared_unit> unit_tmp;
+    std::vector<uint32_t> piece_tmp;
     bool timing = false;
     std::vector<cudaEvent_t> ev_pool;  // pairs: start, stop
     size_t ev_used = 0;
@@ -182,7 +191,7 @@ namespace {
 struct ChainPart { uint64_t k_row, v_row; uint32_t p; };
 struct ChainStrand { uint64_t k_row, v_row; uint32_t cap, len, row_begin, n_rows, key_first; };
 cart_status launch_chains(cart_ctx *ctx, int32_t layer, const std::vector<ChainPart> &parts, const std::vector<ChainStrand> &strands,
-                          uint32_t T, const void *q, void *out, float *lse, cudaStream_t s);
+                          uint32_t T, const void *q, void *out, float *lse, cudaStream_t s, uint32_t n_split = 1);
 
 cart_status fail(cart_ctx *ctx, cart_status st, const char *fmt, ...)
 {
@@ -477,6 +486,14 @@ cart_status cart_set_side_by_side(cart_ctx *ctx, int32_t mode)
     if (mode < 0 || mode >= ctx->n_cta) return fail(ctx, CART_ERR_INVALID_ARG, "side_by_side: out of range");
     ctx->side_by_side = mode;
     ++ctx->epoch;
+    return CART_OK;
+}
+
+cart_status cart_set_prefill_split(cart_ctx *ctx, int32_t pieces)
+{
+    if (!ctx) return CART_ERR_INVALID_ARG;
+    if (pieces < -1 || pieces > 64) return fail(ctx, CART_ERR_INVALID_ARG, "prefill_split: out of range");
+    ctx->prefill_split = pieces;
     return CART_OK;
 }
 
@@ -1047,6 +1064,7 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
             ns.ev_recorded = false;
         }
         ns.valid = false;
+        ns.chain = false;
         // Paged suffixes.  In a fused decode loop every request takes a new page once per 64 steps, each at a step
         // of its own, and a new page means a new plan; so when a plan is built anyway, requests with less than a
         // page of room are given their next page now (if the arena has one), and the plan lasts 64 steps or more.
@@ -1320,27 +1338,47 @@ cart_status cart_prefill_attention(cart_ctx *ctx, int32_t layer, cart_req req, c
 {
     if (!ctx) return CART_ERR_INVALID_ARG;
     if (n_new < 1) return fail(ctx, CART_ERR_INVALID_ARG, "prefill: n_new < 1");
-    // A message long enough to give every SM a chain (an M-tile of 128 / G tokens times a KV head) goes through
-    // chains of masked tiles: one kernel, the diagonal on the tensor cores too (1024 tokens over a 2048-token
-    // Cartridge: 218 us per layer against 256).  Shorter messages have too few chains to fill the device (256
-    // tokens: 110 us against 90) and go, like paged suffixes, through the decode kernels, which split the keys; so
-    // do suffixes beyond 16 k tokens, where every chain re-reads the whole suffix and the decode kernels' shared
-    // steps read it once per group of steps (1024 tokens behind 30 k: 775 us against 680).
+    // A message goes through chains of masked tiles on the tensor-core kernel, the diagonal too: a chain is an M-tile
+    // of 128 / G tokens times a KV head, over the Cartridge(s) and the suffix up to the M-tile's last token.  With a
+    // chain or more per SM, or at least half as many, every chain writes its rows' output itself (1024 tokens over a
+    // 2048-token Cartridge: 194 us per layer against 256 through the decode kernels; 512 tokens: 75 against 122).
+    // A shorter message has too few chains to fill the device, so each chain is cut along its keys into pieces of at
+    // least two tiles, as many as give every SM one, and the merge kernel combines the pieces' partials (64 tokens:
+    // 25 us against 34; 256: 40 against 67).  Paged suffixes, messages of fewer than four tokens (decode in all but
+    // name: 2 tokens take 20 us there, 25 as chains) and suffixes beyond 16 k tokens -- where every chain re-reads the
+    // whole suffix while the decode kernels' shared steps read it once per group of steps (1024 tokens behind 30 k:
+    // 775 us against 680) -- go through the decode kernels.
     Request *r = get_req(ctx, req);
     const int32_t tpt = 128 / ctx->group;
     if (r && !r->paged && !r->evicted && ctx->share_min_readers > 0 && n_new <= ctx->cfg.max_requests &&
-        (int64_t)((n_new + tpt - 1) / tpt) * ctx->cfg.n_kv_heads >= ctx->n_cta && r->len[(size_t)std::max(0, std::min(layer, ctx->cfg.n_layers - 1))] <= 16384 &&
+        r->len[(size_t)std::max(0, std::min(layer, ctx->cfg.n_layers - 1))] <= 16384 &&
         layer >= 0 && layer < ctx->cfg.n_layers && r->len[(size_t)layer] >= n_new && evicted_part(ctx, *r) < 0 && aligned16(q) &&
         aligned16(out)) {
         std::vector<ChainPart> parts;
+        uint32_t chain_tiles = 0;
         if (r->cart != CART_NONE) {
             const Cartridge &c = ctx->carts[(size_t)r->cart];
             if (c.composed) for (int32_t b : c.parts) parts.push_back(ChainPart{ctx->carts[(size_t)b].k_row, ctx->carts[(size_t)b].v_row, (uint32_t)ctx->carts[(size_t)b].p});
             else parts.push_back(ChainPart{c.k_row, c.v_row, (uint32_t)c.p});
         }
+        for (const ChainPart &pt : parts) chain_tiles += (pt.p + 127u) / 128u;
         const uint32_t len = (uint32_t)r->len[(size_t)layer];
-        std::vector<ChainStrand> strands{ChainStrand{r->k_row, r->v_row, (uint32_t)r->cap, len, 0u, (uint32_t)n_new, len - (uint32_t)n_new}};
-        return launch_chains(ctx, layer, parts, strands, (uint32_t)n_new, q, out, lse, static_cast<cudaStream_t>(stream));
+        chain_tiles += (len + 127u) / 128u;
+        const int64_t chains = (int64_t)((n_new + tpt - 1) / tpt) * ctx->cfg.n_kv_heads;
+        uint32_t n_split = 1;
+        if (chains < ctx->n_cta) {
+            const bool chosen = ctx->prefill_split >= 0;
+            n_split = chosen ? (uint32_t)ctx->prefill_split
+                             : (n_new >= 4 ? (uint32_t)std::max<int64_t>(1, std::min<int64_t>(ctx->n_cta / chains, chain_tiles / 2u)) : 0u);
+            // no more pieces than the chain has tiles or the partial slots hold
+            const int64_t rgs = (int64_t)n_new * ctx->cfg.n_kv_heads;
+            n_split = std::min(n_split, std::max(chain_tiles, 1u));
+            while (n_split > 1u && rgs * n_split > ctx->lay.slots_cap) --n_split;
+        }
+        if (n_split >= 1u) {
+            std::vector<ChainStrand> strands{ChainStrand{r->k_row, r->v_row, (uint32_t)r->cap, len, 0u, (uint32_t)n_new, len - (uint32_t)n_new}};
+            return launch_chains(ctx, layer, parts, strands, (uint32_t)n_new, q, out, lse, static_cast<cudaStream_t>(stream), n_split);
+        }
     }
     return decode_impl(ctx, layer, &req, 1, q, out, lse, nullptr, nullptr, stream, &n_new, 1);
 }
@@ -1429,144 +1467,227 @@ extern "C" {
 
 namespace {
 
-// Rows that attend causally, as chains of units on the tensor-core kernel (prefill of a long message; the forward
-// of training attention).  The rows are numbered 0 .. T - 1 (row t = query row t of q / out / lse); every row sees
+// Rows that attend causally, as chains of units on the tensor-core kernel (prefill of a message; the forward of
+// training attention).  The rows are numbered 0 .. T - 1 (row t = query row t of q / out / lse); every row sees
 // all of `parts` (Cartridge blocks, in order) and then its own "strand": strand c owns the rows row_begin ..
 // row_begin + n_rows - 1, its keys are the first key_first + i + 1 tokens of a contiguous suffix buffer for its row i.
-
+//
 // One chain of units per (M-tile of 128 / G consecutive rows' tokens, KV head): the parts' tiles (every row sees all
-// of them), then, strand by strand, the tiles of the strands the M-tile's rows belong to, masked causally; the
-// chain's last unit writes out and lse directly -- no partials, no merge, and no row streams its diagonal by itself.
+// of them), then, strand by strand, the tiles of the strands the M-tile's rows belong to, masked causally.  With
+// n_split = 1 the chain's last unit writes out and lse directly -- no partials, no merge, and no row streams its
+// diagonal by itself.  With n_split > 1 (one strand only: a message too short to give every SM a chain) a chain is cut
+// along its keys into up to n_split pieces, each a chain of its own that ends in a partial, and the merge kernel
+// combines a row's partials; a piece starts no later than the tile that holds the first key which the M-tile's first
+// row sees last, so every row sees at least one key of every piece.
+//
+// The plan is laid out back to back in a buffer of the plan ring -- [block -> first unit][reader -> query row]
+// [reader slots][reader merges][merge items][units] -- so that one copy of just those bytes uploads it, and it is
+// kept: a call with the same parts, strands and split (the next layer of the same step) launches from the buffer as
+// it is.
 cart_status launch_chains(cart_ctx *ctx, int32_t layer, const std::vector<ChainPart> &parts, const std::vector<ChainStrand> &strands,
-                          uint32_t T, const void *q, void *out, float *lse, cudaStream_t s)
+                          uint32_t T, const void *q, void *out, float *lse, cudaStream_t s, uint32_t n_split)
 {
     const int Hkv = ctx->cfg.n_kv_heads, G = ctx->group;
     const uint32_t tpt = 128u / (uint32_t)G;   // tokens (readers) per M-tile
     const uint32_t n_rt = (T + tpt - 1) / tpt;
     const int32_t n_strands = (int32_t)strands.size();
-    PlanSlot *cur = ctx->cur_slot >= 0 ? &ctx->slots[ctx->cur_slot] : nullptr;
-    if (cur && cur->valid) {
-        CART_CUDA(ctx, cudaEventRecord(cur->ev, cur->last_stream));
-        cur->ev_recorded = true;
-    }
-    const int next = (ctx->cur_slot + 1) % kPlanSlots;
-    PlanSlot &ns = ctx->slots[next];
-    if (ns.ev_recorded) {
-        CART_CUDA(ctx, cudaEventSynchronize(ns.ev));
-        ns.ev_recorded = false;
-    }
-    ns.valid = false;
     const ScratchLayout &lay = ctx->lay;
-    cart_shared_unit *units = reinterpret_cast<cart_shared_unit *>(ns.host + lay.units_off);
-    uint32_t *unit_cta_begin = reinterpret_cast<uint32_t *>(ns.host + lay.unit_cta_begin_off);
-    uint32_t *readers = reinterpret_cast<uint32_t *>(ns.host + lay.readers_off);
-    if ((int64_t)T > lay.readers_cap) return fail(ctx, CART_ERR_CAPACITY, "%u rows exceed the reader table", T);
-    for (uint32_t t = 0; t < T; ++t) readers[t] = t;   // reader entry t = query row t
-    uint32_t part_tiles = 0;
-    for (const ChainPart &pt : parts) part_tiles += (pt.p + 127u) / 128u;
-    // keys of strand c that the rows of [a, b) need: up to the last of its rows in the tile
-    auto needed = [&](const ChainStrand &st, uint32_t b) {
-        const uint32_t last_row = std::min(b, st.row_begin + st.n_rows) - 1u;
-        return st.key_first + (last_row - st.row_begin) + 1u;
-    };
-    std::vector<uint32_t> chain_tiles(n_rt, 0);
-    std::vector<int32_t> first_strand(n_rt, 0);
-    {
-        int32_t c = 0;
-        for (uint32_t rt = 0; rt < n_rt; ++rt) {
-            const uint32_t a = rt * tpt, b = std::min(T, a + tpt);
-            while (strands[(size_t)c].row_begin + strands[(size_t)c].n_rows <= a) ++c;
-            first_strand[rt] = c;
-            uint32_t tiles = part_tiles;
-            for (int32_t cc = c; cc < n_strands && strands[(size_t)cc].row_begin < b; ++cc)
-                tiles += (needed(strands[(size_t)cc], b) + 127u) / 128u;
-            chain_tiles[rt] = tiles;
-        }
+    if (n_split < 1u || (n_split > 1u && n_strands != 1)) return fail(ctx, CART_ERR_INVALID_ARG, "chains: bad split");
+
+    std::vector<uint64_t> &key = ctx->chain_key_tmp;
+    key.clear();
+    key.push_back(((uint64_t)T << 32) | n_split);
+    for (const ChainPart &pt : parts) { key.push_back(pt.k_row); key.push_back(pt.v_row); key.push_back(pt.p); }
+    key.push_back(~0ull);
+    for (const ChainStrand &st : strands) {
+        key.push_back(st.k_row); key.push_back(st.v_row);
+        key.push_back(((uint64_t)st.cap << 32) | st.len);
+        key.push_back(((uint64_t)st.row_begin << 32) | st.n_rows);
+        key.push_back(st.key_first);
     }
-    uint64_t total_tiles = 0;
-    for (uint32_t rt = 0; rt < n_rt; ++rt) total_tiles += (uint64_t)chain_tiles[rt] * (uint64_t)Hkv;
-    const uint32_t n_blocks = (uint32_t)std::min<uint64_t>((uint64_t)ctx->n_cta, (uint64_t)n_rt * Hkv);
-    size_t nu = 0;
-    uint32_t blk = 0;
-    uint64_t given = 0;
-    bool full = false;
-    unit_cta_begin[0] = 0;
-    for (int g = 0; g < Hkv && !full; ++g)
-        for (uint32_t rt = 0; rt < n_rt && !full; ++rt) {
-            // a chain goes to the block whose share of the tiles it starts in
-            while (blk + 1 < n_blocks && given * n_blocks >= (uint64_t)(blk + 1) * total_tiles) unit_cta_begin[++blk] = (uint32_t)nu;
-            given += chain_tiles[rt];
-            const uint32_t a = rt * tpt, b = std::min(T, a + tpt);
-            bool first = true;
-            auto emit = [&](cart_shared_unit u, bool last) {
-                if (nu >= (size_t)lay.units_cap) { full = true; return; }
-                u.reader_begin = a;
-                u.n_readers = b - a;
-                u.kv_head = (uint16_t)g;
-                u.chunk = 0;
-                u.reserved = 0;
-                if (!first) u.flags |= CART_UNIT_CONT;
-                u.flags |= last ? CART_UNIT_DIRECT : CART_UNIT_HOLD;
-                first = false;
-                units[nu++] = u;
-            };
-            int32_t c_last = first_strand[rt];
-            while (c_last + 1 < n_strands && strands[(size_t)c_last + 1].row_begin < b) ++c_last;
-            for (const ChainPart &pt : parts) {
-                cart_shared_unit u{};
-                u.k_row = (uint32_t)(pt.k_row + (uint64_t)g * pt.p);
-                u.v_row = (uint32_t)(pt.v_row + (uint64_t)g * pt.p);
-                u.layer_stride = (uint32_t)Hkv * pt.p;
-                u.n_tiles = (pt.p + 127u) / 128u;
-                u.flags = (pt.p % 128u) ? CART_UNIT_MASKED : 0;
-                u.lim_base = (int32_t)pt.p - 1;
-                u.lim_cap = (int32_t)pt.p - 1;
-                u.tr_hi = tpt;
-                emit(u, false);
-            }
-            for (int32_t c = first_strand[rt]; c <= c_last; ++c) {
-                const ChainStrand &st = strands[(size_t)c];
-                cart_shared_unit u{};
-                u.k_row = (uint32_t)(st.k_row + (uint64_t)g * st.cap);
-                u.v_row = (uint32_t)(st.v_row + (uint64_t)g * st.cap);
-                u.layer_stride = (uint32_t)((uint64_t)Hkv * st.cap);
-                u.n_tiles = (needed(st, b) + 127u) / 128u;
-                u.flags = CART_UNIT_MASKED | CART_UNIT_SUFFIX;
-                // token offset 0 of the M-tile is the strand's row a - row_begin (negative: the strand starts inside the tile)
-                u.lim_base = (int32_t)st.key_first + ((int32_t)a - (int32_t)st.row_begin);
-                u.lim_cap = (int32_t)st.len - 1;                   // the strand's last stored key
-                u.tr_hi = st.row_begin + st.n_rows - a;            // tokens from here on belong to later strands
-                emit(u, c == c_last);
+    PlanSlot *cur = ctx->cur_slot >= 0 ? &ctx->slots[ctx->cur_slot] : nullptr;
+    PlanSlot *sl = nullptr;
+    if (cur && cur->chain && cur->chain_key == key) {
+        sl = cur;
+    } else {
+        if (cur && (cur->valid || cur->chain)) {
+            CART_CUDA(ctx, cudaEventRecord(cur->ev, cur->last_stream));
+            cur->ev_recorded = true;
+        }
+        const int next = (ctx->cur_slot + 1) % kPlanSlots;
+        PlanSlot &ns = ctx->slots[next];
+        if (ns.ev_recorded) {
+            CART_CUDA(ctx, cudaEventSynchronize(ns.ev));
+            ns.ev_recorded = false;
+        }
+        ns.valid = false;
+        ns.chain = false;
+        ns.epoch = 0;
+
+        uint32_t part_tiles = 0;
+        for (const ChainPart &pt : parts) part_tiles += (pt.p + 127u) / 128u;
+        // keys of strand c that the rows of [a, b) need: up to the last of its rows in the tile
+        auto needed = [&](const ChainStrand &st, uint32_t b) {
+            const uint32_t last_row = std::min(b, st.row_begin + st.n_rows) - 1u;
+            return st.key_first + (last_row - st.row_begin) + 1u;
+        };
+        std::vector<cart_shared_unit> &units = ctx->unit_tmp;
+        std::vector<uint32_t> &piece_of_rt = ctx->piece_tmp;   // pieces of M-tile rt's chains (the same for every KV head)
+        std::vector<uint32_t> chain_start;                     // index in `units` of every chain's (piece's) first unit
+        units.clear();
+        piece_of_rt.assign(n_rt, 1u);
+        std::vector<cart_shared_unit> cu;   // the units of one chain before it is cut
+        std::vector<uint32_t> cuts;
+        int32_t c0 = 0;
+        for (int g = 0; g < Hkv; ++g) {
+            c0 = 0;
+            for (uint32_t rt = 0; rt < n_rt; ++rt) {
+                const uint32_t a = rt * tpt, b = std::min(T, a + tpt);
+                while (strands[(size_t)c0].row_begin + strands[(size_t)c0].n_rows <= a) ++c0;
+                int32_t c_last = c0;
+                while (c_last + 1 < n_strands && strands[(size_t)c_last + 1].row_begin < b) ++c_last;
+                cu.clear();
+                for (const ChainPart &pt : parts) {
+                    cart_shared_unit u{};
+                    u.k_row = (uint32_t)(pt.k_row + (uint64_t)g * pt.p);
+                    u.v_row = (uint32_t)(pt.v_row + (uint64_t)g * pt.p);
+                    u.layer_stride = (uint32_t)Hkv * pt.p;
+                    u.n_tiles = (pt.p + 127u) / 128u;
+                    u.flags = (pt.p % 128u) ? CART_UNIT_MASKED : 0;
+                    u.lim_base = (int32_t)pt.p - 1;
+                    u.lim_cap = (int32_t)pt.p - 1;
+                    u.tr_hi = tpt;
+                    cu.push_back(u);
+                }
+                for (int32_t c = c0; c <= c_last; ++c) {
+                    const ChainStrand &st = strands[(size_t)c];
+                    cart_shared_unit u{};
+                    u.k_row = (uint32_t)(st.k_row + (uint64_t)g * st.cap);
+                    u.v_row = (uint32_t)(st.v_row + (uint64_t)g * st.cap);
+                    u.layer_stride = (uint32_t)((uint64_t)Hkv * st.cap);
+                    u.n_tiles = (needed(st, b) + 127u) / 128u;
+                    u.flags = CART_UNIT_MASKED | CART_UNIT_SUFFIX;
+                    // token offset 0 of the M-tile is the strand's row a - row_begin (negative: the strand starts inside the tile)
+                    u.lim_base = (int32_t)st.key_first + ((int32_t)a - (int32_t)st.row_begin);
+                    u.lim_cap = (int32_t)st.len - 1;                   // the strand's last stored key
+                    u.tr_hi = st.row_begin + st.n_rows - a;            // tokens from here on belong to later strands
+                    cu.push_back(u);
+                }
+                uint32_t total = 0;
+                for (const cart_shared_unit &u : cu) total += u.n_tiles;
+                // where the chain is cut: piece k starts at tile cuts[k] of the chain
+                cuts.assign(1, 0u);
+                if (n_split > 1u) {
+                    const uint32_t safe = part_tiles + (uint32_t)std::max(cu.back().lim_base, 0) / 128u;
+                    for (uint32_t k = 1; k < n_split; ++k) {
+                        const uint32_t at = std::min((uint32_t)((uint64_t)k * total / n_split), safe);
+                        if (at > cuts.back() && at < total) cuts.push_back(at);
+                    }
+                }
+                piece_of_rt[rt] = (uint32_t)cuts.size();
+                cuts.push_back(total);
+                for (size_t k = 0; k + 1 < cuts.size(); ++k) {
+                    const uint32_t lo = cuts[k], hi = cuts[k + 1];
+                    chain_start.push_back((uint32_t)units.size());
+                    uint32_t u0 = 0;
+                    bool first = true;
+                    for (const cart_shared_unit &src : cu) {
+                        const uint32_t u1 = u0 + src.n_tiles;
+                        const uint32_t x = std::max(lo, u0), y = std::min(hi, u1);
+                        if (x < y) {
+                            cart_shared_unit u = src;
+                            const uint32_t skip = (x - u0) * 128u;   // keys of the unit that earlier pieces hold
+                            u.k_row += skip;
+                            u.v_row += skip;
+                            u.lim_base -= (int32_t)skip;
+                            u.lim_cap -= (int32_t)skip;
+                            u.n_tiles = y - x;
+                            u.reader_begin = a;
+                            u.n_readers = b - a;
+                            u.kv_head = (uint16_t)g;
+                            u.chunk = (uint32_t)k;
+                            u.reserved = 0;
+                            if (!first) u.flags |= CART_UNIT_CONT;
+                            if (y < hi) u.flags |= CART_UNIT_HOLD;
+                            else if (n_split == 1u) u.flags |= CART_UNIT_DIRECT;
+                            first = false;
+                            units.push_back(u);
+                        }
+                        u0 = u1;
+                    }
+                }
             }
         }
-    if (full) return fail(ctx, CART_ERR_CAPACITY, "more than %d units", lay.units_cap);
-    // a chain's first unit names the distance to the next chain (the kernel fetches that chain's query rows ahead)
-    {
-        size_t next_start = nu;
-        for (size_t i = nu; i-- > 0;) {
-            if (units[i].flags & CART_UNIT_CONT) continue;
-            units[i].reserved = next_start < nu ? (uint32_t)(next_start - i) : 0u;
-            next_start = i;
+        const size_t nu = units.size();
+        // a chain's first unit names the distance to the next chain (the kernel fetches that chain's query rows ahead)
+        for (size_t i = 0; i < chain_start.size(); ++i)
+            units[chain_start[i]].reserved = i + 1 < chain_start.size() ? chain_start[i + 1] - chain_start[i] : 0u;
+        // a chain goes to the block whose share of the tiles it starts in (chains of unequal length, no more of them
+        // than blocks, would leave some blocks with two and others with none that way: then every chain gets a block)
+        uint64_t total_tiles = 0;
+        for (const cart_shared_unit &u : units) total_tiles += u.n_tiles;
+        const uint32_t n_blocks = (uint32_t)std::min<uint64_t>((uint64_t)ctx->n_cta, (uint64_t)chain_start.size());
+        const uint32_t n_merges = n_split > 1u ? T * (uint32_t)Hkv : 0u;
+        // the buffer's layout
+        auto up = [](uint64_t x) { return (x + 63u) & ~63ull; };
+        const uint64_t off_ucb = lay.shared_off;
+        const uint64_t off_readers = up(off_ucb + (uint64_t)(n_blocks + 1u) * 4u);
+        const uint64_t off_rslot = up(off_readers + (uint64_t)T * 4u);
+        const uint64_t off_rmerge = up(off_rslot + (uint64_t)n_merges * 4u);
+        const uint64_t off_merges = up(off_rmerge + (uint64_t)n_merges * 4u);
+        const uint64_t off_units = up(off_merges + (uint64_t)n_merges * sizeof(cart_merge_item));
+        const uint64_t end = off_units + (uint64_t)nu * sizeof(cart_shared_unit);
+        if (end > lay.plan_slot_bytes) return fail(ctx, CART_ERR_CAPACITY, "chains: the plan of %u rows does not fit its buffer", T);
+        if ((uint64_t)n_merges * n_split > (uint64_t)lay.slots_cap)
+            return fail(ctx, CART_ERR_CAPACITY, "chains: %u rows in %u pieces exceed the partial slots", T, n_split);
+        uint32_t *unit_cta_begin = reinterpret_cast<uint32_t *>(ns.host + off_ucb);
+        uint32_t *readers = reinterpret_cast<uint32_t *>(ns.host + off_readers);
+        uint32_t blk = 0;
+        uint64_t given = 0;
+        unit_cta_begin[0] = 0;
+        const bool one_each = chain_start.size() <= (size_t)n_blocks;   // no more chains than blocks: a block each
+        for (size_t i = 0; i < chain_start.size(); ++i) {
+            while (blk + 1 < n_blocks && (one_each ? (size_t)blk < i : given * n_blocks >= (uint64_t)(blk + 1) * total_tiles))
+                unit_cta_begin[++blk] = chain_start[i];
+            const size_t e = i + 1 < chain_start.size() ? chain_start[i + 1] : nu;
+            for (size_t j = chain_start[i]; j < e; ++j) given += units[j].n_tiles;
         }
+        while (blk < n_blocks) unit_cta_begin[++blk] = (uint32_t)nu;
+        for (uint32_t t = 0; t < T; ++t) readers[t] = t;   // reader entry t = query row t
+        if (n_split > 1u) {
+            uint32_t *rslot = reinterpret_cast<uint32_t *>(ns.host + off_rslot);
+            uint32_t *rmerge = reinterpret_cast<uint32_t *>(ns.host + off_rmerge);
+            cart_merge_item *merges = reinterpret_cast<cart_merge_item *>(ns.host + off_merges);
+            for (uint32_t t = 0; t < T; ++t)
+                for (uint32_t g = 0; g < (uint32_t)Hkv; ++g) {
+                    const uint32_t rg = t * (uint32_t)Hkv + g;
+                    rslot[rg] = rg * n_split;
+                    rmerge[rg] = rg;
+                    merges[rg] = cart_merge_item{rg, rg * n_split, rg * n_split + piece_of_rt[t / tpt], 0u};
+                }
+        }
+        std::memcpy(ns.host + off_units, units.data(), nu * sizeof(cart_shared_unit));
+        CART_CUDA(ctx, cudaMemcpyAsync(ns.dev + off_ucb, ns.host + off_ucb, end - off_ucb, cudaMemcpyHostToDevice, s));
+        ns.chain = true;
+        ns.chain_key = key;
+        ns.chain_blocks = n_blocks;
+        ns.chain_merges = n_merges;
+        ns.chain_off[0] = off_ucb; ns.chain_off[1] = off_readers; ns.chain_off[2] = off_rslot;
+        ns.chain_off[3] = off_rmerge; ns.chain_off[4] = off_merges; ns.chain_off[5] = off_units;
+        ++ctx->plans_built;
+        ctx->cur_slot = next;
+        sl = &ns;
     }
-    while (blk + 1 <= n_blocks) unit_cta_begin[++blk] = (uint32_t)nu;
-    for (uint32_t b2 = blk; b2 < (uint32_t)kMaxCta; ++b2) unit_cta_begin[b2 + 1] = (uint32_t)nu;
-    const uint64_t sh_bytes = lay.units_off + (uint64_t)nu * sizeof(cart_shared_unit) - lay.shared_off;
-    CART_CUDA(ctx, cudaMemcpyAsync(ns.dev + lay.shared_off, ns.host + lay.shared_off, sh_bytes, cudaMemcpyHostToDevice, s));
-    ns.last_stream = s;
-    ns.epoch = 0;
-    ctx->cur_slot = next;
-    CART_CUDA(ctx, cudaEventRecord(ns.ev, s));
-    ns.ev_recorded = true;
+    sl->last_stream = s;
 
     uint8_t *arena = static_cast<uint8_t *>(ctx->cfg.arena);
     SharedParams sp;
-    sp.unit_cta_begin = reinterpret_cast<const uint32_t *>(ns.dev + lay.unit_cta_begin_off);
-    sp.units = reinterpret_cast<const cart_shared_unit *>(ns.dev + lay.units_off);
-    sp.readers = reinterpret_cast<const uint32_t *>(ns.dev + lay.readers_off);
-    sp.reader_slot = reinterpret_cast<const uint32_t *>(ns.dev + lay.reader_slot_off);
-    sp.reader_merge = reinterpret_cast<const uint32_t *>(ns.dev + lay.reader_merge_off);
-    sp.merges = reinterpret_cast<const cart_merge_item *>(ns.dev + lay.merges_off);
+    sp.unit_cta_begin = reinterpret_cast<const uint32_t *>(sl->dev + sl->chain_off[0]);
+    sp.readers = reinterpret_cast<const uint32_t *>(sl->dev + sl->chain_off[1]);
+    sp.reader_slot = reinterpret_cast<const uint32_t *>(sl->dev + sl->chain_off[2]);
+    sp.reader_merge = reinterpret_cast<const uint32_t *>(sl->dev + sl->chain_off[3]);
+    sp.merges = reinterpret_cast<const cart_merge_item *>(sl->dev + sl->chain_off[4]);
+    sp.units = reinterpret_cast<const cart_shared_unit *>(sl->dev + sl->chain_off[5]);
     sp.q = q;
     sp.out = out;
     sp.lse = lse;
@@ -1580,9 +1701,21 @@ cart_status launch_chains(cart_ctx *ctx, int32_t layer, const std::vector<ChainP
     sp.n_q_heads = ctx->cfg.n_q_heads;
     sp.scale_log2 = ctx->scale * 1.4426950408889634f;
     sp.pages = nullptr;
-    CART_CUDA(ctx, launch_shared(ctx->tmap, sp, (int)n_blocks, s, true));
+    CART_CUDA(ctx, launch_shared(ctx->tmap, sp, (int)sl->chain_blocks, s, true));
     ++ctx->launches;
-    CART_CUDA(ctx, cudaEventRecord(ns.ev, s));
+    if (sl->chain_merges > 0) {
+        MergeParams mp;
+        mp.merges = sp.merges;
+        mp.part_o = sp.part_o;
+        mp.part_lse2 = sp.part_lse2;
+        mp.out = out;
+        mp.lse = lse;
+        mp.group = G;
+        CART_CUDA(ctx, launch_merge(mp, (int)sl->chain_merges, s));
+        ++ctx->launches;
+    }
+    CART_CUDA(ctx, cudaEventRecord(sl->ev, s));   // whoever takes this buffer next waits for these launches
+    sl->ev_recorded = true;
     return CART_OK;
 }
 
@@ -1642,6 +1775,7 @@ cart_status cart_train_attention_bwd(cart_ctx *ctx, int32_t layer, const cart_re
         ns.ev_recorded = false;
     }
     ns.valid = false;
+    ns.chain = false;
     TrainItem *items = reinterpret_cast<TrainItem *>(ns.host + ctx->lay.items_off);
     const size_t items_cap = (size_t)ctx->lay.items_cap * sizeof(cart_work_item) / sizeof(TrainItem);
     size_t n_items = 0;

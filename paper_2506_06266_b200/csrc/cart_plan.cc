@@ -199,7 +199,7 @@ extern "C" cart_status cart_plan_build_shared(const cart_plan_seg *segs, const i
     };
     // Side by side: how many of the n_cta blocks the shared kernel gets.  Estimated times in nanoseconds,
     // fitted to measurements on B200 (launch lists of the two kernels at several divisions of the SMs):
-    //   shared kernel on s blocks   3000 + (1200 per 128-token tile + 4000 per unit) / s
+    //   shared kernel on s blocks   3000 + (1200 per 128-token tile + 4000 per unit) of its heaviest block
     //   stream kernel on c blocks   3000 + max((510 per 64-token tile + 1500 per row-group piece) / c,
     //                                          5.1 per tile)      -- the second term is the HBM bound
     // One after the other costs the sum of the two on all blocks; side by side the larger of the two on their shares.  The division with the smallest estimate is taken if it beats one-after-the-other by 5 %.
@@ -217,11 +217,21 @@ extern "C" cart_status cart_plan_build_shared(const cart_plan_seg *segs, const i
             if (t > 0) st_rgs += (uint64_t)n_kv_heads;
         }
         if (st_tiles > 0) {
-            auto est_shared = [&](uint64_t blocks) {
-                // runs of equal length that divide evenly over the blocks are not cut; otherwise every block
-                // boundary but the last cuts one
-                const uint64_t cuts = combos.size() % blocks == 0 ? 0 : blocks - 1;
-                return 3000 + (W_sh * 1200 + (combos.size() + cuts) * 4000) / blocks;
+            // The heaviest block of the division that step 3 would make of the runs (runs of unequal length do not
+            // divide evenly: a block that holds a long run whole sets the time).  With very many runs the walk per
+            // candidate is not worth its host time and the even share stands in for it.
+            auto est_shared = [&](uint64_t blocks) -> uint64_t {
+                blocks = std::min<uint64_t>(blocks, std::max<uint64_t>(1, W_sh / 2));
+                if (combos.size() > 256) {
+                    const uint64_t cuts = combos.size() % blocks == 0 ? 0 : blocks - 1;
+                    return 3000 + (W_sh * 1200 + (combos.size() + cuts) * 4000) / blocks;
+                }
+                uint64_t at = 0, w = 0, worst = 0;
+                walk(blocks, [&](size_t, uint64_t, uint64_t take, uint32_t, uint64_t c) {
+                    if (c != at) { worst = std::max(worst, w); w = 0; at = c; }
+                    w += take * 1200 + 4000;
+                });
+                return 3000 + std::max(worst, w);
             };
             auto est_stream = [&](uint64_t blocks) {
                 return 3000 + std::max<uint64_t>((st_tiles * 510 + (st_rgs + blocks) * 1500) / blocks, (st_tiles * 51) / 10);

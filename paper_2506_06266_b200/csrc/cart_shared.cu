@@ -664,14 +664,16 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                 }
                 if (wg == 0 && p.lse) p.lse[orow] = (m_run + log2f(l)) * 0.6931471805599453f;
             } else if (alive && valid) {
+                // (a row that saw no key of the unit -- all of them beyond its causal limit -- leaves an empty partial:
+                //  zeros with lse = -inf, which the merge gives no weight)
                 const float l = xchg_l[row] + xchg_l[128 + row];
-                const float inv = 1.f / l;
+                const float inv = l > 0.f ? 1.f / l : 0.f;
                 float4 *dst = reinterpret_cast<float4 *>(p.part_o + ((size_t)slot * G + h) * kHeadDim + col0);
 #pragma unroll
                 for (int q4 = 0; q4 < 16; ++q4)
                     dst[q4] = make_float4(__uint_as_float(o[4 * q4]) * inv, __uint_as_float(o[4 * q4 + 1]) * inv,
                                           __uint_as_float(o[4 * q4 + 2]) * inv, __uint_as_float(o[4 * q4 + 3]) * inv);
-                if (wg == 0) p.part_lse2[(size_t)slot * kMaxGroup + h] = m_run + log2f(l);
+                if (wg == 0) p.part_lse2[(size_t)slot * kMaxGroup + h] = l > 0.f ? m_run + log2f(l) : -INFINITY;
             }
             if (p.tickets == nullptr || direct) {
                 softmax_bar_both();  // the sums have been read: the next unit's maxima may be written

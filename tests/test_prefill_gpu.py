@@ -33,11 +33,13 @@ def prefill(sess, layer, req, q, n_new):
     return out, lse
 
 
-def run(Hq, Hkv, p, s_old, n_new, parts=1, layers=2, seed=0):
+def run(Hq, Hkv, p, s_old, n_new, parts=1, layers=2, seed=0, split=None):
     w = synth.Workload("prefill", 600 + seed + p + s_old + n_new, layers, Hq, Hkv, 1, max(p, 1), s_old, s_old,
                        cartridges="pool" if parts > 1 else ("none" if p == 0 else "private"), pool=parts, compose=parts)
     sess = H.Session(layers, Hq, Hkv, 64 << 20, max_requests=max(n_new, 4))
     try:
+        if split is not None:
+            binding.cart_set_prefill_split(sess.ctx, split)
         if p == 0:
             cart = binding.CART_NONE
         else:
@@ -61,33 +63,40 @@ def run(Hq, Hkv, p, s_old, n_new, parts=1, layers=2, seed=0):
         sess.close()
 
 
+# split: None = the library's choice (chains of masked tiles for four tokens or more), 0 = through the decode kernels
+@pytest.mark.parametrize("split", [None, 0])
 @pytest.mark.parametrize("s_old,n_new", [(0, 1), (0, 3), (5, 4), (130, 37), (260, 64), (127, 129), (300, 5)])
-def test_prefill_over_a_private_cartridge(s_old, n_new):
-    run(32, 8, 300, s_old, n_new, seed=1)
+def test_prefill_over_a_private_cartridge(s_old, n_new, split):
+    run(32, 8, 300, s_old, n_new, seed=1, split=split)
 
 
+@pytest.mark.parametrize("split", [None, 0])
 @pytest.mark.parametrize("Hq,Hkv", [(24, 8), (8, 8), (8, 1)])
-def test_prefill_group_sizes(Hq, Hkv):
-    run(Hq, Hkv, 520, 140, 33, seed=2)
+def test_prefill_group_sizes(Hq, Hkv, split):
+    run(Hq, Hkv, 520, 140, 33, seed=2, split=split)
 
 
-def test_prefill_without_a_cartridge_is_causal_self_attention():
-    run(32, 8, 0, 0, 70, layers=1, seed=3)
+@pytest.mark.parametrize("split", [None, 0])
+def test_prefill_without_a_cartridge_is_causal_self_attention(split):
+    run(32, 8, 0, 0, 70, layers=1, seed=3, split=split)
 
 
-def test_prefill_over_composed_cartridges():
-    run(32, 8, 256, 64, 48, parts=3, seed=4)
+@pytest.mark.parametrize("split", [None, 0])
+def test_prefill_over_composed_cartridges(split):
+    run(32, 8, 256, 64, 48, parts=3, seed=4, split=split)
 
 
-def test_prefill_many_rows_long_cartridge():
-    run(32, 8, 4096, 0, 256, layers=1, seed=5)
+@pytest.mark.parametrize("split", [None, 0])
+def test_prefill_many_rows_long_cartridge(split):
+    run(32, 8, 4096, 0, 256, layers=1, seed=5, split=split)
 
 
 @pytest.mark.parametrize("Hq,Hkv,s_old,n_new", [(32, 8, 100, 300), (24, 8, 77, 200), (64, 8, 0, 150), (8, 1, 250, 140),
                                                 (32, 8, 0, 130), (32, 8, 126, 35)])
 def test_prefill_of_a_long_message_shares_the_suffix_in_causal_steps(Hq, Hkv, s_old, n_new):
-    # the message spans several shared tiles: groups of 128 / G rows share the suffix before their first
-    # token (a staircase along the diagonal); (0, 130) leaves 2 rows on the last step, too few to share it
+    # through the decode kernels the message spans several shared tiles: groups of 128 / G rows share the suffix before
+    # their first token (a staircase along the diagonal); (0, 130) leaves 2 rows on the last step, too few to share it
+    run(Hq, Hkv, 200, s_old, n_new, layers=1, seed=6, split=0)
     run(Hq, Hkv, 200, s_old, n_new, layers=1, seed=6)
 
 
@@ -98,6 +107,49 @@ def test_prefill_of_a_message_that_fills_the_device_runs_as_chains_of_masked_til
     # to each row's own token under a causal mask (Cartridge and suffix ends inside tiles, a group of three heads whose
     # row tiles hold two rows no token owns, no Cartridge at all); with at least one chain per SM the call takes this path
     run(Hq, Hkv, p, s_old, n_new, parts=parts, layers=1, seed=8)
+
+
+@pytest.mark.parametrize("Hq,Hkv,p,parts,s_old,n_new,split", [
+    (24, 8, 2048, 1, 256, 64, -1),      # what a short message gets by default: 16 chains cut into 9 pieces each
+    (32, 8, 300, 1, 100, 70, 3),        # Cartridge and suffix end inside tiles; three M-tiles, the last with 6 rows
+    (32, 8, 300, 1, 100, 70, 64),       # more pieces asked for than the chain has tiles
+    (24, 8, 128, 2, 0, 50, 2),          # nothing before the message: the only safe cut is inside the Cartridges
+    (8, 8, 0, 1, 700, 40, 4),           # no Cartridge: every cut lies in the suffix before the message
+    (8, 8, 0, 1, 0, 140, 5),            # no Cartridge, no suffix: no cut is safe, the chains stay whole
+    (8, 1, 260, 1, 250, 33, 2),         # one KV head with eight query heads
+    (32, 8, 256, 1, 130, 17, -1)])
+def test_prefill_of_a_short_message_cuts_its_chains_along_the_keys(Hq, Hkv, p, parts, s_old, n_new, split):
+    # too few chains to fill the device: each is cut into pieces that end in partials, merged by the merge kernel;
+    # a piece never starts beyond the first key that the M-tile's first row sees last, so no row has an empty piece
+    run(Hq, Hkv, p, s_old, n_new, parts=parts, layers=2, seed=9, split=split)
+
+
+def test_prefill_chain_plan_is_kept_for_the_next_layer_and_dropped_when_the_message_changes():
+    w = synth.Workload("keep", 811, 3, 32, 8, 1, 256, 100, 100)
+    sess = H.Session(3, 32, 8, 64 << 20, max_requests=64)
+    try:
+        req = sess.open(sess.register(*w.cartridge_kv(0, "cuda:0")), 400)
+        sess.extend(req, *w.suffix_kv(0, 100, "cuda:0"))
+        for msg, n_new in enumerate((48, 48, 20)):
+            sess.extend(req, *w.suffix_kv(1 + msg, n_new, "cuda:0"))
+            before = binding.cart_plan_count(sess.ctx)
+            for layer in range(3):
+                q = synth.normal_bf16((n_new, 32, 128), 900 + 10 * msg + layer, "cuda:0")
+                out, lse = prefill(sess, layer, req, q, n_new)
+                ro, rl = oracle_rows(sess, layer, req, q, n_new)
+                H.assert_close(out, lse, ro, rl, "message %d layer %d" % (msg, layer))
+            assert binding.cart_plan_count(sess.ctx) == before + 1      # one plan per message, not per layer
+        # a decode call in between takes another buffer of the ring; the next prefill builds its plan again
+        q1 = synth.normal_bf16((1, 32, 128), 990, "cuda:0")
+        sess.decode(0, [req], q1)
+        before = binding.cart_plan_count(sess.ctx)
+        q = synth.normal_bf16((20, 32, 128), 991, "cuda:0")
+        out, lse = prefill(sess, 0, req, q, 20)
+        ro, rl = oracle_rows(sess, 0, req, q, 20)
+        H.assert_close(out, lse, ro, rl, "after a decode call")
+        assert binding.cart_plan_count(sess.ctx) == before + 1
+    finally:
+        sess.close()
 
 
 def test_prefill_errors():
