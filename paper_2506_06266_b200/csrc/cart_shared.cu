@@ -668,11 +668,17 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                 //  zeros with lse = -inf, which the merge gives no weight)
                 const float l = xchg_l[row] + xchg_l[128 + row];
                 const float inv = l > 0.f ? 1.f / l : 0.f;
-                float4 *dst = reinterpret_cast<float4 *>(p.part_o + ((size_t)slot * G + h) * kHeadDim + col0);
+                // 32 bytes per store: a thread writes a row by itself, so every store of a warp touches 32 rows, and
+                // 16-byte stores fill only half of each 32-byte sector they touch
+                float *dst = p.part_o + ((size_t)slot * G + h) * kHeadDim + col0;
 #pragma unroll
-                for (int q4 = 0; q4 < 16; ++q4)
-                    dst[q4] = make_float4(__uint_as_float(o[4 * q4]) * inv, __uint_as_float(o[4 * q4 + 1]) * inv,
-                                          __uint_as_float(o[4 * q4 + 2]) * inv, __uint_as_float(o[4 * q4 + 3]) * inv);
+                for (int q8 = 0; q8 < 8; ++q8)
+                    asm volatile("st.global.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(dst + 8 * q8),
+                                 "f"(__uint_as_float(o[8 * q8]) * inv), "f"(__uint_as_float(o[8 * q8 + 1]) * inv),
+                                 "f"(__uint_as_float(o[8 * q8 + 2]) * inv), "f"(__uint_as_float(o[8 * q8 + 3]) * inv),
+                                 "f"(__uint_as_float(o[8 * q8 + 4]) * inv), "f"(__uint_as_float(o[8 * q8 + 5]) * inv),
+                                 "f"(__uint_as_float(o[8 * q8 + 6]) * inv), "f"(__uint_as_float(o[8 * q8 + 7]) * inv)
+                                 : "memory");
                 if (wg == 0) p.part_lse2[(size_t)slot * kMaxGroup + h] = l > 0.f ? m_run + log2f(l) : -INFINITY;
             }
             if (p.tickets == nullptr || direct) {
