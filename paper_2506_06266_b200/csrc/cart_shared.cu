@@ -652,15 +652,16 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                 const float l = xchg_l[row] + xchg_l[128 + row];
                 const float inv = 1.f / l;
                 const size_t orow = (size_t)slot * p.n_q_heads + (size_t)u.kv_head * G + h;
-                uint4 *dst = reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(p.out) + orow * kHeadDim + col0);
+                __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(p.out) + orow * kHeadDim + col0;
 #pragma unroll
-                for (int c8 = 0; c8 < 8; ++c8) {
-                    uint4 w;
-                    w.x = pack_bf16(__uint_as_float(o[8 * c8]) * inv, __uint_as_float(o[8 * c8 + 1]) * inv);
-                    w.y = pack_bf16(__uint_as_float(o[8 * c8 + 2]) * inv, __uint_as_float(o[8 * c8 + 3]) * inv);
-                    w.z = pack_bf16(__uint_as_float(o[8 * c8 + 4]) * inv, __uint_as_float(o[8 * c8 + 5]) * inv);
-                    w.w = pack_bf16(__uint_as_float(o[8 * c8 + 6]) * inv, __uint_as_float(o[8 * c8 + 7]) * inv);
-                    dst[c8] = w;
+                for (int c16 = 0; c16 < 4; ++c16) {   // 32 bytes per store (see the partials below)
+                    uint32_t w[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        w[j] = pack_bf16(__uint_as_float(o[16 * c16 + 2 * j]) * inv, __uint_as_float(o[16 * c16 + 2 * j + 1]) * inv);
+                    asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(dst + 16 * c16), "r"(w[0]), "r"(w[1]),
+                                 "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+                                 : "memory");
                 }
                 if (wg == 0 && p.lse) p.lse[orow] = (m_run + log2f(l)) * 0.6931471805599453f;
             } else if (alive && valid) {
