@@ -618,6 +618,10 @@ __global__ void __launch_bounds__(128) cart_append_kernel(const __grid_constant_
 // Token-major [T][Hkv][128] -> head-major suffix rows; one thread per 16-byte chunk.
 __global__ void __launch_bounds__(256) cart_extend_kernel(const ExtendParams p)
 {
+    // launched as a dependent of the kernel before it: its blocks are placed while that kernel drains, and wait
+    // here for it (k and v may be its output, and its tiles may still cover the rows written below)
+    pdl_launch_dependents();
+    pdl_wait();
     const size_t chunks = (size_t)p.n_tokens * p.n_kv_heads * 16;
     uint4 *arena = reinterpret_cast<uint4 *>(p.arena);
     const uint4 *ks = reinterpret_cast<const uint4 *>(p.k);
@@ -671,8 +675,9 @@ cudaError_t launch_extend(const ExtendParams &p, cudaStream_t s)
     int grid = (int)((chunks + 255) / 256);
     if (grid > 148 * 8) grid = 148 * 8;
     if (grid < 1) grid = 1;
-    cart_extend_kernel<<<grid, 256, 0, s>>>(p);
-    return cudaGetLastError();
+    cudaLaunchAttribute attr;
+    const cudaLaunchConfig_t cfg = pdl_config(grid, 256, 0, s, &attr);
+    return cudaLaunchKernelEx(&cfg, cart_extend_kernel, p);
 }
 
 }  // namespace cart
