@@ -219,6 +219,36 @@ CART_API cart_status cart_decode_step(cart_ctx *ctx, int32_t layer, const cart_r
                              const void *k_new /*device*/, const void *v_new /*device*/, const void *q /*device*/,
                              void *out /*device*/, float *lse /*device or NULL*/, void *stream);
 
+/* Sec. 2.3, the decode loop as launches that can be recorded into a CUDA graph.  cart_decode_step does host work
+ * every step (it advances the lengths it mirrors and passes the tokens appended since the plan was built as a
+ * kernel parameter), so its launches cannot be replayed.  These three calls move that count to device memory:
+ *
+ *   cart_graph_begin(ctx, reqs, n_reqs, max_steps, stream)
+ *       plans the batch once and uploads the plan (not capturable: call it before the capture), clears the device
+ *       word that counts the steps, and reserves room for max_steps more tokens per request (paged suffixes take
+ *       their pages now).  Every request must hold the same number of tokens in all layers; a handle may appear
+ *       once; max_steps <= the plan-reuse limit + 1 (cart_set_plan_reuse; 193 by default).
+ *   cart_graph_step(ctx, layer, k_new, v_new, q, out, lse, stream)
+ *       what cart_decode_step computes for `layer` of the batch given to cart_graph_begin, in its order; only
+ *       kernel launches, so the calls for layers 0 .. n_layers - 1 of ONE step can be captured (stream capture or
+ *       explicit nodes) and replayed; after the last layer's kernels a one-thread kernel advances the count.  The
+ *       pointers are recorded: refill the same buffers between replays.  A batch with shared Cartridges runs its
+ *       tensor-core kernel and its stream kernel one after the other here, not side by side.
+ *   cart_graph_end(ctx, steps_run)
+ *       host only: the step ran steps_run times (<= max_steps), every request is that much longer in every layer.
+ *
+ * Between begin and end no other attention, prefill or training call may be made on ctx (it would take the loop's
+ * plan: cart_graph_step then returns INVALID_ARG; replays of a recorded step cannot notice), and the requests
+ * must not be closed, reserved or evicted.  Running more than max_steps steps writes past the reserved room.
+ * Errors: begin: INVALID_ARG, BAD_HANDLE, CAPACITY (room, max_steps), OOM, EVICTED, IN_USE (a loop is open), CUDA;
+ * step: INVALID_ARG (no loop open, plan taken, pointers), BAD_HANDLE (layer), CUDA; end: INVALID_ARG. */
+CART_API cart_status cart_graph_begin(cart_ctx *ctx, const cart_req *reqs /*host*/, int32_t n_reqs, int32_t max_steps,
+                                      void *stream);
+CART_API cart_status cart_graph_step(cart_ctx *ctx, int32_t layer, const void *k_new /*device*/, const void *v_new /*device*/,
+                                     const void *q /*device*/, void *out /*device*/, float *lse /*device or NULL*/,
+                                     void *stream);
+CART_API cart_status cart_graph_end(cart_ctx *ctx, int32_t steps_run);
+
 /* Sec. 2.3, prefill of the user's message over a Cartridge: attention for the LAST n_new tokens of
  * request req's suffix in `layer` (append them first with cart_extend_kv).  Row i of q (device bf16
  * [n_new][n_q_heads][128], token-major as the projection produces it) is the query of the i-th new

@@ -31,7 +31,7 @@ EXPORTS = ["cart_scratch_bytes", "cart_create", "cart_destroy", "cart_register_c
            "cart_append_kv", "cart_extend_kv", "cart_decode_attention", "cart_decode_step", "cart_prefill_attention", "cart_suffix_len",
            "cart_kv_bytes", "cart_sync_status", "cart_set_timing", "cart_get_timing",
            "cart_set_share_min_readers", "cart_set_piece_cost", "cart_plan_build_shared",
-           "cart_set_plan_reuse", "cart_set_prefill_split", "cart_plan_count", "cart_plan_reusable", "cart_set_side_by_side",
+           "cart_set_plan_reuse", "cart_set_prefill_split", "cart_graph_begin", "cart_graph_step", "cart_graph_end", "cart_plan_count", "cart_plan_reusable", "cart_set_side_by_side",
            "cart_request_open_paged", "cart_evict_request", "cart_restore_request", "cart_evict_cartridge",
            "cart_restore_cartridge", "cart_train_attention_fwd", "cart_train_attention_bwd",
            "cart_decode_attention_static", "cart_launch_count", "cart_status_string",
@@ -141,6 +141,9 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.cart_decode_attention.argtypes = [vp, i32, i32p, i32, vp, vp, vp, vp]
     lib.cart_decode_step.argtypes = [vp, i32, i32p, i32, vp, vp, vp, vp, vp, vp]
     lib.cart_prefill_attention.argtypes = [vp, i32, i32, vp, i32, vp, vp, vp]
+    lib.cart_graph_begin.argtypes = [vp, i32p, i32, i32, vp]
+    lib.cart_graph_step.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp]
+    lib.cart_graph_end.argtypes = [vp, i32]
     lib.cart_suffix_len.argtypes = [vp, i32, i32, i32p]
     lib.cart_kv_bytes.argtypes = [vp, i32, u64p, u64p]
     lib.cart_sync_status.argtypes = [vp, vp]
@@ -339,6 +342,20 @@ def cart_decode_step(ctx: int, layer: int, reqs, k_new, v_new, q, out, lse=None,
     arr, n = _reqs(reqs)
     _check(load_library().cart_decode_step(ctx, int(layer), arr, n, _ptr(k_new), _ptr(v_new), _ptr(q), _ptr(out),
                                            _ptr(lse), _stream(stream)), "cart_decode_step", ctx)
+
+
+def cart_graph_begin(ctx: int, reqs, max_steps: int, stream=None) -> None:
+    arr, n = _reqs(reqs)
+    _check(load_library().cart_graph_begin(ctx, arr, n, int(max_steps), _stream(stream)), "cart_graph_begin", ctx)
+
+
+def cart_graph_step(ctx: int, layer: int, k_new, v_new, q, out, lse=None, stream=None) -> None:
+    _check(load_library().cart_graph_step(ctx, int(layer), _ptr(k_new), _ptr(v_new), _ptr(q), _ptr(out), _ptr(lse),
+                                          _stream(stream)), "cart_graph_step", ctx)
+
+
+def cart_graph_end(ctx: int, steps_run: int) -> None:
+    _check(load_library().cart_graph_end(ctx, int(steps_run)), "cart_graph_end", ctx)
 
 
 def cart_prefill_attention(ctx: int, layer: int, req: int, q, n_new: int, out, lse=None, stream=None) -> None:

@@ -157,6 +157,12 @@ struct cart_ctx {
     int max_grow = kMaxGrowTokens;
     int side_by_side = 1;        // shared and stream kernel share the SMs (0: one after the other; > 1: blocks for the shared kernel)
     int prefill_split = -1;      // pieces a short message's chains are cut into along the keys (-1: chosen per call; 0: never)
+    bool plan_only = false;      // decode_impl stops after the plan (cart_graph_begin)
+    // a recorded decode loop (cart_graph_begin .. cart_graph_end): its batch, the ring buffer of its plan, its steps
+    bool graph_active = false;
+    std::vector<int32_t> graph_reqs;
+    int graph_slot = -1;
+    int32_t graph_max_steps = 0;
     uint32_t pair_seq = 0;       // counts side-by-side launches (the value the stream kernel hands to the shared kernel)
     uint64_t plans_built = 0;
     uint64_t n_rows = 0;
@@ -986,6 +992,110 @@ namespace {
 // that share the Cartridge(s) and, group by group, the part of the suffix before the group's first token, so
 // those go through the shared-segment kernel.  (One request: prefill of a user's message.  Many requests
 // that are whole conversations over one Cartridge: the forward of training-time attention.)
+// Launches the kernels of a plan for one layer: the stream kernel, the tensor-core kernel for the shared part and the
+// merge kernel, as the plan needs them.  grow: tokens every request has appended since the plan was built, or, with
+// grow_ctr set, the device word that holds that count (a launch recorded in a CUDA graph: the shared and the stream
+// kernel then run one after the other, since their side-by-side handshake carries a launch number as a parameter).
+cart_status launch_plan(cart_ctx *ctx, PlanSlot *sl, int32_t layer, const void *q, void *out, float *lse, const void *k_new,
+                        const void *v_new, int32_t grow, const uint32_t *grow_ctr, cudaStream_t s)
+{
+    const int Hkv = ctx->cfg.n_kv_heads;
+    sl->last_stream = s;
+
+    uint8_t *arena = static_cast<uint8_t *>(ctx->cfg.arena);
+    DecodeParams dp;
+    dp.cta_begin = reinterpret_cast<const uint32_t *>(sl->dev + ctx->lay.cta_begin_off);
+    dp.items = reinterpret_cast<const cart_work_item *>(sl->dev + ctx->lay.items_off);
+    dp.q = q;
+    dp.k_new = k_new;
+    dp.v_new = v_new;
+    dp.arena = ctx->cfg.arena;
+    dp.out = out;
+    dp.lse = lse;
+    dp.part_o = reinterpret_cast<float *>(arena + ctx->lay.part_o_off);
+    dp.part_lse2 = reinterpret_cast<float *>(arena + ctx->lay.part_lse_off);
+    dp.merges = reinterpret_cast<const cart_merge_item *>(sl->dev + ctx->lay.merges_off);
+    // Few split row groups: the block that delivers the last partial merges (arrival tickets, no extra
+    // launch).  Many (every reader of a shared Cartridge is one): a merge kernel over all of them.
+    const bool merge_after = sl->n_merges > ctx->n_cta;
+    dp.tickets = merge_after ? nullptr : reinterpret_cast<uint32_t *>(arena + ctx->lay.tickets_off);
+    dp.status = reinterpret_cast<uint32_t *>(arena + ctx->lay.status_off);
+    dp.layer = layer;
+    dp.group = ctx->group;
+    dp.scale_log2 = ctx->scale * 1.4426950408889634f;
+    dp.grow = (uint32_t)grow;
+    dp.grow_ctr = grow_ctr;
+    dp.edge_boxes = 1u;
+    dp.pages = reinterpret_cast<const uint32_t *>(sl->dev + ctx->lay.pages_off);
+    const bool timed = ctx->timing && grow_ctr == nullptr && ctx->ev_used + 2 <= kMaxTimedLaunches * 2;
+    if (timed) {
+        while (ctx->ev_pool.size() < ctx->ev_used + 2) {
+            cudaEvent_t e;
+            CART_CUDA(ctx, cudaEventCreate(&e));
+            ctx->ev_pool.push_back(e);
+        }
+        CART_CUDA(ctx, cudaEventRecord(ctx->ev_pool[ctx->ev_used], s));
+    }
+    // A batch with a shared part and a stream part runs the two kernels side by side: the stream kernel
+    // is launched first on its share of the SMs, the shared kernel right behind it on the rest (a dependent
+    // launch starts as soon as every block of the kernel before has started).
+    const bool pair = sl->n_units > 0 && sl->n_items > 0 && ctx->side_by_side > 0 && grow_ctr == nullptr;
+    if (pair) {
+        dp.ready_flag = reinterpret_cast<uint32_t *>(arena + ctx->lay.status_off + 128);
+        dp.seq = ++ctx->pair_seq;
+    }
+    if (pair) {
+        CART_CUDA(ctx, launch_decode(ctx->tmap, ctx->tmap_edge, dp, sl->n_cta_used, s));
+        ++ctx->launches;
+    }
+    if (sl->n_units > 0) {
+        SharedParams sp;
+        sp.unit_cta_begin = reinterpret_cast<const uint32_t *>(sl->dev + ctx->lay.unit_cta_begin_off);
+        sp.units = reinterpret_cast<const cart_shared_unit *>(sl->dev + ctx->lay.units_off);
+        sp.readers = reinterpret_cast<const uint32_t *>(sl->dev + ctx->lay.readers_off);
+        sp.reader_slot = reinterpret_cast<const uint32_t *>(sl->dev + ctx->lay.reader_slot_off);
+        sp.reader_merge = reinterpret_cast<const uint32_t *>(sl->dev + ctx->lay.reader_merge_off);
+        sp.merges = dp.merges;
+        sp.q = q;
+        sp.out = out;
+        sp.lse = lse;
+        sp.part_o = dp.part_o;
+        sp.part_lse2 = dp.part_lse2;
+        sp.tickets = dp.tickets;
+        sp.status = dp.status;
+        sp.layer = layer;
+        sp.group = ctx->group;
+        sp.n_kv_heads = Hkv;
+        sp.n_q_heads = ctx->cfg.n_q_heads;
+        sp.scale_log2 = dp.scale_log2;
+        sp.ready_flag = dp.ready_flag;
+        sp.seq = dp.seq;
+        sp.pages = dp.pages;
+        CART_CUDA(ctx, launch_shared(ctx->tmap, sp, sl->n_unit_cta_used, s));
+        ++ctx->launches;
+    }
+    if (sl->n_items > 0 && !pair) {
+        CART_CUDA(ctx, launch_decode(ctx->tmap, ctx->tmap_edge, dp, sl->n_cta_used, s));
+        ++ctx->launches;
+    }
+    if (merge_after) {
+        MergeParams mp;
+        mp.merges = dp.merges;
+        mp.part_o = dp.part_o;
+        mp.part_lse2 = dp.part_lse2;
+        mp.out = out;
+        mp.lse = lse;
+        mp.group = ctx->group;
+        CART_CUDA(ctx, launch_merge(mp, sl->n_merges, s));
+        ++ctx->launches;
+    }
+    if (timed) {
+        CART_CUDA(ctx, cudaEventRecord(ctx->ev_pool[ctx->ev_used + 1], s));
+        ctx->ev_used += 2;
+    }
+    return CART_OK;
+}
+
 cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int32_t n_reqs, const void *q,
                         void *out, float *lse, const void *k_new, const void *v_new, void *stream,
                         const int32_t *n_new_list = nullptr, int32_t n_pre = 0)
@@ -1045,7 +1155,7 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
 
     PlanSlot *sl = ctx->cur_slot >= 0 ? &ctx->slots[ctx->cur_slot] : nullptr;
     int32_t grow = 0;
-    bool reuse = sl && sl->valid && sl->epoch == ctx->epoch && sl->prefill == prefill;
+    bool reuse = sl && sl->valid && sl->epoch == ctx->epoch && sl->prefill == prefill && !ctx->plan_only;
     if (reuse && prefill) reuse = sl->key == key;
     if (reuse && !prefill)
         reuse = sl->reqs.size() == (size_t)n_reqs && std::memcmp(sl->reqs.data(), reqs, (size_t)n_reqs * sizeof(int32_t)) == 0 &&
@@ -1190,7 +1300,7 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
         po.slots_cap = lay.slots_cap;
         po.piece_cost = ctx->piece_cost;
         po.unit_cost = kUnitCostTiles;
-        po.side_by_side = ctx->side_by_side;
+        po.side_by_side = ctx->plan_only ? 0 : ctx->side_by_side;   // (a recorded loop runs the two kernels in turn)
         po.units = reinterpret_cast<cart_shared_unit *>(ns.host + lay.units_off);
         po.units_cap = lay.units_cap;
         po.unit_cta_begin = reinterpret_cast<uint32_t *>(ns.host + lay.unit_cta_begin_off);
@@ -1227,99 +1337,8 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
         ctx->cur_slot = next;
         sl = &ns;
     }
-    sl->last_stream = s;
-
-    uint8_t *arena = static_cast<uint8_t *>(ctx->cfg.arena);
-    DecodeParams dp;
-    dp.cta_begin = reinterpret_cast<const uint32_t *>(sl->dev + ctx->lay.cta_begin_off);
-    dp.items = reinterpret_cast<const cart_work_item *>(sl->dev + ctx->lay.items_off);
-    dp.q = q;
-    dp.k_new = k_new;
-    dp.v_new = v_new;
-    dp.arena = ctx->cfg.arena;
-    dp.out = out;
-    dp.lse = lse;
-    dp.part_o = reinterpret_cast<float *>(arena + ctx->lay.part_o_off);
-    dp.part_lse2 = reinterpret_cast<float *>(arena + ctx->lay.part_lse_off);
-    dp.merges = reinterpret_cast<const cart_merge_item *>(sl->dev + ctx->lay.merges_off);
-    // Few split row groups: the block that delivers the last partial merges (arrival tickets, no extra
-    // launch).  Many (every reader of a shared Cartridge is one): a merge kernel over all of them.
-    const bool merge_after = sl->n_merges > ctx->n_cta;
-    dp.tickets = merge_after ? nullptr : reinterpret_cast<uint32_t *>(arena + ctx->lay.tickets_off);
-    dp.status = reinterpret_cast<uint32_t *>(arena + ctx->lay.status_off);
-    dp.layer = layer;
-    dp.group = ctx->group;
-    dp.scale_log2 = ctx->scale * 1.4426950408889634f;
-    dp.grow = (uint32_t)grow;
-    dp.edge_boxes = 1u;
-    dp.pages = reinterpret_cast<const uint32_t *>(sl->dev + ctx->lay.pages_off);
-    const bool timed = ctx->timing && ctx->ev_used + 2 <= kMaxTimedLaunches * 2;
-    if (timed) {
-        while (ctx->ev_pool.size() < ctx->ev_used + 2) {
-            cudaEvent_t e;
-            CART_CUDA(ctx, cudaEventCreate(&e));
-            ctx->ev_pool.push_back(e);
-        }
-        CART_CUDA(ctx, cudaEventRecord(ctx->ev_pool[ctx->ev_used], s));
-    }
-    // A batch with a shared part and a stream part runs the two kernels side by side: the stream kernel
-    // is launched first on its share of the SMs, the shared kernel right behind it on the rest (a dependent
-    // launch starts as soon as every block of the kernel before has started).
-    const bool pair = sl->n_units > 0 && sl->n_items > 0 && ctx->side_by_side > 0;
-    if (pair) {
-        dp.ready_flag = reinterpret_cast<uint32_t *>(arena + ctx->lay.status_off + 128);
-        dp.seq = ++ctx->pair_seq;
-    }
-    if (pair) {
-        CART_CUDA(ctx, launch_decode(ctx->tmap, ctx->tmap_edge, dp, sl->n_cta_used, s));
-        ++ctx->launches;
-    }
-    if (sl->n_units > 0) {
-        SharedParams sp;
-        sp.unit_cta_begin = reinterpret_cast<const uint32_t *>(sl->dev + ctx->lay.unit_cta_begin_off);
-        sp.units = reinterpret_cast<const cart_shared_unit *>(sl->dev + ctx->lay.units_off);
-        sp.readers = reinterpret_cast<const uint32_t *>(sl->dev + ctx->lay.readers_off);
-        sp.reader_slot = reinterpret_cast<const uint32_t *>(sl->dev + ctx->lay.reader_slot_off);
-        sp.reader_merge = reinterpret_cast<const uint32_t *>(sl->dev + ctx->lay.reader_merge_off);
-        sp.merges = dp.merges;
-        sp.q = q;
-        sp.out = out;
-        sp.lse = lse;
-        sp.part_o = dp.part_o;
-        sp.part_lse2 = dp.part_lse2;
-        sp.tickets = dp.tickets;
-        sp.status = dp.status;
-        sp.layer = layer;
-        sp.group = ctx->group;
-        sp.n_kv_heads = Hkv;
-        sp.n_q_heads = ctx->cfg.n_q_heads;
-        sp.scale_log2 = dp.scale_log2;
-        sp.ready_flag = dp.ready_flag;
-        sp.seq = dp.seq;
-        sp.pages = dp.pages;
-        CART_CUDA(ctx, launch_shared(ctx->tmap, sp, sl->n_unit_cta_used, s));
-        ++ctx->launches;
-    }
-    if (sl->n_items > 0 && !pair) {
-        CART_CUDA(ctx, launch_decode(ctx->tmap, ctx->tmap_edge, dp, sl->n_cta_used, s));
-        ++ctx->launches;
-    }
-    if (merge_after) {
-        MergeParams mp;
-        mp.merges = dp.merges;
-        mp.part_o = dp.part_o;
-        mp.part_lse2 = dp.part_lse2;
-        mp.out = out;
-        mp.lse = lse;
-        mp.group = ctx->group;
-        CART_CUDA(ctx, launch_merge(mp, sl->n_merges, s));
-        ++ctx->launches;
-    }
-    if (timed) {
-        CART_CUDA(ctx, cudaEventRecord(ctx->ev_pool[ctx->ev_used + 1], s));
-        ctx->ev_used += 2;
-    }
-    return CART_OK;
+    if (ctx->plan_only) return CART_OK;   // (a recorded decode loop launches from the plan later)
+    return launch_plan(ctx, sl, layer, q, out, lse, k_new, v_new, grow, nullptr, s);
 }
 
 }  // namespace
@@ -1412,6 +1431,100 @@ cart_status cart_decode_step(cart_ctx *ctx, int32_t layer, const cart_req *reqs,
     if (st != CART_OK && ctx->launches == launches_before)
         for (int32_t i = 0; i < n_reqs; ++i) --ctx->reqs[(size_t)reqs[i]].len[(size_t)layer];
     return st;
+}
+
+// ---- a decode loop that can be recorded into a CUDA graph ----------------------------------------------------------
+// cart_graph_begin plans the batch once, for the step that appends the first token, and clears a device word that
+// counts the steps since; cart_graph_step launches a layer's kernels from that plan, reading the count from the
+// word, and after the last layer a one-thread kernel advances it: no host work depends on the step, so the launches
+// of one step can be recorded once and replayed.  cart_graph_end tells the host-side mirror how many steps ran.
+
+static uint32_t *graph_counter(cart_ctx *ctx)
+{
+    return reinterpret_cast<uint32_t *>(static_cast<uint8_t *>(ctx->cfg.arena) + ctx->lay.status_off + 192);
+}
+
+cart_status cart_graph_begin(cart_ctx *ctx, const cart_req *reqs, int32_t n_reqs, int32_t max_steps, void *stream)
+{
+    if (!ctx) return CART_ERR_INVALID_ARG;
+    if (ctx->graph_active) return fail(ctx, CART_ERR_IN_USE, "graph_begin: a recorded loop is already open");
+    if (!reqs || n_reqs < 1 || max_steps < 1)
+        return fail(ctx, CART_ERR_INVALID_ARG, "graph_begin: empty batch or max_steps < 1");
+    if (max_steps > ctx->max_grow + 1)
+        return fail(ctx, CART_ERR_CAPACITY, "graph_begin: max_steps %d exceeds what a kept plan covers (%d)", max_steps,
+                    ctx->max_grow + 1);
+    const int L = ctx->cfg.n_layers;
+    const uint64_t stamp = ++ctx->stamp;
+    for (int32_t i = 0; i < n_reqs; ++i) {
+        Request *r = get_req(ctx, reqs[i]);
+        if (!r) return fail(ctx, CART_ERR_BAD_HANDLE, "graph_begin: reqs[%d] is not an open request", i);
+        if (r->stamp == stamp) return fail(ctx, CART_ERR_INVALID_ARG, "graph_begin: reqs[%d] appears twice", i);
+        r->stamp = stamp;
+        if (r->evicted) return fail(ctx, CART_ERR_EVICTED, "graph_begin: reqs[%d] is swapped out", i);
+        for (int l = 1; l < L; ++l)
+            if (r->len[(size_t)l] != r->len[0])
+                return fail(ctx, CART_ERR_INVALID_ARG, "graph_begin: reqs[%d] holds %d tokens in layer %d and %d in layer 0", i,
+                            r->len[(size_t)l], l, r->len[0]);
+        if (!r->paged && r->len[0] + max_steps > r->cap)
+            return fail(ctx, CART_ERR_CAPACITY, "graph_begin: reqs[%d] has room for %d more tokens, fewer than max_steps", i,
+                        r->cap - r->len[0]);
+    }
+    for (int32_t i = 0; i < n_reqs; ++i) {  // paged suffixes take the pages of all the steps now
+        Request &r = ctx->reqs[(size_t)reqs[i]];
+        if (r.paged && !grow_pages(ctx, r, (int64_t)r.len[0] + max_steps))
+            return fail(ctx, CART_ERR_OOM, "graph_begin: arena has no pages left for reqs[%d]", i);
+    }
+    // the plan of the first step: every request one token longer (the fused append writes that token)
+    for (int32_t i = 0; i < n_reqs; ++i) ++ctx->reqs[(size_t)reqs[i]].len[0];
+    ctx->plan_only = true;
+    alignas(16) static const unsigned char dummy[16] = {0};   // (plan only: no pointer is used, they only have to pass the checks)
+    alignas(16) static unsigned char sink[16];
+    const cart_status st = decode_impl(ctx, 0, reqs, n_reqs, dummy, sink, nullptr, dummy, dummy, stream);
+    ctx->plan_only = false;
+    for (int32_t i = 0; i < n_reqs; ++i) --ctx->reqs[(size_t)reqs[i]].len[0];
+    if (st != CART_OK) return st;
+    CART_CUDA(ctx, cudaMemsetAsync(graph_counter(ctx), 0, 4, static_cast<cudaStream_t>(stream)));
+    ctx->graph_active = true;
+    ctx->graph_reqs.assign(reqs, reqs + n_reqs);
+    ctx->graph_slot = ctx->cur_slot;
+    ctx->graph_max_steps = max_steps;
+    return CART_OK;
+}
+
+cart_status cart_graph_step(cart_ctx *ctx, int32_t layer, const void *k_new, const void *v_new, const void *q, void *out,
+                            float *lse, void *stream)
+{
+    if (!ctx) return CART_ERR_INVALID_ARG;
+    if (!ctx->graph_active) return fail(ctx, CART_ERR_INVALID_ARG, "graph_step: no recorded loop is open");
+    if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, CART_ERR_BAD_HANDLE, "graph_step: layer out of range");
+    if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(q) || !aligned16(out) || (lse && (reinterpret_cast<uintptr_t>(lse) & 3u)))
+        return fail(ctx, CART_ERR_INVALID_ARG, "graph_step: null/misaligned pointer");
+    if (ctx->cur_slot != ctx->graph_slot || !ctx->slots[ctx->graph_slot].valid)
+        return fail(ctx, CART_ERR_INVALID_ARG, "graph_step: another attention call has taken the loop's plan");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    PlanSlot *sl = &ctx->slots[ctx->graph_slot];
+    const cart_status st = launch_plan(ctx, sl, layer, q, out, lse, k_new, v_new, 0, graph_counter(ctx), s);
+    if (st != CART_OK) return st;
+    if (layer == ctx->cfg.n_layers - 1) {
+        CART_CUDA(ctx, launch_advance(graph_counter(ctx), s));
+        ++ctx->launches;
+    }
+    return CART_OK;
+}
+
+cart_status cart_graph_end(cart_ctx *ctx, int32_t steps_run)
+{
+    if (!ctx) return CART_ERR_INVALID_ARG;
+    if (!ctx->graph_active) return fail(ctx, CART_ERR_INVALID_ARG, "graph_end: no recorded loop is open");
+    if (steps_run < 0 || steps_run > ctx->graph_max_steps)
+        return fail(ctx, CART_ERR_INVALID_ARG, "graph_end: %d steps, the loop was opened for at most %d", steps_run,
+                    ctx->graph_max_steps);
+    for (int32_t r : ctx->graph_reqs)
+        for (int l = 0; l < ctx->cfg.n_layers; ++l) ctx->reqs[(size_t)r].len[(size_t)l] += steps_run;
+    ctx->graph_active = false;
+    ctx->graph_slot = -1;
+    ++ctx->epoch;   // the kept plan describes the lengths before the loop
+    return CART_OK;
 }
 
 }  // extern "C"

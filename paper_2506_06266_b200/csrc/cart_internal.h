@@ -49,6 +49,9 @@ struct DecodeParams {
     uint32_t seq = 0;
     uint32_t grow = 0;           // tokens every request has appended since the plan was built: added to the token
                                  // count of every item marked CART_ITEM_TAIL
+    const uint32_t *grow_ctr = nullptr;  // if set, that number is read from here instead (a launch recorded in a CUDA
+                                         // graph cannot carry it as a parameter); a kernel earlier on the stream
+                                         // advances it, so it is read only after griddepcontrol.wait
     uint32_t edge_boxes = 0;     // 1: ragged last tiles are fetched in boxes of kEdgeBoxRows rows through the second
                                  // tensor map; 0: every tile is fetched whole
     const uint32_t *pages = nullptr;  // page list of the batch (base row of every page of every paged suffix), read by
@@ -192,6 +195,7 @@ cudaError_t prepare_shared_kernel();
 // chains: the plan holds chained / masked / directly written units (see CART_UNIT_CONT in cart_plan.h)
 cudaError_t launch_shared(const CUtensorMap &tmap, const SharedParams &p, int grid, cudaStream_t s, bool chains = false);
 cudaError_t launch_merge(const MergeParams &p, int n_merges, cudaStream_t s);
+cudaError_t launch_advance(uint32_t *ctr, cudaStream_t s);
 cudaError_t launch_append(const AppendParams &p, cudaStream_t s);
 cudaError_t launch_extend(const ExtendParams &p, cudaStream_t s);
 cudaError_t prepare_train_kernels();

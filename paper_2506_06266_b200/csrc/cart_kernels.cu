@@ -243,6 +243,12 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
         // extend kernels, and the fused append of an earlier decode step, which may be the kernel right
         // before this one -- so the first suffix tile is fetched only after griddepcontrol.wait.
         bool waited = false;
+        uint32_t grow = p.grow;
+        if (p.grow_ctr != nullptr) {  // the count lives in memory that the kernels before this one advance
+            pdl_wait();
+            waited = true;
+            grow = ld_volatile_u32(p.grow_ctr);
+        }
         uint32_t tails_seen = 0;  // tiles met so far that end with a new token
         // The next work item is requested while the copies of this one are issued: read at the item's start, it
         // held the ring back by a memory round trip per item, which short row groups cannot spare.
@@ -251,7 +257,7 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
         for (uint32_t it = item_begin; it < item_end && ok; ++it) {
             cart_work_item w = w_next;
             if (it + 1 < item_end) w_next = p.items[it + 1];
-            if (w.flags & CART_ITEM_TAIL) w.n_tok += p.grow;  // tokens appended since the plan was built
+            if (w.flags & CART_ITEM_TAIL) w.n_tok += grow;  // tokens appended since the plan was built
             const uint32_t k_row = w.k_row + (uint32_t)p.layer * w.layer_stride;
             const uint32_t v_row = w.v_row + (uint32_t)p.layer * w.layer_stride;
             const uint32_t ntiles = (w.n_tok + kTileTokens - 1) / kTileTokens;
@@ -356,6 +362,12 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
             bool waited = false;
             const uint4 *new_rows = reinterpret_cast<const uint4 *>(lane < 16 ? p.k_new : p.v_new);
             uint32_t n_done = 0;
+            uint32_t grow = p.grow;
+            if (p.grow_ctr != nullptr) {
+                pdl_wait();
+                waited = true;
+                grow = ld_volatile_u32(p.grow_ctr);
+            }
             for (uint32_t base_it = item_begin; base_it < item_end; base_it += 32u) {
                 const uint32_t mine = base_it + (uint32_t)lane;
                 cart_work_item a{};
@@ -381,7 +393,7 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
                             const uint32_t a_v = __shfl_sync(0xffffffffu, a.v_row, src_lane);
                             const uint32_t row0 = lane < 16 ? a_k : a_v;
                             const uint32_t a_ls = __shfl_sync(0xffffffffu, a.layer_stride, src_lane);
-                            const uint32_t a_n = __shfl_sync(0xffffffffu, a.n_tok, src_lane) + p.grow;
+                            const uint32_t a_n = __shfl_sync(0xffffffffu, a.n_tok, src_lane) + grow;
                             const uint32_t a_rg = __shfl_sync(0xffffffffu, a.row_group, src_lane);
                             const uint32_t a_fl = __shfl_sync(0xffffffffu, a.flags, src_lane);
                             val[u] = __ldg(new_rows + (size_t)a_rg * 16 + c);
@@ -502,6 +514,7 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
     pdl_wait();  // q, the partial slots and the tickets belong to the kernels before until they are done
     if (p.ready_flag != nullptr && blockIdx.x == 0 && threadIdx.x == 0)  // tell the kernel that runs beside this one
         asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.ready_flag), "r"(p.seq) : "memory");
+    const uint32_t grow = p.grow_ctr != nullptr ? ld_volatile_u32(p.grow_ctr) : p.grow;
     const int G = p.group;
     const int row = lane >> 2;  // query head inside the group that this thread's c0/c1 belong to
     const __nv_bfloat16 *q = reinterpret_cast<const __nv_bfloat16 *>(p.q);
@@ -517,7 +530,7 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
 
     for (uint32_t it = item_begin; it < item_end; ++it) {
         cart_work_item w = p.items[it];
-        if (w.flags & CART_ITEM_TAIL) w.n_tok += p.grow;
+        if (w.flags & CART_ITEM_TAIL) w.n_tok += grow;
         if (w.flags & CART_ITEM_BEGIN) {
             st.m = -INFINITY;
             st.l = 0.f;
@@ -615,6 +628,14 @@ __global__ void __launch_bounds__(128) cart_append_kernel(const __grid_constant_
     }
 }
 
+// Advances the count of tokens appended since the plan was built (one decode step of a recorded loop is over).
+__global__ void cart_advance_kernel(uint32_t *ctr)
+{
+    pdl_launch_dependents();
+    pdl_wait();  // the kernels before still read the old value
+    if (threadIdx.x == 0 && blockIdx.x == 0) *ctr = *ctr + 1u;
+}
+
 // Token-major [T][Hkv][128] -> head-major suffix rows; one thread per 16-byte chunk.
 __global__ void __launch_bounds__(256) cart_extend_kernel(const ExtendParams p)
 {
@@ -661,6 +682,13 @@ cudaError_t launch_merge(const MergeParams &p, int n_merges, cudaStream_t s)
     cudaLaunchAttribute attr;
     const cudaLaunchConfig_t cfg = pdl_config(n_merges, 128, 0, s, &attr);
     return cudaLaunchKernelEx(&cfg, cart_merge_kernel, p);
+}
+
+cudaError_t launch_advance(uint32_t *ctr, cudaStream_t s)
+{
+    cudaLaunchAttribute attr;
+    const cudaLaunchConfig_t cfg = pdl_config(1, 32, 0, s, &attr);
+    return cudaLaunchKernelEx(&cfg, cart_advance_kernel, ctr);
 }
 
 cudaError_t launch_append(const AppendParams &p, cudaStream_t s)
