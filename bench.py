@@ -274,10 +274,42 @@ def measure_side_workload(name: str, dev, stream, warmup: int, steps_per_block: 
             res["tensor_frac"] = roof["tensor"]["frac"]
         if L == 1:
             res["single_call"] = single_call_latency(lw, tensors, stream, dev)
+        res["recorded_loop"] = recorded_loop(lw, tensors, stream, dev, 30)
         return res
     finally:
         lw.close()
         torch.cuda.empty_cache()
+
+
+def recorded_loop(lw, tensors, stream, dev, steps: int) -> dict:
+    """The same decode steps as one CUDA graph per step: recorded once (cart_graph_begin / cart_graph_step), replayed
+    `steps` times back to back; CUDA events around the replays.  Needs room for steps + 3 more tokens per request."""
+    from paper_2506_06266_b200 import binding
+    q, k_new, v_new, out, lse = tensors
+    L = q.shape[0]
+    side = torch.cuda.Stream(device=dev)
+    side.wait_stream(stream)
+    with torch.cuda.stream(side):
+        binding.cart_graph_begin(lw.ctx, lw.req_list, steps + 3, side)
+        side.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            for layer in range(L):
+                binding.cart_graph_step(lw.ctx, layer, k_new[layer], v_new[layer], q[layer], out[layer], lse[layer], side)
+        for _ in range(3):
+            g.replay()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(side)
+        for _ in range(steps):
+            g.replay()
+        b.record(side)
+        b.synchronize()
+    ms = a.elapsed_time(b)
+    binding.cart_graph_end(lw.ctx, steps + 3)
+    lw.appended += steps + 3
+    binding.cart_sync_status(lw.ctx, stream)
+    return {"what": "one CUDA graph per decode step (all layers), recorded once and replayed; shared and stream kernel in turn",
+            "steps": steps, "us_per_step": round(ms * 1e3 / steps, 2), "us_per_layer": round(ms * 1e3 / steps / L, 2)}
 
 
 def single_call_latency(lw, tensors, stream, dev) -> dict:

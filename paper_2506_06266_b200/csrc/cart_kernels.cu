@@ -244,11 +244,7 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
         // before this one -- so the first suffix tile is fetched only after griddepcontrol.wait.
         bool waited = false;
         uint32_t grow = p.grow;
-        if (p.grow_ctr != nullptr) {  // the count lives in memory that the kernels before this one advance
-            pdl_wait();
-            waited = true;
-            grow = ld_volatile_u32(p.grow_ctr);
-        }
+        bool grow_known = p.grow_ctr == nullptr;  // else the count lives in memory that a kernel before this one advances
         uint32_t tails_seen = 0;  // tiles met so far that end with a new token
         // The next work item is requested while the copies of this one are issued: read at the item's start, it
         // held the ring back by a memory round trip per item, which short row groups cannot spare.
@@ -257,7 +253,17 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
         for (uint32_t it = item_begin; it < item_end && ok; ++it) {
             cart_work_item w = w_next;
             if (it + 1 < item_end) w_next = p.items[it + 1];
-            if (w.flags & CART_ITEM_TAIL) w.n_tok += grow;  // tokens appended since the plan was built
+            if (w.flags & CART_ITEM_TAIL) {
+                if (!grow_known) {  // (read at the first item that needs it: the Cartridge tiles before are fetched meanwhile)
+                    if (!waited) {
+                        pdl_wait();
+                        waited = true;
+                    }
+                    grow = ld_volatile_u32(p.grow_ctr);
+                    grow_known = true;
+                }
+                w.n_tok += grow;  // tokens appended since the plan was built
+            }
             const uint32_t k_row = w.k_row + (uint32_t)p.layer * w.layer_stride;
             const uint32_t v_row = w.v_row + (uint32_t)p.layer * w.layer_stride;
             const uint32_t ntiles = (w.n_tok + kTileTokens - 1) / kTileTokens;
