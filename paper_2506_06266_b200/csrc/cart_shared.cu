@@ -10,23 +10,28 @@
 //   producer warps  TMA loads of K tiles (warp 0, three stages) and V tiles (warp 2, two stages), 128 tokens
 //                   x 128 dims, 128-byte swizzle, completion on mbarriers
 //   MMA warp        one thread issues  S = Q K^T  (128 x 128 x 128, both operands from shared memory,
-//                   accumulator in tensor memory) two tiles ahead of the softmax, and  O += P V  (A operand
-//                   P from tensor memory, V from shared memory, one accumulator for the whole unit);
-//                   tcgen05.commit signals mbarriers
+//                   accumulator in tensor memory) one tile ahead of the softmax, and, per half x of the tile's
+//                   tokens,  O_x += P_x V_x  (A operand P_x from tensor memory, V from shared memory, one
+//                   accumulator per half for the whole unit); tcgen05.commit signals mbarriers
 //   2 x 4 softmax   both warpgroups work on every tile: thread (w, r) owns query row r (tensor-memory
-//   warps           lane r) and the 64 score columns of half w.  It reads its 64 scores once, the two
-//                   owners of a row exchange their maxima through shared memory, and each writes
-//                   P = 2^(s - m) as bf16 pairs over its own half of the score buffer (tcgen05.st).  The
-//                   reference m of a row only moves when the row's maximum has outgrown it by more
-//                   than 2^8 (then the two owners rescale their halves of the accumulator in tensor
-//                   memory); sums and accumulator always refer to the same reference, so the result is
-//                   exact.  At the end of a unit each thread reads its 64 columns of the accumulator,
-//                   the two owners add their sums, and the row leaves as a normalised fp32 partial.
+//   warps           lane r) and the 64 score columns (tokens) of half w.  It reads its 64 scores once and writes
+//                   P = 2^(s - m) as bf16 pairs over its own half of the score buffer (tcgen05.st).  Each half
+//                   of the tokens keeps a reference m, a sum and an accumulator of its own, so the two
+//                   warpgroups never wait for each other inside a unit: a half's P V product is issued when its
+//                   probabilities are there, and the warpgroups drift apart instead of meeting at the
+//                   exponential unit every tile (one accumulator and a per-tile exchange of maxima through
+//                   shared memory took 12 % longer per tile).  A reference only moves when the row's maximum
+//                   has outgrown it by more than 2^8 (then the warpgroup rescales its accumulator in tensor
+//                   memory); sum and accumulator always refer to the same reference, so the result is exact.
+//                   At the end of a unit the owners trade references and sums, each mixes its 64 output dims
+//                   from both accumulators by log-sum-exp weights, and the row leaves as a normalised fp32
+//                   partial (or, for a chain's last unit, as the bf16 output).
 //
-// Tensor memory: three score buffers (S0 S1 S2, with P inside) and one accumulator, 128 fp32 columns
-// each.  With three buffers the score products of tiles t+1 and t+2 are complete or in flight while the
-// softmax of tile t runs, so neither side waits for the other's latency: the tile rate is set by the
-// tensor pipe (16 instructions per tile) or by the exponentials (128 x 128 per tile), whichever is slower.
+// Tensor memory: two score buffers (S0 S1, with P inside) and the two accumulators, 128 fp32 columns each.
+// The score product of tile t+1 is complete or in flight while the softmax of tile t runs, and the one of tile
+// t+2 is queued right behind the P V products of tile t (the tensor pipe runs one thread's products in order),
+// so neither side waits for the other's latency: the tile rate is set by the tensor pipe (16 instructions per
+// tile) or by the exponentials (128 x 128 per tile), whichever is slower.
 // The partials of a (request, KV head) row group are merged by log-sum-exp either by the block that
 // delivers the last one -- this kernel's or the stream kernel's -- or, when the batch has more split row
 // groups than blocks, by a merge kernel that runs afterwards.
@@ -47,7 +52,7 @@ constexpr uint32_t kShBlock = 128u * 128u;            // 128 rows x 128 bytes: o
 constexpr uint32_t kShTileBytes = 2u * kShBlock;      // 128 x 128 bf16
 constexpr int kKStages = 3;                           // K tiles in flight (each ring has its own producer warp)
 constexpr int kVStages = 2;
-constexpr int kSBufs = 3;                             // score buffers in tensor memory
+constexpr int kSBufs = 2;                             // score buffers in tensor memory
 constexpr int kShThreads = 384;                       // utility warpgroup (K producer, MMA, V producer, 1 idle) + 2 softmax warpgroups
 // Registers per thread after the warpgroups have re-divided the block's allocation (384 x 168): the
 // utility warps need few, a softmax thread holds 64 scores and 32 packed probabilities.  4 x 32 x 40 + 8 x 32 x 232
@@ -55,8 +60,8 @@ constexpr int kShThreads = 384;                       // utility warpgroup (K pr
 constexpr int kRegsUtility = 40;
 constexpr int kRegsSoftmax = 232;
 constexpr int kSoftmaxThreads = 128;                  // one softmax warpgroup
-constexpr uint32_t kTmemCols = 512;                   // S0 S1 S2 (scores, then P), O (accumulator): 128 fp32 columns each
-constexpr uint32_t kTmemO = 3u * 128u;                // first column of the accumulator
+constexpr uint32_t kTmemCols = 512;                   // S0 S1 (scores, then P), O_a O_b (accumulators): 128 fp32 columns each
+constexpr uint32_t kTmemO = 2u * 128u;                // first column of the accumulators (one per softmax warpgroup)
 constexpr float kRescaleStep = 8.f;                   // how far a row's maximum may outgrow its reference (base-2 units)
 
 // shared-memory layout (offsets from a 1024-byte aligned base)
@@ -66,8 +71,8 @@ constexpr uint32_t kOffV = kOffK + kKStages * kShTileBytes;
 constexpr uint32_t kOffBar = kOffV + kVStages * kShTileBytes;
 constexpr uint32_t kOffMisc = kOffBar + 32 * 8;        // room for 32 barriers; then: tmem address, abort flag, unit flag
 constexpr uint32_t kOffFlags = kOffMisc + 16;          // one word per reader: "merge this row group"
-// what the two owners of a row tell each other: per tile their maxima (bf16 bits, [tile parity][half][row]);
-// at a unit's end their sums (fp32 [half][row], over the same bytes, behind a barrier)
+// what the two owners of a row tell each other at a unit's end: their references, then their sums (fp32 [half][row];
+// one after the other through the same kilobyte: shared memory has no room for both at once)
 constexpr uint32_t kOffXchg = kOffFlags + 128 * 4;
 constexpr uint32_t kShSmemUsed = kOffXchg + 2 * 128 * 4;
 constexpr uint32_t kShSmemBytes = kShSmemUsed + 1024;  // slack to align the base
@@ -75,19 +80,18 @@ static_assert(kShSmemBytes <= 232448, "shared memory budget of one sm_100 block 
 
 enum Bar : int {
     kBarKFull = 0,   // [kKStages] TMA -> MMA
-    kBarKEmpty = 3,  // (unused: the K producer listens on kBarSFull)
+    kBarKEmpty = 3,  // [kKStages] MMA (commit of the score product) -> K producer
     kBarVFull = 6,   // [kVStages]
     kBarVEmpty = 8,  // [kVStages]
     kBarSFull = 10,  // [kSBufs] MMA (commit) -> softmax
     kBarSFree = 13,  // [kSBufs] MMA (commit of P V) -> softmax: the accumulator holds the products up to this tile
-    kBarPReady = 16, // [kSBufs] softmax -> MMA         (8 arrivals: one per softmax warp)
+    kBarPReady = 16, // [kSBufs][2] softmax -> MMA: a warpgroup's half of the probabilities  (4 arrivals: one per warp)
     kBarQReady = 20, // [2] softmax -> MMA: a unit's query rows are in their buffer  (8 arrivals: one per softmax warp)
     kBarDrain = 24,  // MMA (commit) -> MMA, on the way out
 };
-static_assert(kKStages == kSBufs, "the K ring's stages are released through the score buffers' barriers");
 static_assert(kBarKEmpty - kBarKFull >= kKStages && kBarVFull - kBarKEmpty >= kKStages &&
               kBarVEmpty - kBarVFull >= kVStages && kBarSFull - kBarVEmpty >= kVStages &&
-              kBarSFree - kBarSFull >= kSBufs && kBarPReady - kBarSFree >= kSBufs && kBarQReady - kBarPReady >= kSBufs,
+              kBarSFree - kBarSFull >= kSBufs && kBarPReady - kBarSFree >= kSBufs && kBarQReady - kBarPReady >= 2 * kSBufs,
               "barrier indices overlap");
 
 // Instruction descriptor, kind::f16: fp32 accumulator, bf16 A and B, M = 128, N = 128.
@@ -103,14 +107,6 @@ __device__ __forceinline__ void softmax_bar_both()  // both softmax warpgroups
 {
     asm volatile("bar.sync 3, %0;" ::"n"(2 * kSoftmaxThreads) : "memory");
 }
-// A float rounded up to the next bf16 (upper 16 bits), for finite inputs: the exchanged row maxima only
-// have to be the same number for both owners of a row and not below the true maximum.
-__device__ __forceinline__ uint32_t bf16_ceil_bits(float x)
-{
-    const uint32_t b = __float_as_uint(x);
-    return ((b & 0x80000000u) ? b : b + 0xFFFFu) >> 16;  // negative: truncation already rounds up
-}
-
 // "The kernels before this one on the stream are complete and their writes visible."  Alone, that is
 // griddepcontrol.wait.  Side by side with the stream kernel (launched just before, resident at the same
 // time) it is a flag that the stream kernel's block 0 sets after its own griddepcontrol.wait: waiting for
@@ -181,6 +177,7 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
     if (threadIdx.x == 0) {
         for (int i = 0; i < kKStages; ++i) {
             mbar_init(bar(kBarKFull + i), 1);
+            mbar_init(bar(kBarKEmpty + i), 1);
         }
         for (int i = 0; i < kVStages; ++i) {
             mbar_init(bar(kBarVFull + i), 1);
@@ -189,7 +186,8 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
         for (int i = 0; i < kSBufs; ++i) {
             mbar_init(bar(kBarSFull + i), 1);
             mbar_init(bar(kBarSFree + i), 1);
-            mbar_init(bar(kBarPReady + i), 8);
+            mbar_init(bar(kBarPReady + 2 * i), 4);
+            mbar_init(bar(kBarPReady + 2 * i + 1), 4);
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar(kBarQReady + i), 8);
@@ -225,8 +223,7 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
             //  V ring is waiting for)
             if (lane == 0) {
                 const bool is_v = warp == 2;
-                // (a K stage is free once the score product that read it is complete: the barrier of score buffer tt % 3)
-                const int full0 = is_v ? kBarVFull : kBarKFull, empty0 = is_v ? kBarVEmpty : kBarSFull;
+                const int full0 = is_v ? kBarVFull : kBarKFull, empty0 = is_v ? kBarVEmpty : kBarKEmpty;
                 const uint32_t ring = base + (is_v ? kOffV : kOffK);
                 const uint32_t nst = is_v ? (uint32_t)kVStages : (uint32_t)kKStages;
                 asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap)) : "memory");
@@ -309,8 +306,8 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
             };
             uint32_t total = 0;
             for (uint32_t ui = unit_begin; ui < unit_end; ++ui) total += p.units[ui].n_tiles;
-            // S(tt) = Q K^T into score buffer tt % 3.  The buffer last held the probabilities of tile tt - 3,
-            // read by that tile's P V product, which this thread issued earlier: the tensor pipe executes one
+            // S(tt) = Q K^T into score buffer tt % 2.  The buffer last held the probabilities of tile tt - 2,
+            // read by that tile's P V products, which this thread issued earlier: the tensor pipe executes one
             // thread's products in the order of issue, so no completion has to be waited for here.
             auto issue_s = [&](uint32_t tt) -> bool {
                 const uint32_t sb = tt % (uint32_t)kSBufs;
@@ -330,18 +327,20 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                     const uint64_t off16 = (uint64_t)(((k >> 2) * kShBlock + (k & 3u) * 32u) >> 4);
                     umma_bf16(d_s, a0 + off16, b0 + off16, kIdescS, k, issue);
                 }
-                // one commit tells the softmax warps that the scores are there and the K producer that its
-                // stage is free (the K ring and the score buffers are both indexed by tt % 3)
+                // the softmax warps hear that the scores are there, the K producer that its stage is free
                 umma_commit(bar(kBarSFull + (int)sb), issue);
+                umma_commit(bar(kBarKEmpty + (int)kst), issue);
                 advance(qk);
                 return true;
             };
-            // O += P V (O = P V for a unit's first tile)
+            // O_x += P_x V_x for both halves x of the tile's tokens (O_x = P_x V_x for a unit's first tile): each softmax
+            // warpgroup owns 64 tokens of every tile, with a reference, a sum and an accumulator of its own, so
+            // its half of the product goes out as soon as its probabilities are there, whatever the other does
             auto issue_pv = [&](uint32_t tt) -> bool {
                 const uint32_t sb = tt % (uint32_t)kSBufs, spar = (tt / (uint32_t)kSBufs) & 1u;
                 const uint32_t vst = tt % (uint32_t)kVStages, vpar = (tt / (uint32_t)kVStages) & 1u;
                 if (!wait_all(kBarVFull + (int)vst, vpar)) return false;
-                if (!wait_all(kBarPReady + (int)sb, spar)) return false;
+                if (!wait_all(kBarPReady + 2 * (int)sb, spar)) return false;
                 tc_fence_after();
                 const uint32_t v_lo = base + kOffV + vst * kShTileBytes;
                 // P: the A operand comes from tensor memory, where the softmax warps left it inside the
@@ -352,11 +351,16 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                 const uint64_t b0 = umma_desc(v_lo, kShBlock, 1024);
                 const uint32_t p_tm = tmem + sb * 128u;
                 const uint32_t d_o = tmem + kTmemO;
-                const bool first = pv.t == 0u && pv.cont == 0u;  // (a unit that continues a chain adds to its accumulator)
+                const bool first = pv.t == 0u && pv.cont == 0u;  // (a unit that continues a chain adds to its accumulators)
 #pragma unroll
-                for (uint32_t k = 0; k < 8; ++k)  // 16 tokens per instruction
-                    umma_bf16_ts(d_o, p_tm + (k < 4u ? 8u * k : 64u + 8u * (k - 4u)), b0 + (uint64_t)(k * 128u), kIdescPV,
-                                 (first && k == 0u) ? 0u : 1u, issue);
+                for (uint32_t k = 0; k < 4; ++k)  // 16 tokens per instruction
+                    umma_bf16_ts(d_o, p_tm + 8u * k, b0 + (uint64_t)(k * 128u), kIdescPV, (first && k == 0u) ? 0u : 1u, issue);
+                if (!wait_all(kBarPReady + 2 * (int)sb + 1, spar)) return false;
+                tc_fence_after();
+#pragma unroll
+                for (uint32_t k = 4; k < 8; ++k)
+                    umma_bf16_ts(d_o + 128u, p_tm + 64u + 8u * (k - 4u), b0 + (uint64_t)(k * 128u), kIdescPV,
+                                 (first && k == 4u) ? 0u : 1u, issue);
                 umma_commit(bar(kBarVEmpty + (int)vst), issue);
                 umma_commit(bar(kBarSFree + (int)sb), issue);  // the accumulator holds the products up to this tile
                 advance(pv);
@@ -365,21 +369,11 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
             if (total > 0u) ok = issue_s(0u);
             if (ok && total > 1u) ok = issue_s(1u);
             for (uint32_t tt = 0; tt < total && ok; ++tt) {
-                // The score product two tiles on goes first, so that it is queued on the tensor pipe while the
-                // softmax of tile tt still runs -- unless it opens a unit whose query rows are not there yet:
-                // the softmax warps store them while they work on the unit before, which (for units of one
-                // tile) may need this tile's P V product first.
-                bool s_issued = tt + 2u >= total;
-                if (!s_issued) {
-                    const bool q_there = qk.t != 0u || qk.cont != 0u || __all_sync(0xffffffffu, mbar_try_wait(bar(kBarQReady + (int)(qk.unit_no & 1u)),
-                                                                                         (qk.unit_no >> 1) & 1u));
-                    if (q_there) {
-                        ok = issue_s(tt + 2u);
-                        s_issued = true;
-                    }
-                }
-                if (ok) ok = issue_pv(tt);
-                if (ok && !s_issued) ok = issue_s(tt + 2u);
+                // The scores of tile tt + 1 are in the other buffer already (or on the pipe), so the softmax of that
+                // tile starts the moment this tile's is over; the score product two tiles on reuses this tile's
+                // buffer and is queued right behind this tile's P V products.
+                ok = issue_pv(tt);
+                if (ok && tt + 2u < total) ok = issue_s(tt + 2u);
             }
             // products still in flight must finish before the tensor memory is given back
             umma_commit(bar(kBarDrain), issue);
@@ -397,8 +391,7 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
         const int tid = row;                  // index among the 128 threads of the warpgroup
         const uint32_t lane_addr = tmem + ((uint32_t)(32 * sw) << 16);
         const uint32_t col0 = 64u * (uint32_t)wg;
-        uint16_t *xchg_mx = reinterpret_cast<uint16_t *>(smem + kOffXchg);  // [tile parity][half][row]
-        float *xchg_l = reinterpret_cast<float *>(smem + kOffXchg);         // [half][row]
+        float *xchg = reinterpret_cast<float *>(smem + kOffXchg);           // [half][row]
         uint32_t tt = 0;      // tiles of the block so far
         bool alive = true;    // false once the block has given up: work is skipped, barriers are still met
         // the warp's lanes must stay together (the tensor-memory loads are warp-wide): a wait fails for
@@ -406,7 +399,7 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
         auto warp_wait = [&](uint32_t b, uint32_t parity) -> bool {
             return __all_sync(0xffffffffu, mbar_wait(b, parity, abort_flag, p.status, kStatusTimeoutConsumer));
         };
-        const uint32_t o_addr = lane_addr + kTmemO + col0;
+        const uint32_t o_addr = lane_addr + kTmemO + 128u * (uint32_t)wg;   // this warpgroup's accumulator: 128 columns
 
         // Query rows.  Thread (w, r) copies the 64-dim half w of row r (head r % G of the M-tile's reader r / G)
         // into the unit's query buffer, in the swizzled K-major operand layout: block w, row r, 16-byte chunk c
@@ -539,22 +532,17 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                     }
                     mx *= p.scale_log2;
                 }
-                // the row's maximum over the whole tile: the two owners trade their halves' maxima (rounded up to
-                // bf16, the same numbers on both sides, so both keep the same reference)
-                const uint32_t mine = bf16_ceil_bits(mx);
-                xchg_mx[((tt & 1u) * 2u + (uint32_t)wg) * 128u + (uint32_t)row] = (uint16_t)mine;
-                softmax_bar_both();
-                const uint32_t theirs = xchg_mx[((tt & 1u) * 2u + (uint32_t)(wg ^ 1)) * 128u + (uint32_t)row];
+                // the row's maximum over this warpgroup's 64 tokens: the two halves of a tile keep references, sums and
+                // accumulators of their own and only meet at the unit's end, so neither waits for the other per tile
                 if (!alive) continue;
-                const float m_tile = fmaxf(__uint_as_float(mine << 16), __uint_as_float(theirs << 16));
+                const float m_tile = mx;
                 if (fresh) {
                     m_run = m_tile;
                     fresh = false;
                 } else if (__any_sync(0xffffffffu, m_tile > m_run + kRescaleStep)) {
                     // a row of this warp has outgrown its reference: every row of the warp moves up to its
-                    // maximum and the two owners rescale their halves of the accumulator's lanes (tensor-memory
-                    // accesses are warp-wide, so the warp decides together, and its twin in the other warpgroup
-                    // sees the same numbers and decides the same; the other rows' factors are 1 or close to it)
+                    // maximum and rescales its lane of the warpgroup's accumulator (tensor-memory accesses are
+                    // warp-wide, so the warp decides together; the other rows' factors are 1 or close to it)
                     const float m_new = fmaxf(m_run, m_tile);
                     // (a row of a masked run may not have seen a key yet: its reference stays at -inf, factor 1)
                     const float f = m_new == -INFINITY ? 1.f : fast_exp2(m_run - m_new);
@@ -568,7 +556,7 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                     if (!alive) continue;
                     tc_fence_after();
 #pragma unroll
-                    for (int c = 0; c < 2; ++c) {
+                    for (int c = 0; c < 4; ++c) {
                         uint32_t o[32];
                         tmem_ld32_issue(o_addr + (uint32_t)c * 32u, o);
                         tmem_ld_wait(o);
@@ -601,14 +589,16 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                 if (masked && t + 1u == u.n_tiles && (uint32_t)(u.lim_cap + 1) < u.n_tiles * (uint32_t)kShTile) {
                     // The run ends inside this tile.  The rows behind its last key hold whatever follows in memory;
                     // their probabilities are zero, but 0 * NaN would poison the product, so those rows of the V tile
-                    // are cleared (both softmax warpgroups share the work) before the MMA warp hears of the tile.
+                    // are cleared before the MMA warp hears of the tile.
                     const uint32_t vst = tt % (uint32_t)kVStages, vpar = (tt / (uint32_t)kVStages) & 1u;
                     alive = warp_wait(bar(kBarVFull + (int)vst), vpar);
                     if (!alive) continue;
                     const uint32_t first_bad = (uint32_t)(u.lim_cap + 1) - t * (uint32_t)kShTile;   // 1 .. 127
                     const uint32_t v_lo = base + kOffV + vst * kShTileBytes;
-                    for (uint32_t x = (uint32_t)(wg * kSoftmaxThreads + tid); x < (128u - first_bad) * 16u; x += 2u * kSoftmaxThreads) {
-                        const uint32_t r = first_bad + x / 16u, c = x % 16u;
+                    // (this warpgroup's product reads the rows of its own 64 tokens only, and clears those)
+                    const uint32_t r_lo = first_bad > 64u * (uint32_t)wg ? first_bad : 64u * (uint32_t)wg, r_hi = 64u * (uint32_t)wg + 64u;
+                    for (uint32_t x = (uint32_t)tid; r_lo < r_hi && x < (r_hi - r_lo) * 16u; x += (uint32_t)kSoftmaxThreads) {
+                        const uint32_t r = r_lo + x / 16u, c = x % 16u;
                         asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(v_lo + (c >> 3) * kShBlock + r * 128u + ((c & 7u) << 4)),
                                      "r"(0u)
                                      : "memory");
@@ -618,7 +608,7 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                 tmem_st_wait();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(kBarPReady + (int)sb));
+                if (lane == 0) mbar_arrive(bar(kBarPReady + 2 * (int)sb + wg));
                 if (has_next) {
                     if (kChains && t == 0u) {
                         valid_next = (uint32_t)i_reader < uq.n_readers;
@@ -632,24 +622,44 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
             // ---- the unit's rows leave as normalised partials -------------------------------------------
             // (unless the next unit continues the same rows: then the state simply stays)
             if (hold) continue;
-            // Each thread reads its 64 columns of the accumulator once the last product has landed; the two
-            // owners of a row add their sums (in a fixed order, so the result does not depend on timing).
+            // The two halves of the row's keys meet here: the owners trade references and sums, and each writes 64 of
+            // the row's 128 output dims, mixed from both accumulators by log-sum-exp weights (in a fixed order, so
+            // the result does not depend on timing).  o[k]: the unnormalised output, l: the sum it is divided by,
+            // m_all: the reference both refer to.
             uint32_t o[64];
             if (alive) alive = warp_wait(bar(kBarSFree + (int)((tt - 1u) % (uint32_t)kSBufs)), ((tt - 1u) / (uint32_t)kSBufs) & 1u);
+            softmax_bar_both();  // the exchange area is free: the unit before has been read
+            xchg[wg * 128 + row] = m_run;
+            softmax_bar_both();
+            float2 theirs;
+            theirs.x = xchg[(wg ^ 1) * 128 + row];
+            softmax_bar_both();
+            xchg[wg * 128 + row] = l_run;
+            softmax_bar_both();
+            theirs.y = xchg[(wg ^ 1) * 128 + row];
+            const float m_all = fmaxf(m_run, theirs.x);
+            // (a half that saw no key has reference -inf and weight 0; a row that saw none at all has l = 0)
+            const float w_mine = m_all == -INFINITY ? 0.f : fast_exp2(m_run - m_all);
+            const float w_theirs = m_all == -INFINITY ? 0.f : fast_exp2(theirs.x - m_all);
+            const float w_a = wg == 0 ? w_mine : w_theirs, w_b = wg == 0 ? w_theirs : w_mine;
+            const float l = w_a * (wg == 0 ? l_run : theirs.y) + w_b * (wg == 0 ? theirs.y : l_run);
             if (alive) {
                 tc_fence_after();
-                tmem_ld32_issue(o_addr, reinterpret_cast<uint32_t(&)[32]>(o[0]));
-                tmem_ld32_issue(o_addr + 32u, reinterpret_cast<uint32_t(&)[32]>(o[32]));
-                tmem_ld_wait(reinterpret_cast<uint32_t(&)[32]>(o[0]));
-                tmem_ld_wait(reinterpret_cast<uint32_t(&)[32]>(o[32]));
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t a[32], b[32];
+                    tmem_ld32_issue(lane_addr + kTmemO + col0 + 32u * (uint32_t)c, a);
+                    tmem_ld32_issue(lane_addr + kTmemO + 128u + col0 + 32u * (uint32_t)c, b);
+                    tmem_ld_wait(a);
+                    tmem_ld_wait(b);
+#pragma unroll
+                    for (int k = 0; k < 32; ++k)
+                        o[32 * c + k] = __float_as_uint(w_a * __uint_as_float(a[k]) + w_b * __uint_as_float(b[k]));
+                }
                 tc_fence_before();
             }
-            softmax_bar_both();  // nobody reads the maxima of the last tile any more: the sums go over them
-            xchg_l[wg * 128 + row] = l_run;
-            softmax_bar_both();
             if (alive && valid && direct) {
                 // the chain covered the row's whole cache: the final output, rounded to bf16, and the lse
-                const float l = xchg_l[row] + xchg_l[128 + row];
                 const float inv = 1.f / l;
                 const size_t orow = (size_t)slot * p.n_q_heads + (size_t)u.kv_head * G + h;
                 __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(p.out) + orow * kHeadDim + col0;
@@ -663,11 +673,10 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                                  "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
                                  : "memory");
                 }
-                if (wg == 0 && p.lse) p.lse[orow] = (m_run + log2f(l)) * 0.6931471805599453f;
+                if (wg == 0 && p.lse) p.lse[orow] = (m_all + log2f(l)) * 0.6931471805599453f;
             } else if (alive && valid) {
                 // (a row that saw no key of the unit -- all of them beyond its causal limit -- leaves an empty partial:
                 //  zeros with lse = -inf, which the merge gives no weight)
-                const float l = xchg_l[row] + xchg_l[128 + row];
                 const float inv = l > 0.f ? 1.f / l : 0.f;
                 // 32 bytes per store: a thread writes a row by itself, so every store of a warp touches 32 rows, and
                 // 16-byte stores fill only half of each 32-byte sector they touch
@@ -680,7 +689,7 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                                  "f"(__uint_as_float(o[8 * q8 + 4]) * inv), "f"(__uint_as_float(o[8 * q8 + 5]) * inv),
                                  "f"(__uint_as_float(o[8 * q8 + 6]) * inv), "f"(__uint_as_float(o[8 * q8 + 7]) * inv)
                                  : "memory");
-                if (wg == 0) p.part_lse2[(size_t)slot * kMaxGroup + h] = l > 0.f ? m_run + log2f(l) : -INFINITY;
+                if (wg == 0) p.part_lse2[(size_t)slot * kMaxGroup + h] = l > 0.f ? m_all + log2f(l) : -INFINITY;
             }
             if (p.tickets == nullptr || direct) {
                 softmax_bar_both();  // the sums have been read: the next unit's maxima may be written
