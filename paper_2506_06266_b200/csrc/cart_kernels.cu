@@ -612,8 +612,11 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
 __global__ void __launch_bounds__(128) cart_merge_kernel(const MergeParams p)
 {
     pdl_launch_dependents();
+    // (the plan was uploaded before the kernels whose partials are merged here were launched: its entry is read
+    //  while those kernels still run, one memory round trip less behind them)
+    const cart_merge_item mi = p.merges[blockIdx.x];
     pdl_wait();  // the partials come from the kernels before
-    merge_row_group<1, 8>(p.merges[blockIdx.x], p.group, p.part_o, p.part_lse2, p.out, p.lse, (int)threadIdx.x, 128);
+    merge_row_group<1, 8>(mi, p.group, p.part_o, p.part_lse2, p.out, p.lse, (int)threadIdx.x, 128);
 }
 
 // One block per request: copy the new token's K and V rows (Hkv x 256 bytes each) to the suffix end.
