@@ -171,7 +171,9 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
     if (unit_begin < unit_end) {
         u_first = p.units[unit_begin];
         const uint32_t r0 = (threadIdx.x & 127u) / (uint32_t)p.group;
-        if (threadIdx.x >= 128u && r0 < u_first.n_readers) first_batch = p.readers[u_first.reader_begin + r0];
+        // (in a plan of chains reader entry t is query row t: the table is not consulted, one dependent read less)
+        if (threadIdx.x >= 128u && r0 < u_first.n_readers)
+            first_batch = kChains ? u_first.reader_begin + r0 : p.readers[u_first.reader_begin + r0];
     }
 
     if (threadIdx.x == 0) {
@@ -476,14 +478,14 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                 if (valid_next) batch_next = p.readers[uq.reader_begin + (uint32_t)i_reader];
             }
             // the tiles after which the next unit's rows are requested and stored: in a plan with chains the request
-            // hangs on two dependent reads issued above, which get two tiles' time
-            const uint32_t t_load = kChains ? (u.n_tiles > 2u ? 2u : u.n_tiles - 1u) : 0u;
-            const uint32_t t_store = kChains ? (u.n_tiles > 4u ? 4u : u.n_tiles - 1u) : (u.n_tiles > 1u ? 1u : 0u);
+            // hangs on the read of the next chain's first unit issued above, which gets a tile's time
+            const uint32_t t_load = kChains ? (u.n_tiles > 1u ? 1u : 0u) : 0u;
+            const uint32_t t_store = kChains ? (u.n_tiles > 3u ? 3u : u.n_tiles - 1u) : (u.n_tiles > 1u ? 1u : 0u);
             const bool direct = kChains && (u.flags & CART_UNIT_DIRECT) != 0u, hold = kChains && (u.flags & CART_UNIT_HOLD) != 0u;
             const bool masked = kChains && (u.flags & CART_UNIT_MASKED) != 0u;
             uint32_t slot = 0;   // where this row's partial goes, or (direct) its query row: needed at the unit's end
             if (valid && !hold)
-                slot = direct ? p.readers[u.reader_begin + (uint32_t)i_reader]
+                slot = direct ? u.reader_begin + (uint32_t)i_reader
                               : p.reader_slot[(size_t)(u.reader_begin + (uint32_t)i_reader) * p.n_kv_heads + u.kv_head] + u.chunk;
             // m_run: the reference that l_run and the accumulator in tensor memory refer to, the same for both
             // owners of the row.  It only moves when the row's maximum has outgrown it by more than
@@ -612,7 +614,7 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                 if (has_next) {
                     if (kChains && t == 0u) {
                         valid_next = (uint32_t)i_reader < uq.n_readers;
-                        if (valid_next) batch_next = p.readers[uq.reader_begin + (uint32_t)i_reader];
+                        if (valid_next) batch_next = uq.reader_begin + (uint32_t)i_reader;
                     }
                     if (t == t_load) load_q(q_src(uq.kv_head, batch_next), valid_next, (unit_no + 1u) & 1u);
                     if (t == t_store) store_q((unit_no + 1u) & 1u);
