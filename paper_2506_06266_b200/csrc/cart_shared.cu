@@ -693,10 +693,8 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
                                  : "memory");
                 if (wg == 0) p.part_lse2[(size_t)slot * kMaxGroup + h] = l > 0.f ? m_all + log2f(l) : -INFINITY;
             }
-            if (p.tickets == nullptr || direct) {
-                softmax_bar_both();  // the sums have been read: the next unit's maxima may be written
-                continue;
-            }
+            // (the exchange area is written next behind the first barrier of the next unit's end: nothing to wait for here)
+            if (p.tickets == nullptr || direct) continue;
 
             // ---- arrival tickets (when no merge kernel follows) -------------------------------------------
             __threadfence();  // publish the partials before the tickets
