@@ -308,7 +308,7 @@ def recorded_loop(lw, tensors, stream, dev, steps: int) -> dict:
     binding.cart_graph_end(lw.ctx, steps + 3)
     lw.appended += steps + 3
     binding.cart_sync_status(lw.ctx, stream)
-    return {"what": "one CUDA graph per decode step (all layers), recorded once and replayed; shared and stream kernel in turn",
+    return {"what": "one CUDA graph per decode step (all layers), recorded once and replayed",
             "steps": steps, "us_per_step": round(ms * 1e3 / steps, 2), "us_per_layer": round(ms * 1e3 / steps / L, 2)}
 
 

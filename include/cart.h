@@ -232,8 +232,7 @@ CART_API cart_status cart_decode_step(cart_ctx *ctx, int32_t layer, const cart_r
  *       what cart_decode_step computes for `layer` of the batch given to cart_graph_begin, in its order; only
  *       kernel launches, so the calls for layers 0 .. n_layers - 1 of ONE step can be captured (stream capture or
  *       explicit nodes) and replayed; after the last layer's kernels a one-thread kernel advances the count.  The
- *       pointers are recorded: refill the same buffers between replays.  A batch with shared Cartridges runs its
- *       tensor-core kernel and its stream kernel one after the other here, not side by side.
+ *       pointers are recorded: refill the same buffers between replays.
  *   cart_graph_end(ctx, steps_run)
  *       host only: the step ran steps_run times (<= max_steps), every request is that much longer in every layer.
  *

@@ -163,7 +163,6 @@ struct cart_ctx {
     std::vector<int32_t> graph_reqs;
     int graph_slot = -1;
     int32_t graph_max_steps = 0;
-    uint32_t pair_seq = 0;       // counts side-by-side launches (the value the stream kernel hands to the shared kernel)
     uint64_t plans_built = 0;
     uint64_t n_rows = 0;
     alignas(64) CUtensorMap tmap;
@@ -994,8 +993,7 @@ namespace {
 // that are whole conversations over one Cartridge: the forward of training-time attention.)
 // Launches the kernels of a plan for one layer: the stream kernel, the tensor-core kernel for the shared part and the
 // merge kernel, as the plan needs them.  grow: tokens every request has appended since the plan was built, or, with
-// grow_ctr set, the device word that holds that count (a launch recorded in a CUDA graph: the shared and the stream
-// kernel then run one after the other, since their side-by-side handshake carries a launch number as a parameter).
+// grow_ctr set, the device word that holds that count (a launch recorded in a CUDA graph).
 cart_status launch_plan(cart_ctx *ctx, PlanSlot *sl, int32_t layer, const void *q, void *out, float *lse, const void *k_new,
                         const void *v_new, int32_t grow, const uint32_t *grow_ctr, cudaStream_t s)
 {
@@ -1039,10 +1037,9 @@ cart_status launch_plan(cart_ctx *ctx, PlanSlot *sl, int32_t layer, const void *
     // A batch with a shared part and a stream part runs the two kernels side by side: the stream kernel
     // is launched first on its share of the SMs, the shared kernel right behind it on the rest (a dependent
     // launch starts as soon as every block of the kernel before has started).
-    const bool pair = sl->n_units > 0 && sl->n_items > 0 && ctx->side_by_side > 0 && grow_ctr == nullptr;
+    const bool pair = sl->n_units > 0 && sl->n_items > 0 && ctx->side_by_side > 0;
     if (pair) {
         dp.ready_flag = reinterpret_cast<uint32_t *>(arena + ctx->lay.status_off + 128);
-        dp.seq = ++ctx->pair_seq;
     }
     if (pair) {
         CART_CUDA(ctx, launch_decode(ctx->tmap, ctx->tmap_edge, dp, sl->n_cta_used, s));
@@ -1069,7 +1066,6 @@ cart_status launch_plan(cart_ctx *ctx, PlanSlot *sl, int32_t layer, const void *
         sp.n_q_heads = ctx->cfg.n_q_heads;
         sp.scale_log2 = dp.scale_log2;
         sp.ready_flag = dp.ready_flag;
-        sp.seq = dp.seq;
         sp.pages = dp.pages;
         CART_CUDA(ctx, launch_shared(ctx->tmap, sp, sl->n_unit_cta_used, s));
         ++ctx->launches;
@@ -1300,7 +1296,7 @@ cart_status decode_impl(cart_ctx *ctx, int32_t layer, const cart_req *reqs, int3
         po.slots_cap = lay.slots_cap;
         po.piece_cost = ctx->piece_cost;
         po.unit_cost = kUnitCostTiles;
-        po.side_by_side = ctx->plan_only ? 0 : ctx->side_by_side;   // (a recorded loop runs the two kernels in turn)
+        po.side_by_side = ctx->side_by_side;
         po.units = reinterpret_cast<cart_shared_unit *>(ns.host + lay.units_off);
         po.units_cap = lay.units_cap;
         po.unit_cta_begin = reinterpret_cast<uint32_t *>(ns.host + lay.unit_cta_begin_off);

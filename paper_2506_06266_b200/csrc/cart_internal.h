@@ -42,11 +42,10 @@ struct DecodeParams {
     int32_t group;               // G
     float scale_log2;            // softmax scale * log2(e)
     // Side by side with the shared-segment kernel (launched right after this one, resident at the same
-    // time): once this kernel knows that the kernels before it are complete, block 0 stores `seq` here and
+    // time): once this kernel knows that the kernels before it are complete, block 0 stores 1 here and
     // the shared kernel, which cannot learn it from griddepcontrol.wait without waiting for this kernel
-    // too, reads it.  Null otherwise.
+    // too, reads it; the shared kernel's last block clears it on its way out.  Null otherwise.
     uint32_t *ready_flag = nullptr;
-    uint32_t seq = 0;
     uint32_t grow = 0;           // tokens every request has appended since the plan was built: added to the token
                                  // count of every item marked CART_ITEM_TAIL
     const uint32_t *grow_ctr = nullptr;  // if set, that number is read from here instead (a launch recorded in a CUDA
@@ -79,10 +78,11 @@ struct SharedParams {
     int32_t n_q_heads;
     float scale_log2;
     // Side by side with the stream kernel (launched right before this one): "the kernels before the pair
-    // are complete" is read from this flag (>= seq) instead of griddepcontrol.wait, which this kernel then
-    // only executes on its way out, so that it never completes before the stream kernel.  Null: alone.
-    const uint32_t *ready_flag = nullptr;
-    uint32_t seq = 0;
+    // are complete" is read from this flag (1 once they are) instead of griddepcontrol.wait, which this kernel
+    // then only executes on its way out, so that it never completes before the stream kernel; the block that
+    // leaves last (counted in the word behind the flag) clears the flag for the next pair.  No launch number is
+    // involved, so the pair can be recorded into a CUDA graph.  Null: alone.
+    uint32_t *ready_flag = nullptr;
     const uint32_t *pages = nullptr;  // page list (units marked CART_UNIT_PAGED)
 };
 

@@ -519,7 +519,7 @@ cart_decode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
     // ===================== consumers ==============================================================
     pdl_wait();  // q, the partial slots and the tickets belong to the kernels before until they are done
     if (p.ready_flag != nullptr && blockIdx.x == 0 && threadIdx.x == 0)  // tell the kernel that runs beside this one
-        asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.ready_flag), "r"(p.seq) : "memory");
+        asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.ready_flag), "r"(1u) : "memory");
     const uint32_t grow = p.grow_ctr != nullptr ? ld_volatile_u32(p.grow_ctr) : p.grow;
     const int G = p.group;
     const int row = lane >> 2;  // query head inside the group that this thread's c0/c1 belong to

@@ -125,7 +125,7 @@ __device__ __forceinline__ bool wait_for_prior_kernels(const SharedParams &p, vo
     for (;;) {
         uint32_t v;
         asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p.ready_flag) : "memory");
-        if ((int32_t)(v - p.seq) >= 0) return true;
+        if (v == 1u) return true;
         if ((++spins & 0xFFu) == 0) {
             if (*abort_flag) return false;
             const long long now = clock64();
@@ -736,7 +736,15 @@ cart_shared_kernel(const __grid_constant__ CUtensorMap tmap, const SharedParams 
     }
     // Side by side: this kernel must not complete before the stream kernel does, because the kernel after
     // this one takes this kernel's completion for that of everything before it.
-    if (p.ready_flag != nullptr && threadIdx.x == 0) pdl_wait();
+    if (p.ready_flag != nullptr && threadIdx.x == 0) {
+        pdl_wait();
+        // every block has read the flag by the time it gets here; the last one clears it (and the count) for the next
+        // pair, whose stream kernel sets it only after this kernel is complete
+        if (atomicAdd(p.ready_flag + 1, 1u) == gridDim.x - 1u) {
+            p.ready_flag[1] = 0u;
+            p.ready_flag[0] = 0u;
+        }
+    }
 }
 
 }  // namespace

@@ -79,7 +79,7 @@ def test_replayed_step_grows_private_caches_across_a_tile_boundary():
     run_loop(synth.Workload("graph_priv", 511, 3, 24, 8, 6, 300, 60, 66), steps=8)
 
 
-def test_replayed_step_over_a_shared_cartridge_runs_its_two_kernels_in_turn():
+def test_replayed_step_over_a_shared_cartridge():
     run_loop(synth.shrink(synth.config3(), n_layers=2, batch=21, p=512, suffix_lo=1, suffix_hi=140), steps=4)
 
 
